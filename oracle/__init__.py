@@ -1,0 +1,305 @@
+"""ctypes front end of the CPU oracle (oracle/twn_oracle.c).  TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg import
+this package.  It shares nothing with the CUDA library.  Arrays are numpy;
+bf16 tensors are uint16 bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_DIR = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_DIR, "twn_oracle.c")
+_LIB = os.path.join(_DIR, "libtwn_oracle.so")
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (OpenMP, -O2, strict IEEE: no -ffast-math)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared",
+                               "-ffp-contract=off", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+class ConvDesc(C.Structure):
+    _fields_ = [("B", C.c_int64), ("H", C.c_int64), ("W", C.c_int64), ("Cin", C.c_int64),
+                ("Cout", C.c_int64), ("kh", C.c_int32), ("kw", C.c_int32),
+                ("stride_h", C.c_int32), ("stride_w", C.c_int32),
+                ("pad_h", C.c_int32), ("pad_w", C.c_int32)]
+
+    @property
+    def Ho(self):
+        return (self.H + 2 * self.pad_h - self.kh) // self.stride_h + 1
+
+    @property
+    def Wo(self):
+        return (self.W + 2 * self.pad_w - self.kw) // self.stride_w + 1
+
+
+def conv_desc(B, H, W, Cin, Cout, k, stride=1, pad=0) -> ConvDesc:
+    kh, kw = (k, k) if isinstance(k, int) else k
+    return ConvDesc(B, H, W, Cin, Cout, kh, kw, stride, stride, pad, pad)
+
+
+class _Stats(C.Structure):
+    _fields_ = [("delta", C.c_double), ("alpha", C.c_double), ("sum_abs", C.c_double),
+                ("sum_abs_kept", C.c_double), ("n_neg", C.c_int64), ("n_zero", C.c_int64),
+                ("n_pos", C.c_int64), ("n_boundary", C.c_int64), ("nonfinite", C.c_int32),
+                ("pad_", C.c_int32)]
+
+
+class _Epi(C.Structure):
+    _fields_ = [("scale", C.c_void_p), ("shift", C.c_void_p), ("residual", C.c_void_p),
+                ("relu", C.c_int32), ("pad_", C.c_int32)]
+
+
+@dataclass
+class Stats:
+    delta: float
+    alpha: float
+    sum_abs: float
+    sum_abs_kept: float
+    n_neg: int
+    n_zero: int
+    n_pos: int
+    n_boundary: int
+    nonfinite: bool
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.ref_alpha_alg1.restype = C.c_double
+        _lib.ref_sum_abs_ld.restype = C.c_double
+        _lib.ref_objective.restype = C.c_double
+        _lib.ref_num_threads.restype = C.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().ref_num_threads())
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _f32(a):
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def _u16(a):
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.uint16, "bf16 tensors are passed as uint16 bit patterns"
+    return a
+
+
+def _i8(a):
+    return np.ascontiguousarray(a, dtype=np.int8)
+
+
+def _epi(N, scale=None, shift=None, residual=None, relu=False):
+    keep = []
+    e = _Epi()
+    if scale is not None:
+        s = _f32(scale); assert s.size == N; keep.append(s); e.scale = s.ctypes.data
+    if shift is not None:
+        s = _f32(shift); assert s.size == N; keep.append(s); e.shift = s.ctypes.data
+    if residual is not None:
+        r = np.ascontiguousarray(residual, dtype=np.float64); keep.append(r); e.residual = r.ctypes.data
+    e.relu = int(bool(relu))
+    return e, keep
+
+
+# ---------------------------------------------------------------- ternarize
+def ternarize(W, delta_factor: float = 0.7, want_codes: bool = True):
+    """Eq. 3, Eq. 5 and the threshold rule on the flattened tensor W (fp32).
+    Returns (Stats, int8 codes shaped like W or None)."""
+    w = _f32(W)
+    st = _Stats()
+    codes = np.empty(w.shape, dtype=np.int8) if want_codes else None
+    lib().ref_ternarize(_p(w), C.c_int64(w.size), C.c_double(delta_factor), C.byref(st), _p(codes))
+    return Stats(st.delta, st.alpha, st.sum_abs, st.sum_abs_kept, st.n_neg, st.n_zero, st.n_pos,
+                 st.n_boundary, bool(st.nonfinite)), codes
+
+
+def alpha_alg1(W, codes) -> float:
+    w, c = _f32(W), _i8(codes)
+    return float(lib().ref_alpha_alg1(_p(w), _p(c), C.c_int64(w.size)))
+
+
+def sum_abs_ld(W) -> float:
+    w = _f32(W)
+    return float(lib().ref_sum_abs_ld(_p(w), C.c_int64(w.size)))
+
+
+def objective(W, codes, alpha) -> float:
+    w, c = _f32(W), _i8(codes)
+    return float(lib().ref_objective(_p(w), _p(c), C.c_double(alpha), C.c_int64(w.size)))
+
+
+def bruteforce_threshold(W):
+    w = _f32(W)
+    d, a, j, f = C.c_double(), C.c_double(), C.c_double(), C.c_double()
+    rc = lib().ref_bruteforce_threshold(_p(w), C.c_int64(w.size), C.byref(d), C.byref(a),
+                                        C.byref(j), C.byref(f))
+    assert rc == 0
+    return d.value, a.value, j.value, f.value
+
+
+def bruteforce_enum(W):
+    w = _f32(W)
+    codes = np.zeros(w.size, dtype=np.int8)
+    a, j = C.c_double(), C.c_double()
+    rc = lib().ref_bruteforce_enum(_p(w), C.c_int64(w.size), _p(codes), C.byref(a), C.byref(j))
+    assert rc == 0
+    return codes, a.value, j.value
+
+
+# --------------------------------------------------------------------- pack
+def ld_for(cols: int, multiple: int = 64) -> int:
+    return (cols + multiple - 1) // multiple * multiple
+
+
+def pack(codes, ld_codes: int | None = None):
+    c = _i8(codes)
+    c2 = c.reshape(1, -1) if c.ndim == 1 else c.reshape(c.shape[0], -1)
+    rows, cols = c2.shape
+    ld = ld_for(cols) if ld_codes is None else ld_codes
+    out = np.empty((rows, ld // 16), dtype=np.uint32)
+    rc = lib().ref_pack(_p(c2), C.c_int64(rows), C.c_int64(cols), C.c_int64(ld), _p(out))
+    if rc != 0:
+        raise ValueError(f"ref_pack failed ({rc})")
+    return out
+
+
+def unpack(packed, rows: int, cols: int, ld_codes: int):
+    p = np.ascontiguousarray(packed, dtype=np.uint32)
+    out = np.empty((rows, cols), dtype=np.int8)
+    rc = lib().ref_unpack(_p(p), C.c_int64(rows), C.c_int64(cols), C.c_int64(ld_codes), _p(out))
+    if rc != 0:
+        raise ValueError(f"ref_unpack failed ({rc})")
+    return out
+
+
+# ------------------------------------------------------------- contractions
+def gemm(X, T, alpha, scale=None, shift=None, residual=None, relu=False):
+    """X: uint16 [M, K] bf16 bits; T: int8 [N, K].  Returns (Y, A) fp64 [M, N]."""
+    x, t = _u16(X), _i8(T)
+    M, K = x.shape
+    N = t.shape[0]
+    assert t.shape[1] == K
+    e, keep = _epi(N, scale, shift, residual, relu)
+    Y = np.empty((M, N)); A = np.empty((M, N))
+    lib().ref_gemm(_p(x), C.c_int64(K), _p(t), C.c_double(alpha), C.c_int64(M), C.c_int64(N),
+                   C.c_int64(K), C.byref(e), _p(Y), _p(A))
+    return Y, A
+
+
+def conv2d_fwd(d: ConvDesc, X, T, alpha, scale=None, shift=None, residual=None, relu=False,
+               pixels=None):
+    """X: uint16 [B,H,W,Cin]; T: int8 [Cout,kh,kw,Cin].  Returns (Y, A) fp64
+    [B,Ho,Wo,Cout], or [len(pixels), Cout] when a list of flat output pixels is given."""
+    x, t = _u16(X), _i8(T)
+    assert x.size == d.B * d.H * d.W * d.Cin and t.size == d.Cout * d.kh * d.kw * d.Cin
+    e, keep = _epi(d.Cout, scale, shift, residual, relu)
+    if pixels is None:
+        shape = (d.B, d.Ho, d.Wo, d.Cout)
+        Y = np.empty(shape); A = np.empty(shape)
+        lib().ref_conv2d_fwd(C.byref(d), _p(x), _p(t), C.c_double(alpha), C.byref(e), _p(Y), _p(A))
+    else:
+        pix = np.ascontiguousarray(pixels, dtype=np.int64)
+        Y = np.empty((pix.size, d.Cout)); A = np.empty((pix.size, d.Cout))
+        lib().ref_conv2d_fwd_pixels(C.byref(d), _p(x), _p(t), C.c_double(alpha), C.byref(e),
+                                    _p(pix), C.c_int64(pix.size), _p(Y), _p(A))
+    return Y, A
+
+
+def conv2d_bwd_data(d: ConvDesc, dZ, T, alpha, pixels=None):
+    """dZ: uint16 [B,Ho,Wo,Cout]; returns (dX, A) fp64 [B,H,W,Cin] (scatter form) or
+    [len(pixels), Cin] (gather form) for flat input pixels."""
+    g, t = _u16(dZ), _i8(T)
+    assert g.size == d.B * d.Ho * d.Wo * d.Cout
+    if pixels is None:
+        shape = (d.B, d.H, d.W, d.Cin)
+        dX = np.empty(shape); A = np.empty(shape)
+        lib().ref_conv2d_bwd_data(C.byref(d), _p(g), _p(t), C.c_double(alpha), _p(dX), _p(A))
+    else:
+        pix = np.ascontiguousarray(pixels, dtype=np.int64)
+        dX = np.empty((pix.size, d.Cin)); A = np.empty((pix.size, d.Cin))
+        lib().ref_conv2d_bwd_data_pixels(C.byref(d), _p(g), _p(t), C.c_double(alpha), _p(pix),
+                                         C.c_int64(pix.size), _p(dX), _p(A))
+    return dX, A
+
+
+def conv2d_bwd_weight(d: ConvDesc, X, dZ, entries=None):
+    """Straight-through dW, fp64 [Cout,kh,kw,Cin] or one value per flat entry index."""
+    x, g = _u16(X), _u16(dZ)
+    if entries is None:
+        shape = (d.Cout, d.kh, d.kw, d.Cin)
+        dW = np.empty(shape); A = np.empty(shape)
+        lib().ref_conv2d_bwd_weight(C.byref(d), _p(x), _p(g), None, C.c_int64(0), _p(dW), _p(A))
+    else:
+        idx = np.ascontiguousarray(entries, dtype=np.int64)
+        dW = np.empty(idx.size); A = np.empty(idx.size)
+        lib().ref_conv2d_bwd_weight(C.byref(d), _p(x), _p(g), _p(idx), C.c_int64(idx.size),
+                                    _p(dW), _p(A))
+    return dW, A
+
+
+# --------------------------------------------------- glue (textbook, numpy)
+def maxpool(x, k: int, stride: int, pad: int = 0):
+    """x: fp64 [B,H,W,C]; window k x k, -inf padding.  Returns (y, argmax flat
+    index into the H*W plane of each image) with the first maximum in scan order."""
+    B, H, W, Cc = x.shape
+    Ho = (H + 2 * pad - k) // stride + 1
+    Wo = (W + 2 * pad - k) // stride + 1
+    y = np.full((B, Ho, Wo, Cc), -np.inf)
+    arg = np.zeros((B, Ho, Wo, Cc), dtype=np.int64)
+    for r in range(k):
+        for s in range(k):
+            for ho in range(Ho):
+                h = ho * stride - pad + r
+                if h < 0 or h >= H:
+                    continue
+                wo_lo = max(0, -(-(pad - s) // stride))
+                wo_hi = min(Wo, (W - 1 + pad - s) // stride + 1)
+                if wo_hi <= wo_lo:
+                    continue
+                ws = np.arange(wo_lo, wo_hi) * stride - pad + s
+                cand = x[:, h, ws, :]
+                cur = y[:, ho, wo_lo:wo_hi, :]
+                better = cand > cur
+                y[:, ho, wo_lo:wo_hi, :] = np.where(better, cand, cur)
+                a = arg[:, ho, wo_lo:wo_hi, :]
+                arg[:, ho, wo_lo:wo_hi, :] = np.where(better, (h * W + ws)[None, :, None], a)
+    return y, arg
+
+
+def maxpool_bwd(dy, arg, H: int, W: int):
+    """Route each output gradient to the input position recorded in arg."""
+    B, Ho, Wo, Cc = dy.shape
+    dx = np.zeros((B, H * W, Cc))
+    b = np.arange(B)[:, None, None, None]
+    c = np.arange(Cc)[None, None, None, :]
+    np.add.at(dx, (np.broadcast_to(b, arg.shape), arg, np.broadcast_to(c, arg.shape)), dy)
+    return dx.reshape(B, H, W, Cc)
+
+
+def global_avgpool(x):
+    return x.mean(axis=(1, 2))
+
+
+def global_avgpool_bwd(dy, H: int, W: int):
+    return np.broadcast_to(dy[:, None, None, :] / (H * W), (dy.shape[0], H, W, dy.shape[1])).copy()
