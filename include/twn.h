@@ -1,0 +1,155 @@
+/*
+ * twn.h -- C ABI of the Ternary Weight Networks hot path for NVIDIA B200 (sm_100a).
+ *
+ * Threshold ternarization of fp32 master weights with 2-bit packing, and the
+ * ternary-weight contractions (inner product, convolution forward, backward
+ * for data, straight-through weight gradient) that consume the packed codes.
+ *
+ * General rules
+ *   - Every pointer is a DEVICE pointer unless its comment says "host".
+ *   - The caller owns every buffer.  Unless a function says otherwise it
+ *     allocates nothing, frees nothing and keeps no pointer after it returns.
+ *   - Work is enqueued on `stream` (a cudaStream_t) and the call returns after
+ *     the launch; results are ready when the stream reaches that point.
+ *   - Return value: TWN_OK or a negative twn_status.  Errors that the host can
+ *     see (bad sizes, misalignment, NULL) are returned before anything is
+ *     launched.  Errors only the device can see (non-finite weights, invalid
+ *     codes, a bounded wait that ran out) are written to `status` of the
+ *     twn_stats_t / status word the call was given and read back with
+ *     twn_read_status() after the caller synchronises.
+ *   - Results are deterministic: same inputs, same bits.
+ *   - bf16 tensors are passed as `const void*` / `void*`; conv tensors are
+ *     NHWC; filters are [Cout][kh][kw][Cin] with Cin fastest.
+ *   - There is no CPU path.  On a device that is not sm_100 every compute
+ *     call returns TWN_ERR_UNSUPPORTED_ARCH.
+ */
+#ifndef TWN_H_
+#define TWN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st *twn_stream_t; /* == cudaStream_t */
+
+typedef enum {
+    TWN_OK = 0,
+    TWN_ERR_INVALID_ARG = -1,
+    TWN_ERR_MISALIGNED = -2,
+    TWN_ERR_WORKSPACE = -3,
+    TWN_ERR_NONFINITE = -4,   /* device: a master weight is NaN or +-Inf           */
+    TWN_ERR_TIMEOUT = -5,     /* device: a bounded wait inside a kernel ran out    */
+    TWN_ERR_CUDA = -6,        /* a CUDA runtime / driver call failed               */
+    TWN_ERR_UNSUPPORTED_ARCH = -7,
+    TWN_ERR_BAD_CODE = -8     /* device: an int8 code outside {-1,0,+1}            */
+} twn_status;
+
+enum { TWN_F32 = 0, TWN_BF16 = 1 };
+
+/* Result of one ternarization; lives in device memory so that the contraction
+ * kernels read alpha without a host round trip.  64 bytes. */
+typedef struct {
+    double delta;        /* threshold: delta_factor * (1/n) * sum |W_i|  (Sec. 2.3)     */
+    double alpha;        /* scale: mean of |W_i| over |W_i| > delta, 0 if none (Eq. 5)  */
+    double sum_abs;      /* sum |W_i|                                                  */
+    double sum_abs_kept; /* sum of |W_i| over |W_i| > delta                            */
+    uint64_t n_neg, n_zero, n_pos; /* code counts, padding excluded                    */
+    int32_t status;      /* twn_status written by the device                           */
+    int32_t reserved;
+} twn_stats_t;
+
+/* Convolution geometry.  Output extent Ho = (H + 2*pad_h - kh)/stride_h + 1. */
+typedef struct {
+    int64_t B, H, W, Cin, Cout;
+    int32_t kh, kw, stride_h, stride_w, pad_h, pad_w;
+} twn_conv_desc_t;
+
+/* What follows the contraction, per output element with channel n:
+ *   y = acc * alpha;  y = y * scale[n] + shift[n];  y += residual;  y = max(y, 0)
+ * each step only if its field is set.  (Eq. 2 puts alpha on the input; a scalar
+ * commutes with the sum, so it is applied once per output here.) */
+typedef struct {
+    const float *scale;    /* fp32 [N] or NULL (folded batch-norm scale)            */
+    const float *shift;    /* fp32 [N] or NULL                                      */
+    const void *residual;  /* same shape and leading dimension as Y, or NULL        */
+    int32_t residual_dtype;/* TWN_F32 | TWN_BF16                                    */
+    int32_t relu;          /* 0 | 1                                                 */
+    int32_t out_dtype;     /* TWN_F32 | TWN_BF16 (round to nearest even)            */
+    int32_t reserved;
+} twn_epilogue_t;
+
+/* ---- library ---------------------------------------------------------- */
+
+/* Text for a twn_status.  Host; static storage. */
+const char *twn_strerror(int status);
+
+/* Copies the device status word at `dev_status` (e.g. &stats->status) to
+ * *host_out with a blocking copy on `stream`.  Returns TWN_OK or TWN_ERR_CUDA. */
+int twn_read_status(const int32_t *dev_status, int32_t *host_out, twn_stream_t stream);
+
+/* ---- ternarization (Sec. 2.3: Eq. 3, Eq. 5, threshold rule; Algorithm 1) -- */
+
+/* Bytes of scratch twn_ternarize needs (independent of the tensor size). */
+size_t twn_ternarize_workspace_bytes(void);
+
+/*
+ * Per-layer threshold ternarization fused with 2-bit packing.
+ *   delta  = delta_factor * (1/n) * sum_i |W_i|,  n = rows*cols (zeros count)
+ *   code_i = +1 if W_i > delta, -1 if W_i < -delta, 0 if |W_i| <= delta   (Eq. 3)
+ *   alpha  = mean of |W_i| over { i : |W_i| > delta }                      (Eq. 5)
+ * The paper's rule of thumb is delta_factor = 0.75; any value >= 0 is accepted.
+ *
+ * W        fp32 [rows, cols], contiguous, 16-byte aligned.  rows = filters
+ *          (output channels), cols = fan-in.
+ * stats    one twn_stats_t, 8-byte aligned; written completely.
+ * packed   uint32 [rows][ld_codes/16].  Code j of a row occupies bits
+ *          [2*(j%16)+1 : 2*(j%16)] of word j/16: 00 = 0, 01 = +1, 11 = -1.
+ *          ld_codes is a multiple of 64 (rows start 16-byte aligned),
+ *          ld_codes >= cols; the padding is written as 00.  16-byte aligned.
+ * codes_i8 optional int8 [rows, cols] copy of the codes (16-byte aligned), or NULL.
+ * workspace/workspace_bytes  scratch of at least twn_ternarize_workspace_bytes(),
+ *          256-byte aligned; contents need not be preserved or initialised.
+ *          Two calls that overlap on the device must not share it.
+ * The sums are fp64 with a fixed reduction order.  The comparison is done in
+ * fp32 against delta rounded toward -inf, which decides exactly as the fp64
+ * comparison does.  n = 0 gives delta = alpha = 0.
+ * Device status: TWN_ERR_NONFINITE if any W_i is NaN/Inf (other outputs
+ * are then unspecified).
+ */
+int twn_ternarize(const float *W, int64_t rows, int64_t cols, double delta_factor,
+                  twn_stats_t *stats, uint32_t *packed, int64_t ld_codes,
+                  int8_t *codes_i8, void *workspace, size_t workspace_bytes,
+                  twn_stream_t stream);
+
+/* ---- 2-bit storage (Sec. 2.1, model compression) ------------------------- */
+
+/*
+ * Packs int8 codes in {-1,0,+1} ([rows, cols], contiguous) into the layout
+ * described at twn_ternarize.  `counts` (optional) receives n_neg/n_zero/n_pos
+ * and a status; its other fields are zeroed.  A code outside {-1,0,+1} sets
+ * TWN_ERR_BAD_CODE there (and packs as 0).
+ */
+int twn_pack(const int8_t *codes, int64_t rows, int64_t cols, uint32_t *packed,
+             int64_t ld_codes, twn_stats_t *counts, twn_stream_t stream);
+
+/* Inverse of twn_pack: int8 [rows, cols] from packed rows.  The unused field
+ * 10 unpacks as 0 and sets TWN_ERR_BAD_CODE in *dev_status (optional). */
+int twn_unpack(const uint32_t *packed, int64_t rows, int64_t cols, int64_t ld_codes,
+               int8_t *codes, int32_t *dev_status, twn_stream_t stream);
+
+/*
+ * Re-lays the packed filters of a convolution for the backward-for-data pass:
+ * from [Cout][kh][kw][Cin] (rows of ld_fwd codes) to [Cin][kh][kw][Cout]
+ * (rows of ld_bwd codes, same tap order, no spatial flip; padding 00).
+ * For an inner-product layer use kh = kw = 1: a plain transpose.
+ */
+int twn_transpose_codes(const uint32_t *packed_fwd, int64_t ld_fwd, const twn_conv_desc_t *desc,
+                        uint32_t *packed_bwd, int64_t ld_bwd, twn_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TWN_H_ */

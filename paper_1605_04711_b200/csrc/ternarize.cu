@@ -1,0 +1,518 @@
+// Threshold ternarization fused with 2-bit packing (Sec. 2.3: Eq. 3, Eq. 5 and the
+// threshold rule; Algorithm 1, first loop), plus the standalone pack / unpack /
+// re-layout kernels.
+//
+// Two sweeps over the fp32 master weights, both bound by HBM bandwidth:
+//   sweep 1  S = sum |W_i| in fp64  ->  delta = factor * S / n
+//   sweep 2  codes by Eq. 3, packed 16 per word; sum and count of the kept set
+//            ->  alpha (Eq. 5)
+// Sweep 2 walks the tensor back to front so that what sweep 1 read last is still
+// in L2.  Both reductions have a fixed order: per-thread strided partial sums,
+// a shuffle tree per warp, a shared-memory tree per block, one partial per block
+// in the workspace, and the block that finishes last folds the partials in index
+// order.  No floating-point atomics, no waiting on other blocks.
+#include "common.cuh"
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kMaxBlocks = 2048;
+// workspace: [0,256) tickets, then four arrays of kMaxBlocks 8-byte partials
+constexpr size_t kWorkspaceBytes = 256 + 4 * size_t(kMaxBlocks) * 8;
+
+struct Workspace {
+    unsigned int *ticket1;
+    unsigned int *ticket2;
+    double *part_sum;
+    double *part_kept;
+    unsigned long long *part_pos;
+    unsigned long long *part_neg;
+};
+
+__host__ __device__ inline Workspace carve(void *ws)
+{
+    char *b = static_cast<char *>(ws);
+    Workspace w;
+    w.ticket1 = reinterpret_cast<unsigned int *>(b);
+    w.ticket2 = reinterpret_cast<unsigned int *>(b + 64);
+    w.part_sum = reinterpret_cast<double *>(b + 256);
+    w.part_kept = w.part_sum + kMaxBlocks;
+    w.part_pos = reinterpret_cast<unsigned long long *>(w.part_kept + kMaxBlocks);
+    w.part_neg = w.part_pos + kMaxBlocks;
+    return w;
+}
+
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ unsigned long long warp_sum(unsigned long long v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Block-wide sum with a fixed order; the result is valid in thread 0.
+template <typename T>
+__device__ __forceinline__ T block_sum(T v, T *smem /* kWarps entries */)
+{
+    v = warp_sum(v);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __syncthreads();
+    if (lane == 0) smem[warp] = v;
+    __syncthreads();
+    T r = T(0);
+    if (warp == 0) {
+        r = lane < kWarps ? smem[lane] : T(0);
+        r = warp_sum(r);
+    }
+    return r;
+}
+
+// Returns true in every thread of the block that took the last ticket.
+__device__ __forceinline__ bool last_block(unsigned int *ticket)
+{
+    __shared__ bool is_last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+    __syncthreads();
+    return is_last;
+}
+
+// ---- sweep 1 -------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+sum_abs_kernel(const float *__restrict__ W, long long n, double factor, void *ws_raw,
+               twn_stats_t *__restrict__ stats)
+{
+    __shared__ double red[kWarps];
+    const Workspace ws = carve(ws_raw);
+    const long long n4 = n >> 2;
+    const float4 *W4 = reinterpret_cast<const float4 *>(W);
+    const long long stride = (long long)gridDim.x * kThreads;
+    long long i = (long long)blockIdx.x * kThreads + threadIdx.x;
+
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+    for (; i + 3 * stride < n4; i += 4 * stride) {
+        const float4 v0 = __ldg(W4 + i);
+        const float4 v1 = __ldg(W4 + i + stride);
+        const float4 v2 = __ldg(W4 + i + 2 * stride);
+        const float4 v3 = __ldg(W4 + i + 3 * stride);
+        a0 += (double)fabsf(v0.x); a1 += (double)fabsf(v0.y); a2 += (double)fabsf(v0.z); a3 += (double)fabsf(v0.w);
+        a0 += (double)fabsf(v1.x); a1 += (double)fabsf(v1.y); a2 += (double)fabsf(v1.z); a3 += (double)fabsf(v1.w);
+        a0 += (double)fabsf(v2.x); a1 += (double)fabsf(v2.y); a2 += (double)fabsf(v2.z); a3 += (double)fabsf(v2.w);
+        a0 += (double)fabsf(v3.x); a1 += (double)fabsf(v3.y); a2 += (double)fabsf(v3.z); a3 += (double)fabsf(v3.w);
+    }
+    for (; i < n4; i += stride) {
+        const float4 v = __ldg(W4 + i);
+        a0 += (double)fabsf(v.x); a1 += (double)fabsf(v.y); a2 += (double)fabsf(v.z); a3 += (double)fabsf(v.w);
+    }
+    // scalar tail (n % 4 elements), by the first threads of block 0
+    if (blockIdx.x == 0) {
+        const long long t = (n4 << 2) + threadIdx.x;
+        if (t < n) a0 += (double)fabsf(__ldg(W + t));
+    }
+    const double bsum = block_sum((a0 + a1) + (a2 + a3), red);
+    if (threadIdx.x == 0) ws.part_sum[blockIdx.x] = bsum;
+
+    if (last_block(ws.ticket1)) {
+        double s = 0.0;
+        for (int b = threadIdx.x; b < (int)gridDim.x; b += kThreads) s += __ldcg(ws.part_sum + b);
+        s = block_sum(s, red);
+        if (threadIdx.x == 0) {
+            const double delta = n > 0 ? factor * (s / (double)n) : 0.0;
+            stats->sum_abs = s;
+            stats->delta = delta;
+            stats->status = isfinite(s) ? TWN_OK : TWN_ERR_NONFINITE;
+            stats->reserved = 0;
+            *ws.ticket1 = 0u;
+        }
+    }
+}
+
+// ---- sweep 2 -------------------------------------------------------------
+// 2-bit field of one weight: bit 0 = kept, bit 1 = negative  (00 / 01 / 11).
+__device__ __forceinline__ uint32_t code2(float w, float thr, double &kept_sum)
+{
+    const float a = fabsf(w);
+    const bool keep = a > thr;
+    if (keep) kept_sum += (double)a;
+    return keep ? (w < 0.0f ? 3u : 1u) : 0u;
+}
+
+__device__ __forceinline__ uint32_t code8(const float4 v, float thr, double &k0, double &k1)
+{
+    uint32_t c = code2(v.x, thr, k0);
+    c |= code2(v.y, thr, k1) << 2;
+    c |= code2(v.z, thr, k0) << 4;
+    c |= code2(v.w, thr, k1) << 6;
+    return c;
+}
+
+// int8 image of four packed fields: 00 -> 0x00, 01 -> 0x01, 11 -> 0xFF
+__device__ __forceinline__ uint32_t fields_to_i8x4(uint32_t c8)
+{
+    uint32_t r = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const uint32_t f = (c8 >> (2 * e)) & 3u;
+        const uint32_t b = (f & 1u) ? ((f & 2u) ? 0xFFu : 0x01u) : 0u;
+        r |= b << (8 * e);
+    }
+    return r;
+}
+
+// Fast path geometry: a "unit" is 512 consecutive weights = 128 float4 = 32 words,
+// handled by one warp: lane l loads float4 (unit*128 + j*32 + l) for j = 0..3, so
+// every load instruction covers 512 contiguous bytes.  A 4x4 byte transpose inside
+// each group of four lanes then leaves lane l with the complete word
+// unit*32 + (l%4)*8 + l/4, and the warp stores one contiguous 128-byte line.
+__global__ void __launch_bounds__(kThreads)
+code_pack_kernel(const float *__restrict__ W, long long rows, long long cols, long long ld_codes,
+                 long long fast_units, uint32_t *__restrict__ packed, int8_t *__restrict__ codes_i8,
+                 void *ws_raw, twn_stats_t *__restrict__ stats)
+{
+    __shared__ double red[kWarps];
+    __shared__ unsigned long long redu[kWarps];
+    const Workspace ws = carve(ws_raw);
+    const long long n = rows * cols;
+    // delta rounded toward -inf: for any float w,  w > delta  <=>  w > thr
+    const float thr = __double2float_rd(stats->delta);
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    double k0 = 0.0, k1 = 0.0;
+    unsigned long long npos = 0, nneg = 0;
+
+    // -- fast units, back to front
+    const long long gwarps = (long long)gridDim.x * kWarps;
+    const float4 *W4 = reinterpret_cast<const float4 *>(W);
+    for (long long u = fast_units - 1 - ((long long)blockIdx.x * kWarps + warp); u >= 0; u -= gwarps) {
+        const long long f0 = u * 128 + lane;
+        const float4 v0 = __ldg(W4 + f0);
+        const float4 v1 = __ldg(W4 + f0 + 32);
+        const float4 v2 = __ldg(W4 + f0 + 64);
+        const float4 v3 = __ldg(W4 + f0 + 96);
+        const uint32_t c0 = code8(v0, thr, k0, k1);
+        const uint32_t c1 = code8(v1, thr, k0, k1);
+        const uint32_t c2 = code8(v2, thr, k0, k1);
+        const uint32_t c3 = code8(v3, thr, k0, k1);
+        uint32_t r = c0 | (c1 << 8) | (c2 << 16) | (c3 << 24);
+        const uint32_t neg = __popc((r >> 1) & 0x55555555u);
+        nneg += neg;
+        npos += __popc(r & 0x55555555u) - neg;
+        if (codes_i8) {
+            uint32_t *o = reinterpret_cast<uint32_t *>(codes_i8) + f0;
+            o[0] = fields_to_i8x4(c0);
+            o[32] = fields_to_i8x4(c1);
+            o[64] = fields_to_i8x4(c2);
+            o[96] = fields_to_i8x4(c3);
+        }
+        // 4x4 byte transpose across lanes l^2 then l^1
+        const uint32_t y = __shfl_xor_sync(0xffffffffu, r, 2);
+        r = __byte_perm(r, y, (lane & 2) ? 0x3276 : 0x5410);
+        const uint32_t z = __shfl_xor_sync(0xffffffffu, r, 1);
+        r = __byte_perm(r, z, (lane & 1) ? 0x3715 : 0x6240);
+        packed[u * 32 + (lane & 3) * 8 + (lane >> 2)] = r;
+    }
+
+    // -- everything else, one thread per word: the tail of a flat tensor, ragged rows, padding
+    const long long wpr = ld_codes >> 4;
+    const long long total_words = rows * wpr;
+    const long long first_word = fast_units * 32;
+    for (long long w = first_word + (long long)blockIdx.x * kThreads + threadIdx.x; w < total_words;
+         w += (long long)gridDim.x * kThreads) {
+        const long long r = w / wpr;
+        const long long j0 = (w - r * wpr) << 4;
+        uint32_t word = 0;
+#pragma unroll 4
+        for (int e = 0; e < 16; ++e) {
+            const long long j = j0 + e;
+            if (j < cols) {
+                const float v = __ldg(W + r * cols + j);
+                const uint32_t c = code2(v, thr, k0);
+                word |= c << (2 * e);
+                if (codes_i8) codes_i8[r * cols + j] = (int8_t)((c & 1u) ? ((c & 2u) ? -1 : 1) : 0);
+            }
+        }
+        const uint32_t neg = __popc((word >> 1) & 0x55555555u);
+        nneg += neg;
+        npos += __popc(word & 0x55555555u) - neg;
+        packed[w] = word;
+    }
+
+    const double bk = block_sum(k0 + k1, red);
+    const unsigned long long bp = block_sum(npos, redu);
+    const unsigned long long bn = block_sum(nneg, redu);
+    if (threadIdx.x == 0) {
+        ws.part_kept[blockIdx.x] = bk;
+        ws.part_pos[blockIdx.x] = bp;
+        ws.part_neg[blockIdx.x] = bn;
+    }
+    if (last_block(ws.ticket2)) {
+        double s = 0.0;
+        unsigned long long p = 0, q = 0;
+        for (int b = threadIdx.x; b < (int)gridDim.x; b += kThreads) {
+            s += __ldcg(ws.part_kept + b);
+            p += __ldcg(ws.part_pos + b);
+            q += __ldcg(ws.part_neg + b);
+        }
+        s = block_sum(s, red);
+        p = block_sum(p, redu);
+        q = block_sum(q, redu);
+        if (threadIdx.x == 0) {
+            const unsigned long long kept = p + q;
+            stats->sum_abs_kept = s;
+            stats->alpha = kept > 0 ? s / (double)kept : 0.0;
+            stats->n_pos = p;
+            stats->n_neg = q;
+            stats->n_zero = (unsigned long long)n - kept;
+            *ws.ticket2 = 0u;
+        }
+    }
+}
+
+// ---- standalone pack / unpack / re-layout ----------------------------------
+__device__ __forceinline__ uint32_t i8x4_to_fields(uint32_t x, uint32_t &bad)
+{
+    // a byte is valid iff (byte + 1) mod 256 <= 2
+    const uint32_t inval = __vcmpgtu4(__vadd4(x, 0x01010101u), 0x02020202u);
+    bad |= inval;
+    x &= ~inval;
+    const uint32_t y = x & 0x03030303u;
+    const uint32_t t = y | (y >> 6);
+    return (t & 0xFu) | ((t >> 12) & 0xF0u);
+}
+
+__global__ void __launch_bounds__(kThreads)
+pack_kernel(const int8_t *__restrict__ codes, long long rows, long long cols, long long ld_codes,
+            int vec_ok, uint32_t *__restrict__ packed, twn_stats_t *__restrict__ counts)
+{
+    __shared__ unsigned long long redu[kWarps];
+    const long long wpr = ld_codes >> 4;
+    const long long total_words = rows * wpr;
+    unsigned long long npos = 0, nneg = 0;
+    uint32_t bad = 0;
+    for (long long w = (long long)blockIdx.x * kThreads + threadIdx.x; w < total_words;
+         w += (long long)gridDim.x * kThreads) {
+        const long long r = w / wpr;
+        const long long j0 = (w - r * wpr) << 4;
+        uint32_t word = 0;
+        if (vec_ok && j0 + 16 <= cols) {
+            const uint4 v = __ldg(reinterpret_cast<const uint4 *>(codes + r * cols + j0));
+            word = i8x4_to_fields(v.x, bad) | (i8x4_to_fields(v.y, bad) << 8) |
+                   (i8x4_to_fields(v.z, bad) << 16) | (i8x4_to_fields(v.w, bad) << 24);
+        } else {
+            for (int e = 0; e < 16; ++e) {
+                const long long j = j0 + e;
+                if (j < cols) {
+                    const uint32_t b = (uint8_t)codes[r * cols + j];
+                    word |= i8x4_to_fields(b, bad) << (2 * e);
+                }
+            }
+        }
+        const uint32_t neg = __popc((word >> 1) & 0x55555555u);
+        nneg += neg;
+        npos += __popc(word & 0x55555555u) - neg;
+        packed[w] = word;
+    }
+    if (counts) {
+        const unsigned long long bp = block_sum(npos, redu);
+        const unsigned long long bn = block_sum(nneg, redu);
+        const int any_bad = __syncthreads_or(bad != 0);
+        if (threadIdx.x == 0) {
+            // integer atomics: order-independent, hence still deterministic
+            atomicAdd(reinterpret_cast<unsigned long long *>(&counts->n_pos), bp);
+            atomicAdd(reinterpret_cast<unsigned long long *>(&counts->n_neg), bn);
+            if (any_bad) atomicMin(&counts->status, (int)TWN_ERR_BAD_CODE);
+        }
+    }
+}
+
+__global__ void finish_counts_kernel(twn_stats_t *counts, unsigned long long n)
+{
+    counts->n_zero = n - counts->n_pos - counts->n_neg;
+}
+
+__global__ void __launch_bounds__(kThreads)
+unpack_kernel(const uint32_t *__restrict__ packed, long long rows, long long cols, long long ld_codes,
+              int vec_ok, int8_t *__restrict__ codes, int32_t *__restrict__ dev_status)
+{
+    const long long wpr = ld_codes >> 4;
+    const long long wpr_used = (cols + 15) >> 4;
+    const long long total = rows * wpr_used;
+    bool bad = false;
+    for (long long t = (long long)blockIdx.x * kThreads + threadIdx.x; t < total;
+         t += (long long)gridDim.x * kThreads) {
+        const long long r = t / wpr_used;
+        const long long wi = t - r * wpr_used;
+        const uint32_t word = __ldg(packed + r * wpr + wi);
+        // field 10: bit 1 set while bit 0 is clear
+        const uint32_t inval = (word >> 1) & ~word & 0x55555555u;
+        const long long j0 = wi << 4;
+        const long long valid = cols - j0 >= 16 ? 16 : cols - j0;
+        const uint32_t vmask = valid >= 16 ? 0xFFFFFFFFu : ((1u << (2 * valid)) - 1u);
+        if (inval & vmask) bad = true;
+        const uint32_t clean = word & ~(inval << 1);
+        if (vec_ok && valid == 16) {
+            uint4 o;
+            o.x = fields_to_i8x4(clean & 0xFFu);
+            o.y = fields_to_i8x4((clean >> 8) & 0xFFu);
+            o.z = fields_to_i8x4((clean >> 16) & 0xFFu);
+            o.w = fields_to_i8x4(clean >> 24);
+            *reinterpret_cast<uint4 *>(codes + r * cols + j0) = o;
+        } else {
+            for (int e = 0; e < valid; ++e) {
+                const uint32_t f = (clean >> (2 * e)) & 3u;
+                codes[r * cols + j0 + e] = (int8_t)((f & 1u) ? ((f & 2u) ? -1 : 1) : 0);
+            }
+        }
+    }
+    if (dev_status && __syncthreads_or(bad) && threadIdx.x == 0) atomicMin(dev_status, (int)TWN_ERR_BAD_CODE);
+}
+
+// out row c, column t*Cout + o  <-  in row o, column t*Cin + c   (t = tap index)
+__global__ void __launch_bounds__(kThreads)
+transpose_codes_kernel(const uint32_t *__restrict__ in, long long ld_in, long long Cout, long long Cin,
+                       long long taps, uint32_t *__restrict__ out, long long ld_out)
+{
+    const long long wpr_out = ld_out >> 4, wpr_in = ld_in >> 4;
+    const long long total = Cin * wpr_out;
+    const long long cols_out = taps * Cout;
+    for (long long w = (long long)blockIdx.x * kThreads + threadIdx.x; w < total;
+         w += (long long)gridDim.x * kThreads) {
+        const long long c = w / wpr_out;
+        const long long j0 = (w - c * wpr_out) << 4;
+        uint32_t word = 0;
+        for (int e = 0; e < 16; ++e) {
+            const long long j = j0 + e;
+            if (j < cols_out) {
+                const long long t = j / Cout, o = j - t * Cout;
+                const long long src = t * Cin + c;
+                const uint32_t f = (__ldg(in + o * wpr_in + (src >> 4)) >> (2 * (src & 15))) & 3u;
+                word |= f << (2 * e);
+            }
+        }
+        out[w] = word;
+    }
+}
+
+int grid_for(long long items_per_thread_units, int sm_count)
+{
+    long long blocks = (items_per_thread_units + kThreads - 1) / kThreads;
+    const long long cap = (long long)sm_count * 8 < kMaxBlocks ? (long long)sm_count * 8 : kMaxBlocks;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return (int)blocks;
+}
+
+}  // namespace
+
+extern "C" size_t twn_ternarize_workspace_bytes(void) { return kWorkspaceBytes; }
+
+extern "C" int twn_ternarize(const float *W, int64_t rows, int64_t cols, double delta_factor,
+                             twn_stats_t *stats, uint32_t *packed, int64_t ld_codes,
+                             int8_t *codes_i8, void *workspace, size_t workspace_bytes,
+                             twn_stream_t stream)
+{
+    TWN_REQUIRE(rows >= 0 && cols >= 0, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(stats != nullptr && workspace != nullptr, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(delta_factor >= 0.0 && delta_factor == delta_factor, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(ld_codes >= cols && ld_codes % 64 == 0, TWN_ERR_INVALID_ARG);
+    const long long n = (long long)rows * cols;
+    TWN_REQUIRE(n == 0 || (W != nullptr && packed != nullptr), TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(workspace_bytes >= kWorkspaceBytes, TWN_ERR_WORKSPACE);
+    TWN_REQUIRE(twn_aligned(W, 16) && twn_aligned(packed, 16) && twn_aligned(stats, 8) &&
+                    twn_aligned(workspace, 256) && twn_aligned(codes_i8, 16), TWN_ERR_MISALIGNED);
+    twn_device_info dev;
+    const int rc = twn_current_device(&dev);
+    if (rc != TWN_OK) return rc;
+    cudaStream_t s = twn_cu(stream);
+
+    // the two tickets must start at zero
+    TWN_CUDA_OK(cudaMemsetAsync(workspace, 0, 128, s));
+
+    const int g1 = grid_for((n / 4 + 3) / 4, dev.sm_count);
+    sum_abs_kernel<<<g1, kThreads, 0, s>>>(W, n, delta_factor, workspace, stats);
+
+    // a flat run of whole 512-weight units exists when rows are stored back to back
+    const bool flat = (rows <= 1) || (ld_codes == cols);
+    const long long fast_units = flat ? n / 512 : 0;
+    const long long rest_words = (long long)rows * (ld_codes / 16) - fast_units * 32;
+    long long work = fast_units * 32 / 4;  // threads: each warp-iteration covers one unit
+    if (rest_words > work) work = rest_words;
+    const int g2 = grid_for(work, dev.sm_count);
+    code_pack_kernel<<<g2, kThreads, 0, s>>>(W, rows, cols, ld_codes, fast_units, packed, codes_i8,
+                                             workspace, stats);
+    TWN_CUDA_OK(cudaGetLastError());
+    return TWN_OK;
+}
+
+extern "C" int twn_pack(const int8_t *codes, int64_t rows, int64_t cols, uint32_t *packed,
+                        int64_t ld_codes, twn_stats_t *counts, twn_stream_t stream)
+{
+    TWN_REQUIRE(rows >= 0 && cols >= 0, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(ld_codes >= cols && ld_codes % 64 == 0, TWN_ERR_INVALID_ARG);
+    const long long n = (long long)rows * cols;
+    TWN_REQUIRE(n == 0 || (codes != nullptr && packed != nullptr), TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(twn_aligned(packed, 16) && twn_aligned(counts, 8), TWN_ERR_MISALIGNED);
+    twn_device_info dev;
+    const int rc = twn_current_device(&dev);
+    if (rc != TWN_OK) return rc;
+    const long long words = (long long)rows * (ld_codes / 16);
+    if (words == 0) {
+        if (counts) TWN_CUDA_OK(cudaMemsetAsync(counts, 0, sizeof(twn_stats_t), twn_cu(stream)));
+        return TWN_OK;
+    }
+    const int vec_ok = twn_aligned(codes, 16) && (cols % 16 == 0);
+    if (counts) TWN_CUDA_OK(cudaMemsetAsync(counts, 0, sizeof(twn_stats_t), twn_cu(stream)));
+    pack_kernel<<<grid_for(words, dev.sm_count), kThreads, 0, twn_cu(stream)>>>(
+        codes, rows, cols, ld_codes, vec_ok, packed, counts);
+    if (counts) finish_counts_kernel<<<1, 1, 0, twn_cu(stream)>>>(counts, (unsigned long long)n);
+    TWN_CUDA_OK(cudaGetLastError());
+    return TWN_OK;
+}
+
+extern "C" int twn_unpack(const uint32_t *packed, int64_t rows, int64_t cols, int64_t ld_codes,
+                          int8_t *codes, int32_t *dev_status, twn_stream_t stream)
+{
+    TWN_REQUIRE(rows >= 0 && cols >= 0, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(ld_codes >= cols && ld_codes % 64 == 0, TWN_ERR_INVALID_ARG);
+    const long long n = (long long)rows * cols;
+    TWN_REQUIRE(n == 0 || (codes != nullptr && packed != nullptr), TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(twn_aligned(packed, 16) && twn_aligned(dev_status, 4), TWN_ERR_MISALIGNED);
+    twn_device_info dev;
+    const int rc = twn_current_device(&dev);
+    if (rc != TWN_OK) return rc;
+    if (n == 0) return TWN_OK;
+    const int vec_ok = twn_aligned(codes, 16) && (cols % 16 == 0);
+    const long long items = (long long)rows * ((cols + 15) / 16);
+    unpack_kernel<<<grid_for(items, dev.sm_count), kThreads, 0, twn_cu(stream)>>>(
+        packed, rows, cols, ld_codes, vec_ok, codes, dev_status);
+    TWN_CUDA_OK(cudaGetLastError());
+    return TWN_OK;
+}
+
+extern "C" int twn_transpose_codes(const uint32_t *packed_fwd, int64_t ld_fwd,
+                                   const twn_conv_desc_t *d, uint32_t *packed_bwd, int64_t ld_bwd,
+                                   twn_stream_t stream)
+{
+    TWN_REQUIRE(d != nullptr && packed_fwd != nullptr && packed_bwd != nullptr, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(d->Cin > 0 && d->Cout > 0 && d->kh > 0 && d->kw > 0, TWN_ERR_INVALID_ARG);
+    const long long taps = (long long)d->kh * d->kw;
+    TWN_REQUIRE(ld_fwd % 64 == 0 && ld_fwd >= taps * d->Cin, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(ld_bwd % 64 == 0 && ld_bwd >= taps * d->Cout, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(twn_aligned(packed_fwd, 16) && twn_aligned(packed_bwd, 16), TWN_ERR_MISALIGNED);
+    twn_device_info dev;
+    const int rc = twn_current_device(&dev);
+    if (rc != TWN_OK) return rc;
+    const long long words = d->Cin * (ld_bwd / 16);
+    transpose_codes_kernel<<<grid_for(words, dev.sm_count), kThreads, 0, twn_cu(stream)>>>(
+        packed_fwd, ld_fwd, d->Cout, d->Cin, taps, packed_bwd, ld_bwd);
+    TWN_CUDA_OK(cudaGetLastError());
+    return TWN_OK;
+}

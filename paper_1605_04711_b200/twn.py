@@ -1,0 +1,150 @@
+"""ctypes binding of libtwn.so: the same entry points as include/twn.h.
+
+Argument marshalling only.  Tensors are torch tensors on the current CUDA
+device (torch provides memory and streams); every step of the computation runs
+in the library's kernels.  There is no fallback: if the library is missing or
+the device is not sm_100 the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libtwn.so")
+
+OK = 0
+F32, BF16 = 0, 1
+STATS_BYTES = 64
+
+
+class TwnError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+class ConvDesc(C.Structure):
+    _fields_ = [("B", C.c_int64), ("H", C.c_int64), ("W", C.c_int64), ("Cin", C.c_int64),
+                ("Cout", C.c_int64), ("kh", C.c_int32), ("kw", C.c_int32),
+                ("stride_h", C.c_int32), ("stride_w", C.c_int32),
+                ("pad_h", C.c_int32), ("pad_w", C.c_int32)]
+
+    @property
+    def Ho(self):
+        return (self.H + 2 * self.pad_h - self.kh) // self.stride_h + 1
+
+    @property
+    def Wo(self):
+        return (self.W + 2 * self.pad_w - self.kw) // self.stride_w + 1
+
+
+def conv_desc(B, H, W, Cin, Cout, k, stride=1, pad=0) -> ConvDesc:
+    kh, kw = (k, k) if isinstance(k, int) else k
+    return ConvDesc(B, H, W, Cin, Cout, kh, kw, stride, stride, pad, pad)
+
+
+class Epilogue(C.Structure):
+    _fields_ = [("scale", C.c_void_p), ("shift", C.c_void_p), ("residual", C.c_void_p),
+                ("residual_dtype", C.c_int32), ("relu", C.c_int32), ("out_dtype", C.c_int32),
+                ("reserved", C.c_int32)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Opens libtwn.so (built by paper_1605_04711_b200/build.py).  Raises if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} not found: build it with `python -m paper_1605_04711_b200.build`")
+        l = C.CDLL(LIB_PATH)
+        l.twn_strerror.restype = C.c_char_p
+        l.twn_ternarize_workspace_bytes.restype = C.c_size_t
+        _lib = l
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().twn_strerror(C.c_int(code)).decode()
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise TwnError(code, where)
+
+
+def _ptr(t) -> C.c_void_p:
+    if t is None:
+        return C.c_void_p(0)
+    assert t.is_cuda and t.is_contiguous(), "device tensors must be contiguous CUDA tensors"
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None) -> C.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def ld_for(cols: int) -> int:
+    """Smallest legal row pitch (in codes) for rows of `cols` codes."""
+    return (cols + 63) // 64 * 64
+
+
+def new_stats(device="cuda") -> torch.Tensor:
+    """A zeroed device twn_stats_t (64 bytes, as 8 int64 words)."""
+    return torch.zeros(8, dtype=torch.int64, device=device)
+
+
+def stats_to_host(stats: torch.Tensor) -> dict:
+    """Synchronises and decodes a device twn_stats_t."""
+    h = stats.cpu()
+    d = h.view(torch.float64)
+    return {"delta": float(d[0]), "alpha": float(d[1]), "sum_abs": float(d[2]),
+            "sum_abs_kept": float(d[3]), "n_neg": int(h[4]), "n_zero": int(h[5]),
+            "n_pos": int(h[6]), "status": int(h.view(torch.int32)[14])}
+
+
+def read_status(dev_status: torch.Tensor, stream=None) -> int:
+    out = C.c_int32(0)
+    _check(lib().twn_read_status(_ptr(dev_status), C.byref(out), _stream(stream)), "twn_read_status")
+    return out.value
+
+
+def ternarize_workspace_bytes() -> int:
+    return int(lib().twn_ternarize_workspace_bytes())
+
+
+def ternarize(W: torch.Tensor, delta_factor: float, stats: torch.Tensor, packed: torch.Tensor,
+              ld_codes: int, codes_i8, workspace: torch.Tensor, stream=None,
+              rows: int | None = None, cols: int | None = None) -> None:
+    """twn_ternarize.  W fp32 [rows, cols] (or any shape with rows/cols given)."""
+    if rows is None:
+        rows, cols = (W.shape[0], W.numel() // W.shape[0]) if W.dim() > 1 else (1, W.numel())
+    _check(lib().twn_ternarize(_ptr(W), C.c_int64(rows), C.c_int64(cols), C.c_double(delta_factor),
+                               _ptr(stats), _ptr(packed), C.c_int64(ld_codes), _ptr(codes_i8),
+                               _ptr(workspace), C.c_size_t(workspace.numel() * workspace.element_size()),
+                               _stream(stream)), "twn_ternarize")
+
+
+def pack(codes: torch.Tensor, rows: int, cols: int, packed: torch.Tensor, ld_codes: int,
+         counts=None, stream=None) -> None:
+    _check(lib().twn_pack(_ptr(codes), C.c_int64(rows), C.c_int64(cols), _ptr(packed),
+                          C.c_int64(ld_codes), _ptr(counts), _stream(stream)), "twn_pack")
+
+
+def unpack(packed: torch.Tensor, rows: int, cols: int, ld_codes: int, codes: torch.Tensor,
+           dev_status=None, stream=None) -> None:
+    _check(lib().twn_unpack(_ptr(packed), C.c_int64(rows), C.c_int64(cols), C.c_int64(ld_codes),
+                            _ptr(codes), _ptr(dev_status), _stream(stream)), "twn_unpack")
+
+
+def transpose_codes(packed_fwd: torch.Tensor, ld_fwd: int, desc: ConvDesc, packed_bwd: torch.Tensor,
+                    ld_bwd: int, stream=None) -> None:
+    _check(lib().twn_transpose_codes(_ptr(packed_fwd), C.c_int64(ld_fwd), C.byref(desc),
+                                     _ptr(packed_bwd), C.c_int64(ld_bwd), _stream(stream)),
+           "twn_transpose_codes")
