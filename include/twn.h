@@ -105,8 +105,13 @@ size_t twn_ternarize_workspace_bytes(void);
  * W        fp32 [rows, cols], contiguous, 16-byte aligned.  rows = filters
  *          (output channels), cols = fan-in.
  * stats    one twn_stats_t, 8-byte aligned; written completely.
- * packed   uint32 [rows][ld_codes/16].  Code j of a row occupies bits
- *          [2*(j%16)+1 : 2*(j%16)] of word j/16: 00 = 0, 01 = +1, 11 = -1.
+ * packed   uint32 [rows][ld_codes/16].  A field is two bits: 00 = 0, 01 = +1,
+ *          11 = -1 (10 is never written).  Code j of a row lives in word j/16;
+ *          inside the word the even elements fill the low half-word and the odd
+ *          elements the high half-word: element e = j%16 is at bit position
+ *          2*(e/2) + 16*(e%2).  (The paper fixes no encoding; this one lets a
+ *          shift, one logic op and one bf16x2 subtract turn two fields into a
+ *          pair of bf16 tensor-core operands.)
  *          ld_codes is a multiple of 64 (rows start 16-byte aligned),
  *          ld_codes >= cols; the padding is written as 00.  16-byte aligned.
  * codes_i8 optional int8 [rows, cols] copy of the codes (16-byte aligned), or NULL.
@@ -148,6 +153,59 @@ int twn_unpack(const uint32_t *packed, int64_t rows, int64_t cols, int64_t ld_co
  */
 int twn_transpose_codes(const uint32_t *packed_fwd, int64_t ld_fwd, const twn_conv_desc_t *desc,
                         uint32_t *packed_bwd, int64_t ld_bwd, twn_stream_t stream);
+
+/* ---- ternary-weight contractions (Eq. 2; Algorithm 1, TernaryForward/Backward) ---- */
+
+/*
+ * Inner product (fully-connected layer):  Y[M,N] = epi( alpha * X[M,K] * T^T ).
+ *   X         bf16 [M, ldx], row-major, 16-byte aligned, ldx >= K, ldx % 8 == 0.
+ *   T_packed  N rows of K codes (row n = output unit n, the [out, in] order of the
+ *             master weights) in the layout of twn_ternarize, row pitch ld_codes.
+ *   stats     the twn_stats_t of the ternarization; only alpha is read, on the
+ *             device.  NULL means alpha = 1.
+ *   epi       optional epilogue (NULL: none, fp32 output).
+ *   Y         [M, ldy] fp32 or bf16 (epi->out_dtype), ldy >= N, 4-byte aligned.
+ *   dev_status optional device int32 that receives TWN_ERR_TIMEOUT if a bounded
+ *             wait inside the kernel runs out (the kernel then exits early and the
+ *             output is unspecified).  Must be zero (TWN_OK) before the call.
+ * Products are exact (the codes are exactly -1/0/+1 in bf16); accumulation is fp32
+ * on the tensor cores; alpha and the epilogue are applied in fp32.
+ */
+int twn_gemm(const void *X, int64_t ldx, const uint32_t *T_packed, int64_t ld_codes,
+             const twn_stats_t *stats, int64_t M, int64_t N, int64_t K,
+             const twn_epilogue_t *epi, void *Y, int64_t ldy, int32_t *dev_status,
+             twn_stream_t stream);
+
+/*
+ * Convolution forward (cross-correlation, zero padding):
+ *   Y[b,ho,wo,o] = epi( alpha * sum_{r,s,c} X[b, ho*stride_h - pad_h + r, wo*stride_w - pad_w + s, c]
+ *                                           * T[o,r,s,c] )
+ *   X      bf16 NHWC [B,H,W,Cin], contiguous, 16-byte aligned.
+ *   T_fwd  Cout rows of kh*kw*Cin codes ([Cout][kh][kw][Cin]), row pitch ld_codes.
+ *   Y      NHWC [B,Ho,Wo,Cout], contiguous, fp32 or bf16.
+ * Requires Cin % 16 == 0 (Cin % 8 == 0 for a 1x1 filter) and kh*kw <= 64; other
+ * layers go through twn_im2col + twn_gemm.  Other arguments as in twn_gemm.
+ */
+int twn_conv2d_fwd(const twn_conv_desc_t *desc, const void *X, const uint32_t *T_fwd, int64_t ld_codes,
+                   const twn_stats_t *stats, const twn_epilogue_t *epi, void *Y,
+                   int32_t *dev_status, twn_stream_t stream);
+
+/*
+ * Convolution backward for data (Algorithm 1: ordinary back-propagation with
+ * T = alpha * W~ in place of W), the adjoint of twn_conv2d_fwd:
+ *   dX[b,h,w,c] = epi( alpha * sum over (r,s,o) with ho*stride_h - pad_h + r == h,
+ *                      wo*stride_w - pad_w + s == w  of  dZ[b,ho,wo,o] * T[o,r,s,c] )
+ *   dZ     bf16 NHWC [B,Ho,Wo,Cout], contiguous.
+ *   T_bwd  the output of twn_transpose_codes: Cin rows of kh*kw*Cout codes.
+ *   dX     NHWC [B,H,W,Cin], fp32 or bf16; every element is written.
+ *   epi    scale/shift are indexed by the input channel c; `residual` (shape of dX)
+ *          lets a second gradient branch be added in the same pass.
+ * Requires Cout % 16 == 0 (Cout % 8 == 0 for a 1x1 filter).  A strided layer runs as
+ * stride_h*stride_w launches, one per residue class of (h, w) modulo the stride.
+ */
+int twn_conv2d_bwd_data(const twn_conv_desc_t *desc, const void *dZ, const uint32_t *T_bwd, int64_t ld_codes,
+                        const twn_stats_t *stats, const twn_epilogue_t *epi, void *dX,
+                        int32_t *dev_status, twn_stream_t stream);
 
 #ifdef __cplusplus
 }

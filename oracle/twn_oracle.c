@@ -152,11 +152,17 @@ double ref_objective(const float *W, const int8_t *codes, double alpha, int64_t 
 
 /* ------------------------------------------------------------------------
  * 2-bit storage (Section 2.1, "2-bit storage requirement ... for a unit of
- * weight").  The paper fixes no encoding; this library's is two's complement
- * in two bits: 0 -> 00, +1 -> 01, -1 -> 11 (10 is never produced).  Element j
- * of a row sits in bits [2*(j%16)+1 : 2*(j%16)] of 32-bit word j/16; a row
- * occupies ld_codes/16 words (ld_codes a multiple of 16 here), padded with 00.
+ * weight").  The paper fixes no encoding; this library's is:
+ *   field   two's complement in two bits: 0 -> 00, +1 -> 01, -1 -> 11
+ *           (10 is never produced);
+ *   word    a row is cut into groups of 16 codes, one 32-bit word per group.
+ *           Inside a group the even elements fill the low half-word and the
+ *           odd elements the high half-word: element e (0..15) sits at bit
+ *           position 2*(e/2) + 16*(e%2);
+ *   row     ld_codes/16 words (ld_codes a multiple of 16 here), padded with 00.
  * ---------------------------------------------------------------------- */
+static int field_pos(int64_t e) { return (int)(2 * (e / 2) + 16 * (e % 2)); }
+
 int ref_pack(const int8_t *codes, int64_t rows, int64_t cols, int64_t ld_codes, uint32_t *packed)
 {
     if (ld_codes % 16 != 0 || ld_codes < cols) return -1;
@@ -167,7 +173,7 @@ int ref_pack(const int8_t *codes, int64_t rows, int64_t cols, int64_t ld_codes, 
             int8_t t = codes[r * cols + j];
             uint32_t f;
             if (t == 0) f = 0u; else if (t == 1) f = 1u; else if (t == -1) f = 3u; else return -2;
-            packed[r * wpr + j / 16] |= f << (2 * (j % 16));
+            packed[r * wpr + j / 16] |= f << field_pos(j % 16);
         }
     }
     return 0;
@@ -179,7 +185,7 @@ int ref_unpack(const uint32_t *packed, int64_t rows, int64_t cols, int64_t ld_co
     int64_t wpr = ld_codes / 16;
     for (int64_t r = 0; r < rows; ++r)
         for (int64_t j = 0; j < cols; ++j) {
-            uint32_t f = (packed[r * wpr + j / 16] >> (2 * (j % 16))) & 3u;
+            uint32_t f = (packed[r * wpr + j / 16] >> field_pos(j % 16)) & 3u;
             if (f == 2u) return -2;
             codes[r * cols + j] = (f == 0u) ? 0 : (f == 1u ? 1 : -1);
         }

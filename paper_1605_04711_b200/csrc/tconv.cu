@@ -1,0 +1,711 @@
+// Ternary-weight contraction on the 5th-generation tensor cores (Eq. 2 forward block;
+// Algorithm 1 TernaryForward / TernaryBackward):  Y = epilogue(alpha * X (*) T).
+//
+// One persistent, warp-specialised kernel serves the inner product, the convolution
+// forward pass and the backward-for-data pass.  All three are written as a sum over
+// "taps": for output pixel p and output channel n
+//     acc[n, p] = sum_t sum_c  T[n, koff_t + c] * X[pixel(p) * stride + (dh_t, dw_t), c]
+// with X an NHWC bf16 tensor addressed through a 4-D TMA tensor map (out-of-range
+// pixels and channels read as zero) and T the packed 2-bit codes, one row per n.
+//
+// The weights are the A operand of tcgen05.mma and live in tensor memory: decode
+// warps turn the packed codes into exact bf16 {-1, 0, +1} in registers and write them
+// with tcgen05.st.  The activations are the B operand, staged by TMA into 128-byte
+// swizzled shared memory.  The accumulator (fp32, tensor memory) therefore holds
+// D[n, p]: a lane is an output channel, a column a pixel.  In the epilogue each thread
+// owns one channel, so alpha, the per-channel affine and ReLU cost one register each,
+// and a warp's store of one pixel covers 32 consecutive channels (128 contiguous bytes).
+//
+//   warp 0      TMA producer: X tile and packed-code tile per k-block
+//   warp 1      allocates tensor memory, issues tcgen05.mma, commits to mbarriers
+//   warps 2-5   decode: packed codes (smem) -> bf16 pairs -> tensor memory
+//   warps 6-9   epilogue: tensor memory -> registers -> global
+//
+// Every wait on an mbarrier is bounded (about a second); on expiry the kernel records
+// TWN_ERR_TIMEOUT, all roles leave their loops, tensor memory is freed and the grid exits.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+namespace {
+
+constexpr int kStages = 8;          // smem / tensor-memory operand ring depth
+constexpr int kChan = 128;          // output channels per tile (UMMA M)
+constexpr int kPix = 128;           // pixels per tile (UMMA N)
+constexpr int kBlockK = 64;         // reduction elements per k-block (128 bytes of bf16)
+constexpr int kXBytes = kPix * kBlockK * 2;    // 16 KB
+constexpr int kCodeRowBytes = 32;              // 8 words per channel row per k-block (4 used)
+constexpr int kCodeBytes = kChan * kCodeRowBytes;  // 4 KB
+constexpr int kThreadsConv = 320;
+constexpr int kMaxTaps = 64;
+constexpr int kAccCols = kPix;                 // fp32 accumulator columns per buffer
+constexpr int kAColsPerStage = kBlockK / 2;    // 32 columns of bf16 pairs
+constexpr uint32_t kTmemCols = 512;
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;
+
+struct Tap {
+    int16_t dh, dw;   // input pixel offset of this tap
+    int32_t koff;     // first code column of this tap in a packed row
+};
+
+struct ConvParams {
+    // tiles
+    int n_tiles, tw, th, tb, total_tiles;
+    int lgBW, lgBH;               // pixel tile = BB x BH x BW, powers of two, product kPix
+    // reduction
+    int n_taps, n_cblk;           // k-blocks per tile = n_taps * n_cblk
+    int sw, sh;                   // input pixel = output pixel * (sh, sw) + (dh, dw)
+    // virtual output grid and its embedding in the output tensor
+    int Bv, Hv, Wv;
+    int OH, OW, osh, osw, ooh, oow;
+    long long ldy;                // output pixel pitch in elements
+    int Cout;
+    // epilogue
+    const double *alpha;          // device scalar (twn_stats_t::alpha) or nullptr for 1
+    const float *scale, *shift;
+    const void *residual;
+    int res_dtype, relu, out_dtype;
+    void *Y;
+    int32_t *status;
+    Tap taps[kMaxTaps];
+};
+
+struct __align__(1024) SmemLayout {
+    uint8_t x[kStages][kXBytes];           // swizzled activation tiles
+    uint8_t codes[kStages][kCodeBytes];    // packed code tiles, row = channel
+    unsigned long long full[kStages];      // TMA -> decode + MMA
+    unsigned long long ready_a[kStages];   // decode -> MMA
+    unsigned long long empty[kStages];     // MMA commit -> TMA + decode
+    unsigned long long acc_full[2];        // MMA commit -> epilogue
+    unsigned long long acc_empty[2];       // epilogue -> MMA
+    long long pix_off[4][kPix];            // per epilogue warp: output element offset, -1 = skip
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(void *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(void *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(void *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(void *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait.  Returns false when the limit ran out or another role gave up.
+__device__ __forceinline__ bool mbar_wait(void *bar, uint32_t parity, SmemLayout *sm, int32_t *status)
+{
+    if (mbar_try(bar, parity)) return true;
+    unsigned long long t0 = 0;
+    for (uint32_t spin = 1;; ++spin) {
+        if (mbar_try(bar, parity)) return true;
+        if ((spin & 255u) == 0) {
+            if (sm->abort_flag) return false;
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) {
+                sm->abort_flag = 1;
+                if (status) atomicMin(status, (int)TWN_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, void *bar, int c0, int c1, int c2, int c3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, void *bar, int c0, int c1)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(void *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// D[tmem] (+)= A[tmem] * B[smem]^T, bf16 x bf16 -> fp32, one thread issues.
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// K-major, 128-byte swizzled operand tile: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);   // start address
+    d |= (uint64_t)1 << 16;                     // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;           // stride byte offset
+    d |= (uint64_t)1 << 46;                     // descriptor version for sm_100
+    d |= (uint64_t)2 << 61;                     // 128-byte swizzle
+    return d;
+}
+
+// kind::f16 instruction descriptor: bf16 A and B (both K-major), fp32 accumulate.
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N)
+{
+    return (1u << 4)              // D format fp32
+           | (1u << 7)            // A format bf16
+           | (1u << 10)           // B format bf16
+           | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr),
+          "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+
+// Two 2-bit fields (bits 1:0 and 17:16 of x) -> two exact bf16 values in {-1, 0, +1}.
+// field ^ 2 is the field's value + 2 (00 -> 2, 01 -> 3, 11 -> 1); or-ing it into the
+// mantissa of 128.0 gives 130 + value, and subtracting 130.0 leaves the value.
+__device__ __forceinline__ uint32_t fields_to_bf16x2(uint32_t x)
+{
+    const uint32_t t = (x & 0x00030003u) ^ 0x43024302u;
+    uint32_t r;
+    asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(t), "r"(0x43024302u));
+    return r;
+}
+
+// ---------------------------------------------------------------- the kernel
+__global__ void __launch_bounds__(kThreadsConv, 1)
+tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_t,
+             const __grid_constant__ ConvParams P)
+{
+    extern __shared__ uint8_t smem_raw[];
+    SmemLayout *sm = reinterpret_cast<SmemLayout *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int kbpt = P.n_taps * P.n_cblk;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&sm->full[s], 1);
+            mbar_init(&sm->ready_a[s], 4);
+            mbar_init(&sm->empty[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&sm->acc_full[b], 1);
+            mbar_init(&sm->acc_empty[b], 4);
+        }
+        sm->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sm->tmem_base;
+    const uint32_t tmem_acc = tmem;                       // 2 x kAccCols columns
+    const uint32_t tmem_a = tmem + 2 * kAccCols;          // kStages x kAColsPerStage columns
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
+                const int nt = tile % P.n_tiles;
+                int pt = tile / P.n_tiles;
+                const int twi = pt % P.tw; pt /= P.tw;
+                const int thi = pt % P.th;
+                const int tbi = pt / P.th;
+                const int w0 = (twi << P.lgBW) * P.sw;
+                const int h0 = (thi << P.lgBH) * P.sh;
+                const int b0 = tbi * (kPix >> (P.lgBW + P.lgBH));
+                for (int t = 0; t < P.n_taps && ok; ++t) {
+                    const Tap tap = P.taps[t];
+                    for (int cb = 0; cb < P.n_cblk; ++cb, ++it) {
+                        const int s = it % kStages;
+                        const uint32_t ph = (it / kStages) & 1u;
+                        if (!mbar_wait(&sm->empty[s], ph ^ 1u, sm, P.status)) { ok = false; break; }
+                        mbar_expect_tx(&sm->full[s], kXBytes + kCodeBytes);
+                        tma_load_4d(sm->x[s], &map_x, &sm->full[s], cb * kBlockK, w0 + tap.dw, h0 + tap.dh, b0);
+                        const int word = (tap.koff >> 4) + cb * (kBlockK / 16);
+                        tma_load_2d(sm->codes[s], &map_t, &sm->full[s], word & ~3, nt * kChan);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(kChan, kPix);
+            uint32_t it = 0, lt = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x, ++lt) {
+                const int buf = lt & 1;
+                if (!mbar_wait(&sm->acc_empty[buf], ((lt >> 1) & 1u) ^ 1u, sm, P.status)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_acc + buf * kAccCols;
+                for (int kb = 0; kb < kbpt; ++kb, ++it) {
+                    const int s = it % kStages;
+                    const uint32_t ph = (it / kStages) & 1u;
+                    if (!mbar_wait(&sm->full[s], ph, sm, P.status) ||
+                        !mbar_wait(&sm->ready_a[s], ph, sm, P.status)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t bdesc = smem_desc_sw128(smem_u32(sm->x[s]));
+#pragma unroll
+                    for (int k = 0; k < kBlockK / 16; ++k) {
+                        // 16 reduction elements = 8 tensor-memory columns of A, 32 bytes of a B row
+                        tc_mma_ts(d_tmem, tmem_a + s * kAColsPerStage + k * 8, bdesc + (uint64_t)(k * 2),
+                                  idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    }
+                    tc_commit(&sm->empty[s]);
+                }
+                if (ok) tc_commit(&sm->acc_full[buf]);
+            }
+        }
+    } else if (warp < 6) {
+        // ------------------------------------------------ decode: codes -> bf16 -> tensor memory
+        const int q = warp & 3;                 // tensor-memory lane quadrant of this warp
+        const int row = q * 32 + lane;          // channel row inside the tile
+        uint32_t it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
+            for (int t = 0; t < P.n_taps && ok; ++t) {
+                const int koff = P.taps[t].koff;
+                for (int cb = 0; cb < P.n_cblk; ++cb, ++it) {
+                    const int s = it % kStages;
+                    const uint32_t ph = (it / kStages) & 1u;
+                    // the codes have landed; the producer refilled this slot only after the MMAs that
+                    // read its previous contents (shared and tensor memory) had completed
+                    bool w = mbar_wait(&sm->full[s], ph, sm, P.status);
+                    if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
+                    tc_fence_after();
+                    const int word = (koff >> 4) + cb * (kBlockK / 16);
+                    const uint32_t *src = reinterpret_cast<const uint32_t *>(sm->codes[s] + row * kCodeRowBytes) + (word & 3);
+                    uint32_t out[32];
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        const uint32_t wv = src[g];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) out[g * 8 + i] = fields_to_bf16x2(wv >> (2 * i));
+                    }
+                    tmem_st32(tmem_a + ((uint32_t)(q * 32) << 16) + s * kAColsPerStage, out);
+                    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm->ready_a[s]);
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------ epilogue
+        const int q = warp & 3;
+        const int ew = warp - 6;
+        long long *pix_off = sm->pix_off[ew];
+        const float alpha = P.alpha ? (float)(*P.alpha) : 1.0f;
+        const int BWm = (1 << P.lgBW) - 1, BHm = (1 << P.lgBH) - 1;
+        uint32_t lt = 0;
+        for (int tile = blockIdx.x; tile < P.total_tiles; tile += gridDim.x, ++lt) {
+            const int nt = tile % P.n_tiles;
+            int pt = tile / P.n_tiles;
+            const int twi = pt % P.tw; pt /= P.tw;
+            const int thi = pt % P.th;
+            const int tbi = pt / P.th;
+            const int n = nt * kChan + q * 32 + lane;
+            const bool n_ok = n < P.Cout;
+            const float sc = (P.scale && n_ok) ? __ldg(P.scale + n) : 1.0f;
+            const float sf = (P.shift && n_ok) ? __ldg(P.shift + n) : 0.0f;
+            // output offsets of the tile's pixels (same for every channel)
+#pragma unroll
+            for (int j = 0; j < kPix / 32; ++j) {
+                const int p = j * 32 + lane;
+                const int wv = (twi << P.lgBW) + (p & BWm);
+                const int hv = (thi << P.lgBH) + ((p >> P.lgBW) & BHm);
+                const int bv = tbi * (kPix >> (P.lgBW + P.lgBH)) + (p >> (P.lgBW + P.lgBH));
+                long long off = -1;
+                if (wv < P.Wv && hv < P.Hv && bv < P.Bv)
+                    off = (((long long)bv * P.OH + (hv * P.osh + P.ooh)) * P.OW + (wv * P.osw + P.oow)) * P.ldy;
+                pix_off[p] = off;
+            }
+            __syncwarp();
+            const int buf = lt & 1;
+            bool w = true;
+            if (kbpt > 0) w = mbar_wait(&sm->acc_full[buf], (lt >> 1) & 1u, sm, P.status);
+            if (!__all_sync(0xffffffffu, w)) break;
+            tc_fence_after();
+#pragma unroll 1
+            for (int c = 0; c < kPix / 32; ++c) {
+                uint32_t v[32];
+                if (kbpt > 0) {
+                    tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + buf * kAccCols + c * 32, v);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = 0u;
+                }
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const long long off = pix_off[c * 32 + j];
+                    if (off < 0 || !n_ok) continue;
+                    float y = __uint_as_float(v[j]) * alpha;
+                    y = fmaf(y, sc, sf);
+                    if (P.residual) {
+                        y += P.res_dtype == TWN_BF16
+                                 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(P.residual)[off + n])
+                                 : reinterpret_cast<const float *>(P.residual)[off + n];
+                    }
+                    if (P.relu) y = fmaxf(y, 0.0f);
+                    if (P.out_dtype == TWN_BF16) reinterpret_cast<__nv_bfloat16 *>(P.Y)[off + n] = __float2bfloat16_rn(y);
+                    else reinterpret_cast<float *>(P.Y)[off + n] = y;
+                }
+            }
+            if (kbpt > 0) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm->acc_empty[buf]);
+            }
+            __syncwarp();
+        }
+    }
+
+    // ---------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (sm->abort_flag) {
+        // give copies and MMAs still in flight time to land before the memory is released
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &p, 12000, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+struct Geometry {
+    // input tensor X: NHWC [XB, XH, XW, XC] with pixel pitch ldx (elements)
+    long long XB, XH, XW, XC, ldx;
+    // virtual output grid and embedding
+    int Bv, Hv, Wv, OH, OW, osh, osw, ooh, oow;
+    long long ldy;
+    int sh, sw;      // input step per virtual output pixel
+    int Cout;
+    long long ld_codes, code_cols;  // packed row pitch and used columns
+    int n_taps;
+    Tap taps[kMaxTaps];
+    long long Cin;   // channels per tap
+};
+
+// Picks the pixel-tile shape (powers of two, product kPix) that wastes the fewest pixels.
+void pick_tile(const Geometry &g, int *lgBW, int *lgBH)
+{
+    long long best = -1;
+    int bw = 0, bh = 0;
+    for (int a = 0; a <= 7; ++a)
+        for (int b = 0; a + b <= 7; ++b) {
+            const int BW = 1 << a, BH = 1 << b, BB = kPix >> (a + b);
+            if (BW * g.sw > 256 || BH * g.sh > 256) continue;
+            const long long tiles = ((g.Wv + BW - 1) / BW) * (long long)((g.Hv + BH - 1) / BH) * ((g.Bv + BB - 1) / BB);
+            // prefer fewer tiles, then wider rows
+            if (best < 0 || tiles < best || (tiles == best && a > bw)) { best = tiles; bw = a; bh = b; }
+        }
+    *lgBW = bw; *lgBH = bh;
+}
+
+int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_stats_t *stats,
+                const twn_epilogue_t *epi, void *Y, int out_dtype_default, int32_t *dev_status, cudaStream_t s)
+{
+    twn_device_info dev;
+    int rc = twn_current_device(&dev);
+    if (rc != TWN_OK) return rc;
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return TWN_ERR_CUDA;
+
+    static bool attr_set[64] = {false};
+    const int smem_bytes = (int)sizeof(SmemLayout) + 1024;
+    if (!attr_set[dev.ordinal]) {
+        TWN_CUDA_OK(cudaFuncSetAttribute(tconv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
+        attr_set[dev.ordinal] = true;
+    }
+
+    ConvParams P;
+    memset(&P, 0, sizeof P);
+    pick_tile(g, &P.lgBW, &P.lgBH);
+    const int BW = 1 << P.lgBW, BH = 1 << P.lgBH, BB = kPix >> (P.lgBW + P.lgBH);
+    P.n_tiles = (g.Cout + kChan - 1) / kChan;
+    P.tw = (g.Wv + BW - 1) / BW;
+    P.th = (g.Hv + BH - 1) / BH;
+    P.tb = (g.Bv + BB - 1) / BB;
+    const long long total = (long long)P.n_tiles * P.tw * P.th * P.tb;
+    if (total <= 0 || total > 0x7fffffffLL) return TWN_ERR_INVALID_ARG;
+    P.total_tiles = (int)total;
+    P.n_taps = g.n_taps;
+    P.n_cblk = (int)((g.Cin + kBlockK - 1) / kBlockK);
+    P.sw = g.sw; P.sh = g.sh;
+    P.Bv = g.Bv; P.Hv = g.Hv; P.Wv = g.Wv;
+    P.OH = g.OH; P.OW = g.OW; P.osh = g.osh; P.osw = g.osw; P.ooh = g.ooh; P.oow = g.oow;
+    P.ldy = g.ldy;
+    P.Cout = g.Cout;
+    P.alpha = stats ? &stats->alpha : nullptr;
+    P.scale = epi ? epi->scale : nullptr;
+    P.shift = epi ? epi->shift : nullptr;
+    P.residual = epi ? epi->residual : nullptr;
+    P.res_dtype = epi ? epi->residual_dtype : TWN_F32;
+    P.relu = epi ? epi->relu : 0;
+    P.out_dtype = epi ? epi->out_dtype : out_dtype_default;
+    P.Y = Y;
+    P.status = dev_status;
+    for (int t = 0; t < g.n_taps; ++t) P.taps[t] = g.taps[t];
+
+    // activations: (C, W, H, B), 64-channel boxes with 128-byte swizzle, zero fill outside
+    CUtensorMap map_x, map_t;
+    {
+        cuuint64_t dims[4] = {(cuuint64_t)g.XC, (cuuint64_t)g.XW, (cuuint64_t)g.XH, (cuuint64_t)g.XB};
+        cuuint64_t strides[3] = {(cuuint64_t)g.ldx * 2, (cuuint64_t)g.XW * g.ldx * 2, (cuuint64_t)g.XH * g.XW * g.ldx * 2};
+        cuuint32_t box[4] = {(cuuint32_t)kBlockK, (cuuint32_t)(BW * g.sw), (cuuint32_t)(BH * g.sh), (cuuint32_t)BB};
+        // with a traversal stride the box counts traversed elements: N loaded elements need N * stride
+        cuuint32_t estr[4] = {1, (cuuint32_t)g.sw, (cuuint32_t)g.sh, 1};
+        if (enc(&map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(X), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return TWN_ERR_INVALID_ARG;
+    }
+    // packed codes: (words, rows), boxes of 8 words x 128 rows, zero fill outside
+    {
+        cuuint64_t dims[2] = {(cuuint64_t)(g.ld_codes / 16), (cuuint64_t)g.Cout};
+        cuuint64_t strides[1] = {(cuuint64_t)(g.ld_codes / 4)};
+        cuuint32_t box[2] = {8, (cuuint32_t)kChan};
+        cuuint32_t estr[2] = {1, 1};
+        if (enc(&map_t, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t *>(T), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return TWN_ERR_INVALID_ARG;
+    }
+    int grid = dev.sm_count < P.total_tiles ? dev.sm_count : P.total_tiles;
+    tconv_kernel<<<grid, kThreadsConv, smem_bytes, s>>>(map_x, map_t, P);
+    TWN_CUDA_OK(cudaGetLastError());
+    return TWN_OK;
+}
+
+int check_epilogue(const twn_epilogue_t *e)
+{
+    if (!e) return TWN_OK;
+    TWN_REQUIRE(e->out_dtype == TWN_F32 || e->out_dtype == TWN_BF16, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(e->residual_dtype == TWN_F32 || e->residual_dtype == TWN_BF16, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(e->relu == 0 || e->relu == 1, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(twn_aligned(e->scale, 4) && twn_aligned(e->shift, 4) && twn_aligned(e->residual, 4), TWN_ERR_MISALIGNED);
+    return TWN_OK;
+}
+
+}  // namespace
+
+extern "C" int twn_gemm(const void *X, int64_t ldx, const uint32_t *T_packed, int64_t ld_codes,
+                        const twn_stats_t *stats, int64_t M, int64_t N, int64_t K,
+                        const twn_epilogue_t *epi, void *Y, int64_t ldy, int32_t *dev_status,
+                        twn_stream_t stream)
+{
+    TWN_REQUIRE(M >= 0 && N >= 0 && K >= 0, TWN_ERR_INVALID_ARG);
+    if (M == 0 || N == 0) return TWN_OK;
+    TWN_REQUIRE(X && T_packed && Y && K > 0, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(ldx >= K && ldy >= N && ld_codes >= K && ld_codes % 64 == 0, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(M <= 0x7fffffffLL && N <= 0x7fffffffLL && K <= 0x7fffffffLL, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(ldx % 8 == 0, TWN_ERR_MISALIGNED);
+    TWN_REQUIRE(twn_aligned(X, 16) && twn_aligned(T_packed, 16) && twn_aligned(Y, 4) && twn_aligned(stats, 8) &&
+                    twn_aligned(dev_status, 4), TWN_ERR_MISALIGNED);
+    int rc = check_epilogue(epi);
+    if (rc != TWN_OK) return rc;
+    Geometry g;
+    memset(&g, 0, sizeof g);
+    g.XB = 1; g.XH = 1; g.XW = M; g.XC = K; g.ldx = ldx;
+    g.Bv = 1; g.Hv = 1; g.Wv = (int)M; g.OH = 1; g.OW = (int)M;
+    g.osh = g.osw = 1; g.ooh = g.oow = 0; g.ldy = ldy;
+    g.sh = g.sw = 1;
+    g.Cout = (int)N; g.ld_codes = ld_codes; g.code_cols = K;
+    g.n_taps = 1; g.taps[0] = Tap{0, 0, 0};
+    g.Cin = K;
+    return launch_conv(g, X, T_packed, stats, epi, Y, TWN_F32, dev_status, twn_cu(stream));
+}
+
+namespace {
+
+int conv_common_checks(const twn_conv_desc_t *d)
+{
+    TWN_REQUIRE(d != nullptr, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(d->B > 0 && d->H > 0 && d->W > 0 && d->Cin > 0 && d->Cout > 0, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(d->kh > 0 && d->kw > 0 && d->stride_h > 0 && d->stride_w > 0 && d->pad_h >= 0 && d->pad_w >= 0,
+                TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(d->stride_h <= 8 && d->stride_w <= 8, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(d->kh * d->kw <= kMaxTaps, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(d->H + 2 * d->pad_h >= d->kh && d->W + 2 * d->pad_w >= d->kw, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(d->B <= 0x7fffffffLL && d->H <= 0x7fffffffLL && d->W <= 0x7fffffffLL && d->Cin <= 0x7fffffffLL &&
+                    d->Cout <= 0x7fffffffLL, TWN_ERR_INVALID_ARG);
+    return TWN_OK;
+}
+
+}  // namespace
+
+extern "C" int twn_conv2d_fwd(const twn_conv_desc_t *d, const void *X, const uint32_t *T_fwd, int64_t ld_codes,
+                              const twn_stats_t *stats, const twn_epilogue_t *epi, void *Y,
+                              int32_t *dev_status, twn_stream_t stream)
+{
+    int rc = conv_common_checks(d);
+    if (rc != TWN_OK) return rc;
+    TWN_REQUIRE(X && T_fwd && Y, TWN_ERR_INVALID_ARG);
+    const long long taps = (long long)d->kh * d->kw;
+    TWN_REQUIRE(ld_codes % 64 == 0 && ld_codes >= taps * d->Cin, TWN_ERR_INVALID_ARG);
+    // channel runs must start on 16-byte boundaries for TMA, tap columns on word boundaries
+    TWN_REQUIRE(d->Cin % 8 == 0 && (taps == 1 || d->Cin % 16 == 0), TWN_ERR_MISALIGNED);
+    TWN_REQUIRE(twn_aligned(X, 16) && twn_aligned(T_fwd, 16) && twn_aligned(Y, 4) && twn_aligned(stats, 8) &&
+                    twn_aligned(dev_status, 4), TWN_ERR_MISALIGNED);
+    rc = check_epilogue(epi);
+    if (rc != TWN_OK) return rc;
+    const long long Ho = (d->H + 2 * d->pad_h - d->kh) / d->stride_h + 1;
+    const long long Wo = (d->W + 2 * d->pad_w - d->kw) / d->stride_w + 1;
+    Geometry g;
+    memset(&g, 0, sizeof g);
+    g.XB = d->B; g.XH = d->H; g.XW = d->W; g.XC = d->Cin; g.ldx = d->Cin;
+    g.Bv = (int)d->B; g.Hv = (int)Ho; g.Wv = (int)Wo; g.OH = (int)Ho; g.OW = (int)Wo;
+    g.osh = g.osw = 1; g.ooh = g.oow = 0; g.ldy = d->Cout;
+    g.sh = d->stride_h; g.sw = d->stride_w;
+    g.Cout = (int)d->Cout; g.ld_codes = ld_codes; g.code_cols = taps * d->Cin;
+    g.Cin = d->Cin;
+    for (int r = 0; r < d->kh; ++r)
+        for (int s = 0; s < d->kw; ++s) {
+            Tap &t = g.taps[g.n_taps++];
+            t.dh = (int16_t)(r - d->pad_h);
+            t.dw = (int16_t)(s - d->pad_w);
+            t.koff = (int32_t)((r * d->kw + s) * d->Cin);
+        }
+    return launch_conv(g, X, T_fwd, stats, epi, Y, TWN_F32, dev_status, twn_cu(stream));
+}
+
+extern "C" int twn_conv2d_bwd_data(const twn_conv_desc_t *d, const void *dZ, const uint32_t *T_bwd, int64_t ld_codes,
+                                   const twn_stats_t *stats, const twn_epilogue_t *epi, void *dX,
+                                   int32_t *dev_status, twn_stream_t stream)
+{
+    int rc = conv_common_checks(d);
+    if (rc != TWN_OK) return rc;
+    TWN_REQUIRE(dZ && T_bwd && dX, TWN_ERR_INVALID_ARG);
+    const long long taps = (long long)d->kh * d->kw;
+    TWN_REQUIRE(ld_codes % 64 == 0 && ld_codes >= taps * d->Cout, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(d->Cout % 8 == 0 && (taps == 1 || d->Cout % 16 == 0), TWN_ERR_MISALIGNED);
+    TWN_REQUIRE(twn_aligned(dZ, 16) && twn_aligned(T_bwd, 16) && twn_aligned(dX, 4) && twn_aligned(stats, 8) &&
+                    twn_aligned(dev_status, 4), TWN_ERR_MISALIGNED);
+    rc = check_epilogue(epi);
+    if (rc != TWN_OK) return rc;
+    const long long Ho = (d->H + 2 * d->pad_h - d->kh) / d->stride_h + 1;
+    const long long Wo = (d->W + 2 * d->pad_w - d->kw) / d->stride_w + 1;
+    // One launch per residue class (ph, pw) of the input pixel modulo the stride: inside a
+    // class the adjoint is a stride-1 sum over the taps r with (ph + pad - r) divisible by
+    // the stride, reading dZ at ho = h' + (ph + pad - r)/stride.
+    for (int ph = 0; ph < d->stride_h; ++ph)
+        for (int pw = 0; pw < d->stride_w; ++pw) {
+            if (ph >= d->H || pw >= d->W) continue;
+            Geometry g;
+            memset(&g, 0, sizeof g);
+            g.XB = d->B; g.XH = Ho; g.XW = Wo; g.XC = d->Cout; g.ldx = d->Cout;
+            g.Bv = (int)d->B;
+            g.Hv = (int)((d->H - ph + d->stride_h - 1) / d->stride_h);
+            g.Wv = (int)((d->W - pw + d->stride_w - 1) / d->stride_w);
+            g.OH = (int)d->H; g.OW = (int)d->W;
+            g.osh = d->stride_h; g.osw = d->stride_w; g.ooh = ph; g.oow = pw;
+            g.ldy = d->Cin;
+            g.sh = g.sw = 1;
+            g.Cout = (int)d->Cin; g.ld_codes = ld_codes; g.code_cols = taps * d->Cout;
+            g.Cin = d->Cout;
+            for (int r = 0; r < d->kh; ++r) {
+                const int xh = ph + d->pad_h - r;
+                if (((xh % d->stride_h) + d->stride_h) % d->stride_h != 0) continue;
+                for (int s = 0; s < d->kw; ++s) {
+                    const int xw = pw + d->pad_w - s;
+                    if (((xw % d->stride_w) + d->stride_w) % d->stride_w != 0) continue;
+                    Tap &t = g.taps[g.n_taps++];
+                    t.dh = (int16_t)(xh / d->stride_h);
+                    t.dw = (int16_t)(xw / d->stride_w);
+                    t.koff = (int32_t)((r * d->kw + s) * d->Cout);
+                }
+            }
+            rc = launch_conv(g, dZ, T_bwd, stats, epi, dX, TWN_F32, dev_status, twn_cu(stream));
+            if (rc != TWN_OK) return rc;
+        }
+    return TWN_OK;
+}

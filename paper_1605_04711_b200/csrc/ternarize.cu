@@ -145,22 +145,52 @@ __device__ __forceinline__ uint32_t code2(float w, float thr, double &kept_sum)
     return keep ? (w < 0.0f ? 3u : 1u) : 0u;
 }
 
+// Bit position of element e (0..15) inside its word: even elements fill the low
+// half-word, odd elements the high half-word.
+__host__ __device__ __forceinline__ int field_pos(int e) { return 2 * (e >> 1) + 16 * (e & 1); }
+
+// Four consecutive weights -> one byte: low nibble = fields of elements 0 and 2,
+// high nibble = fields of elements 1 and 3.
 __device__ __forceinline__ uint32_t code8(const float4 v, float thr, double &k0, double &k1)
 {
     uint32_t c = code2(v.x, thr, k0);
-    c |= code2(v.y, thr, k1) << 2;
-    c |= code2(v.z, thr, k0) << 4;
+    c |= code2(v.z, thr, k0) << 2;
+    c |= code2(v.y, thr, k1) << 4;
     c |= code2(v.w, thr, k1) << 6;
     return c;
 }
 
-// int8 image of four packed fields: 00 -> 0x00, 01 -> 0x01, 11 -> 0xFF
+// Bytes B0..B3 (as produced by code8 for four consecutive float4) -> the word of
+// those 16 elements: low half = low nibbles, high half = high nibbles.
+__device__ __forceinline__ uint32_t bytes_to_word(uint32_t r)
+{
+    uint32_t lo = r & 0x0F0F0F0Fu, hi = (r >> 4) & 0x0F0F0F0Fu;
+    lo = (lo | (lo >> 4)) & 0x00FF00FFu;
+    lo = (lo | (lo >> 8)) & 0x0000FFFFu;
+    hi = (hi | (hi >> 4)) & 0x00FF00FFu;
+    hi = (hi | (hi >> 8)) & 0x0000FFFFu;
+    return lo | (hi << 16);
+}
+
+// inverse: word -> bytes B0..B3
+__device__ __forceinline__ uint32_t word_to_bytes(uint32_t w)
+{
+    uint32_t lo = w & 0xFFFFu, hi = w >> 16;
+    lo = (lo | (lo << 8)) & 0x00FF00FFu;
+    lo = (lo | (lo << 4)) & 0x0F0F0F0Fu;
+    hi = (hi | (hi << 8)) & 0x00FF00FFu;
+    hi = (hi | (hi << 4)) & 0x0F0F0F0Fu;
+    return lo | (hi << 4);
+}
+
+// int8 image of the four fields of a code8 byte, in element order:
+// 00 -> 0x00, 01 -> 0x01, 11 -> 0xFF
 __device__ __forceinline__ uint32_t fields_to_i8x4(uint32_t c8)
 {
     uint32_t r = 0;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-        const uint32_t f = (c8 >> (2 * e)) & 3u;
+        const uint32_t f = (c8 >> (2 * (e >> 1) + 4 * (e & 1))) & 3u;
         const uint32_t b = (f & 1u) ? ((f & 2u) ? 0xFFu : 0x01u) : 0u;
         r |= b << (8 * e);
     }
@@ -170,7 +200,7 @@ __device__ __forceinline__ uint32_t fields_to_i8x4(uint32_t c8)
 // Fast path geometry: a "unit" is 512 consecutive weights = 128 float4 = 32 words,
 // handled by one warp: lane l loads float4 (unit*128 + j*32 + l) for j = 0..3, so
 // every load instruction covers 512 contiguous bytes.  A 4x4 byte transpose inside
-// each group of four lanes then leaves lane l with the complete word
+// each group of four lanes then leaves lane l with the four bytes of word
 // unit*32 + (l%4)*8 + l/4, and the warp stores one contiguous 128-byte line.
 __global__ void __launch_bounds__(kThreads)
 code_pack_kernel(const float *__restrict__ W, long long rows, long long cols, long long ld_codes,
@@ -217,7 +247,7 @@ code_pack_kernel(const float *__restrict__ W, long long rows, long long cols, lo
         r = __byte_perm(r, y, (lane & 2) ? 0x3276 : 0x5410);
         const uint32_t z = __shfl_xor_sync(0xffffffffu, r, 1);
         r = __byte_perm(r, z, (lane & 1) ? 0x3715 : 0x6240);
-        packed[u * 32 + (lane & 3) * 8 + (lane >> 2)] = r;
+        packed[u * 32 + (lane & 3) * 8 + (lane >> 2)] = bytes_to_word(r);
     }
 
     // -- everything else, one thread per word: the tail of a flat tensor, ragged rows, padding
@@ -235,7 +265,7 @@ code_pack_kernel(const float *__restrict__ W, long long rows, long long cols, lo
             if (j < cols) {
                 const float v = __ldg(W + r * cols + j);
                 const uint32_t c = code2(v, thr, k0);
-                word |= c << (2 * e);
+                word |= c << field_pos(e);
                 if (codes_i8) codes_i8[r * cols + j] = (int8_t)((c & 1u) ? ((c & 2u) ? -1 : 1) : 0);
             }
         }
@@ -283,9 +313,9 @@ __device__ __forceinline__ uint32_t i8x4_to_fields(uint32_t x, uint32_t &bad)
     const uint32_t inval = __vcmpgtu4(__vadd4(x, 0x01010101u), 0x02020202u);
     bad |= inval;
     x &= ~inval;
+    // low two bits of bytes 0..3 -> fields in code8 order (e0, e2 | e1, e3)
     const uint32_t y = x & 0x03030303u;
-    const uint32_t t = y | (y >> 6);
-    return (t & 0xFu) | ((t >> 12) & 0xF0u);
+    return (y & 3u) | ((y >> 14) & 0xCu) | ((y >> 4) & 0x30u) | ((y >> 18) & 0xC0u);
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -304,14 +334,14 @@ pack_kernel(const int8_t *__restrict__ codes, long long rows, long long cols, lo
         uint32_t word = 0;
         if (vec_ok && j0 + 16 <= cols) {
             const uint4 v = __ldg(reinterpret_cast<const uint4 *>(codes + r * cols + j0));
-            word = i8x4_to_fields(v.x, bad) | (i8x4_to_fields(v.y, bad) << 8) |
-                   (i8x4_to_fields(v.z, bad) << 16) | (i8x4_to_fields(v.w, bad) << 24);
+            word = bytes_to_word(i8x4_to_fields(v.x, bad) | (i8x4_to_fields(v.y, bad) << 8) |
+                                 (i8x4_to_fields(v.z, bad) << 16) | (i8x4_to_fields(v.w, bad) << 24));
         } else {
             for (int e = 0; e < 16; ++e) {
                 const long long j = j0 + e;
                 if (j < cols) {
                     const uint32_t b = (uint8_t)codes[r * cols + j];
-                    word |= i8x4_to_fields(b, bad) << (2 * e);
+                    word |= (i8x4_to_fields(b, bad) & 3u) << field_pos(e);
                 }
             }
         }
@@ -355,19 +385,23 @@ unpack_kernel(const uint32_t *__restrict__ packed, long long rows, long long col
         const uint32_t inval = (word >> 1) & ~word & 0x55555555u;
         const long long j0 = wi << 4;
         const long long valid = cols - j0 >= 16 ? 16 : cols - j0;
-        const uint32_t vmask = valid >= 16 ? 0xFFFFFFFFu : ((1u << (2 * valid)) - 1u);
+        // fields of elements < valid: ceil(valid/2) in the low half, floor(valid/2) in the high half
+        const uint32_t vmask = valid >= 16 ? 0xFFFFFFFFu
+                                           : (((1u << (2 * ((valid + 1) >> 1))) - 1u) |
+                                              (((1u << (2 * (valid >> 1))) - 1u) << 16));
         if (inval & vmask) bad = true;
         const uint32_t clean = word & ~(inval << 1);
         if (vec_ok && valid == 16) {
+            const uint32_t by = word_to_bytes(clean);
             uint4 o;
-            o.x = fields_to_i8x4(clean & 0xFFu);
-            o.y = fields_to_i8x4((clean >> 8) & 0xFFu);
-            o.z = fields_to_i8x4((clean >> 16) & 0xFFu);
-            o.w = fields_to_i8x4(clean >> 24);
+            o.x = fields_to_i8x4(by & 0xFFu);
+            o.y = fields_to_i8x4((by >> 8) & 0xFFu);
+            o.z = fields_to_i8x4((by >> 16) & 0xFFu);
+            o.w = fields_to_i8x4(by >> 24);
             *reinterpret_cast<uint4 *>(codes + r * cols + j0) = o;
         } else {
             for (int e = 0; e < valid; ++e) {
-                const uint32_t f = (clean >> (2 * e)) & 3u;
+                const uint32_t f = (clean >> field_pos(e)) & 3u;
                 codes[r * cols + j0 + e] = (int8_t)((f & 1u) ? ((f & 2u) ? -1 : 1) : 0);
             }
         }
@@ -393,8 +427,8 @@ transpose_codes_kernel(const uint32_t *__restrict__ in, long long ld_in, long lo
             if (j < cols_out) {
                 const long long t = j / Cout, o = j - t * Cout;
                 const long long src = t * Cin + c;
-                const uint32_t f = (__ldg(in + o * wpr_in + (src >> 4)) >> (2 * (src & 15))) & 3u;
-                word |= f << (2 * e);
+                const uint32_t f = (__ldg(in + o * wpr_in + (src >> 4)) >> field_pos((int)(src & 15))) & 3u;
+                word |= f << field_pos(e);
             }
         }
         out[w] = word;

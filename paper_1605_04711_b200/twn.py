@@ -148,3 +148,41 @@ def transpose_codes(packed_fwd: torch.Tensor, ld_fwd: int, desc: ConvDesc, packe
     _check(lib().twn_transpose_codes(_ptr(packed_fwd), C.c_int64(ld_fwd), C.byref(desc),
                                      _ptr(packed_bwd), C.c_int64(ld_bwd), _stream(stream)),
            "twn_transpose_codes")
+
+
+def epilogue(scale=None, shift=None, residual=None, relu=False, out_dtype=F32):
+    """Builds a twn_epilogue_t; keeps no reference, the caller keeps the tensors alive."""
+    e = Epilogue()
+    e.scale = _ptr(scale).value or None
+    e.shift = _ptr(shift).value or None
+    e.residual = _ptr(residual).value or None
+    e.residual_dtype = BF16 if (residual is not None and residual.dtype == torch.bfloat16) else F32
+    e.relu = int(bool(relu))
+    e.out_dtype = out_dtype
+    return e
+
+
+def _alpha_stats(stats):
+    return _ptr(stats)
+
+
+def gemm(X: torch.Tensor, ldx: int, T_packed: torch.Tensor, ld_codes: int, stats, M: int, N: int,
+         K: int, epi, Y: torch.Tensor, ldy: int, dev_status=None, stream=None) -> None:
+    _check(lib().twn_gemm(_ptr(X), C.c_int64(ldx), _ptr(T_packed), C.c_int64(ld_codes), _ptr(stats),
+                          C.c_int64(M), C.c_int64(N), C.c_int64(K),
+                          C.byref(epi) if epi is not None else None, _ptr(Y), C.c_int64(ldy),
+                          _ptr(dev_status), _stream(stream)), "twn_gemm")
+
+
+def conv2d_fwd(desc: ConvDesc, X: torch.Tensor, T_fwd: torch.Tensor, ld_codes: int, stats, epi,
+               Y: torch.Tensor, dev_status=None, stream=None) -> None:
+    _check(lib().twn_conv2d_fwd(C.byref(desc), _ptr(X), _ptr(T_fwd), C.c_int64(ld_codes), _ptr(stats),
+                                C.byref(epi) if epi is not None else None, _ptr(Y), _ptr(dev_status),
+                                _stream(stream)), "twn_conv2d_fwd")
+
+
+def conv2d_bwd_data(desc: ConvDesc, dZ: torch.Tensor, T_bwd: torch.Tensor, ld_codes: int, stats, epi,
+                    dX: torch.Tensor, dev_status=None, stream=None) -> None:
+    _check(lib().twn_conv2d_bwd_data(C.byref(desc), _ptr(dZ), _ptr(T_bwd), C.c_int64(ld_codes),
+                                     _ptr(stats), C.byref(epi) if epi is not None else None, _ptr(dX),
+                                     _ptr(dev_status), _stream(stream)), "twn_conv2d_bwd_data")

@@ -218,14 +218,16 @@ def test_golden_closed_forms_file():
 
 # ----------------------------------------------------------- 2-bit storage
 def test_pack_hand_worked_word():
-    # element j -> bits [2j+1:2j]; 0 -> 00, +1 -> 01, -1 -> 11
+    # element e of a 16-group -> bit 2*(e//2) + 16*(e%2); 0 -> 00, +1 -> 01, -1 -> 11
+    # e0 = +1 -> bits 1:0 = 01 ; e1 = 0 ; e2 = -1 -> bits 3:2 = 11 ; e3 = +1 -> bits 19:18 = 01
     codes = np.array([1, 0, -1, 1], dtype=np.int8)
     p = oracle.pack(codes, 16)
-    assert p.shape == (1, 1) and int(p[0, 0]) == 0b01_11_00_01
-    codes = np.zeros(32, dtype=np.int8); codes[15] = -1; codes[16] = 1
+    assert p.shape == (1, 1) and int(p[0, 0]) == (0b1101 | (0b0100 << 16))
+    # e15 (odd, pair 7) -> bits 31:30 ; e16 = element 0 of the next word -> bits 1:0
+    codes = np.zeros(32, dtype=np.int8); codes[15] = -1; codes[16] = 1; codes[14] = 1
     p = oracle.pack(codes, 64)
     assert p.shape == (1, 4)
-    assert [int(v) for v in p[0]] == [0xC0000000, 0x00000001, 0, 0]
+    assert [int(v) for v in p[0]] == [0xC0004000, 0x00000001, 0, 0]
 
 
 def test_pack_round_trip_all_3_pow_16_words():
