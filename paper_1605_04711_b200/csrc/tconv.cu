@@ -30,17 +30,21 @@
 
 namespace {
 
-constexpr int kStages = 8;          // smem / tensor-memory operand ring depth
+constexpr int kStages = 4;          // smem / tensor-memory operand ring depth
+constexpr int kSub = 2;             // k-blocks per stage: one wait and one commit per 8 MMAs
 constexpr int kChan = 128;          // output channels per tile (UMMA M)
 constexpr int kPix = 128;           // pixels per tile (UMMA N)
 constexpr int kBlockK = 64;         // reduction elements per k-block (128 bytes of bf16)
 constexpr int kXBytes = kPix * kBlockK * 2;    // 16 KB
-constexpr int kCodeRowBytes = 32;              // 8 words per channel row per k-block (4 used)
-constexpr int kCodeBytes = kChan * kCodeRowBytes;  // 4 KB
-constexpr int kThreadsConv = 320;
+constexpr int kCodeRowBytesMax = 32;           // up to 8 words per channel row per k-block (4 used)
+constexpr int kCodeBytes = kChan * kCodeRowBytesMax;  // 4 KB
+constexpr int kDecodeSets = 2;      // groups of 4 decode warps; a group takes every other stage
+constexpr int kFirstEpiWarp = 2 + 4 * kDecodeSets;
+constexpr int kThreadsConv = 32 * (kFirstEpiWarp + 4);
 constexpr int kMaxTaps = 64;
 constexpr int kAccCols = kPix;                 // fp32 accumulator columns per buffer
-constexpr int kAColsPerStage = kBlockK / 2;    // 32 columns of bf16 pairs
+constexpr int kAColsPerBlock = kBlockK / 2;    // 32 columns of bf16 pairs per k-block
+constexpr int kAColsPerStage = kSub * kAColsPerBlock;
 constexpr uint32_t kTmemCols = 512;
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;
 
@@ -55,6 +59,8 @@ struct ConvParams {
     int lgBW, lgBH;               // pixel tile = BB x BH x BW, powers of two, product kPix
     // reduction
     int n_taps, n_cblk;           // k-blocks per tile = n_taps * n_cblk
+    int code_row_words;           // words per channel row in a staged code tile: 4 (every k-block
+                                  // starts on a 16-byte boundary of the packed row) or 8
     int sw, sh;                   // input pixel = output pixel * (sh, sw) + (dh, dw)
     // virtual output grid and its embedding in the output tensor
     int Bv, Hv, Wv;
@@ -72,10 +78,10 @@ struct ConvParams {
 };
 
 struct __align__(1024) SmemLayout {
-    uint8_t x[kStages][kXBytes];           // swizzled activation tiles
-    uint8_t codes[kStages][kCodeBytes];    // packed code tiles, row = channel
-    unsigned long long full[kStages];      // TMA -> decode + MMA
-    unsigned long long ready_a[kStages];   // decode -> MMA
+    uint8_t x[kStages][kSub][kXBytes];           // swizzled activation tiles
+    uint8_t codes[kStages][kSub][kCodeBytes];    // packed code tiles, row = channel
+    unsigned long long full[kStages];      // TMA -> decode
+    unsigned long long ready_a[kStages];   // decode -> MMA (implies full: the decode warps saw it)
     unsigned long long empty[kStages];     // MMA commit -> TMA + decode
     unsigned long long acc_full[2];        // MMA commit -> epilogue
     unsigned long long acc_empty[2];       // epilogue -> MMA
@@ -170,6 +176,18 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint
         : "memory");
 }
 
+// One k-block: four K=16 MMAs.  FIRST clears the accumulator with the first of them.  The
+// accumulate flag is a compile-time constant so that no predicate has to be built at run time:
+// whatever the issuing thread executes between two MMAs is time the tensor core may sit idle.
+template <bool FIRST>
+__device__ __forceinline__ void tc_mma_block(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc)
+{
+    tc_mma_ts(d_tmem, a_tmem, b_desc, idesc, FIRST ? 0u : 1u);
+    tc_mma_ts(d_tmem, a_tmem + 8, b_desc + 2, idesc, 1u);
+    tc_mma_ts(d_tmem, a_tmem + 16, b_desc + 4, idesc, 1u);
+    tc_mma_ts(d_tmem, a_tmem + 24, b_desc + 6, idesc, 1u);
+}
+
 // K-major, 128-byte swizzled operand tile: rows of 128 bytes, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr)
 {
@@ -239,7 +257,8 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
     SmemLayout *sm = reinterpret_cast<SmemLayout *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int kbpt = P.n_taps * P.n_cblk;
+    const int kbpt = P.n_taps * P.n_cblk;               // k-blocks per tile
+    const int spt = (kbpt + kSub - 1) / kSub;           // stages per tile (the last may hold one k-block)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -270,6 +289,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
+            const uint32_t block_bytes = kXBytes + kChan * 4 * P.code_row_words;
             for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
                 const int nt = tile % P.n_tiles;
                 int pt = tile / P.n_tiles;
@@ -279,87 +299,104 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 const int w0 = (twi << P.lgBW) * P.sw;
                 const int h0 = (thi << P.lgBH) * P.sh;
                 const int b0 = tbi * (kPix >> (P.lgBW + P.lgBH));
-                for (int t = 0; t < P.n_taps && ok; ++t) {
-                    const Tap tap = P.taps[t];
-                    for (int cb = 0; cb < P.n_cblk; ++cb, ++it) {
-                        const int s = it % kStages;
-                        const uint32_t ph = (it / kStages) & 1u;
-                        if (!mbar_wait(&sm->empty[s], ph ^ 1u, sm, P.status)) { ok = false; break; }
-                        mbar_expect_tx(&sm->full[s], kXBytes + kCodeBytes);
-                        tma_load_4d(sm->x[s], &map_x, &sm->full[s], cb * kBlockK, w0 + tap.dw, h0 + tap.dh, b0);
+                int t = 0, cb = 0;
+                for (int st = 0; st < spt; ++st, ++it) {
+                    const int s = it % kStages;
+                    const uint32_t ph = (it / kStages) & 1u;
+                    const int nsb = (kbpt - st * kSub) < kSub ? (kbpt - st * kSub) : kSub;
+                    if (!mbar_wait(&sm->empty[s], ph ^ 1u, sm, P.status)) { ok = false; break; }
+                    mbar_expect_tx(&sm->full[s], nsb * block_bytes);
+                    for (int sb = 0; sb < nsb; ++sb) {
+                        const Tap tap = P.taps[t];
+                        tma_load_4d(sm->x[s][sb], &map_x, &sm->full[s], cb * kBlockK, w0 + tap.dw, h0 + tap.dh, b0);
                         const int word = (tap.koff >> 4) + cb * (kBlockK / 16);
-                        tma_load_2d(sm->codes[s], &map_t, &sm->full[s], word & ~3, nt * kChan);
+                        // word % 4 == 0 whenever code_row_words == 4
+                        tma_load_2d(sm->codes[s][sb], &map_t, &sm->full[s], word & ~3, nt * kChan);
+                        if (++cb == P.n_cblk) { cb = 0; ++t; }
                     }
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // Kept as lean as possible: one wait and one commit per stage, constant accumulate flags.
+        // With no taps at all (kbpt == 0) nothing is accumulated and the epilogue does not wait.
+        if (lane == 0 && kbpt > 0) {
             constexpr uint32_t idesc = make_idesc(kChan, kPix);
+            const uint64_t bdesc0 = smem_desc_sw128(smem_u32(sm->x[0][0]));
             uint32_t it = 0, lt = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x, ++lt) {
                 const int buf = lt & 1;
                 if (!mbar_wait(&sm->acc_empty[buf], ((lt >> 1) & 1u) ^ 1u, sm, P.status)) break;
-                tc_fence_after();
                 const uint32_t d_tmem = tmem_acc + buf * kAccCols;
-                for (int kb = 0; kb < kbpt; ++kb, ++it) {
+                for (int st = 0; st < spt; ++st, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
-                    if (!mbar_wait(&sm->full[s], ph, sm, P.status) ||
-                        !mbar_wait(&sm->ready_a[s], ph, sm, P.status)) { ok = false; break; }
+                    if (!mbar_wait(&sm->ready_a[s], ph, sm, P.status)) { ok = false; break; }
                     tc_fence_after();
-                    const uint64_t bdesc = smem_desc_sw128(smem_u32(sm->x[s]));
-#pragma unroll
-                    for (int k = 0; k < kBlockK / 16; ++k) {
-                        // 16 reduction elements = 8 tensor-memory columns of A, 32 bytes of a B row
-                        tc_mma_ts(d_tmem, tmem_a + s * kAColsPerStage + k * 8, bdesc + (uint64_t)(k * 2),
-                                  idesc, (kb > 0 || k > 0) ? 1u : 0u);
-                    }
+                    const uint64_t bdesc = bdesc0 + (uint64_t)(s * ((kSub * kXBytes) >> 4));
+                    const uint32_t a_tmem = tmem_a + s * kAColsPerStage;
+                    if (st == 0) tc_mma_block<true>(d_tmem, a_tmem, bdesc, idesc);
+                    else tc_mma_block<false>(d_tmem, a_tmem, bdesc, idesc);
+                    if (kbpt - st * kSub > 1)
+                        tc_mma_block<false>(d_tmem, a_tmem + kAColsPerBlock, bdesc + (kXBytes >> 4), idesc);
                     tc_commit(&sm->empty[s]);
                 }
                 if (ok) tc_commit(&sm->acc_full[buf]);
             }
         }
-    } else if (warp < 6) {
+    } else if (warp < kFirstEpiWarp) {
         // ------------------------------------------------ decode: codes -> bf16 -> tensor memory
+        // Two groups of four warps; a group handles every other stage, so the latency of the
+        // tensor-memory store of one stage overlaps the decoding of the next by the other group.
         const int q = warp & 3;                 // tensor-memory lane quadrant of this warp
+        const int set = (warp - 2) >> 2;
         const int row = q * 32 + lane;          // channel row inside the tile
+        const uint32_t lane_base = tmem_a + ((uint32_t)(q * 32) << 16);
         uint32_t it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
-            for (int t = 0; t < P.n_taps && ok; ++t) {
-                const int koff = P.taps[t].koff;
-                for (int cb = 0; cb < P.n_cblk; ++cb, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (it / kStages) & 1u;
-                    // the codes have landed; the producer refilled this slot only after the MMAs that
-                    // read its previous contents (shared and tensor memory) had completed
-                    bool w = mbar_wait(&sm->full[s], ph, sm, P.status);
-                    if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
-                    tc_fence_after();
-                    const int word = (koff >> 4) + cb * (kBlockK / 16);
-                    const uint32_t *src = reinterpret_cast<const uint32_t *>(sm->codes[s] + row * kCodeRowBytes) + (word & 3);
+            for (int st = 0; st < spt; ++st, ++it) {
+                if ((int)(it % kDecodeSets) != set) continue;
+                const int s = it % kStages;
+                const uint32_t ph = (it / kStages) & 1u;
+                const int nsb = (kbpt - st * kSub) < kSub ? (kbpt - st * kSub) : kSub;
+                // the codes have landed; the producer refilled this slot only after the MMAs that
+                // read its previous contents (shared and tensor memory) had completed
+                const bool w = mbar_wait(&sm->full[s], ph, sm, P.status);
+                if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
+                tc_fence_after();
+                for (int sb = 0; sb < nsb; ++sb) {
+                    uint32_t wv[4];
+                    if (P.code_row_words == 4) {
+                        const uint4 v = *reinterpret_cast<const uint4 *>(sm->codes[s][sb] + row * 16);
+                        wv[0] = v.x; wv[1] = v.y; wv[2] = v.z; wv[3] = v.w;
+                    } else {
+                        const int u = st * kSub + sb;
+                        const int t = u / P.n_cblk, cb = u - t * P.n_cblk;
+                        const int word = (P.taps[t].koff >> 4) + cb * (kBlockK / 16);
+                        const uint32_t *src = reinterpret_cast<const uint32_t *>(sm->codes[s][sb] + row * 32) + (word & 3);
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) wv[g] = src[g];
+                    }
                     uint32_t out[32];
 #pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        const uint32_t wv = src[g];
+                    for (int g = 0; g < 4; ++g)
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) out[g * 8 + i] = fields_to_bf16x2(wv >> (2 * i));
-                    }
-                    tmem_st32(tmem_a + ((uint32_t)(q * 32) << 16) + s * kAColsPerStage, out);
-                    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&sm->ready_a[s]);
+                        for (int e = 0; e < 8; ++e) out[g * 8 + e] = fields_to_bf16x2(wv[g] >> (2 * e));
+                    tmem_st32(lane_base + s * kAColsPerStage + sb * kAColsPerBlock, out);
                 }
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm->ready_a[s]);
             }
         }
     } else {
         // ------------------------------------------------ epilogue
         const int q = warp & 3;
-        const int ew = warp - 6;
+        const int ew = warp - kFirstEpiWarp;
         long long *pix_off = sm->pix_off[ew];
         const float alpha = P.alpha ? (float)(*P.alpha) : 1.0f;
         const int BWm = (1 << P.lgBW) - 1, BHm = (1 << P.lgBH) - 1;
@@ -520,6 +557,9 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     P.total_tiles = (int)total;
     P.n_taps = g.n_taps;
     P.n_cblk = (int)((g.Cin + kBlockK - 1) / kBlockK);
+    P.code_row_words = 4;
+    for (int t = 0; t < g.n_taps; ++t)
+        if (g.taps[t].koff % kBlockK != 0) P.code_row_words = 8;
     P.sw = g.sw; P.sh = g.sh;
     P.Bv = g.Bv; P.Hv = g.Hv; P.Wv = g.Wv;
     P.OH = g.OH; P.OW = g.OW; P.osh = g.osh; P.osw = g.osw; P.ooh = g.ooh; P.oow = g.oow;
@@ -553,7 +593,7 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     {
         cuuint64_t dims[2] = {(cuuint64_t)(g.ld_codes / 16), (cuuint64_t)g.Cout};
         cuuint64_t strides[1] = {(cuuint64_t)(g.ld_codes / 4)};
-        cuuint32_t box[2] = {8, (cuuint32_t)kChan};
+        cuuint32_t box[2] = {(cuuint32_t)P.code_row_words, (cuuint32_t)kChan};
         cuuint32_t estr[2] = {1, 1};
         if (enc(&map_t, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t *>(T), dims, strides, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
