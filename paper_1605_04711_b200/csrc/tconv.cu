@@ -16,37 +16,53 @@
 // owns one channel, so alpha, the per-channel affine and ReLU cost one register each,
 // and a warp's store of one pixel covers 32 consecutive channels (128 contiguous bytes).
 //
-//   warp 0      TMA producer: X tile and packed-code tile per k-block
-//   warp 1      allocates tensor memory, issues tcgen05.mma, commits to mbarriers
-//   warps 2-5   decode: packed codes (smem) -> bf16 pairs -> tensor memory
-//   warps 6-9   epilogue: tensor memory -> registers -> global
+//   warp 0        TMA producer: X tile and packed-code tile per k-block
+//   warp 1        allocates tensor memory, issues tcgen05.mma, commits to mbarriers
+//   warps 2-9     decode: packed codes (smem) -> bf16 pairs -> tensor memory
+//   warps 10-13   epilogue: tensor memory -> registers -> global
+//
+// Two tile shapes.  Measured on B200: one thread can issue a tcgen05.mma about every
+// 50-90 cycles whatever its size, and waits or commits between MMAs are not hidden
+// unless the MMA itself is long.  A 128x256x16 MMA (128 cycles) hides that; a 128x128x16
+// one (64 cycles) does not.  So the large shape uses 256-pixel tiles with a single
+// accumulator (tensor memory holds 512 columns: 256 for it, the rest for the decoded
+// weights), and the epilogue of a tile is not overlapped with the next tile's MMAs.
+// Small problems use 128-pixel tiles, two accumulators and two k-blocks per stage.
 //
 // Every wait on an mbarrier is bounded (about a second); on expiry the kernel records
 // TWN_ERR_TIMEOUT, all roles leave their loops, tensor memory is freed and the grid exits.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <cstddef>
+
 #include "common.cuh"
 
 namespace {
 
-constexpr int kStages = 4;          // smem / tensor-memory operand ring depth
-constexpr int kSub = 2;             // k-blocks per stage: one wait and one commit per 8 MMAs
 constexpr int kChan = 128;          // output channels per tile (UMMA M)
-constexpr int kPix = 128;           // pixels per tile (UMMA N)
 constexpr int kBlockK = 64;         // reduction elements per k-block (128 bytes of bf16)
-constexpr int kXBytes = kPix * kBlockK * 2;    // 16 KB
 constexpr int kCodeRowBytesMax = 32;           // up to 8 words per channel row per k-block (4 used)
 constexpr int kCodeBytes = kChan * kCodeRowBytesMax;  // 4 KB
 constexpr int kDecodeSets = 2;      // groups of 4 decode warps; a group takes every other stage
 constexpr int kFirstEpiWarp = 2 + 4 * kDecodeSets;
 constexpr int kThreadsConv = 32 * (kFirstEpiWarp + 4);
 constexpr int kMaxTaps = 64;
-constexpr int kAccCols = kPix;                 // fp32 accumulator columns per buffer
 constexpr int kAColsPerBlock = kBlockK / 2;    // 32 columns of bf16 pairs per k-block
-constexpr int kAColsPerStage = kSub * kAColsPerBlock;
 constexpr uint32_t kTmemCols = 512;
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;
+
+template <int PIX> struct Cfg;
+template <> struct Cfg<128> {
+    static constexpr int kStages = 4;   // operand ring depth (shared and tensor memory)
+    static constexpr int kSub = 2;      // k-blocks per stage: one wait and one commit per 8 MMAs
+    static constexpr int kAccBufs = 2;  // the epilogue of a tile overlaps the MMAs of the next
+};
+template <> struct Cfg<256> {
+    static constexpr int kStages = 5;
+    static constexpr int kSub = 1;
+    static constexpr int kAccBufs = 1;
+};
 
 struct Tap {
     int16_t dh, dw;   // input pixel offset of this tap
@@ -56,7 +72,7 @@ struct Tap {
 struct ConvParams {
     // tiles
     int n_tiles, tw, th, tb, total_tiles;
-    int lgBW, lgBH;               // pixel tile = BB x BH x BW, powers of two, product kPix
+    int lgBW, lgBH;               // pixel tile = BB x BH x BW, powers of two, product PIX
     // reduction
     int n_taps, n_cblk;           // k-blocks per tile = n_taps * n_cblk
     int code_row_words;           // words per channel row in a staged code tile: 4 (every k-block
@@ -74,20 +90,28 @@ struct ConvParams {
     int res_dtype, relu, out_dtype;
     void *Y;
     int32_t *status;
+    // output path: 1 = the tile is staged in shared memory 32 pixels at a time and written with
+    // TMA stores (box = 128 channels x sbw x sbh x sbb pixels); 0 = per-thread stores
+    int tma_store, lg_sbw, lg_sbh;
     Tap taps[kMaxTaps];
 };
 
+template <int PIX>
 struct __align__(1024) SmemLayout {
+    static constexpr int kStages = Cfg<PIX>::kStages, kSub = Cfg<PIX>::kSub;
+    static constexpr int kXBytes = PIX * kBlockK * 2;
     uint8_t x[kStages][kSub][kXBytes];           // swizzled activation tiles
     uint8_t codes[kStages][kSub][kCodeBytes];    // packed code tiles, row = channel
     unsigned long long full[kStages];      // TMA -> decode
     unsigned long long ready_a[kStages];   // decode -> MMA (implies full: the decode warps saw it)
-    unsigned long long empty[kStages];     // MMA commit -> TMA + decode
+    unsigned long long empty[kStages];     // MMA commit -> TMA
     unsigned long long acc_full[2];        // MMA commit -> epilogue
     unsigned long long acc_empty[2];       // epilogue -> MMA
-    long long pix_off[4][kPix];            // per epilogue warp: output element offset, -1 = skip
+    alignas(16) uint32_t pix_off[4][PIX];  // per epilogue warp: output element offset of a pixel, ~0 = skip
+    alignas(128) float stage_out[2][32 * kChan];  // output staging for TMA stores: [32 pixels][128 channels]
     uint32_t tmem_base;
     volatile int abort_flag;
+    volatile int epi_ok;                   // outcome of the epilogue's wait, shared by its four warps
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -110,9 +134,9 @@ __device__ __forceinline__ bool mbar_try(void *bar, uint32_t parity)
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(2000u) : "memory");
     return ok != 0;
 }
 __device__ __forceinline__ unsigned long long global_ns()
@@ -123,23 +147,40 @@ __device__ __forceinline__ unsigned long long global_ns()
 }
 
 // Bounded wait.  Returns false when the limit ran out or another role gave up.
-__device__ __forceinline__ bool mbar_wait(void *bar, uint32_t parity, SmemLayout *sm, int32_t *status)
+// Waiting warps share their scheduler with the warps that do the work, so a waiter backs
+// off with nanosleep instead of polling flat out (`backoff_ns` = 0 for the latency-critical
+// waits of the MMA warp, which rely on the suspend time of try_wait alone).
+__device__ __forceinline__ bool mbar_wait(void *bar, uint32_t parity, volatile int *abort_flag, int32_t *status,
+                                          uint32_t backoff_ns = 64)
 {
     if (mbar_try(bar, parity)) return true;
     unsigned long long t0 = 0;
     for (uint32_t spin = 1;; ++spin) {
         if (mbar_try(bar, parity)) return true;
+        if (backoff_ns) __nanosleep(backoff_ns);
         if ((spin & 255u) == 0) {
-            if (sm->abort_flag) return false;
+            if (*abort_flag) return false;
             const unsigned long long now = global_ns();
             if (t0 == 0) t0 = now;
             else if (now - t0 > kWaitLimitNs) {
-                sm->abort_flag = 1;
+                *abort_flag = 1;
                 if (status) atomicMin(status, (int)TWN_ERR_TIMEOUT);
                 return false;
             }
         }
     }
+}
+
+// Warp-wide wait: lane 0 polls, the result is broadcast.  One polling lane instead of 32
+// keeps the shared-memory pipe free for the warps that are working.
+__device__ __forceinline__ bool mbar_wait_warp(void *bar, uint32_t parity, volatile int *abort_flag, int32_t *status,
+                                               uint32_t backoff_ns = 64)
+{
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status, backoff_ns) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    __syncwarp();
+    return ok != 0;
 }
 
 __device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, void *bar, int c0, int c1, int c2, int c3)
@@ -157,23 +198,44 @@ __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, v
         : "memory");
 }
 
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap *map, const void *src, int c0, int c1, int c2, int c3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+        ::"l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// named barrier of the four epilogue warps
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void tc_commit(void *bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
 
-// D[tmem] (+)= A[tmem] * B[smem]^T, bf16 x bf16 -> fp32, one thread issues.
-__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+// The MMA warp runs its loops converged; tcgen05.mma and tcgen05.commit are issued by the
+// lane that elect.sync picks, with the predicate applied inside the asm block (measured to be
+// the cheapest way to issue: no divergent region around the instruction).
+// D[tmem] (+)= A[tmem] * B[smem]^T, bf16 x bf16 -> fp32.
+template <bool ACC>
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
+        "{\n\t.reg .pred p, pe;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "elect.sync _|pe, 0xffffffff;\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "n"(ACC ? 1 : 0)
         : "memory");
+}
+
+__device__ __forceinline__ void tc_commit(void *bar)
+{
+    asm volatile(
+        "{\n\t.reg .pred pe;\n\t"
+        "elect.sync _|pe, 0xffffffff;\n\t"
+        "@pe tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(smem_u32(bar)) : "memory");
 }
 
 // One k-block: four K=16 MMAs.  FIRST clears the accumulator with the first of them.  The
@@ -182,10 +244,10 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint
 template <bool FIRST>
 __device__ __forceinline__ void tc_mma_block(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc)
 {
-    tc_mma_ts(d_tmem, a_tmem, b_desc, idesc, FIRST ? 0u : 1u);
-    tc_mma_ts(d_tmem, a_tmem + 8, b_desc + 2, idesc, 1u);
-    tc_mma_ts(d_tmem, a_tmem + 16, b_desc + 4, idesc, 1u);
-    tc_mma_ts(d_tmem, a_tmem + 24, b_desc + 6, idesc, 1u);
+    tc_mma_ts<!FIRST>(d_tmem, a_tmem, b_desc, idesc);
+    tc_mma_ts<true>(d_tmem, a_tmem + 8, b_desc + 2, idesc);
+    tc_mma_ts<true>(d_tmem, a_tmem + 16, b_desc + 4, idesc);
+    tc_mma_ts<true>(d_tmem, a_tmem + 24, b_desc + 6, idesc);
 }
 
 // K-major, 128-byte swizzled operand tile: rows of 128 bytes, 8-row groups 1024 bytes apart.
@@ -249,16 +311,30 @@ __device__ __forceinline__ uint32_t fields_to_bf16x2(uint32_t x)
 }
 
 // ---------------------------------------------------------------- the kernel
+static_assert(offsetof(SmemLayout<128>, stage_out) % 128 == 0 && offsetof(SmemLayout<256>, stage_out) % 128 == 0 &&
+                  offsetof(SmemLayout<128>, pix_off) % 16 == 0 && offsetof(SmemLayout<256>, pix_off) % 16 == 0 &&
+                  offsetof(SmemLayout<128>, codes) % 128 == 0 && offsetof(SmemLayout<256>, codes) % 128 == 0,
+              "TMA and vector accesses need aligned shared-memory regions");
+
+template <int PIX>
 __global__ void __launch_bounds__(kThreadsConv, 1)
 tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_t,
-             const __grid_constant__ ConvParams P)
+             const __grid_constant__ CUtensorMap map_y, const __grid_constant__ ConvParams P)
 {
+    using L = SmemLayout<PIX>;
+    constexpr int kStages = Cfg<PIX>::kStages, kSub = Cfg<PIX>::kSub, kAccBufs = Cfg<PIX>::kAccBufs;
+    constexpr int kXBytes = L::kXBytes;
+    constexpr int kAColsPerStage = kSub * kAColsPerBlock;
+    static_assert(kAccBufs * PIX + kStages * kAColsPerStage <= (int)kTmemCols, "tensor memory budget");
+    
+
     extern __shared__ uint8_t smem_raw[];
-    SmemLayout *sm = reinterpret_cast<SmemLayout *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    L *sm = reinterpret_cast<L *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    volatile int *abort_flag = &sm->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int kbpt = P.n_taps * P.n_cblk;               // k-blocks per tile
-    const int spt = (kbpt + kSub - 1) / kSub;           // stages per tile (the last may hold one k-block)
+    const int spt = (kbpt + kSub - 1) / kSub;           // stages per tile (the last may hold fewer k-blocks)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -281,8 +357,8 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sm->tmem_base;
-    const uint32_t tmem_acc = tmem;                       // 2 x kAccCols columns
-    const uint32_t tmem_a = tmem + 2 * kAccCols;          // kStages x kAColsPerStage columns
+    const uint32_t tmem_acc = tmem;                       // kAccBufs x PIX columns
+    const uint32_t tmem_a = tmem + kAccBufs * PIX;        // kStages x kAColsPerStage columns
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
@@ -298,13 +374,13 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 const int tbi = pt / P.th;
                 const int w0 = (twi << P.lgBW) * P.sw;
                 const int h0 = (thi << P.lgBH) * P.sh;
-                const int b0 = tbi * (kPix >> (P.lgBW + P.lgBH));
+                const int b0 = tbi * (PIX >> (P.lgBW + P.lgBH));
                 int t = 0, cb = 0;
                 for (int st = 0; st < spt; ++st, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
                     const int nsb = (kbpt - st * kSub) < kSub ? (kbpt - st * kSub) : kSub;
-                    if (!mbar_wait(&sm->empty[s], ph ^ 1u, sm, P.status)) { ok = false; break; }
+                    if (!mbar_wait(&sm->empty[s], ph ^ 1u, abort_flag, P.status)) { ok = false; break; }
                     mbar_expect_tx(&sm->full[s], nsb * block_bytes);
                     for (int sb = 0; sb < nsb; ++sb) {
                         const Tap tap = P.taps[t];
@@ -318,28 +394,30 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------ MMA issuer
-        // Kept as lean as possible: one wait and one commit per stage, constant accumulate flags.
-        // With no taps at all (kbpt == 0) nothing is accumulated and the epilogue does not wait.
-        if (lane == 0 && kbpt > 0) {
-            constexpr uint32_t idesc = make_idesc(kChan, kPix);
+        // ------------------------------------------------ MMA issuer (whole warp, converged)
+        // One wait and one commit per stage, constant accumulate flags.  With no taps at all
+        // (kbpt == 0) nothing is accumulated and the epilogue does not wait.
+        if (kbpt > 0) {
+            constexpr uint32_t idesc = make_idesc(kChan, PIX);
             const uint64_t bdesc0 = smem_desc_sw128(smem_u32(sm->x[0][0]));
             uint32_t it = 0, lt = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x, ++lt) {
-                const int buf = lt & 1;
-                if (!mbar_wait(&sm->acc_empty[buf], ((lt >> 1) & 1u) ^ 1u, sm, P.status)) break;
-                const uint32_t d_tmem = tmem_acc + buf * kAccCols;
+                const int buf = lt % kAccBufs;
+                const uint32_t aph = (lt / kAccBufs) & 1u;
+                if (!mbar_wait_warp(&sm->acc_empty[buf], aph ^ 1u, abort_flag, P.status, 0)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_acc + buf * PIX;
                 for (int st = 0; st < spt; ++st, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
-                    if (!mbar_wait(&sm->ready_a[s], ph, sm, P.status)) { ok = false; break; }
+                    if (!mbar_wait_warp(&sm->ready_a[s], ph, abort_flag, P.status, 0)) { ok = false; break; }
                     tc_fence_after();
                     const uint64_t bdesc = bdesc0 + (uint64_t)(s * ((kSub * kXBytes) >> 4));
                     const uint32_t a_tmem = tmem_a + s * kAColsPerStage;
                     if (st == 0) tc_mma_block<true>(d_tmem, a_tmem, bdesc, idesc);
                     else tc_mma_block<false>(d_tmem, a_tmem, bdesc, idesc);
-                    if (kbpt - st * kSub > 1)
+                    if (kSub > 1 && kbpt - st * kSub > 1)
                         tc_mma_block<false>(d_tmem, a_tmem + kAColsPerBlock, bdesc + (kXBytes >> 4), idesc);
                     tc_commit(&sm->empty[s]);
                 }
@@ -364,8 +442,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 const int nsb = (kbpt - st * kSub) < kSub ? (kbpt - st * kSub) : kSub;
                 // the codes have landed; the producer refilled this slot only after the MMAs that
                 // read its previous contents (shared and tensor memory) had completed
-                const bool w = mbar_wait(&sm->full[s], ph, sm, P.status);
-                if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
+                if (!mbar_wait_warp(&sm->full[s], ph, abort_flag, P.status)) { ok = false; break; }
                 tc_fence_after();
                 for (int sb = 0; sb < nsb; ++sb) {
                     uint32_t wv[4];
@@ -397,9 +474,10 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         // ------------------------------------------------ epilogue
         const int q = warp & 3;
         const int ew = warp - kFirstEpiWarp;
-        long long *pix_off = sm->pix_off[ew];
+        uint32_t *pix_off = sm->pix_off[ew];
         const float alpha = P.alpha ? (float)(*P.alpha) : 1.0f;
         const int BWm = (1 << P.lgBW) - 1, BHm = (1 << P.lgBH) - 1;
+        const bool out_bf16 = P.out_dtype == TWN_BF16, res_bf16 = P.res_dtype == TWN_BF16;
         uint32_t lt = 0;
         for (int tile = blockIdx.x; tile < P.total_tiles; tile += gridDim.x, ++lt) {
             const int nt = tile % P.n_tiles;
@@ -409,59 +487,105 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
             const int tbi = pt / P.th;
             const int n = nt * kChan + q * 32 + lane;
             const bool n_ok = n < P.Cout;
-            const float sc = (P.scale && n_ok) ? __ldg(P.scale + n) : 1.0f;
+            const float sc = ((P.scale && n_ok) ? __ldg(P.scale + n) : 1.0f) * alpha;
             const float sf = (P.shift && n_ok) ? __ldg(P.shift + n) : 0.0f;
-            // output offsets of the tile's pixels (same for every channel)
+            // output offsets of the tile's pixels (the same for every channel), before the wait
 #pragma unroll
-            for (int j = 0; j < kPix / 32; ++j) {
+            for (int j = 0; j < PIX / 32; ++j) {
                 const int p = j * 32 + lane;
                 const int wv = (twi << P.lgBW) + (p & BWm);
                 const int hv = (thi << P.lgBH) + ((p >> P.lgBW) & BHm);
-                const int bv = tbi * (kPix >> (P.lgBW + P.lgBH)) + (p >> (P.lgBW + P.lgBH));
-                long long off = -1;
+                const int bv = tbi * (PIX >> (P.lgBW + P.lgBH)) + (p >> (P.lgBW + P.lgBH));
+                uint32_t off = 0xFFFFFFFFu;
                 if (wv < P.Wv && hv < P.Hv && bv < P.Bv)
-                    off = (((long long)bv * P.OH + (hv * P.osh + P.ooh)) * P.OW + (wv * P.osw + P.oow)) * P.ldy;
+                    off = (uint32_t)((((long long)bv * P.OH + (hv * P.osh + P.ooh)) * P.OW + (wv * P.osw + P.oow)) * P.ldy);
                 pix_off[p] = off;
             }
             __syncwarp();
-            const int buf = lt & 1;
-            bool w = true;
-            if (kbpt > 0) w = mbar_wait(&sm->acc_full[buf], (lt >> 1) & 1u, sm, P.status);
-            if (!__all_sync(0xffffffffu, w)) break;
+            const int buf = lt % kAccBufs;
+            if (kbpt > 0) {
+                // one thread waits for the accumulator; the four warps then decide together, so that
+                // they always execute the same number of named barriers
+                if (ew == 0 && lane == 0)
+                    sm->epi_ok = mbar_wait(&sm->acc_full[buf], (lt / kAccBufs) & 1u, abort_flag, P.status, 32) ? 1 : 0;
+                epi_bar();
+                if (!sm->epi_ok) break;
+            }
             tc_fence_after();
+            float *const y32 = reinterpret_cast<float *>(P.Y) + n;
+            __nv_bfloat16 *const y16 = reinterpret_cast<__nv_bfloat16 *>(P.Y) + n;
+            const int p_w0 = twi << P.lgBW, p_h0 = thi << P.lgBH, p_b0 = tbi * (PIX >> (P.lgBW + P.lgBH));
 #pragma unroll 1
-            for (int c = 0; c < kPix / 32; ++c) {
+            for (int c = 0; c < PIX / 32; ++c) {
+                // the 32 offsets of this chunk: eight 16-byte broadcast loads, issued before the
+                // tensor-memory load is waited for (needed for per-thread stores and for the residual)
+                uint32_t off[32];
+                if (!P.tma_store || P.residual) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const uint4 o = *reinterpret_cast<const uint4 *>(pix_off + c * 32 + i * 4);
+                        off[i * 4 + 0] = o.x; off[i * 4 + 1] = o.y; off[i * 4 + 2] = o.z; off[i * 4 + 3] = o.w;
+                    }
+                }
                 uint32_t v[32];
                 if (kbpt > 0) {
-                    tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + buf * kAccCols + c * 32, v);
+                    tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + buf * PIX + c * 32, v);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (c == PIX / 32 - 1) {
+                        // the accumulator is in registers: hand it back before the last stores
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&sm->acc_empty[buf]);
+                    }
                 } else {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
                 }
+                if (P.tma_store) {
+                    // staging buffer (c & 1) was last read by the store issued two chunks ago
+                    if (ew == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    epi_bar();
+                    const int nl = q * 32 + lane;
+                    float *const st32 = sm->stage_out[c & 1] + nl;
+                    __nv_bfloat16 *const st16 = reinterpret_cast<__nv_bfloat16 *>(sm->stage_out[c & 1]) + nl;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const long long off = pix_off[c * 32 + j];
-                    if (off < 0 || !n_ok) continue;
-                    float y = __uint_as_float(v[j]) * alpha;
-                    y = fmaf(y, sc, sf);
-                    if (P.residual) {
-                        y += P.res_dtype == TWN_BF16
-                                 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(P.residual)[off + n])
-                                 : reinterpret_cast<const float *>(P.residual)[off + n];
+                    for (int j = 0; j < 32; ++j) {
+                        float y = fmaf(__uint_as_float(v[j]), sc, sf);
+                        if (P.residual && off[j] != 0xFFFFFFFFu && n_ok) {
+                            y += res_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(P.residual)[(size_t)off[j] + n])
+                                          : reinterpret_cast<const float *>(P.residual)[(size_t)off[j] + n];
+                        }
+                        if (P.relu) y = fmaxf(y, 0.0f);
+                        if (out_bf16) st16[j * kChan] = __float2bfloat16_rn(y);
+                        else st32[j * kChan] = y;
                     }
-                    if (P.relu) y = fmaxf(y, 0.0f);
-                    if (P.out_dtype == TWN_BF16) reinterpret_cast<__nv_bfloat16 *>(P.Y)[off + n] = __float2bfloat16_rn(y);
-                    else reinterpret_cast<float *>(P.Y)[off + n] = y;
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    epi_bar();
+                    if (ew == 0 && lane == 0) {
+                        const int p0 = c * 32;
+                        tma_store_4d(&map_y, sm->stage_out[c & 1], nt * kChan, p_w0 + (p0 & BWm),
+                                     p_h0 + ((p0 >> P.lgBW) & BHm), p_b0 + (p0 >> (P.lgBW + P.lgBH)));
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        if (off[j] != 0xFFFFFFFFu && n_ok) {
+                            float y = fmaf(__uint_as_float(v[j]), sc, sf);
+                            if (P.residual) {
+                                y += res_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(P.residual)[(size_t)off[j] + n])
+                                              : reinterpret_cast<const float *>(P.residual)[(size_t)off[j] + n];
+                            }
+                            if (P.relu) y = fmaxf(y, 0.0f);
+                            if (out_bf16) y16[off[j]] = __float2bfloat16_rn(y);
+                            else y32[off[j]] = y;
+                        }
+                    }
                 }
-            }
-            if (kbpt > 0) {
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sm->acc_empty[buf]);
             }
             __syncwarp();
         }
+        // all bulk stores of this thread have been written before the block may exit
+        if (P.tma_store && ew == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 
     // ---------------------------------------------------- teardown
@@ -512,20 +636,93 @@ struct Geometry {
     long long Cin;   // channels per tap
 };
 
-// Picks the pixel-tile shape (powers of two, product kPix) that wastes the fewest pixels.
-void pick_tile(const Geometry &g, int *lgBW, int *lgBH)
+// Picks the pixel-tile shape (powers of two, product `pix`) that needs the fewest tiles.
+long long pick_tile(const Geometry &g, int pix, int *lgBW, int *lgBH)
 {
+    int lg = 0;
+    while ((1 << lg) < pix) ++lg;
     long long best = -1;
     int bw = 0, bh = 0;
-    for (int a = 0; a <= 7; ++a)
-        for (int b = 0; a + b <= 7; ++b) {
-            const int BW = 1 << a, BH = 1 << b, BB = kPix >> (a + b);
-            if (BW * g.sw > 256 || BH * g.sh > 256) continue;
+    for (int a = 0; a <= lg; ++a)
+        for (int b = 0; a + b <= lg; ++b) {
+            const int BW = 1 << a, BH = 1 << b, BB = pix >> (a + b);
+            if (BW * g.sw > 256 || BH * g.sh > 256 || BB > 256) continue;
             const long long tiles = ((g.Wv + BW - 1) / BW) * (long long)((g.Hv + BH - 1) / BH) * ((g.Bv + BB - 1) / BB);
             // prefer fewer tiles, then wider rows
             if (best < 0 || tiles < best || (tiles == best && a > bw)) { best = tiles; bw = a; bh = b; }
         }
     *lgBW = bw; *lgBH = bh;
+    return best;
+}
+
+template <int PIX>
+int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const uint32_t *T, const twn_device_info &dev,
+                  EncodeTiledFn enc, cudaStream_t s)
+{
+    static bool attr_set[64] = {false};
+    const int smem_bytes = (int)sizeof(SmemLayout<PIX>) + 1024;
+    if (!attr_set[dev.ordinal]) {
+        TWN_CUDA_OK(cudaFuncSetAttribute(tconv_kernel<PIX>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
+        attr_set[dev.ordinal] = true;
+    }
+    pick_tile(g, PIX, &P.lgBW, &P.lgBH);
+    const int BW = 1 << P.lgBW, BH = 1 << P.lgBH, BB = PIX >> (P.lgBW + P.lgBH);
+    P.tw = (g.Wv + BW - 1) / BW;
+    P.th = (g.Hv + BH - 1) / BH;
+    P.tb = (g.Bv + BB - 1) / BB;
+    const long long total = (long long)P.n_tiles * P.tw * P.th * P.tb;
+    if (total <= 0 || total > 0x7fffffffLL) return TWN_ERR_INVALID_ARG;
+    P.total_tiles = (int)total;
+
+    // activations: (C, W, H, B), 64-channel boxes with 128-byte swizzle, zero fill outside
+    CUtensorMap map_x, map_t;
+    {
+        cuuint64_t dims[4] = {(cuuint64_t)g.XC, (cuuint64_t)g.XW, (cuuint64_t)g.XH, (cuuint64_t)g.XB};
+        cuuint64_t strides[3] = {(cuuint64_t)g.ldx * 2, (cuuint64_t)g.XW * g.ldx * 2, (cuuint64_t)g.XH * g.XW * g.ldx * 2};
+        // with a traversal stride the box counts traversed elements: N loaded elements need N * stride
+        cuuint32_t box[4] = {(cuuint32_t)kBlockK, (cuuint32_t)(BW * g.sw), (cuuint32_t)(BH * g.sh), (cuuint32_t)BB};
+        cuuint32_t estr[4] = {1, (cuuint32_t)g.sw, (cuuint32_t)g.sh, 1};
+        if (enc(&map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(X), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return TWN_ERR_INVALID_ARG;
+    }
+    // packed codes: (words, rows), boxes of 4 or 8 words x 128 rows, zero fill outside
+    {
+        cuuint64_t dims[2] = {(cuuint64_t)(g.ld_codes / 16), (cuuint64_t)g.Cout};
+        cuuint64_t strides[1] = {(cuuint64_t)(g.ld_codes / 4)};
+        cuuint32_t box[2] = {(cuuint32_t)P.code_row_words, (cuuint32_t)kChan};
+        cuuint32_t estr[2] = {1, 1};
+        if (enc(&map_t, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t *>(T), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return TWN_ERR_INVALID_ARG;
+    }
+    // output: TMA stores when the tile is a plain box of the output tensor and the pitch allows it
+    CUtensorMap map_y = map_t;
+    const int es = P.out_dtype == TWN_BF16 ? 2 : 4;
+    P.tma_store = 0;
+    // (the channel extent must be a whole number of 16-byte units: the store clips at that granularity)
+    if (g.osh == 1 && g.osw == 1 && g.ooh == 0 && g.oow == 0 && (g.ldy * es) % 16 == 0 &&
+        ((long long)g.Cout * es) % 16 == 0 && (reinterpret_cast<uintptr_t>(P.Y) % 16) == 0) {
+        // a chunk of 32 consecutive tile pixels is a sub-box sbw x sbh x sbb of the tile box
+        const int lg_sbw = P.lgBW < 5 ? P.lgBW : 5;
+        const int lg_sbh = P.lgBH < 5 - lg_sbw ? P.lgBH : 5 - lg_sbw;
+        const int lg_sbb = 5 - lg_sbw - lg_sbh;
+        P.lg_sbw = lg_sbw; P.lg_sbh = lg_sbh;
+        cuuint64_t dims[4] = {(cuuint64_t)g.Cout, (cuuint64_t)g.OW, (cuuint64_t)g.OH, (cuuint64_t)g.Bv};
+        cuuint64_t strides[3] = {(cuuint64_t)g.ldy * es, (cuuint64_t)g.OW * g.ldy * es, (cuuint64_t)g.OH * g.OW * g.ldy * es};
+        cuuint32_t box[4] = {(cuuint32_t)kChan, 1u << lg_sbw, 1u << lg_sbh, 1u << lg_sbb};
+        cuuint32_t estr[4] = {1, 1, 1, 1};
+        if (enc(&map_y, es == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, P.Y, dims,
+                strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
+            P.tma_store = 1;
+    }
+    const int grid = dev.sm_count < P.total_tiles ? dev.sm_count : P.total_tiles;
+    tconv_kernel<PIX><<<grid, kThreadsConv, smem_bytes, s>>>(map_x, map_t, map_y, P);
+    TWN_CUDA_OK(cudaGetLastError());
+    return TWN_OK;
 }
 
 int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_stats_t *stats,
@@ -537,24 +734,11 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     EncodeTiledFn enc = encode_fn();
     if (!enc) return TWN_ERR_CUDA;
 
-    static bool attr_set[64] = {false};
-    const int smem_bytes = (int)sizeof(SmemLayout) + 1024;
-    if (!attr_set[dev.ordinal]) {
-        TWN_CUDA_OK(cudaFuncSetAttribute(tconv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
-        attr_set[dev.ordinal] = true;
-    }
-
+    // the epilogue keeps output offsets in 32 bits
+    if ((long long)g.Bv * g.OH * g.OW * g.ldy >= 0xFFFFFFFFLL) return TWN_ERR_INVALID_ARG;
     ConvParams P;
     memset(&P, 0, sizeof P);
-    pick_tile(g, &P.lgBW, &P.lgBH);
-    const int BW = 1 << P.lgBW, BH = 1 << P.lgBH, BB = kPix >> (P.lgBW + P.lgBH);
     P.n_tiles = (g.Cout + kChan - 1) / kChan;
-    P.tw = (g.Wv + BW - 1) / BW;
-    P.th = (g.Hv + BH - 1) / BH;
-    P.tb = (g.Bv + BB - 1) / BB;
-    const long long total = (long long)P.n_tiles * P.tw * P.th * P.tb;
-    if (total <= 0 || total > 0x7fffffffLL) return TWN_ERR_INVALID_ARG;
-    P.total_tiles = (int)total;
     P.n_taps = g.n_taps;
     P.n_cblk = (int)((g.Cin + kBlockK - 1) / kBlockK);
     P.code_row_words = 4;
@@ -576,34 +760,11 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     P.status = dev_status;
     for (int t = 0; t < g.n_taps; ++t) P.taps[t] = g.taps[t];
 
-    // activations: (C, W, H, B), 64-channel boxes with 128-byte swizzle, zero fill outside
-    CUtensorMap map_x, map_t;
-    {
-        cuuint64_t dims[4] = {(cuuint64_t)g.XC, (cuuint64_t)g.XW, (cuuint64_t)g.XH, (cuuint64_t)g.XB};
-        cuuint64_t strides[3] = {(cuuint64_t)g.ldx * 2, (cuuint64_t)g.XW * g.ldx * 2, (cuuint64_t)g.XH * g.XW * g.ldx * 2};
-        cuuint32_t box[4] = {(cuuint32_t)kBlockK, (cuuint32_t)(BW * g.sw), (cuuint32_t)(BH * g.sh), (cuuint32_t)BB};
-        // with a traversal stride the box counts traversed elements: N loaded elements need N * stride
-        cuuint32_t estr[4] = {1, (cuuint32_t)g.sw, (cuuint32_t)g.sh, 1};
-        if (enc(&map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(X), dims, strides, box, estr,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return TWN_ERR_INVALID_ARG;
-    }
-    // packed codes: (words, rows), boxes of 8 words x 128 rows, zero fill outside
-    {
-        cuuint64_t dims[2] = {(cuuint64_t)(g.ld_codes / 16), (cuuint64_t)g.Cout};
-        cuuint64_t strides[1] = {(cuuint64_t)(g.ld_codes / 4)};
-        cuuint32_t box[2] = {(cuuint32_t)P.code_row_words, (cuuint32_t)kChan};
-        cuuint32_t estr[2] = {1, 1};
-        if (enc(&map_t, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t *>(T), dims, strides, box, estr,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return TWN_ERR_INVALID_ARG;
-    }
-    int grid = dev.sm_count < P.total_tiles ? dev.sm_count : P.total_tiles;
-    tconv_kernel<<<grid, kThreadsConv, smem_bytes, s>>>(map_x, map_t, P);
-    TWN_CUDA_OK(cudaGetLastError());
-    return TWN_OK;
+    // 256-pixel tiles once they still fill the machine; otherwise 128-pixel tiles
+    int a, b;
+    const long long tiles256 = pick_tile(g, 256, &a, &b) * P.n_tiles;
+    if (tiles256 >= dev.sm_count) return launch_conv_t<256>(g, P, X, T, dev, enc, s);
+    return launch_conv_t<128>(g, P, X, T, dev, enc, s);
 }
 
 int check_epilogue(const twn_epilogue_t *e)

@@ -43,6 +43,8 @@ def assert_within(y, y_ref, A, alpha, scale=None):
 GEMM_SHAPES = [
     (128, 128, 64), (1, 1, 8), (7, 3, 16), (100, 10, 512), (129, 257, 200), (300, 200, 136),
     (128, 512, 1024), (1000, 130, 72), (64, 1000, 512), (128, 1024, 8192), (515, 64, 576),
+    # enough tiles for the 256-pixel kernel, with ragged edges in both dimensions
+    (8192, 640, 512), (40000, 130, 200), (20001, 257, 1152),
 ]
 
 
@@ -131,6 +133,10 @@ CONV_CASES = [
     (1, 33, 20, 80, 130, 3, 1, 1),
     (2, 10, 10, 48, 16, 3, 1, 0),
     (1, 15, 15, 16, 32, 7, 2, 3),
+    # enough pixels for the 256-pixel kernel
+    (8, 64, 64, 64, 256, 3, 1, 1),
+    (37, 28, 28, 128, 256, 3, 2, 1),
+    (64, 14, 14, 64, 384, 3, 1, 1),
 ]
 
 
