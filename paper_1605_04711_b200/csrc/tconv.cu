@@ -16,9 +16,9 @@
 // owns one channel, so alpha, the per-channel affine and ReLU cost one register each,
 // and a warp's store of one pixel covers 32 consecutive channels (128 contiguous bytes).
 //
-//   warp 0        TMA producer: X tile and packed-code tile per k-block
+//   warp 0        TMA producer: activation tile per k-block
 //   warp 1        allocates tensor memory, issues tcgen05.mma, commits to mbarriers
-//   warps 2-9     decode: packed codes (smem) -> bf16 pairs -> tensor memory
+//   warps 2-9     decode: packed codes (global, L2) -> bf16 pairs -> tensor memory
 //   warps 10-13   epilogue: tensor memory -> registers -> global
 //
 // Two tile shapes.  Measured on B200: one thread can issue a tcgen05.mma about every
@@ -42,8 +42,6 @@ namespace {
 
 constexpr int kChan = 128;          // output channels per tile (UMMA M)
 constexpr int kBlockK = 64;         // reduction elements per k-block (128 bytes of bf16)
-constexpr int kCodeRowBytesMax = 32;           // up to 8 words per channel row per k-block (4 used)
-constexpr int kCodeBytes = kChan * kCodeRowBytesMax;  // 4 KB
 constexpr int kDecodeSets = 2;      // groups of 4 decode warps; a group takes every other stage
 constexpr int kFirstEpiWarp = 2 + 4 * kDecodeSets;
 constexpr int kThreadsConv = 32 * (kFirstEpiWarp + 4);
@@ -75,8 +73,9 @@ struct ConvParams {
     int lgBW, lgBH;               // pixel tile = BB x BH x BW, powers of two, product PIX
     // reduction
     int n_taps, n_cblk;           // k-blocks per tile = n_taps * n_cblk
-    int code_row_words;           // words per channel row in a staged code tile: 4 (every k-block
-                                  // starts on a 16-byte boundary of the packed row) or 8
+    int codes_aligned;            // 1: every k-block starts on a 16-byte boundary of the packed row
+    const uint32_t *T;            // packed codes, one row of `wpr` words per output channel
+    long long wpr;
     int sw, sh;                   // input pixel = output pixel * (sh, sw) + (dh, dw)
     // virtual output grid and its embedding in the output tensor
     int Bv, Hv, Wv;
@@ -101,10 +100,9 @@ struct __align__(1024) SmemLayout {
     static constexpr int kStages = Cfg<PIX>::kStages, kSub = Cfg<PIX>::kSub;
     static constexpr int kXBytes = PIX * kBlockK * 2;
     uint8_t x[kStages][kSub][kXBytes];           // swizzled activation tiles
-    uint8_t codes[kStages][kSub][kCodeBytes];    // packed code tiles, row = channel
-    unsigned long long full[kStages];      // TMA -> decode
-    unsigned long long ready_a[kStages];   // decode -> MMA (implies full: the decode warps saw it)
-    unsigned long long empty[kStages];     // MMA commit -> TMA
+    unsigned long long full[kStages];      // TMA -> MMA: activation tile landed
+    unsigned long long ready_a[kStages];   // decode -> MMA: weights of the stage are in tensor memory
+    unsigned long long empty[kStages];     // MMA commit -> TMA and decode: both operand slots are free
     unsigned long long acc_full[2];        // MMA commit -> epilogue
     unsigned long long acc_empty[2];       // epilogue -> MMA
     alignas(16) uint32_t pix_off[4][PIX];  // per epilogue warp: output element offset of a pixel, ~0 = skip
@@ -188,13 +186,6 @@ __device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, v
     asm volatile(
         "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-        : "memory");
-}
-__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, void *bar, int c0, int c1)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
         : "memory");
 }
 
@@ -312,14 +303,13 @@ __device__ __forceinline__ uint32_t fields_to_bf16x2(uint32_t x)
 
 // ---------------------------------------------------------------- the kernel
 static_assert(offsetof(SmemLayout<128>, stage_out) % 128 == 0 && offsetof(SmemLayout<256>, stage_out) % 128 == 0 &&
-                  offsetof(SmemLayout<128>, pix_off) % 16 == 0 && offsetof(SmemLayout<256>, pix_off) % 16 == 0 &&
-                  offsetof(SmemLayout<128>, codes) % 128 == 0 && offsetof(SmemLayout<256>, codes) % 128 == 0,
+                  offsetof(SmemLayout<128>, pix_off) % 16 == 0 && offsetof(SmemLayout<256>, pix_off) % 16 == 0,
               "TMA and vector accesses need aligned shared-memory regions");
 
 template <int PIX>
 __global__ void __launch_bounds__(kThreadsConv, 1)
-tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_t,
-             const __grid_constant__ CUtensorMap map_y, const __grid_constant__ ConvParams P)
+tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
+             const __grid_constant__ ConvParams P)
 {
     using L = SmemLayout<PIX>;
     constexpr int kStages = Cfg<PIX>::kStages, kSub = Cfg<PIX>::kSub, kAccBufs = Cfg<PIX>::kAccBufs;
@@ -365,9 +355,8 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            const uint32_t block_bytes = kXBytes + kChan * 4 * P.code_row_words;
+            const uint32_t block_bytes = kXBytes;
             for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
-                const int nt = tile % P.n_tiles;
                 int pt = tile / P.n_tiles;
                 const int twi = pt % P.tw; pt /= P.tw;
                 const int thi = pt % P.th;
@@ -385,9 +374,6 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     for (int sb = 0; sb < nsb; ++sb) {
                         const Tap tap = P.taps[t];
                         tma_load_4d(sm->x[s][sb], &map_x, &sm->full[s], cb * kBlockK, w0 + tap.dw, h0 + tap.dh, b0);
-                        const int word = (tap.koff >> 4) + cb * (kBlockK / 16);
-                        // word % 4 == 0 whenever code_row_words == 4
-                        tma_load_2d(sm->codes[s][sb], &map_t, &sm->full[s], word & ~3, nt * kChan);
                         if (++cb == P.n_cblk) { cb = 0; ++t; }
                     }
                 }
@@ -411,7 +397,8 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 for (int st = 0; st < spt; ++st, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
-                    if (!mbar_wait_warp(&sm->ready_a[s], ph, abort_flag, P.status, 0)) { ok = false; break; }
+                    if (!mbar_wait_warp(&sm->ready_a[s], ph, abort_flag, P.status, 0) ||
+                        !mbar_wait_warp(&sm->full[s], ph, abort_flag, P.status, 0)) { ok = false; break; }
                     tc_fence_after();
                     const uint64_t bdesc = bdesc0 + (uint64_t)(s * ((kSub * kXBytes) >> 4));
                     const uint32_t a_tmem = tmem_a + s * kAColsPerStage;
@@ -426,48 +413,83 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         }
     } else if (warp < kFirstEpiWarp) {
         // ------------------------------------------------ decode: codes -> bf16 -> tensor memory
-        // Two groups of four warps; a group handles every other stage, so the latency of the
-        // tensor-memory store of one stage overlaps the decoding of the next by the other group.
+        // Two groups of four warps; a group handles every other stage.  Each thread owns one
+        // channel row: it reads the row's 16 bytes of codes per k-block straight from global
+        // memory (L2-resident, fetched two of its stages ahead), so decoding depends only on a
+        // free tensor-memory slot, not on the activation pipeline.
         const int q = warp & 3;                 // tensor-memory lane quadrant of this warp
         const int set = (warp - 2) >> 2;
         const int row = q * 32 + lane;          // channel row inside the tile
         const uint32_t lane_base = tmem_a + ((uint32_t)(q * 32) << 16);
-        uint32_t it = 0;
-        bool ok = true;
-        for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
-            for (int st = 0; st < spt; ++st, ++it) {
-                if ((int)(it % kDecodeSets) != set) continue;
+
+        struct Codes { uint4 v[kSub]; };
+        auto fetch = [&](int tile, int st) -> Codes {
+            Codes c;
+#pragma unroll
+            for (int sb = 0; sb < kSub; ++sb) c.v[sb] = make_uint4(0u, 0u, 0u, 0u);
+            if (tile >= P.total_tiles) return c;
+            const long long n = (long long)(tile % P.n_tiles) * kChan + row;
+            if (n >= P.Cout) return c;
+            const uint32_t *rowp = P.T + n * P.wpr;
+#pragma unroll
+            for (int sb = 0; sb < kSub; ++sb) {
+                const int u = st * kSub + sb;
+                if (u >= kbpt) break;
+                const int t = u / P.n_cblk, cb = u - t * P.n_cblk;
+                const long long word = (P.taps[t].koff >> 4) + cb * (kBlockK / 16);
+                if (P.codes_aligned) {
+                    c.v[sb] = __ldg(reinterpret_cast<const uint4 *>(rowp + word));
+                } else {
+                    uint32_t w4[4];
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) w4[g] = (word + g < P.wpr) ? __ldg(rowp + word + g) : 0u;
+                    c.v[sb] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                }
+            }
+            return c;
+        };
+        // position of this group's next stages: (tile, st), advanced kDecodeSets stages at a time
+        auto advance = [&](int &tile, int &st, int steps) {
+            for (int i = 0; i < steps; ++i)
+                if (++st >= spt) { st = 0; tile += gridDim.x; }
+        };
+        if (spt > 0) {
+            int tile0 = blockIdx.x, st0 = 0;
+            advance(tile0, st0, set);                       // this group's first stage
+            int tile1 = tile0, st1 = st0;
+            advance(tile1, st1, kDecodeSets);
+            int tile2 = tile1, st2 = st1;
+            advance(tile2, st2, kDecodeSets);
+            Codes cur = fetch(tile0, st0), nxt = fetch(tile1, st1);
+            uint32_t it = set;
+            while (tile0 < P.total_tiles) {
+                const Codes nn = fetch(tile2, st2);         // two stages ahead
                 const int s = it % kStages;
                 const uint32_t ph = (it / kStages) & 1u;
-                const int nsb = (kbpt - st * kSub) < kSub ? (kbpt - st * kSub) : kSub;
-                // the codes have landed; the producer refilled this slot only after the MMAs that
-                // read its previous contents (shared and tensor memory) had completed
-                if (!mbar_wait_warp(&sm->full[s], ph, abort_flag, P.status)) { ok = false; break; }
+                const int nsb = (kbpt - st0 * kSub) < kSub ? (kbpt - st0 * kSub) : kSub;
+                // the MMAs that read this slot's previous contents have completed
+                if (!mbar_wait_warp(&sm->empty[s], ph ^ 1u, abort_flag, P.status, 32)) break;
                 tc_fence_after();
-                for (int sb = 0; sb < nsb; ++sb) {
-                    uint32_t wv[4];
-                    if (P.code_row_words == 4) {
-                        const uint4 v = *reinterpret_cast<const uint4 *>(sm->codes[s][sb] + row * 16);
-                        wv[0] = v.x; wv[1] = v.y; wv[2] = v.z; wv[3] = v.w;
-                    } else {
-                        const int u = st * kSub + sb;
-                        const int t = u / P.n_cblk, cb = u - t * P.n_cblk;
-                        const int word = (P.taps[t].koff >> 4) + cb * (kBlockK / 16);
-                        const uint32_t *src = reinterpret_cast<const uint32_t *>(sm->codes[s][sb] + row * 32) + (word & 3);
 #pragma unroll
-                        for (int g = 0; g < 4; ++g) wv[g] = src[g];
+                for (int sb = 0; sb < kSub; ++sb) {
+                    if (sb < nsb) {
+                        const uint32_t wv[4] = {cur.v[sb].x, cur.v[sb].y, cur.v[sb].z, cur.v[sb].w};
+                        uint32_t out[32];
+#pragma unroll
+                        for (int g = 0; g < 4; ++g)
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) out[g * 8 + e] = fields_to_bf16x2(wv[g] >> (2 * e));
+                        tmem_st32(lane_base + s * kAColsPerStage + sb * kAColsPerBlock, out);
                     }
-                    uint32_t out[32];
-#pragma unroll
-                    for (int g = 0; g < 4; ++g)
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) out[g * 8 + e] = fields_to_bf16x2(wv[g] >> (2 * e));
-                    tmem_st32(lane_base + s * kAColsPerStage + sb * kAColsPerBlock, out);
                 }
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sm->ready_a[s]);
+                cur = nxt; nxt = nn;
+                tile0 = tile1; st0 = st1; tile1 = tile2; st1 = st2;
+                advance(tile2, st2, kDecodeSets);
+                it += kDecodeSets;
             }
         }
     } else {
@@ -541,23 +563,36 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
                 }
+                // The inner loops are kept free of conditionals: one warp per scheduler runs this
+                // code, so every instruction fetched and issued here is exposed latency.
+                const float floor_v = P.relu ? 0.0f : -INFINITY;
+                if (P.residual) {
+                    // y = acc * scale' + shift + residual (residual fetched with the per-pixel offsets)
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        float r = 0.0f;
+                        if (off[j] != 0xFFFFFFFFu && n_ok)
+                            r = res_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(P.residual)[(size_t)off[j] + n])
+                                         : reinterpret_cast<const float *>(P.residual)[(size_t)off[j] + n];
+                        v[j] = __float_as_uint(fmaxf(fmaf(__uint_as_float(v[j]), sc, sf) + r, floor_v));
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(fmaxf(fmaf(__uint_as_float(v[j]), sc, sf), floor_v));
+                }
                 if (P.tma_store) {
                     // staging buffer (c & 1) was last read by the store issued two chunks ago
                     if (ew == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                     epi_bar();
                     const int nl = q * 32 + lane;
-                    float *const st32 = sm->stage_out[c & 1] + nl;
-                    __nv_bfloat16 *const st16 = reinterpret_cast<__nv_bfloat16 *>(sm->stage_out[c & 1]) + nl;
+                    if (out_bf16) {
+                        __nv_bfloat16 *const st16 = reinterpret_cast<__nv_bfloat16 *>(sm->stage_out[c & 1]) + nl;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        float y = fmaf(__uint_as_float(v[j]), sc, sf);
-                        if (P.residual && off[j] != 0xFFFFFFFFu && n_ok) {
-                            y += res_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(P.residual)[(size_t)off[j] + n])
-                                          : reinterpret_cast<const float *>(P.residual)[(size_t)off[j] + n];
-                        }
-                        if (P.relu) y = fmaxf(y, 0.0f);
-                        if (out_bf16) st16[j * kChan] = __float2bfloat16_rn(y);
-                        else st32[j * kChan] = y;
+                        for (int j = 0; j < 32; ++j) st16[j * kChan] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                    } else {
+                        uint32_t *const st32 = reinterpret_cast<uint32_t *>(sm->stage_out[c & 1]) + nl;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) st32[j * kChan] = v[j];
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     epi_bar();
@@ -566,19 +601,15 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                         tma_store_4d(&map_y, sm->stage_out[c & 1], nt * kChan, p_w0 + (p0 & BWm),
                                      p_h0 + ((p0 >> P.lgBW) & BHm), p_b0 + (p0 >> (P.lgBW + P.lgBH)));
                     }
-                } else {
+                } else if (n_ok) {
+                    if (out_bf16) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        if (off[j] != 0xFFFFFFFFu && n_ok) {
-                            float y = fmaf(__uint_as_float(v[j]), sc, sf);
-                            if (P.residual) {
-                                y += res_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(P.residual)[(size_t)off[j] + n])
-                                              : reinterpret_cast<const float *>(P.residual)[(size_t)off[j] + n];
-                            }
-                            if (P.relu) y = fmaxf(y, 0.0f);
-                            if (out_bf16) y16[off[j]] = __float2bfloat16_rn(y);
-                            else y32[off[j]] = y;
-                        }
+                        for (int j = 0; j < 32; ++j)
+                            if (off[j] != 0xFFFFFFFFu) y16[off[j]] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (off[j] != 0xFFFFFFFFu) y32[off[j]] = __uint_as_float(v[j]);
                     }
                 }
             }
@@ -656,7 +687,7 @@ long long pick_tile(const Geometry &g, int pix, int *lgBW, int *lgBH)
 }
 
 template <int PIX>
-int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const uint32_t *T, const twn_device_info &dev,
+int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const twn_device_info &dev,
                   EncodeTiledFn enc, cudaStream_t s)
 {
     static bool attr_set[64] = {false};
@@ -675,7 +706,7 @@ int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const uint32_
     P.total_tiles = (int)total;
 
     // activations: (C, W, H, B), 64-channel boxes with 128-byte swizzle, zero fill outside
-    CUtensorMap map_x, map_t;
+    CUtensorMap map_x;
     {
         cuuint64_t dims[4] = {(cuuint64_t)g.XC, (cuuint64_t)g.XW, (cuuint64_t)g.XH, (cuuint64_t)g.XB};
         cuuint64_t strides[3] = {(cuuint64_t)g.ldx * 2, (cuuint64_t)g.XW * g.ldx * 2, (cuuint64_t)g.XH * g.XW * g.ldx * 2};
@@ -687,19 +718,8 @@ int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const uint32_
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return TWN_ERR_INVALID_ARG;
     }
-    // packed codes: (words, rows), boxes of 4 or 8 words x 128 rows, zero fill outside
-    {
-        cuuint64_t dims[2] = {(cuuint64_t)(g.ld_codes / 16), (cuuint64_t)g.Cout};
-        cuuint64_t strides[1] = {(cuuint64_t)(g.ld_codes / 4)};
-        cuuint32_t box[2] = {(cuuint32_t)P.code_row_words, (cuuint32_t)kChan};
-        cuuint32_t estr[2] = {1, 1};
-        if (enc(&map_t, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t *>(T), dims, strides, box, estr,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return TWN_ERR_INVALID_ARG;
-    }
     // output: TMA stores when the tile is a plain box of the output tensor and the pitch allows it
-    CUtensorMap map_y = map_t;
+    CUtensorMap map_y = map_x;
     const int es = P.out_dtype == TWN_BF16 ? 2 : 4;
     P.tma_store = 0;
     // (the channel extent must be a whole number of 16-byte units: the store clips at that granularity)
@@ -720,7 +740,7 @@ int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const uint32_
             P.tma_store = 1;
     }
     const int grid = dev.sm_count < P.total_tiles ? dev.sm_count : P.total_tiles;
-    tconv_kernel<PIX><<<grid, kThreadsConv, smem_bytes, s>>>(map_x, map_t, map_y, P);
+    tconv_kernel<PIX><<<grid, kThreadsConv, smem_bytes, s>>>(map_x, map_y, P);
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }
@@ -741,9 +761,11 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     P.n_tiles = (g.Cout + kChan - 1) / kChan;
     P.n_taps = g.n_taps;
     P.n_cblk = (int)((g.Cin + kBlockK - 1) / kBlockK);
-    P.code_row_words = 4;
+    P.codes_aligned = 1;
     for (int t = 0; t < g.n_taps; ++t)
-        if (g.taps[t].koff % kBlockK != 0) P.code_row_words = 8;
+        if (g.taps[t].koff % kBlockK != 0) P.codes_aligned = 0;
+    P.T = T;
+    P.wpr = g.ld_codes / 16;
     P.sw = g.sw; P.sh = g.sh;
     P.Bv = g.Bv; P.Hv = g.Hv; P.Wv = g.Wv;
     P.OH = g.OH; P.OW = g.OW; P.osh = g.osh; P.osw = g.osw; P.ooh = g.ooh; P.oow = g.oow;
@@ -763,8 +785,8 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     // 256-pixel tiles once they still fill the machine; otherwise 128-pixel tiles
     int a, b;
     const long long tiles256 = pick_tile(g, 256, &a, &b) * P.n_tiles;
-    if (tiles256 >= dev.sm_count) return launch_conv_t<256>(g, P, X, T, dev, enc, s);
-    return launch_conv_t<128>(g, P, X, T, dev, enc, s);
+    if (tiles256 >= dev.sm_count) return launch_conv_t<256>(g, P, X, dev, enc, s);
+    return launch_conv_t<128>(g, P, X, dev, enc, s);
 }
 
 int check_epilogue(const twn_epilogue_t *e)
