@@ -44,7 +44,8 @@ typedef enum {
     TWN_ERR_TIMEOUT = -5,     /* device: a bounded wait inside a kernel ran out    */
     TWN_ERR_CUDA = -6,        /* a CUDA runtime / driver call failed               */
     TWN_ERR_UNSUPPORTED_ARCH = -7,
-    TWN_ERR_BAD_CODE = -8     /* device: an int8 code outside {-1,0,+1}            */
+    TWN_ERR_BAD_CODE = -8,    /* device: an int8 code outside {-1,0,+1}            */
+    TWN_ERR_TOO_LARGE = -9    /* a size beyond what a fixed-capacity entry point takes */
 } twn_status;
 
 enum { TWN_F32 = 0, TWN_BF16 = 1 };
@@ -128,6 +129,38 @@ int twn_ternarize(const float *W, int64_t rows, int64_t cols, double delta_facto
                   twn_stats_t *stats, uint32_t *packed, int64_t ld_codes,
                   int8_t *codes_i8, void *workspace, size_t workspace_bytes,
                   twn_stream_t stream);
+
+/*
+ * twn_ternarize for callers that may not allocate.  (The paper has no counterpart;
+ * this is a packaging variant of the call above, same arithmetic, same results.)
+ *
+ * Some hosts of this library cannot obtain device memory for the scratch buffer
+ * twn_ternarize asks for: code that runs inside another framework's memory plan
+ * and is handed exactly its input and output tensors, plugins loaded by a serving
+ * process whose allocator is frozen once the model is up, and callers on a path
+ * where cudaMalloc's implicit device synchronisation is not acceptable.  For them
+ * the scratch lives inside the library: a static device array of
+ * TWN_TERNARIZE_STATIC_SCRATCH_BYTES that every GPU which loads the library holds
+ * until the process exits.  This call allocates and frees nothing, on the host or
+ * on the device, and calls no routine that does.
+ *
+ * Arguments and results are those of twn_ternarize without workspace/workspace_bytes.
+ * Limits and rules:
+ *   - rows*cols may not exceed TWN_TERNARIZE_STATIC_MAX_WEIGHTS; a larger tensor is
+ *     refused with TWN_ERR_TOO_LARGE before anything is launched.
+ *   - The first call on each device looks up the array's device address (once per
+ *     device, with that device current).  Make that first call outside any stream
+ *     capture.
+ *   - All calls share the one array.  It keeps whatever the previous call left; the
+ *     words that must start at zero are cleared on `stream` at the start of every
+ *     call.  Two calls whose kernels can overlap on the GPU (different streams,
+ *     no dependency between them) race on it and give wrong results: order them.
+ */
+#define TWN_TERNARIZE_STATIC_SCRATCH_BYTES 65792u
+#define TWN_TERNARIZE_STATIC_MAX_WEIGHTS 2147483648LL /* 2^31 weights = 8 GiB of fp32 */
+int twn_ternarize_static(const float *W, int64_t rows, int64_t cols, double delta_factor,
+                         twn_stats_t *stats, uint32_t *packed, int64_t ld_codes,
+                         int8_t *codes_i8, twn_stream_t stream);
 
 /* ---- 2-bit storage (Sec. 2.1, model compression) ------------------------- */
 

@@ -34,6 +34,7 @@ extern "C" const char *twn_strerror(int status)
         case TWN_ERR_CUDA: return "a CUDA call failed";
         case TWN_ERR_UNSUPPORTED_ARCH: return "the current device is not sm_100";
         case TWN_ERR_BAD_CODE: return "a ternary code outside {-1,0,+1}";
+        case TWN_ERR_TOO_LARGE: return "size beyond the fixed capacity of this entry point";
         default: return "unknown status";
     }
 }

@@ -486,6 +486,68 @@ extern "C" int twn_ternarize(const float *W, int64_t rows, int64_t cols, double 
     return TWN_OK;
 }
 
+// ---- the variant that allocates nothing ------------------------------------------------
+// Scratch for twn_ternarize_static: tickets and per-block partials, same layout as a caller's
+// workspace.  File-scope device storage, one copy per GPU that loads the library.  In host
+// code the name `g_static_scratch` is only a handle for cudaGetSymbolAddress, never a pointer
+// a kernel may be given.
+static __device__ __align__(256) unsigned char g_static_scratch[TWN_TERNARIZE_STATIC_SCRATCH_BYTES];
+static_assert(TWN_TERNARIZE_STATIC_SCRATCH_BYTES >= kWorkspaceBytes, "static scratch too small");
+
+// Device address of g_static_scratch on the current device, looked up once per device.
+static int static_scratch_ptr(int ordinal, void **out)
+{
+    static void *cached[64] = {nullptr};
+    if (ordinal < 0 || ordinal >= 64) return TWN_ERR_CUDA;
+    if (cached[ordinal] == nullptr) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return TWN_ERR_CUDA;
+        cached[ordinal] = p;
+    }
+    *out = cached[ordinal];
+    return TWN_OK;
+}
+
+extern "C" int twn_ternarize_static(const float *W, int64_t rows, int64_t cols, double delta_factor,
+                                    twn_stats_t *stats, uint32_t *packed, int64_t ld_codes,
+                                    int8_t *codes_i8, twn_stream_t stream)
+{
+    TWN_REQUIRE(rows >= 0 && cols >= 0, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(stats != nullptr, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(delta_factor >= 0.0 && delta_factor == delta_factor, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(ld_codes >= cols && ld_codes % 64 == 0, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(cols == 0 || rows <= TWN_TERNARIZE_STATIC_MAX_WEIGHTS / cols, TWN_ERR_TOO_LARGE);
+    const long long n = (long long)rows * cols;
+    TWN_REQUIRE(n <= TWN_TERNARIZE_STATIC_MAX_WEIGHTS, TWN_ERR_TOO_LARGE);
+    TWN_REQUIRE(n == 0 || (W != nullptr && packed != nullptr), TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(twn_aligned(W, 16) && twn_aligned(packed, 16) && twn_aligned(stats, 8) &&
+                    twn_aligned(codes_i8, 16), TWN_ERR_MISALIGNED);
+    twn_device_info dev;
+    int rc = twn_current_device(&dev);
+    if (rc != TWN_OK) return rc;
+    void *scratch = nullptr;
+    rc = static_scratch_ptr(dev.ordinal, &scratch);
+    if (rc != TWN_OK) return rc;
+    cudaStream_t s = twn_cu(stream);
+
+    // the array still holds the previous call's partials; only the two tickets must start at zero
+    TWN_CUDA_OK(cudaMemsetAsync(scratch, 0, 128, s));
+
+    const int g1 = grid_for((n / 4 + 3) / 4, dev.sm_count);
+    sum_abs_kernel<<<g1, kThreads, 0, s>>>(W, n, delta_factor, scratch, stats);
+
+    const bool flat = (rows <= 1) || (ld_codes == cols);
+    const long long fast_units = flat ? n / 512 : 0;
+    const long long rest_words = (long long)rows * (ld_codes / 16) - fast_units * 32;
+    long long work = fast_units * 32 / 4;
+    if (rest_words > work) work = rest_words;
+    const int g2 = grid_for(work, dev.sm_count);
+    code_pack_kernel<<<g2, kThreads, 0, s>>>(W, rows, cols, ld_codes, fast_units, packed, codes_i8,
+                                             scratch, stats);
+    TWN_CUDA_OK(cudaGetLastError());
+    return TWN_OK;
+}
+
 extern "C" int twn_pack(const int8_t *codes, int64_t rows, int64_t cols, uint32_t *packed,
                         int64_t ld_codes, twn_stats_t *counts, twn_stream_t stream)
 {

@@ -131,6 +131,22 @@ def ternarize(W: torch.Tensor, delta_factor: float, stats: torch.Tensor, packed:
                                _stream(stream)), "twn_ternarize")
 
 
+TERNARIZE_STATIC_MAX_WEIGHTS = 1 << 31
+
+
+def ternarize_static(W: torch.Tensor, delta_factor: float, stats: torch.Tensor, packed: torch.Tensor,
+                     ld_codes: int, codes_i8, stream=None, rows: int | None = None,
+                     cols: int | None = None) -> None:
+    """twn_ternarize_static: the same ternarization with the scratch held inside the library,
+    for callers that cannot allocate device memory.  Calls on one device must not overlap."""
+    if rows is None:
+        rows, cols = (W.shape[0], W.numel() // W.shape[0]) if W.dim() > 1 else (1, W.numel())
+    _check(lib().twn_ternarize_static(_ptr(W), C.c_int64(rows), C.c_int64(cols),
+                                      C.c_double(delta_factor), _ptr(stats), _ptr(packed),
+                                      C.c_int64(ld_codes), _ptr(codes_i8), _stream(stream)),
+           "twn_ternarize_static")
+
+
 def pack(codes: torch.Tensor, rows: int, cols: int, packed: torch.Tensor, ld_codes: int,
          counts=None, stream=None) -> None:
     _check(lib().twn_pack(_ptr(codes), C.c_int64(rows), C.c_int64(cols), _ptr(packed),
