@@ -240,6 +240,58 @@ int twn_conv2d_bwd_data(const twn_conv_desc_t *desc, const void *dZ, const uint3
                         const twn_stats_t *stats, const twn_epilogue_t *epi, void *dX,
                         int32_t *dev_status, twn_stream_t stream);
 
+/*
+ * Straight-through weight gradient (Algorithm 1, UpdateParameters; Fig. 1 caption): the
+ * gradient with respect to T = alpha*W~, applied to the fp32 master weights unchanged.  No
+ * alpha factor and no mask enter:
+ *   dW[o,r,s,c] = sum_{b,ho,wo} dZ[b,ho,wo,o] * X[b, ho*stride_h - pad_h + r, wo*stride_w - pad_w + s, c]
+ *   X   bf16 NHWC [B,H,W,Cin];  dZ  bf16 NHWC [B,Ho,Wo,Cout];  both contiguous, 16-byte aligned.
+ *   dW  fp32 [Cout][kh][kw][Cin], overwritten.
+ *   workspace  at least twn_conv2d_bwd_weight_workspace_bytes(desc) bytes, 16-byte aligned:
+ *              per-split partial sums, added in a fixed order (deterministic).
+ * Requires Cin % 8 == 0 and Cout % 8 == 0 (layers with fewer channels: run it on the
+ * twn_im2col matrix as a 1x1 convolution).  bf16 products, fp32 accumulation.
+ * dev_status as in twn_gemm.
+ */
+size_t twn_conv2d_bwd_weight_workspace_bytes(const twn_conv_desc_t *desc);
+int twn_conv2d_bwd_weight(const twn_conv_desc_t *desc, const void *X, const void *dZ, float *dW,
+                          void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                          twn_stream_t stream);
+
+/* ---- layer glue (Sec. 2.4: conv, affine, ReLU, pooling; standard back-propagation) ---- */
+
+/*
+ * Patch matrix for layers whose channel count is too small for twn_conv2d_fwd (Cin = 1, 3):
+ *   Xcol[m, (r*kw + s)*Cin + c] = X[b, ho*stride_h - pad_h + r, wo*stride_w - pad_w + s, c]
+ * with m = (b*Ho + ho)*Wo + wo, zero outside the image and in columns K..ldk-1.
+ * Xcol is bf16 [B*Ho*Wo, ldk], ldk >= kh*kw*Cin, ldk % 8 == 0, 16-byte aligned.  The
+ * convolution is then twn_gemm(Xcol, ldk, T_fwd, ...) with K = kh*kw*Cin.
+ */
+int twn_im2col(const twn_conv_desc_t *desc, const void *X, void *Xcol, int64_t ldk, twn_stream_t stream);
+
+/* Max pooling, window k x k (k <= 15), padding with -inf.  X, Y bf16 NHWC; `argmax` (optional,
+ * one byte per output element) records the window position r*k+s of the first maximum in
+ * scan order, for the backward pass. */
+int twn_maxpool2d_fwd(const void *X, int64_t B, int64_t H, int64_t W, int64_t C, int k, int stride,
+                      int pad, void *Y, uint8_t *argmax, twn_stream_t stream);
+/* dX[b,h,w,c] = sum of dY over the windows whose recorded maximum is (h,w).  Deterministic. */
+int twn_maxpool2d_bwd(const void *dY, const uint8_t *argmax, int64_t B, int64_t H, int64_t W, int64_t C,
+                      int k, int stride, int pad, void *dX, twn_stream_t stream);
+
+/* Global average pooling: X bf16 [B, HW, C] -> Y bf16 [B, C]; backward dX = dY / HW. */
+int twn_avgpool_fwd(const void *X, int64_t B, int64_t HW, int64_t C, void *Y, twn_stream_t stream);
+int twn_avgpool_bwd(const void *dY, int64_t B, int64_t HW, int64_t C, void *dX, twn_stream_t stream);
+
+/*
+ * Backward through the epilogue y = relu(z*scale[c] + shift[c] (+ residual)):
+ *   dPre = dY * [Y > 0]   (Y = the block's bf16 output; Y NULL: no ReLU, dPre = dY)
+ *   dZ   = dPre * scale[c]  (scale NULL: 1)
+ * n elements with channel c = index % C.  dZ and dPre are bf16; either may be NULL.
+ * dPre is what flows into a residual branch, dZ into the convolution's backward passes.
+ */
+int twn_act_bwd(const void *dY, const void *Y, const float *scale, int64_t n, int64_t C, void *dZ,
+                void *dPre, twn_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -1,0 +1,366 @@
+// Straight-through weight gradient (Algorithm 1, UpdateParameters; Fig. 1 caption): the
+// gradient with respect to T = alpha * W~ computed by ordinary back-propagation and applied
+// to the fp32 master weights unchanged,
+//     dW[o, r, s, c] = sum_{b,ho,wo} dZ[b,ho,wo,o] * X[b, ho*stride - pad + r, wo*stride - pad + s, c].
+// A dense bf16 x bf16 -> fp32 contraction whose reduction runs over the pixels, i.e. over the
+// slow dimension of both NHWC operands.  tcgen05 takes such operands directly ("MN-major"
+// shared-memory descriptors), so the dZ tile and the tap-shifted X tile go from TMA straight
+// into the MMA: D[o, c] += dZ_tile^T * X_tile, 64 pixels per k-block.
+//
+// The output has few tiles (Cout/128 x taps x Cin/256) but a long reduction (up to 8e5 pixels),
+// so the pixels are split across CTAs; each CTA writes its fp32 partial tile to the workspace
+// and a second kernel adds the partials in split order (deterministic, no atomics).
+//
+//   warp 0     TMA producer        warp 1     MMA issuer (whole warp, elected lane issues)
+//   warps 2-5  epilogue: tensor memory -> workspace
+#include <cstddef>
+
+#include "common.cuh"
+#include "tc_ptx.cuh"
+
+namespace {
+
+constexpr int kDwStages = 4;
+constexpr int kDwPix = 64;                       // pixels per k-block
+constexpr int kDwBlockBytes = kDwPix * 128;      // one 64-channel x 64-pixel swizzled block: 8 KB
+constexpr int kDwMaxCb = 4;                      // up to 256 input channels per tile
+constexpr int kDwThreads = 192;
+constexpr int kDwMaxTaps = 64;
+constexpr int kDwAccCols = 256;
+
+struct DwTap { int16_t dh, dw; int32_t koff; };
+
+struct DwParams {
+    int n_otiles, n_taps, n_ctiles, splits, total_units;
+    int lgBW, lgBH, tw, th, tb, pix_tiles, tiles_per_split;
+    int sw, sh, ncb;
+    int Cout, Cin;
+    long long K;                 // row length of dW and of a partial
+    long long split_stride;      // elements between partials of consecutive splits
+    float *partial;
+    int vec_ok;
+    int32_t *status;
+    DwTap taps[kDwMaxTaps];
+};
+
+struct __align__(1024) DwSmem {
+    uint8_t a[kDwStages][2][kDwBlockBytes];            // dZ: two 64-channel blocks
+    uint8_t b[kDwStages][kDwMaxCb][kDwBlockBytes];     // X: up to four 64-channel blocks
+    unsigned long long full[kDwStages], empty[kDwStages], acc_full[2], acc_empty[2];
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+
+__global__ void __launch_bounds__(kDwThreads, 1)
+dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CUtensorMap map_x,
+          const __grid_constant__ DwParams P)
+{
+    extern __shared__ uint8_t smem_raw[];
+    DwSmem *sm = reinterpret_cast<DwSmem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    volatile int *abort_flag = &sm->abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kDwStages; ++s) { mbar_init(&sm->full[s], 1); mbar_init(&sm->empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&sm->acc_full[b], 1); mbar_init(&sm->acc_empty[b], 4); }
+        sm->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sm->tmem_base;
+
+    // unit -> (o tile, tap, c tile, split); the split covers pixel tiles [p0, p1)
+    auto unit_range = [&](int u, int &ot, int &t, int &ct, int &sp, int &p0, int &p1) {
+        sp = u % P.splits; u /= P.splits;
+        ct = u % P.n_ctiles; u /= P.n_ctiles;
+        t = u % P.n_taps;
+        ot = u / P.n_taps;
+        p0 = sp * P.tiles_per_split;
+        p1 = p0 + P.tiles_per_split;
+        if (p1 > P.pix_tiles) p1 = P.pix_tiles;
+        if (p0 > p1) p0 = p1;
+    };
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            const uint32_t bytes = (2 + P.ncb) * kDwBlockBytes;
+            for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
+                int ot, t, ct, sp, p0, p1;
+                unit_range(u, ot, t, ct, sp, p0, p1);
+                const DwTap tap = P.taps[t];
+                for (int p = p0; p < p1; ++p, ++it) {
+                    const int s = it % kDwStages;
+                    const uint32_t ph = (it / kDwStages) & 1u;
+                    int q = p;
+                    const int twi = q % P.tw; q /= P.tw;
+                    const int thi = q % P.th;
+                    const int tbi = q / P.th;
+                    const int w0 = twi << P.lgBW, h0 = thi << P.lgBH, b0 = tbi * (kDwPix >> (P.lgBW + P.lgBH));
+                    if (!mbar_wait(&sm->empty[s], ph ^ 1u, abort_flag, P.status, 32)) { ok = false; break; }
+                    mbar_expect_tx(&sm->full[s], bytes);
+                    tma_load_4d(sm->a[s][0], &map_dz, &sm->full[s], ot * 128, w0, h0, b0);
+                    tma_load_4d(sm->a[s][1], &map_dz, &sm->full[s], ot * 128 + 64, w0, h0, b0);
+                    for (int j = 0; j < P.ncb; ++j)
+                        tma_load_4d(sm->b[s][j], &map_x, &sm->full[s], (ct * kDwMaxCb + j) * 64, w0 * P.sw + tap.dw,
+                                    h0 * P.sh + tap.dh, b0);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        const uint32_t idesc = make_idesc_mn(128, 64 * P.ncb);
+        uint32_t it = 0, lu = 0;     // lu counts the units that accumulate something
+        bool ok = true;
+        for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
+            int ot, t, ct, sp, p0, p1;
+            unit_range(u, ot, t, ct, sp, p0, p1);
+            if (p1 <= p0) continue;                      // the epilogue writes zeros for an empty split
+            const int buf = lu & 1;
+            if (!mbar_wait_warp(&sm->acc_empty[buf], ((lu >> 1) & 1u) ^ 1u, abort_flag, P.status, 0)) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem + buf * kDwAccCols;
+            for (int p = p0; p < p1; ++p, ++it) {
+                const int s = it % kDwStages;
+                const uint32_t ph = (it / kDwStages) & 1u;
+                if (!mbar_wait_warp(&sm->full[s], ph, abort_flag, P.status, 0)) { ok = false; break; }
+                tc_fence_after();
+                const uint64_t adesc = smem_desc_mn_sw128(smem_u32(sm->a[s][0]), kDwBlockBytes);
+                const uint64_t bdesc = smem_desc_mn_sw128(smem_u32(sm->b[s][0]), kDwBlockBytes);
+                // 16 pixels per MMA = 16 rows of 128 bytes = 2048 bytes
+                if (p == p0) tc_mma_ss<false>(d_tmem, adesc, bdesc, idesc);
+                else tc_mma_ss<true>(d_tmem, adesc, bdesc, idesc);
+                tc_mma_ss<true>(d_tmem, adesc + 128, bdesc + 128, idesc);
+                tc_mma_ss<true>(d_tmem, adesc + 256, bdesc + 256, idesc);
+                tc_mma_ss<true>(d_tmem, adesc + 384, bdesc + 384, idesc);
+                tc_commit(&sm->empty[s]);
+            }
+            if (ok) tc_commit(&sm->acc_full[buf]);
+            ++lu;
+        }
+    } else {
+        const int q = warp & 3;
+        uint32_t lu = 0;
+        for (int u = blockIdx.x; u < P.total_units; u += gridDim.x) {
+            int ot, t, ct, sp, p0, p1;
+            unit_range(u, ot, t, ct, sp, p0, p1);
+            const bool have = p1 > p0;
+            const int buf = lu & 1;
+            if (have && !mbar_wait_warp(&sm->acc_full[buf], (lu >> 1) & 1u, abort_flag, P.status, 32)) break;
+            tc_fence_after();
+            const int o = ot * 128 + q * 32 + lane;
+            const int c_base = ct * (kDwMaxCb * 64);
+            float *dst = P.partial + (long long)sp * P.split_stride + (long long)o * P.K + P.taps[t].koff + c_base;
+#pragma unroll 1
+            for (int c = 0; c < P.ncb * 2; ++c) {
+                uint32_t v[32];
+                if (have) {
+                    tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + buf * kDwAccCols + c * 32, v);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = 0u;
+                }
+                if (o < P.Cout) {
+                    if (P.vec_ok && c_base + c * 32 + 32 <= P.Cin) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            reinterpret_cast<uint4 *>(dst + c * 32)[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (c_base + c * 32 + j < P.Cin) dst[c * 32 + j] = __uint_as_float(v[j]);
+                    }
+                }
+            }
+            if (have) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm->acc_empty[buf]);
+                ++lu;
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (sm->abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+    }
+}
+
+__global__ void __launch_bounds__(256)
+dw_reduce_kernel(const float *__restrict__ partial, long long n, int splits, float *__restrict__ dW)
+{
+    for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256) {
+        float s = 0.0f;
+        for (int k = 0; k < splits; ++k) s += __ldg(partial + (long long)k * n + i);
+        dW[i] = s;
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn dw_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &p, 12000, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+struct DwPlan {
+    DwParams P;
+    long long Ho, Wo;
+    size_t ws_bytes;
+};
+
+int dw_plan(const twn_conv_desc_t *d, int sm_count, DwPlan *plan)
+{
+    TWN_REQUIRE(d != nullptr, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(d->B > 0 && d->H > 0 && d->W > 0 && d->Cin > 0 && d->Cout > 0 && d->kh > 0 && d->kw > 0 &&
+                    d->stride_h > 0 && d->stride_w > 0 && d->stride_h <= 8 && d->stride_w <= 8 && d->pad_h >= 0 &&
+                    d->pad_w >= 0 && d->kh * d->kw <= kDwMaxTaps, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(d->Cin % 8 == 0 && d->Cout % 8 == 0, TWN_ERR_MISALIGNED);
+    DwParams &P = plan->P;
+    memset(&P, 0, sizeof P);
+    plan->Ho = (d->H + 2 * d->pad_h - d->kh) / d->stride_h + 1;
+    plan->Wo = (d->W + 2 * d->pad_w - d->kw) / d->stride_w + 1;
+    TWN_REQUIRE(plan->Ho > 0 && plan->Wo > 0, TWN_ERR_INVALID_ARG);
+    // pixel box: 64 = BB x BH x BW, fewest tiles
+    long long best = -1;
+    for (int a = 0; a <= 6; ++a)
+        for (int b = 0; a + b <= 6; ++b) {
+            const int BW = 1 << a, BH = 1 << b, BB = kDwPix >> (a + b);
+            if (BW * d->stride_w > 256 || BH * d->stride_h > 256) continue;
+            const long long tiles = ((plan->Wo + BW - 1) / BW) * ((plan->Ho + BH - 1) / BH) * ((d->B + BB - 1) / BB);
+            if (best < 0 || tiles < best || (tiles == best && a > P.lgBW)) { best = tiles; P.lgBW = a; P.lgBH = b; }
+        }
+    const int BW = 1 << P.lgBW, BH = 1 << P.lgBH, BB = kDwPix >> (P.lgBW + P.lgBH);
+    P.tw = (int)((plan->Wo + BW - 1) / BW);
+    P.th = (int)((plan->Ho + BH - 1) / BH);
+    P.tb = (int)((d->B + BB - 1) / BB);
+    TWN_REQUIRE(best > 0 && best <= 0x7fffffffLL, TWN_ERR_INVALID_ARG);
+    P.pix_tiles = (int)best;
+    P.n_otiles = (int)((d->Cout + 127) / 128);
+    P.n_taps = d->kh * d->kw;
+    const int cblocks = (int)((d->Cin + 63) / 64);
+    P.n_ctiles = (cblocks + kDwMaxCb - 1) / kDwMaxCb;
+    P.ncb = cblocks < kDwMaxCb ? cblocks : kDwMaxCb;
+    const long long units = (long long)P.n_otiles * P.n_taps * P.n_ctiles;
+    long long splits = (2LL * sm_count + units - 1) / units;
+    if (splits > P.pix_tiles) splits = P.pix_tiles;
+    if (splits < 1) splits = 1;
+    P.tiles_per_split = (int)((P.pix_tiles + splits - 1) / splits);
+    splits = (P.pix_tiles + P.tiles_per_split - 1) / P.tiles_per_split;
+    P.splits = (int)splits;
+    TWN_REQUIRE(units * splits <= 0x7fffffffLL, TWN_ERR_INVALID_ARG);
+    P.total_units = (int)(units * splits);
+    P.sw = d->stride_w; P.sh = d->stride_h;
+    P.Cout = (int)d->Cout; P.Cin = (int)d->Cin;
+    P.K = (long long)P.n_taps * d->Cin;
+    P.split_stride = d->Cout * P.K;
+    P.vec_ok = (d->Cin % 4 == 0) ? 1 : 0;
+    for (int r = 0; r < d->kh; ++r)
+        for (int s = 0; s < d->kw; ++s) {
+            DwTap &t = P.taps[r * d->kw + s];
+            t.dh = (int16_t)(r - d->pad_h);
+            t.dw = (int16_t)(s - d->pad_w);
+            t.koff = (int32_t)((r * d->kw + s) * d->Cin);
+        }
+    plan->ws_bytes = (size_t)P.splits * (size_t)P.split_stride * sizeof(float);
+    return TWN_OK;
+}
+
+}  // namespace
+
+extern "C" size_t twn_conv2d_bwd_weight_workspace_bytes(const twn_conv_desc_t *d)
+{
+    DwPlan plan;
+    // the split count depends on the SM count; size for the largest part in use (148 SMs)
+    int sms = 148;
+    twn_device_info dev;
+    if (twn_current_device(&dev) == TWN_OK) sms = dev.sm_count;
+    if (dw_plan(d, sms, &plan) != TWN_OK) return 0;
+    return plan.ws_bytes;
+}
+
+extern "C" int twn_conv2d_bwd_weight(const twn_conv_desc_t *d, const void *X, const void *dZ, float *dW,
+                                     void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                     twn_stream_t stream)
+{
+    TWN_REQUIRE(X && dZ && dW && workspace, TWN_ERR_INVALID_ARG);
+    twn_device_info dev;
+    int rc = twn_current_device(&dev);
+    if (rc != TWN_OK) return rc;
+    DwPlan plan;
+    rc = dw_plan(d, dev.sm_count, &plan);
+    if (rc != TWN_OK) return rc;
+    TWN_REQUIRE(workspace_bytes >= plan.ws_bytes, TWN_ERR_WORKSPACE);
+    TWN_REQUIRE(twn_aligned(X, 16) && twn_aligned(dZ, 16) && twn_aligned(dW, 16) && twn_aligned(workspace, 16) &&
+                    twn_aligned(dev_status, 4), TWN_ERR_MISALIGNED);
+    EncodeTiledFn enc = dw_encode_fn();
+    if (!enc) return TWN_ERR_CUDA;
+    DwParams &P = plan.P;
+    P.partial = static_cast<float *>(workspace);
+    P.status = dev_status;
+    const int BW = 1 << P.lgBW, BH = 1 << P.lgBH, BB = kDwPix >> (P.lgBW + P.lgBH);
+
+    CUtensorMap map_dz, map_x;
+    {
+        cuuint64_t dims[4] = {(cuuint64_t)d->Cout, (cuuint64_t)plan.Wo, (cuuint64_t)plan.Ho, (cuuint64_t)d->B};
+        cuuint64_t strides[3] = {(cuuint64_t)d->Cout * 2, (cuuint64_t)plan.Wo * d->Cout * 2,
+                                 (cuuint64_t)plan.Ho * plan.Wo * d->Cout * 2};
+        cuuint32_t box[4] = {64, (cuuint32_t)BW, (cuuint32_t)BH, (cuuint32_t)BB};
+        cuuint32_t estr[4] = {1, 1, 1, 1};
+        if (enc(&map_dz, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(dZ), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return TWN_ERR_INVALID_ARG;
+    }
+    {
+        cuuint64_t dims[4] = {(cuuint64_t)d->Cin, (cuuint64_t)d->W, (cuuint64_t)d->H, (cuuint64_t)d->B};
+        cuuint64_t strides[3] = {(cuuint64_t)d->Cin * 2, (cuuint64_t)d->W * d->Cin * 2, (cuuint64_t)d->H * d->W * d->Cin * 2};
+        cuuint32_t box[4] = {64, (cuuint32_t)(BW * d->stride_w), (cuuint32_t)(BH * d->stride_h), (cuuint32_t)BB};
+        cuuint32_t estr[4] = {1, (cuuint32_t)d->stride_w, (cuuint32_t)d->stride_h, 1};
+        if (enc(&map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(X), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return TWN_ERR_INVALID_ARG;
+    }
+    static bool attr_set[64] = {false};
+    const int smem_bytes = (int)sizeof(DwSmem) + 1024;
+    if (!attr_set[dev.ordinal]) {
+        TWN_CUDA_OK(cudaFuncSetAttribute(dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
+        attr_set[dev.ordinal] = true;
+    }
+    cudaStream_t s = twn_cu(stream);
+    const int grid = dev.sm_count < P.total_units ? dev.sm_count : P.total_units;
+    dw_kernel<<<grid, kDwThreads, smem_bytes, s>>>(map_dz, map_x, P);
+    const long long n = P.split_stride;
+    long long rb = (n + 255) / 256;
+    if (rb > dev.sm_count * 8) rb = dev.sm_count * 8;
+    dw_reduce_kernel<<<(int)rb, 256, 0, s>>>(P.partial, n, P.splits, dW);
+    TWN_CUDA_OK(cudaGetLastError());
+    return TWN_OK;
+}

@@ -37,6 +37,7 @@
 #include <cstddef>
 
 #include "common.cuh"
+#include "tc_ptx.cuh"
 
 namespace {
 
@@ -48,7 +49,6 @@ constexpr int kThreadsConv = 32 * (kFirstEpiWarp + 4);
 constexpr int kMaxTaps = 64;
 constexpr int kAColsPerBlock = kBlockK / 2;    // 32 columns of bf16 pairs per k-block
 constexpr uint32_t kTmemCols = 512;
-constexpr unsigned long long kWaitLimitNs = 1000000000ull;
 
 template <int PIX> struct Cfg;
 template <> struct Cfg<128> {
@@ -112,196 +112,6 @@ struct __align__(1024) SmemLayout {
     volatile int epi_ok;                   // outcome of the epilogue's wait, shared by its four warps
 };
 
-// ---------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(void *bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(void *bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(void *bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(void *bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(2000u) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-
-// Bounded wait.  Returns false when the limit ran out or another role gave up.
-// Waiting warps share their scheduler with the warps that do the work, so a waiter backs
-// off with nanosleep instead of polling flat out (`backoff_ns` = 0 for the latency-critical
-// waits of the MMA warp, which rely on the suspend time of try_wait alone).
-__device__ __forceinline__ bool mbar_wait(void *bar, uint32_t parity, volatile int *abort_flag, int32_t *status,
-                                          uint32_t backoff_ns = 64)
-{
-    if (mbar_try(bar, parity)) return true;
-    unsigned long long t0 = 0;
-    for (uint32_t spin = 1;; ++spin) {
-        if (mbar_try(bar, parity)) return true;
-        if (backoff_ns) __nanosleep(backoff_ns);
-        if ((spin & 255u) == 0) {
-            if (*abort_flag) return false;
-            const unsigned long long now = global_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                if (status) atomicMin(status, (int)TWN_ERR_TIMEOUT);
-                return false;
-            }
-        }
-    }
-}
-
-// Warp-wide wait: lane 0 polls, the result is broadcast.  One polling lane instead of 32
-// keeps the shared-memory pipe free for the warps that are working.
-__device__ __forceinline__ bool mbar_wait_warp(void *bar, uint32_t parity, volatile int *abort_flag, int32_t *status,
-                                               uint32_t backoff_ns = 64)
-{
-    int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status, backoff_ns) ? 1 : 0;
-    ok = __shfl_sync(0xffffffffu, ok, 0);
-    __syncwarp();
-    return ok != 0;
-}
-
-__device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, void *bar, int c0, int c1, int c2, int c3)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-        : "memory");
-}
-
-__device__ __forceinline__ void tma_store_4d(const CUtensorMap *map, const void *src, int c0, int c1, int c2, int c3)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
-        ::"l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-        : "memory");
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-// named barrier of the four epilogue warps
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-
-// The MMA warp runs its loops converged; tcgen05.mma and tcgen05.commit are issued by the
-// lane that elect.sync picks, with the predicate applied inside the asm block (measured to be
-// the cheapest way to issue: no divergent region around the instruction).
-// D[tmem] (+)= A[tmem] * B[smem]^T, bf16 x bf16 -> fp32.
-template <bool ACC>
-__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc)
-{
-    asm volatile(
-        "{\n\t.reg .pred p, pe;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "elect.sync _|pe, 0xffffffff;\n\t"
-        "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "n"(ACC ? 1 : 0)
-        : "memory");
-}
-
-__device__ __forceinline__ void tc_commit(void *bar)
-{
-    asm volatile(
-        "{\n\t.reg .pred pe;\n\t"
-        "elect.sync _|pe, 0xffffffff;\n\t"
-        "@pe tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
-        ::"r"(smem_u32(bar)) : "memory");
-}
-
-// One k-block: four K=16 MMAs.  FIRST clears the accumulator with the first of them.  The
-// accumulate flag is a compile-time constant so that no predicate has to be built at run time:
-// whatever the issuing thread executes between two MMAs is time the tensor core may sit idle.
-template <bool FIRST>
-__device__ __forceinline__ void tc_mma_block(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc)
-{
-    tc_mma_ts<!FIRST>(d_tmem, a_tmem, b_desc, idesc);
-    tc_mma_ts<true>(d_tmem, a_tmem + 8, b_desc + 2, idesc);
-    tc_mma_ts<true>(d_tmem, a_tmem + 16, b_desc + 4, idesc);
-    tc_mma_ts<true>(d_tmem, a_tmem + 24, b_desc + 6, idesc);
-}
-
-// K-major, 128-byte swizzled operand tile: rows of 128 bytes, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);   // start address
-    d |= (uint64_t)1 << 16;                     // leading byte offset (unused for swizzled K-major)
-    d |= (uint64_t)(1024 >> 4) << 32;           // stride byte offset
-    d |= (uint64_t)1 << 46;                     // descriptor version for sm_100
-    d |= (uint64_t)2 << 61;                     // 128-byte swizzle
-    return d;
-}
-
-// kind::f16 instruction descriptor: bf16 A and B (both K-major), fp32 accumulate.
-__host__ __device__ constexpr uint32_t make_idesc(int M, int N)
-{
-    return (1u << 4)              // D format fp32
-           | (1u << 7)            // A format bf16
-           | (1u << 10)           // B format bf16
-           | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
-
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32])
-{
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
-        ::"r"(taddr),
-          "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
-          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
-          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-        : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-}
-
-// Two 2-bit fields (bits 1:0 and 17:16 of x) -> two exact bf16 values in {-1, 0, +1}.
-// field ^ 2 is the field's value + 2 (00 -> 2, 01 -> 3, 11 -> 1); or-ing it into the
-// mantissa of 128.0 gives 130 + value, and subtracting 130.0 leaves the value.
-__device__ __forceinline__ uint32_t fields_to_bf16x2(uint32_t x)
-{
-    const uint32_t t = (x & 0x00030003u) ^ 0x43024302u;
-    uint32_t r;
-    asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(t), "r"(0x43024302u));
-    return r;
-}
-
-// ---------------------------------------------------------------- the kernel
 static_assert(offsetof(SmemLayout<128>, stage_out) % 128 == 0 && offsetof(SmemLayout<256>, stage_out) % 128 == 0 &&
                   offsetof(SmemLayout<128>, pix_off) % 16 == 0 && offsetof(SmemLayout<256>, pix_off) % 16 == 0,
               "TMA and vector accesses need aligned shared-memory regions");

@@ -65,6 +65,7 @@ def lib() -> C.CDLL:
         l = C.CDLL(LIB_PATH)
         l.twn_strerror.restype = C.c_char_p
         l.twn_ternarize_workspace_bytes.restype = C.c_size_t
+        l.twn_conv2d_bwd_weight_workspace_bytes.restype = C.c_size_t
         _lib = l
     return _lib
 
@@ -202,3 +203,44 @@ def conv2d_bwd_data(desc: ConvDesc, dZ: torch.Tensor, T_bwd: torch.Tensor, ld_co
     _check(lib().twn_conv2d_bwd_data(C.byref(desc), _ptr(dZ), _ptr(T_bwd), C.c_int64(ld_codes),
                                      _ptr(stats), C.byref(epi) if epi is not None else None, _ptr(dX),
                                      _ptr(dev_status), _stream(stream)), "twn_conv2d_bwd_data")
+
+
+def im2col(desc: ConvDesc, X: torch.Tensor, Xcol: torch.Tensor, ldk: int, stream=None) -> None:
+    _check(lib().twn_im2col(C.byref(desc), _ptr(X), _ptr(Xcol), C.c_int64(ldk), _stream(stream)), "twn_im2col")
+
+
+def maxpool2d_fwd(X, B, H, W, Cc, k, stride, pad, Y, argmax=None, stream=None) -> None:
+    _check(lib().twn_maxpool2d_fwd(_ptr(X), C.c_int64(B), C.c_int64(H), C.c_int64(W), C.c_int64(Cc),
+                                   C.c_int(k), C.c_int(stride), C.c_int(pad), _ptr(Y), _ptr(argmax),
+                                   _stream(stream)), "twn_maxpool2d_fwd")
+
+
+def maxpool2d_bwd(dY, argmax, B, H, W, Cc, k, stride, pad, dX, stream=None) -> None:
+    _check(lib().twn_maxpool2d_bwd(_ptr(dY), _ptr(argmax), C.c_int64(B), C.c_int64(H), C.c_int64(W),
+                                   C.c_int64(Cc), C.c_int(k), C.c_int(stride), C.c_int(pad), _ptr(dX),
+                                   _stream(stream)), "twn_maxpool2d_bwd")
+
+
+def avgpool_fwd(X, B, HW, Cc, Y, stream=None) -> None:
+    _check(lib().twn_avgpool_fwd(_ptr(X), C.c_int64(B), C.c_int64(HW), C.c_int64(Cc), _ptr(Y),
+                                 _stream(stream)), "twn_avgpool_fwd")
+
+
+def avgpool_bwd(dY, B, HW, Cc, dX, stream=None) -> None:
+    _check(lib().twn_avgpool_bwd(_ptr(dY), C.c_int64(B), C.c_int64(HW), C.c_int64(Cc), _ptr(dX),
+                                 _stream(stream)), "twn_avgpool_bwd")
+
+
+def act_bwd(dY, Y, scale, n, Cc, dZ, dPre=None, stream=None) -> None:
+    _check(lib().twn_act_bwd(_ptr(dY), _ptr(Y), _ptr(scale), C.c_int64(n), C.c_int64(Cc), _ptr(dZ),
+                             _ptr(dPre), _stream(stream)), "twn_act_bwd")
+
+
+def conv2d_bwd_weight_workspace_bytes(desc: ConvDesc) -> int:
+    return int(lib().twn_conv2d_bwd_weight_workspace_bytes(C.byref(desc)))
+
+
+def conv2d_bwd_weight(desc: ConvDesc, X, dZ, dW, workspace, dev_status=None, stream=None) -> None:
+    _check(lib().twn_conv2d_bwd_weight(C.byref(desc), _ptr(X), _ptr(dZ), _ptr(dW), _ptr(workspace),
+                                       C.c_size_t(workspace.numel() * workspace.element_size()),
+                                       _ptr(dev_status), _stream(stream)), "twn_conv2d_bwd_weight")
