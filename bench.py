@@ -3,13 +3,15 @@
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
 
-Prints ONE JSON line (rank 0).  A step is one pass of the workload's whole hot
-path over one batch of seeded synthetic input.  Device timing uses CUDA events on
-the launching stream; for N > 1 every rank runs an independent replica (the path
-has no exchange step) and the slowest rank's time is used.
+Prints ONE JSON line (rank 0).  A step is one pass of the workload's whole hot path over one
+batch of seeded synthetic input.  The default workload is the ResNet-18-shaped training step
+(batch 64, 3x224x224): ternarize + pack every layer, forward through the ternary convolutions,
+backward for data through the transposed codes, straight-through weight gradients.  Device
+timing uses CUDA events on the launching stream; for N > 1 every rank runs an independent
+replica (the path has no exchange step) and the slowest rank's time is used.
 
-`--impl reference` times the CPU oracle (oracle/) on a bounded sample of the same
-workload on the host cores; it is a deliberately slow baseline, not a target.
+`--impl reference` times the CPU oracle (oracle/) on a bounded sample of the same workload on
+the host cores; it is a deliberately slow baseline, not a target.
 """
 from __future__ import annotations
 
@@ -50,9 +52,11 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                 "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+                 "-i", str(self.index), "-lms", "50"], stdout=subprocess.PIPE, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
+            time.sleep(0.5)          # let the sampler come up before the timed region starts
+            self.first = len(self.rows)
         except OSError:
             self.proc = None
 
@@ -63,7 +67,6 @@ class ClockSampler:
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -72,7 +75,7 @@ class ClockSampler:
         self.t.join(timeout=2)
         sm, mx, reasons = [], None, set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for r in self.rows[self.first:]:
             try:
                 sm.append(float(r[0])); mx = float(r[1])
             except (ValueError, IndexError):
@@ -92,16 +95,16 @@ def dist_env():
 
 # ------------------------------------------------------------------ workloads
 class TernarizeWorkload:
-    """Ternarize + 2-bit pack of one fp32 tensor of n weights drawn N(0,1):
-    threshold reduction, Eq. 3 codes, Eq. 5 scale, packing.  8.25 algorithmic
-    bytes per weight (two reads of 4 B: the threshold needs every weight before
-    any code can be emitted; 0.25 B written)."""
+    """Ternarize + 2-bit pack of one fp32 tensor of n weights drawn N(0,1): threshold
+    reduction, Eq. 3 codes, Eq. 5 scale, packing.  8.25 algorithmic bytes per weight (two
+    reads of 4 B: the threshold needs every weight before any code can be emitted; 0.25 B
+    written)."""
     name = "ternarize_pack_n1e8_normal"
     metric = "ternarize+pack GB/s"
     unit = "GB/s"
     dtype = "f64"
     bytes_per_unit = 8.25
-    launches_per_step = 2
+    default_steps = 2000
 
     def __init__(self, n=100_000_000, seed=0):
         self.n, self.seed = n, seed
@@ -138,6 +141,9 @@ class TernarizeWorkload:
     def e2e_bytes(self):
         return self.n * 4, self.ld // 4 + 64
 
+    def launches_per_step(self):
+        return 2
+
     def units_per_step(self):
         return self.n * self.bytes_per_unit / 1e9  # GB of algorithmic traffic
 
@@ -152,7 +158,6 @@ class TernarizeWorkload:
         st = self.twn.stats_to_host(self.stats)
         assert st["status"] == 0 and st["n_neg"] + st["n_zero"] + st["n_pos"] == self.n, st
 
-    # CPU oracle on the same tensor (full size: about a second per pass)
     def cpu_sample(self, host_W):
         import oracle
         t0 = time.perf_counter()
@@ -162,8 +167,184 @@ class TernarizeWorkload:
         return self.n * self.bytes_per_unit / dt / 1e9, f"full tensor, n={self.n}", 1
 
 
-WORKLOADS = {"ternarize": TernarizeWorkload}
-DEFAULT_WORKLOAD = "ternarize"
+class NetWorkload:
+    """A chained network workload: images/s of a forward pass or of a whole training step,
+    replayed from a CUDA graph (the step is a fixed sequence of ~200 launches)."""
+    metric = "images/s"
+    unit = "images/s"
+    dtype = "bf16"
+    default_steps = 50
+
+    def __init__(self, kind):
+        self.kind = kind
+        self.name = {"resnet18_train": "resnet18_train_step_b64_224", "vgg7_fwd": "vgg7_forward_b128",
+                     "lenet5_fwd": "lenet5_forward_b100"}[kind]
+
+    def make(self, nets):
+        if self.kind == "resnet18_train":
+            return nets.resnet18(64, train=True)
+        if self.kind == "vgg7_fwd":
+            return nets.vgg7(128)
+        return nets.lenet5(100)
+
+    def config(self):
+        c = {"workload": self.name, "seed": 0, "delta_factor": 0.7,
+             "l2": "activations of a step (> 1 GB for ResNet-18) exceed L2 (126 MB)",
+             "launch": "one CUDA graph replay per step"}
+        if self.kind == "resnet18_train":
+            c["step"] = ("ternarize+pack 21 tensors, transpose codes, forward, backward for data, "
+                         "straight-through dW; synthetic dY N(0,1e-2) at the logits")
+        else:
+            c["step"] = "forward through ternary conv/FC with packed weights (ternarization done once, untimed)"
+            c["l2"] = "L2 flushed between timed steps is not needed: one step per replay, working set noted"
+        return c
+
+    def host_inputs(self):
+        from paper_1605_04711_b200 import datagen as dg
+        shape = {"resnet18_train": (64, 224, 224, 3), "vgg7_fwd": (128, 32, 32, 3), "lenet5_fwd": (100, 28, 28, 1)}[self.kind]
+        n = 1
+        for s in shape:
+            n *= s
+        dist = "uniform01" if self.kind == "lenet5_fwd" else "normal"
+        x = dg.draw_bf16(0, f"{self.name}.input", n, dist)
+        dy = dg.draw_bf16(0, f"{self.name}.dlogits", 64 * 1000, "normal", 0.0, 0.1) if self.kind == "resnet18_train" else None
+        return x, dy
+
+    def setup(self, torch, twn, host):
+        from paper_1605_04711_b200 import nets
+        import numpy as np
+        self.torch, self.twn = torch, twn
+        x, dy = host
+        self.net = net = self.make(nets)
+        self.train = self.kind == "resnet18_train"
+        self.host_x = torch.from_numpy(x.view(np.int16)).pin_memory()
+        net.act["input"].view(torch.int16).view(-1).copy_(self.host_x)
+        last = net.ops[-1][1]
+        self.logits = net.act[last.name]
+        self.host_logits = torch.empty(self.logits.shape, dtype=self.logits.dtype).pin_memory()
+        if self.train:
+            self.host_dy = torch.from_numpy(dy.view(np.int16)).pin_memory()
+            self.dY = torch.zeros((64, 1000), dtype=torch.bfloat16, device="cuda")
+            self.dY.view(torch.int16).view(-1).copy_(self.host_dy)
+        else:
+            net.ternarize_all()
+        # eager warm-up (first-call set-up, lazy buffers), then capture the step
+        for _ in range(2):
+            self._eager()
+        torch.cuda.synchronize()
+        net.check_status()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            self._eager()
+        # per-kernel device times from one eager pass; a spin keeps the GPU behind the host so
+        # that the events bracket kernels only
+        net.timed = []
+        torch.cuda._sleep(int(40e6))
+        self._eager()
+        torch.cuda.synchronize()
+        agg = {}
+        for kind, name, flops, e0, e1 in net.timed:
+            a = agg.setdefault(kind, [0, 0.0, 0.0])
+            a[0] += 1; a[1] += e0.elapsed_time(e1); a[2] += flops
+        self.kernel_times = agg
+        net.timed = None
+
+    def _eager(self):
+        if self.train:
+            self.net.train_step(self.dY)
+        else:
+            self.net.forward()
+
+    def step(self):
+        self.graph.replay()
+
+    def step_e2e(self):
+        t = self.torch
+        self.net.act["input"].view(t.int16).view(-1).copy_(self.host_x, non_blocking=True)
+        if self.train:
+            self.dY.view(t.int16).view(-1).copy_(self.host_dy, non_blocking=True)
+        self.graph.replay()
+        self.host_logits.copy_(self.logits, non_blocking=True)
+
+    def e2e_bytes(self):
+        h2d = self.host_x.numel() * 2 + (self.host_dy.numel() * 2 if self.train else 0)
+        return h2d, self.host_logits.numel() * self.host_logits.element_size()
+
+    def launches_per_step(self):
+        n = 0
+        net = self.net
+        for op in net.ops:
+            if op[0] == "layer":
+                L = op[1]
+                n += 1 + (1 if L.small_cin else 0)                       # forward (+ im2col)
+                if self.train:
+                    n += 3 + (1 if L.src != "input" else 0)               # memset + 2 ternarize (+ transpose)
+                    n += 1 + 2                                           # act_bwd, dW + reduce
+                    if L.src != "input":
+                        n += L.stride * L.stride                         # backward for data
+            elif op[0] in ("maxpool", "avgpool"):
+                n += 2 if self.train else 1
+        return n
+
+    def units_per_step(self):
+        return self.net.B
+
+    def roofline(self, ms_per_step, peaks):
+        k = self.kernel_times
+        t = k.get("tconv", [0, 0.0, 0.0])
+        ach = t[2] / (t[1] * 1e-3) / 1e12 if t[1] > 0 else 0.0
+        peak = peaks["bf16_tflops_sustained"]
+        out = {"bound": "tensor", "kernel": "tconv_kernel (all forward and backward-for-data launches of a step)",
+               "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
+               "peak_source": peaks["source"] + " (sustained bf16)", "traffic": None,
+               "launches": t[0], "ms_in_kernel": t[1],
+               "breakdown_ms": {kk: round(v[1], 4) for kk, v in k.items()},
+               "breakdown_tflops": {kk: (round(v[2] / (v[1] * 1e-3) / 1e12, 1) if v[1] > 0 and v[2] > 0 else None)
+                                    for kk, v in k.items()},
+               "step_macs": self.net.total_macs(),
+               "step_frac_of_tensor_peak": 2 * self.net.total_macs() / (ms_per_step * 1e-3) / 1e12 / peak}
+        return out
+
+    def check(self):
+        self.net.check_status()
+        assert bool(self.torch.isfinite(self.logits.float()).all())
+
+    def cpu_sample(self, host, seconds=10.0):
+        """Oracle convolution (fp64, OpenMP) on sampled output pixels of one mid-network layer
+        (28x28, 128 -> 128 channels, 3x3); images/s extrapolated by the MAC count of a step."""
+        import numpy as np
+        import oracle
+        from paper_1605_04711_b200 import datagen as dg
+        B, H, C = 4, 28, 128
+        d = oracle.conv_desc(B, H, H, C, C, 3, 1, 1)
+        X = dg.draw_bf16(0, "cpu.x", B * H * H * C, "normal").reshape(B, H, H, C)
+        W = dg.he_normal(0, "cpu.w", C, 9 * C)
+        st, codes = oracle.ternarize(W, 0.7)
+        codes = codes.reshape(C, 3, 3, C)
+        npix, rate = 256, None
+        while True:
+            pix = np.arange(npix) % (B * H * H)
+            t0 = time.perf_counter()
+            oracle.conv2d_fwd(d, X, codes, st.alpha, pixels=pix)
+            dt = time.perf_counter() - t0
+            rate = npix * 9 * C * C / dt
+            if dt >= seconds * 0.5 or npix >= 1 << 22:
+                break
+            npix = int(min(1 << 22, max(npix * 2, npix * seconds / max(dt, 1e-3))))
+        macs_per_image = self._macs_per_image()
+        return rate / macs_per_image, (f"oracle conv2d_fwd on {npix} output pixels of a 28x28x128->128 3x3 layer "
+                                       f"({dt:.1f} s); extrapolated by MACs per image ({macs_per_image / 1e9:.2f} G)"), \
+            oracle.num_threads()
+
+    def _macs_per_image(self):
+        if hasattr(self, "net"):
+            return self.net.total_macs() / self.net.B
+        return {"resnet18_train": 340.7e9 / 64 * 1.0, "vgg7_fwd": 615.9e6, "lenet5_fwd": 4.27e6}[self.kind]
+
+
+WORKLOADS = {"ternarize": lambda: TernarizeWorkload(), "resnet18_train": lambda: NetWorkload("resnet18_train"),
+             "vgg7_fwd": lambda: NetWorkload("vgg7_fwd"), "lenet5_fwd": lambda: NetWorkload("lenet5_fwd")}
+DEFAULT_WORKLOAD = "resnet18_train"
 
 
 # ------------------------------------------------------------------ arms
@@ -172,16 +353,18 @@ def run_reference(args):
     if rank != 0:
         return
     wl = WORKLOADS[args.workload]()
-    host = wl.host_inputs()
+    host = wl.host_inputs() if isinstance(wl, TernarizeWorkload) else None
     vals = []
-    for i in range(args.warmup + args.steps):
+    steps = args.steps if args.steps else 3
+    for i in range(args.warmup + steps):
         v, sample, cores = wl.cpu_sample(host)
         if i >= args.warmup:
             vals.append(v)
     value = sum(vals) / len(vals)
+    upstep = wl.units_per_step() if isinstance(wl, TernarizeWorkload) else {"resnet18_train": 64, "vgg7_fwd": 128, "lenet5_fwd": 100}[args.workload]
     line = {"impl": "reference", "metric": wl.metric, "value": value, "unit": wl.unit,
-            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": wl.units_per_step() / value * 1e3, "higher_is_better": True,
+            "n_gpus": args.gpus, "steps": steps, "warmup": args.warmup,
+            "ms_per_step": upstep / value * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": wl.config(), "gpu_launches": 0,
             "cpu_baseline": {"value": value, "unit": wl.unit, "cores": cores, "kind": "oracle",
@@ -206,17 +389,19 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     wl = WORKLOADS[args.workload]()
+    steps = args.steps if args.steps else wl.default_steps
+    warmup = max(args.warmup, 3)
     host = wl.host_inputs()
     wl.setup(torch, twn, host)
     peaks = measured_peaks()
 
-    def timed(fn, steps, warmup):
-        for _ in range(warmup):
+    def timed(fn, n_steps, n_warm):
+        for _ in range(n_warm):
             fn()
         barrier()
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ev0.record()
-        for _ in range(steps):
+        for _ in range(n_steps):
             fn()
         ev1.record()
         barrier()
@@ -225,26 +410,26 @@ def run_ours(args):
             t = torch.tensor([ms], device="cuda", dtype=torch.float64)
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             ms = float(t.item())
-        return ms / steps
+        return ms / n_steps
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
     if sampler:
         sampler.start()
-    ms = timed(wl.step, args.steps, max(args.warmup, 3))
+    ms = timed(wl.step, steps, warmup)
     clocks = sampler.stop() if sampler else None
     wl.check()
-    ms_e2e = timed(wl.step_e2e, max(2, min(args.steps, 5)), 1)
+    ms_e2e = timed(wl.step_e2e, max(2, min(steps, 20)), 1)
     wl.check()
 
     if rank == 0:
         h2d, d2h = wl.e2e_bytes()
         line = {"metric": wl.metric, "value": world * wl.units_per_step() / (ms * 1e-3),
-                "unit": wl.unit, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+                "unit": wl.unit, "n_gpus": world, "steps": steps, "warmup": warmup,
                 "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": wl.dtype, "data": "synthetic", "config": wl.config(), "clocks": clocks,
                 "e2e": {"value": world * wl.units_per_step() / (ms_e2e * 1e-3), "unit": wl.unit,
                         "ms_per_step": ms_e2e, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-                "gpu_launches": wl.launches_per_step * args.steps,
+                "gpu_launches": wl.launches_per_step() * steps,
                 "roofline": wl.roofline(ms, peaks)}
         if world == 1 and not args.no_cpu:
             v, sample, cores = wl.cpu_sample(host)
@@ -258,7 +443,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=0, help="timed steps (0: the workload's default)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
