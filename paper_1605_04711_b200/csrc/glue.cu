@@ -19,88 +19,160 @@ inline int blocks_for(long long items, int sm_count)
     return (int)b;
 }
 
+// Index arithmetic is 32-bit whenever the tensors allow it (64-bit division is an order of
+// magnitude slower on the GPU); `I` is int or long long.
+
 // ---- im2col: rows = output pixels, columns = (r, s, c), zero outside the image and past K
+template <typename I>
 __global__ void __launch_bounds__(kT)
-im2col_kernel(const __nv_bfloat16 *__restrict__ X, twn_conv_desc_t d, long long Ho, long long Wo,
-              __nv_bfloat16 *__restrict__ out, long long ldk)
+im2col_kernel(const __nv_bfloat16 *__restrict__ X, twn_conv_desc_t d, I Ho, I Wo,
+              __nv_bfloat16 *__restrict__ out, I ldk)
 {
-    const long long K = (long long)d.kh * d.kw * d.Cin;
-    const long long chunks = ldk / 8;                 // 8 columns (16 bytes) per thread
-    const long long total = d.B * Ho * Wo * chunks;
-    for (long long i = (long long)blockIdx.x * kT + threadIdx.x; i < total; i += (long long)gridDim.x * kT) {
-        const long long m = i / chunks;
+    const int K = d.kh * d.kw * (int)d.Cin, Cin = (int)d.Cin;
+    const I chunks = ldk / 8;                 // 8 columns (16 bytes) per thread
+    const I total = (I)d.B * Ho * Wo * chunks;
+    const I H = (I)d.H, W = (I)d.W;
+    for (I i = (I)blockIdx.x * kT + threadIdx.x; i < total; i += (I)gridDim.x * kT) {
+        const I m = i / chunks;
         const int k0 = (int)(i - m * chunks) * 8;
-        const long long wo = m % Wo, ho = (m / Wo) % Ho, b = m / (Wo * Ho);
+        const I wo = m % Wo, t1 = m / Wo, ho = t1 % Ho, b = t1 / Ho;
+        int t = k0 / Cin, c = k0 - t * Cin;
+        int r = t / d.kw, sx = t - r * d.kw;
         __align__(16) __nv_bfloat16 v[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-            const int k = k0 + e;
             __nv_bfloat16 x = __float2bfloat16_rn(0.0f);
-            if (k < K) {
-                const int c = k % (int)d.Cin, t = k / (int)d.Cin;
-                const int s = t % d.kw, r = t / d.kw;
-                const long long h = ho * d.stride_h - d.pad_h + r, w = wo * d.stride_w - d.pad_w + s;
-                if (h >= 0 && h < d.H && w >= 0 && w < d.W) x = X[((b * d.H + h) * d.W + w) * d.Cin + c];
+            if (k0 + e < K) {
+                const I h = ho * d.stride_h - d.pad_h + r, w = wo * d.stride_w - d.pad_w + sx;
+                if (h >= 0 && h < H && w >= 0 && w < W) x = X[((b * H + h) * W + w) * Cin + c];
             }
             v[e] = x;
+            if (++c == Cin) { c = 0; if (++sx == d.kw) { sx = 0; ++r; } }
         }
         *reinterpret_cast<uint4 *>(out + m * ldk + k0) = *reinterpret_cast<const uint4 *>(v);
     }
 }
 
-// ---- max pooling, window k x k, -inf padding; the first maximum in scan order wins
+__device__ __forceinline__ void unpack8(const uint4 v, float (&f)[8])
+{
+    const __nv_bfloat162 *p = reinterpret_cast<const __nv_bfloat162 *>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { const float2 t = __bfloat1622float2(p[i]); f[2 * i] = t.x; f[2 * i + 1] = t.y; }
+}
+__device__ __forceinline__ uint4 pack8(const float (&f)[8])
+{
+    uint4 v;
+    __nv_bfloat162 *p = reinterpret_cast<__nv_bfloat162 *>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) p[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+    return v;
+}
+
+// ---- max pooling, window k x k, -inf padding; the first maximum in scan order wins.
+// V = 8: eight channels per thread with 16-byte accesses (C % 8 == 0); V = 1: any C.
+template <typename I, int V>
 __global__ void __launch_bounds__(kT)
-maxpool_fwd_kernel(const __nv_bfloat16 *__restrict__ X, long long B, long long H, long long W, long long C,
-                   int k, int stride, int pad, long long Ho, long long Wo,
+maxpool_fwd_kernel(const __nv_bfloat16 *__restrict__ X, I B, I H, I W, I C,
+                   int k, int stride, int pad, I Ho, I Wo,
                    __nv_bfloat16 *__restrict__ Y, uint8_t *__restrict__ idx)
 {
-    const long long total = B * Ho * Wo * C;
-    for (long long i = (long long)blockIdx.x * kT + threadIdx.x; i < total; i += (long long)gridDim.x * kT) {
-        const long long c = i % C, wo = (i / C) % Wo, ho = (i / (C * Wo)) % Ho, b = i / (C * Wo * Ho);
-        float best = -INFINITY;
-        int arg = 0;
-        __nv_bfloat16 bestv = __float2bfloat16_rn(0.0f);
+    const I Cv = C / V;
+    const I total = B * Ho * Wo * Cv;
+    for (I i = (I)blockIdx.x * kT + threadIdx.x; i < total; i += (I)gridDim.x * kT) {
+        const I cv = i % Cv, t1 = i / Cv, wo = t1 % Wo, t2 = t1 / Wo, ho = t2 % Ho, b = t2 / Ho;
+        float best[V];
+        int arg[V];
+#pragma unroll
+        for (int e = 0; e < V; ++e) { best[e] = -INFINITY; arg[e] = 0; }
         for (int r = 0; r < k; ++r) {
-            const long long h = ho * stride - pad + r;
+            const I h = ho * stride - pad + r;
             if (h < 0 || h >= H) continue;
             for (int s = 0; s < k; ++s) {
-                const long long w = wo * stride - pad + s;
+                const I w = wo * stride - pad + s;
                 if (w < 0 || w >= W) continue;
-                const __nv_bfloat16 xv = X[((b * H + h) * W + w) * C + c];
-                const float x = __bfloat162float(xv);
-                if (x > best) { best = x; bestv = xv; arg = r * k + s; }
+                const __nv_bfloat16 *src = X + ((b * H + h) * W + w) * C + cv * V;
+                float x[V];
+                if (V == 8) {
+                    float t8[8];
+                    unpack8(__ldg(reinterpret_cast<const uint4 *>(src)), t8);
+#pragma unroll
+                    for (int e = 0; e < V; ++e) x[e] = t8[e];
+                } else {
+                    x[0] = __bfloat162float(src[0]);
+                }
+#pragma unroll
+                for (int e = 0; e < V; ++e)
+                    if (x[e] > best[e]) { best[e] = x[e]; arg[e] = r * k + s; }
             }
         }
-        Y[i] = bestv;
-        if (idx) idx[i] = (uint8_t)arg;
+        const I o = ((b * Ho + ho) * Wo + wo) * C + cv * V;
+        if (V == 8) {
+            float t8[8];
+#pragma unroll
+            for (int e = 0; e < V; ++e) t8[e] = best[e] == -INFINITY ? 0.0f : best[e];
+            *reinterpret_cast<uint4 *>(Y + o) = pack8(t8);     // exact: the values are bf16 already
+            if (idx) {
+                uint2 a;
+                a.x = arg[0] | (arg[1 % V] << 8) | (arg[2 % V] << 16) | (arg[3 % V] << 24);
+                a.y = arg[4 % V] | (arg[5 % V] << 8) | (arg[6 % V] << 16) | (arg[7 % V] << 24);
+                *reinterpret_cast<uint2 *>(idx + o) = a;
+            }
+        } else {
+            Y[o] = __float2bfloat16_rn(best[0] == -INFINITY ? 0.0f : best[0]);
+            if (idx) idx[o] = (uint8_t)arg[0];
+        }
     }
 }
 
 // gather form: an input pixel collects the gradient of every window whose maximum it was
+template <typename I, int V>
 __global__ void __launch_bounds__(kT)
-maxpool_bwd_kernel(const __nv_bfloat16 *__restrict__ dY, const uint8_t *__restrict__ idx, long long B, long long H,
-                   long long W, long long C, int k, int stride, int pad, long long Ho, long long Wo,
+maxpool_bwd_kernel(const __nv_bfloat16 *__restrict__ dY, const uint8_t *__restrict__ idx, I B, I H,
+                   I W, I C, int k, int stride, int pad, I Ho, I Wo,
                    __nv_bfloat16 *__restrict__ dX)
 {
-    const long long total = B * H * W * C;
-    for (long long i = (long long)blockIdx.x * kT + threadIdx.x; i < total; i += (long long)gridDim.x * kT) {
-        const long long c = i % C, w = (i / C) % W, h = (i / (C * W)) % H, b = i / (C * W * H);
-        float g = 0.0f;
+    const I Cv = C / V;
+    const I total = B * H * W * Cv;
+    for (I i = (I)blockIdx.x * kT + threadIdx.x; i < total; i += (I)gridDim.x * kT) {
+        const I cv = i % Cv, t1 = i / Cv, w = t1 % W, t2 = t1 / W, h = t2 % H, b = t2 / H;
+        float g[V];
+#pragma unroll
+        for (int e = 0; e < V; ++e) g[e] = 0.0f;
         for (int r = 0; r < k; ++r) {
-            const long long hn = h + pad - r;
+            const I hn = h + pad - r;
             if (hn < 0 || hn % stride != 0) continue;
-            const long long ho = hn / stride;
+            const I ho = hn / stride;
             if (ho >= Ho) continue;
             for (int s = 0; s < k; ++s) {
-                const long long wn = w + pad - s;
+                const I wn = w + pad - s;
                 if (wn < 0 || wn % stride != 0) continue;
-                const long long wo = wn / stride;
+                const I wo = wn / stride;
                 if (wo >= Wo) continue;
-                const long long o = ((b * Ho + ho) * Wo + wo) * C + c;
-                if (idx[o] == r * k + s) g += __bfloat162float(dY[o]);
+                const I o = ((b * Ho + ho) * Wo + wo) * C + cv * V;
+                const int want = r * k + s;
+                if (V == 8) {
+                    const uint2 a = __ldg(reinterpret_cast<const uint2 *>(idx + o));
+                    float t8[8];
+                    unpack8(__ldg(reinterpret_cast<const uint4 *>(dY + o)), t8);
+#pragma unroll
+                    for (int e = 0; e < V; ++e) {
+                        const int ai = ((e < 4 ? a.x : a.y) >> (8 * (e & 3))) & 0xFF;
+                        if (ai == want) g[e] += t8[e];
+                    }
+                } else {
+                    if (idx[o] == want) g[0] += __bfloat162float(dY[o]);
+                }
             }
         }
-        dX[i] = __float2bfloat16_rn(g);
+        const I o = ((b * H + h) * W + w) * C + cv * V;
+        if (V == 8) {
+            float t8[8];
+#pragma unroll
+            for (int e = 0; e < V; ++e) t8[e] = g[e];
+            *reinterpret_cast<uint4 *>(dX + o) = pack8(t8);
+        } else {
+            dX[o] = __float2bfloat16_rn(g[0]);
+        }
     }
 }
 
@@ -145,6 +217,34 @@ act_bwd_kernel(const __nv_bfloat16 *__restrict__ dY, const __nv_bfloat16 *__rest
     }
 }
 
+// eight elements per thread (C % 8 == 0, 16-byte aligned tensors)
+__global__ void __launch_bounds__(kT)
+act_bwd_vec_kernel(const uint4 *__restrict__ dY, const uint4 *__restrict__ Y, const float *__restrict__ scale,
+                   long long n8, int C8, uint4 *__restrict__ dZ, uint4 *__restrict__ dPre)
+{
+    for (long long i = (long long)blockIdx.x * kT + threadIdx.x; i < n8; i += (long long)gridDim.x * kT) {
+        float g[8];
+        unpack8(__ldg(dY + i), g);
+        if (Y) {
+            float y[8];
+            unpack8(__ldg(Y + i), y);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) if (!(y[e] > 0.0f)) g[e] = 0.0f;
+        }
+        if (dPre) dPre[i] = pack8(g);
+        if (dZ) {
+            if (scale) {
+                const int c0 = (int)(i % C8) * 8;
+                const float4 s0 = __ldg(reinterpret_cast<const float4 *>(scale + c0));
+                const float4 s1 = __ldg(reinterpret_cast<const float4 *>(scale + c0 + 4));
+                g[0] *= s0.x; g[1] *= s0.y; g[2] *= s0.z; g[3] *= s0.w;
+                g[4] *= s1.x; g[5] *= s1.y; g[6] *= s1.z; g[7] *= s1.w;
+            }
+            dZ[i] = pack8(g);
+        }
+    }
+}
+
 int pool_extent(long long in, int k, int stride, int pad) { return (int)((in + 2 * pad - k) / stride + 1); }
 
 }  // namespace
@@ -163,8 +263,13 @@ extern "C" int twn_im2col(const twn_conv_desc_t *d, const void *X, void *Xcol, i
     const long long Ho = (d->H + 2 * d->pad_h - d->kh) / d->stride_h + 1, Wo = (d->W + 2 * d->pad_w - d->kw) / d->stride_w + 1;
     TWN_REQUIRE(Ho > 0 && Wo > 0, TWN_ERR_INVALID_ARG);
     const long long items = d->B * Ho * Wo * (ldk / 8);
-    im2col_kernel<<<blocks_for(items, dev.sm_count), kT, 0, twn_cu(stream)>>>(
-        static_cast<const __nv_bfloat16 *>(X), *d, Ho, Wo, static_cast<__nv_bfloat16 *>(Xcol), ldk);
+    const bool small = items * 8 < 0x7fffffffLL && d->B * d->H * d->W * d->Cin < 0x7fffffffLL;
+    if (small)
+        im2col_kernel<int><<<blocks_for(items, dev.sm_count), kT, 0, twn_cu(stream)>>>(
+            static_cast<const __nv_bfloat16 *>(X), *d, (int)Ho, (int)Wo, static_cast<__nv_bfloat16 *>(Xcol), (int)ldk);
+    else
+        im2col_kernel<long long><<<blocks_for(items, dev.sm_count), kT, 0, twn_cu(stream)>>>(
+            static_cast<const __nv_bfloat16 *>(X), *d, Ho, Wo, static_cast<__nv_bfloat16 *>(Xcol), (long long)ldk);
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }
@@ -179,8 +284,20 @@ extern "C" int twn_maxpool2d_fwd(const void *X, int64_t B, int64_t H, int64_t W,
     if (rc != TWN_OK) return rc;
     const long long Ho = pool_extent(H, k, stride, pad), Wo = pool_extent(W, k, stride, pad);
     TWN_REQUIRE(Ho > 0 && Wo > 0, TWN_ERR_INVALID_ARG);
-    maxpool_fwd_kernel<<<blocks_for(B * Ho * Wo * C, dev.sm_count), kT, 0, twn_cu(stream)>>>(
-        static_cast<const __nv_bfloat16 *>(X), B, H, W, C, k, stride, pad, Ho, Wo, static_cast<__nv_bfloat16 *>(Y), argmax);
+    const __nv_bfloat16 *x = static_cast<const __nv_bfloat16 *>(X);
+    __nv_bfloat16 *y = static_cast<__nv_bfloat16 *>(Y);
+    const bool small = B * H * W * C < 0x7fffffffLL;
+    const bool vec = C % 8 == 0 && twn_aligned(X, 16) && twn_aligned(Y, 16) && twn_aligned(argmax, 8);
+    cudaStream_t s = twn_cu(stream);
+    if (vec && small)
+        maxpool_fwd_kernel<int, 8><<<blocks_for(B * Ho * Wo * C / 8, dev.sm_count), kT, 0, s>>>(
+            x, (int)B, (int)H, (int)W, (int)C, k, stride, pad, (int)Ho, (int)Wo, y, argmax);
+    else if (vec)
+        maxpool_fwd_kernel<long long, 8><<<blocks_for(B * Ho * Wo * C / 8, dev.sm_count), kT, 0, s>>>(
+            x, B, H, W, C, k, stride, pad, Ho, Wo, y, argmax);
+    else
+        maxpool_fwd_kernel<long long, 1><<<blocks_for(B * Ho * Wo * C, dev.sm_count), kT, 0, s>>>(
+            x, B, H, W, C, k, stride, pad, Ho, Wo, y, argmax);
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }
@@ -195,8 +312,20 @@ extern "C" int twn_maxpool2d_bwd(const void *dY, const uint8_t *argmax, int64_t 
     if (rc != TWN_OK) return rc;
     const long long Ho = pool_extent(H, k, stride, pad), Wo = pool_extent(W, k, stride, pad);
     TWN_REQUIRE(Ho > 0 && Wo > 0, TWN_ERR_INVALID_ARG);
-    maxpool_bwd_kernel<<<blocks_for(B * H * W * C, dev.sm_count), kT, 0, twn_cu(stream)>>>(
-        static_cast<const __nv_bfloat16 *>(dY), argmax, B, H, W, C, k, stride, pad, Ho, Wo, static_cast<__nv_bfloat16 *>(dX));
+    const __nv_bfloat16 *dy = static_cast<const __nv_bfloat16 *>(dY);
+    __nv_bfloat16 *dx = static_cast<__nv_bfloat16 *>(dX);
+    const bool small = B * H * W * C < 0x7fffffffLL;
+    const bool vec = C % 8 == 0 && twn_aligned(dY, 16) && twn_aligned(dX, 16) && twn_aligned(argmax, 8);
+    cudaStream_t s = twn_cu(stream);
+    if (vec && small)
+        maxpool_bwd_kernel<int, 8><<<blocks_for(B * H * W * C / 8, dev.sm_count), kT, 0, s>>>(
+            dy, argmax, (int)B, (int)H, (int)W, (int)C, k, stride, pad, (int)Ho, (int)Wo, dx);
+    else if (vec)
+        maxpool_bwd_kernel<long long, 8><<<blocks_for(B * H * W * C / 8, dev.sm_count), kT, 0, s>>>(
+            dy, argmax, B, H, W, C, k, stride, pad, Ho, Wo, dx);
+    else
+        maxpool_bwd_kernel<long long, 1><<<blocks_for(B * H * W * C, dev.sm_count), kT, 0, s>>>(
+            dy, argmax, B, H, W, C, k, stride, pad, Ho, Wo, dx);
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }
@@ -233,9 +362,16 @@ extern "C" int twn_act_bwd(const void *dY, const void *Y, const float *scale, in
     const int rc = twn_current_device(&dev);
     if (rc != TWN_OK) return rc;
     if (n == 0) return TWN_OK;
-    act_bwd_kernel<<<blocks_for(n, dev.sm_count), kT, 0, twn_cu(stream)>>>(
-        static_cast<const __nv_bfloat16 *>(dY), static_cast<const __nv_bfloat16 *>(Y), scale, n, C,
-        static_cast<__nv_bfloat16 *>(dZ), static_cast<__nv_bfloat16 *>(dPre));
+    const bool vec = C % 8 == 0 && n % 8 == 0 && twn_aligned(dY, 16) && twn_aligned(Y, 16) && twn_aligned(dZ, 16) &&
+                     twn_aligned(dPre, 16) && twn_aligned(scale, 16);
+    if (vec)
+        act_bwd_vec_kernel<<<blocks_for(n / 8, dev.sm_count), kT, 0, twn_cu(stream)>>>(
+            static_cast<const uint4 *>(dY), static_cast<const uint4 *>(Y), scale, n / 8, (int)(C / 8),
+            static_cast<uint4 *>(dZ), static_cast<uint4 *>(dPre));
+    else
+        act_bwd_kernel<<<blocks_for(n, dev.sm_count), kT, 0, twn_cu(stream)>>>(
+            static_cast<const __nv_bfloat16 *>(dY), static_cast<const __nv_bfloat16 *>(Y), scale, n, C,
+            static_cast<__nv_bfloat16 *>(dZ), static_cast<__nv_bfloat16 *>(dPre));
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }

@@ -92,6 +92,7 @@ struct ConvParams {
     // output path: 1 = the tile is staged in shared memory 32 pixels at a time and written with
     // TMA stores (box = 128 channels x sbw x sbh x sbb pixels); 0 = per-thread stores
     int tma_store, lg_sbw, lg_sbh;
+    int res_tma;                  // 1: the residual (bf16) is staged by TMA loads, three chunks deep
     Tap taps[kMaxTaps];
 };
 
@@ -107,19 +108,23 @@ struct __align__(1024) SmemLayout {
     unsigned long long acc_empty[2];       // epilogue -> MMA
     alignas(16) uint32_t pix_off[4][PIX];  // per epilogue warp: output element offset of a pixel, ~0 = skip
     alignas(128) float stage_out[2][32 * kChan];  // output staging for TMA stores: [32 pixels][128 channels]
+    alignas(128) __nv_bfloat16 stage_res[3][32 * kChan];  // residual staging, same chunk shape
+    unsigned long long res_full[3];
     uint32_t tmem_base;
     volatile int abort_flag;
     volatile int epi_ok;                   // outcome of the epilogue's wait, shared by its four warps
 };
 
-static_assert(offsetof(SmemLayout<128>, stage_out) % 128 == 0 && offsetof(SmemLayout<256>, stage_out) % 128 == 0 &&
+static_assert(offsetof(SmemLayout<128>, stage_res) % 128 == 0 && offsetof(SmemLayout<256>, stage_res) % 128 == 0 &&
+                  sizeof(SmemLayout<256>) + 1024 <= 232448 &&
+                  offsetof(SmemLayout<128>, stage_out) % 128 == 0 && offsetof(SmemLayout<256>, stage_out) % 128 == 0 &&
                   offsetof(SmemLayout<128>, pix_off) % 16 == 0 && offsetof(SmemLayout<256>, pix_off) % 16 == 0,
               "TMA and vector accesses need aligned shared-memory regions");
 
 template <int PIX>
 __global__ void __launch_bounds__(kThreadsConv, 1)
 tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
-             const __grid_constant__ ConvParams P)
+             const __grid_constant__ CUtensorMap map_r, const __grid_constant__ ConvParams P)
 {
     using L = SmemLayout<PIX>;
     constexpr int kStages = Cfg<PIX>::kStages, kSub = Cfg<PIX>::kSub, kAccBufs = Cfg<PIX>::kAccBufs;
@@ -146,6 +151,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
             mbar_init(&sm->acc_full[b], 1);
             mbar_init(&sm->acc_empty[b], 4);
         }
+        for (int b = 0; b < 3; ++b) mbar_init(&sm->res_full[b], 1);
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -347,12 +353,22 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
             float *const y32 = reinterpret_cast<float *>(P.Y) + n;
             __nv_bfloat16 *const y16 = reinterpret_cast<__nv_bfloat16 *>(P.Y) + n;
             const int p_w0 = twi << P.lgBW, p_h0 = thi << P.lgBH, p_b0 = tbi * (PIX >> (P.lgBW + P.lgBH));
+            const uint32_t g0 = lt * (PIX / 32);     // running chunk count: selects the residual buffer
+            auto res_load = [&](int c) {             // one thread: stage the residual of chunk c
+                const uint32_t g = g0 + c;
+                const int p0 = c * 32;
+                mbar_expect_tx(&sm->res_full[g % 3], 32 * kChan * 2);
+                tma_load_4d(sm->stage_res[g % 3], &map_r, &sm->res_full[g % 3], nt * kChan,
+                            (p_w0 + (p0 & BWm)) * P.osw, (p_h0 + ((p0 >> P.lgBW) & BHm)) * P.osh,
+                            p_b0 + (p0 >> (P.lgBW + P.lgBH)));
+            };
+            if (P.res_tma && ew == 0 && lane == 0) { res_load(0); res_load(1); }
 #pragma unroll 1
             for (int c = 0; c < PIX / 32; ++c) {
                 // the 32 offsets of this chunk: eight 16-byte broadcast loads, issued before the
                 // tensor-memory load is waited for (needed for per-thread stores and for the residual)
                 uint32_t off[32];
-                if (!P.tma_store || P.residual) {
+                if (!P.tma_store || (P.residual && !P.res_tma)) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         const uint4 o = *reinterpret_cast<const uint4 *>(pix_off + c * 32 + i * 4);
@@ -376,7 +392,27 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 // The inner loops are kept free of conditionals: one warp per scheduler runs this
                 // code, so every instruction fetched and issued here is exposed latency.
                 const float floor_v = P.relu ? 0.0f : -INFINITY;
-                if (P.residual) {
+                if (P.tma_store) {
+                    // staging buffer (c & 1) was last read by the store issued two chunks ago; the
+                    // residual of this chunk has landed.  One thread waits, all four warps follow.
+                    if (ew == 0 && lane == 0) {
+                        asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                        if (P.res_tma)
+                            sm->epi_ok = mbar_wait(&sm->res_full[(g0 + c) % 3], ((g0 + c) / 3) & 1u, abort_flag, P.status, 32) ? 1 : 0;
+                    }
+                    epi_bar();
+                    if (P.res_tma) {
+                        if (!sm->epi_ok) break;
+                        // the buffer two chunks ahead was last read in the previous chunk
+                        if (ew == 0 && lane == 0 && c + 2 < PIX / 32) res_load(c + 2);
+                    }
+                }
+                if (P.res_tma) {
+                    const __nv_bfloat16 *rs = sm->stage_res[(g0 + c) % 3] + q * 32 + lane;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        v[j] = __float_as_uint(fmaxf(fmaf(__uint_as_float(v[j]), sc, sf) + __bfloat162float(rs[j * kChan]), floor_v));
+                } else if (P.residual) {
                     // y = acc * scale' + shift + residual (residual fetched with the per-pixel offsets)
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
@@ -391,9 +427,6 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(fmaxf(fmaf(__uint_as_float(v[j]), sc, sf), floor_v));
                 }
                 if (P.tma_store) {
-                    // staging buffer (c & 1) was last read by the store issued two chunks ago
-                    if (ew == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                    epi_bar();
                     const int nl = q * 32 + lane;
                     if (out_bf16) {
                         __nv_bfloat16 *const st16 = reinterpret_cast<__nv_bfloat16 *>(sm->stage_out[c & 1]) + nl;
@@ -408,8 +441,8 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     epi_bar();
                     if (ew == 0 && lane == 0) {
                         const int p0 = c * 32;
-                        tma_store_4d(&map_y, sm->stage_out[c & 1], nt * kChan, p_w0 + (p0 & BWm),
-                                     p_h0 + ((p0 >> P.lgBW) & BHm), p_b0 + (p0 >> (P.lgBW + P.lgBH)));
+                        tma_store_4d(&map_y, sm->stage_out[c & 1], nt * kChan, (p_w0 + (p0 & BWm)) * P.osw,
+                                     (p_h0 + ((p0 >> P.lgBW) & BHm)) * P.osh, p_b0 + (p0 >> (P.lgBW + P.lgBH)));
                     }
                 } else if (n_ok) {
                     if (out_bf16) {
@@ -528,29 +561,46 @@ int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const twn_dev
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return TWN_ERR_INVALID_ARG;
     }
-    // output: TMA stores when the tile is a plain box of the output tensor and the pitch allows it
-    CUtensorMap map_y = map_x;
+    // output: TMA stores when the pitch allows it.  The virtual output grid may be embedded in
+    // the tensor with a stride and an offset (backward for data of a strided layer): the map
+    // then starts at the offset pixel and traverses with that stride.
+    // (the channel extent must be a whole number of 16-byte units: the store clips at that granularity)
+    CUtensorMap map_y = map_x, map_r = map_x;
     const int es = P.out_dtype == TWN_BF16 ? 2 : 4;
     P.tma_store = 0;
-    // (the channel extent must be a whole number of 16-byte units: the store clips at that granularity)
-    if (g.osh == 1 && g.osw == 1 && g.ooh == 0 && g.oow == 0 && (g.ldy * es) % 16 == 0 &&
-        ((long long)g.Cout * es) % 16 == 0 && (reinterpret_cast<uintptr_t>(P.Y) % 16) == 0) {
+    P.res_tma = 0;
+    const long long base_pix = (long long)g.ooh * g.OW + g.oow;
+    if ((g.ldy * es) % 16 == 0 && ((long long)g.Cout * es) % 16 == 0 && (reinterpret_cast<uintptr_t>(P.Y) % 16) == 0 &&
+        g.OW > g.oow && g.OH > g.ooh) {
         // a chunk of 32 consecutive tile pixels is a sub-box sbw x sbh x sbb of the tile box
         const int lg_sbw = P.lgBW < 5 ? P.lgBW : 5;
         const int lg_sbh = P.lgBH < 5 - lg_sbw ? P.lgBH : 5 - lg_sbw;
         const int lg_sbb = 5 - lg_sbw - lg_sbh;
         P.lg_sbw = lg_sbw; P.lg_sbh = lg_sbh;
-        cuuint64_t dims[4] = {(cuuint64_t)g.Cout, (cuuint64_t)g.OW, (cuuint64_t)g.OH, (cuuint64_t)g.Bv};
-        cuuint64_t strides[3] = {(cuuint64_t)g.ldy * es, (cuuint64_t)g.OW * g.ldy * es, (cuuint64_t)g.OH * g.OW * g.ldy * es};
-        cuuint32_t box[4] = {(cuuint32_t)kChan, 1u << lg_sbw, 1u << lg_sbh, 1u << lg_sbb};
-        cuuint32_t estr[4] = {1, 1, 1, 1};
-        if (enc(&map_y, es == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, P.Y, dims,
-                strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-                CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
-            P.tma_store = 1;
+        cuuint64_t dims[4] = {(cuuint64_t)g.Cout, (cuuint64_t)(g.OW - g.oow), (cuuint64_t)(g.OH - g.ooh), (cuuint64_t)g.Bv};
+        cuuint32_t box[4] = {(cuuint32_t)kChan, (cuuint32_t)((1 << lg_sbw) * g.osw), (cuuint32_t)((1 << lg_sbh) * g.osh), 1u << lg_sbb};
+        cuuint32_t estr[4] = {1, (cuuint32_t)g.osw, (cuuint32_t)g.osh, 1};
+        if (box[1] <= 256 && box[2] <= 256) {
+            cuuint64_t strides[3] = {(cuuint64_t)g.ldy * es, (cuuint64_t)g.OW * g.ldy * es, (cuuint64_t)g.OH * g.OW * g.ldy * es};
+            void *ybase = static_cast<char *>(P.Y) + base_pix * g.ldy * es;
+            if (enc(&map_y, es == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, ybase, dims,
+                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                    CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
+                P.tma_store = 1;
+            // a bf16 residual of the same geometry is staged the same way
+            if (P.tma_store && P.residual && P.res_dtype == TWN_BF16 && (g.ldy * 2) % 16 == 0 &&
+                ((long long)g.Cout * 2) % 16 == 0 && (reinterpret_cast<uintptr_t>(P.residual) % 16) == 0) {
+                cuuint64_t rstrides[3] = {(cuuint64_t)g.ldy * 2, (cuuint64_t)g.OW * g.ldy * 2, (cuuint64_t)g.OH * g.OW * g.ldy * 2};
+                void *rbase = const_cast<char *>(static_cast<const char *>(P.residual)) + base_pix * g.ldy * 2;
+                if (enc(&map_r, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, rbase, dims, rstrides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
+                    P.res_tma = 1;
+            }
+        }
     }
     const int grid = dev.sm_count < P.total_tiles ? dev.sm_count : P.total_tiles;
-    tconv_kernel<PIX><<<grid, kThreadsConv, smem_bytes, s>>>(map_x, map_y, P);
+    tconv_kernel<PIX><<<grid, kThreadsConv, smem_bytes, s>>>(map_x, map_y, map_r, P);
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }

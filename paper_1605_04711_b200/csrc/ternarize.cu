@@ -410,26 +410,27 @@ unpack_kernel(const uint32_t *__restrict__ packed, long long rows, long long col
 }
 
 // out row c, column t*Cout + o  <-  in row o, column t*Cin + c   (t = tap index)
+// (32-bit index arithmetic: a filter bank has far fewer than 2^31 codes)
 __global__ void __launch_bounds__(kThreads)
-transpose_codes_kernel(const uint32_t *__restrict__ in, long long ld_in, long long Cout, long long Cin,
-                       long long taps, uint32_t *__restrict__ out, long long ld_out)
+transpose_codes_kernel(const uint32_t *__restrict__ in, int ld_in, int Cout, int Cin,
+                       int taps, uint32_t *__restrict__ out, int ld_out)
 {
-    const long long wpr_out = ld_out >> 4, wpr_in = ld_in >> 4;
-    const long long total = Cin * wpr_out;
-    const long long cols_out = taps * Cout;
-    for (long long w = (long long)blockIdx.x * kThreads + threadIdx.x; w < total;
-         w += (long long)gridDim.x * kThreads) {
-        const long long c = w / wpr_out;
-        const long long j0 = (w - c * wpr_out) << 4;
+    const int wpr_out = ld_out >> 4, wpr_in = ld_in >> 4;
+    const int total = Cin * wpr_out;
+    const int cols_out = taps * Cout;
+    for (int w = blockIdx.x * kThreads + threadIdx.x; w < total; w += gridDim.x * kThreads) {
+        const int c = w / wpr_out;
+        const int j0 = (w - c * wpr_out) << 4;
+        int t = j0 / Cout, o = j0 - t * Cout;
         uint32_t word = 0;
+#pragma unroll
         for (int e = 0; e < 16; ++e) {
-            const long long j = j0 + e;
-            if (j < cols_out) {
-                const long long t = j / Cout, o = j - t * Cout;
-                const long long src = t * Cin + c;
-                const uint32_t f = (__ldg(in + o * wpr_in + (src >> 4)) >> field_pos((int)(src & 15))) & 3u;
+            if (j0 + e < cols_out) {
+                const int src = t * Cin + c;
+                const uint32_t f = (__ldg(in + (size_t)o * wpr_in + (src >> 4)) >> field_pos(src & 15)) & 3u;
                 word |= f << field_pos(e);
             }
+            if (++o == Cout) { o = 0; ++t; }
         }
         out[w] = word;
     }
@@ -607,8 +608,10 @@ extern "C" int twn_transpose_codes(const uint32_t *packed_fwd, int64_t ld_fwd,
     const int rc = twn_current_device(&dev);
     if (rc != TWN_OK) return rc;
     const long long words = d->Cin * (ld_bwd / 16);
+    TWN_REQUIRE(words < 0x7fffffffLL && d->Cout * (ld_fwd / 16) < 0x7fffffffLL && ld_fwd < 0x7fffffffLL &&
+                    ld_bwd < 0x7fffffffLL, TWN_ERR_INVALID_ARG);
     transpose_codes_kernel<<<grid_for(words, dev.sm_count), kThreads, 0, twn_cu(stream)>>>(
-        packed_fwd, ld_fwd, d->Cout, d->Cin, taps, packed_bwd, ld_bwd);
+        packed_fwd, (int)ld_fwd, (int)d->Cout, (int)d->Cin, (int)taps, packed_bwd, (int)ld_bwd);
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }
