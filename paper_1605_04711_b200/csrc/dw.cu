@@ -7,7 +7,9 @@
 // shared-memory descriptors), so the dZ tile and the tap-shifted X tile go from TMA straight
 // into the MMA: D[o, c] += dZ_tile^T * X_tile, 64 pixels per k-block.
 //
-// The output has few tiles (Cout/128 x taps x Cin/256) but a long reduction (up to 8e5 pixels),
+// One MMA covers up to four 64-channel column blocks of dW, taken in (tap, channel block)
+// order, so narrow layers (Cin = 64) process four taps per pass over the dZ tile.
+// The output has few tiles (Cout/128 x taps*Cin/256) but a long reduction (up to 8e5 pixels),
 // so the pixels are split across CTAs; each CTA writes its fp32 partial tile to the workspace
 // and a second kernel adds the partials in split order (deterministic, no atomics).
 //
@@ -31,9 +33,10 @@ constexpr int kDwAccCols = 256;
 struct DwTap { int16_t dh, dw; int32_t koff; };
 
 struct DwParams {
-    int n_otiles, n_taps, n_ctiles, splits, total_units;
+    int n_otiles, n_taps, n_groups, splits, total_units;
+    int cblocks, n_colblocks;    // 64-channel blocks per tap; column blocks = taps * cblocks, 4 per group
     int lgBW, lgBH, tw, th, tb, pix_tiles, tiles_per_split;
-    int sw, sh, ncb;
+    int sw, sh;
     int Cout, Cin;
     long long K;                 // row length of dW and of a partial
     long long split_stride;      // elements between partials of consecutive splits
@@ -75,12 +78,13 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
     tc_fence_after();
     const uint32_t tmem = sm->tmem_base;
 
-    // unit -> (o tile, tap, c tile, split); the split covers pixel tiles [p0, p1)
-    auto unit_range = [&](int u, int &ot, int &t, int &ct, int &sp, int &p0, int &p1) {
+    // unit -> (o tile, group of column blocks, split); the split covers pixel tiles [p0, p1)
+    auto unit_range = [&](int u, int &ot, int &gi, int &nb, int &sp, int &p0, int &p1) {
         sp = u % P.splits; u /= P.splits;
-        ct = u % P.n_ctiles; u /= P.n_ctiles;
-        t = u % P.n_taps;
-        ot = u / P.n_taps;
+        gi = u % P.n_groups;
+        ot = u / P.n_groups;
+        nb = P.n_colblocks - gi * kDwMaxCb;
+        if (nb > kDwMaxCb) nb = kDwMaxCb;
         p0 = sp * P.tiles_per_split;
         p1 = p0 + P.tiles_per_split;
         if (p1 > P.pix_tiles) p1 = P.pix_tiles;
@@ -91,11 +95,10 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            const uint32_t bytes = (2 + P.ncb) * kDwBlockBytes;
             for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
-                int ot, t, ct, sp, p0, p1;
-                unit_range(u, ot, t, ct, sp, p0, p1);
-                const DwTap tap = P.taps[t];
+                int ot, gi, nb, sp, p0, p1;
+                unit_range(u, ot, gi, nb, sp, p0, p1);
+                const uint32_t bytes = (2 + nb) * kDwBlockBytes;
                 for (int p = p0; p < p1; ++p, ++it) {
                     const int s = it % kDwStages;
                     const uint32_t ph = (it / kDwStages) & 1u;
@@ -108,20 +111,23 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
                     mbar_expect_tx(&sm->full[s], bytes);
                     tma_load_4d(sm->a[s][0], &map_dz, &sm->full[s], ot * 128, w0, h0, b0);
                     tma_load_4d(sm->a[s][1], &map_dz, &sm->full[s], ot * 128 + 64, w0, h0, b0);
-                    for (int j = 0; j < P.ncb; ++j)
-                        tma_load_4d(sm->b[s][j], &map_x, &sm->full[s], (ct * kDwMaxCb + j) * 64, w0 * P.sw + tap.dw,
+                    for (int j = 0; j < nb; ++j) {
+                        const int i = gi * kDwMaxCb + j, t = i / P.cblocks, cb = i - t * P.cblocks;
+                        const DwTap tap = P.taps[t];
+                        tma_load_4d(sm->b[s][j], &map_x, &sm->full[s], cb * 64, w0 * P.sw + tap.dw,
                                     h0 * P.sh + tap.dh, b0);
+                    }
                 }
             }
         }
     } else if (warp == 1) {
-        const uint32_t idesc = make_idesc_mn(128, 64 * P.ncb);
         uint32_t it = 0, lu = 0;     // lu counts the units that accumulate something
         bool ok = true;
         for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
-            int ot, t, ct, sp, p0, p1;
-            unit_range(u, ot, t, ct, sp, p0, p1);
+            int ot, gi, nb, sp, p0, p1;
+            unit_range(u, ot, gi, nb, sp, p0, p1);
             if (p1 <= p0) continue;                      // the epilogue writes zeros for an empty split
+            const uint32_t idesc = make_idesc_mn(128, 64 * nb);
             const int buf = lu & 1;
             if (!mbar_wait_warp(&sm->acc_empty[buf], ((lu >> 1) & 1u) ^ 1u, abort_flag, P.status, 0)) break;
             tc_fence_after();
@@ -148,17 +154,20 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
         const int q = warp & 3;
         uint32_t lu = 0;
         for (int u = blockIdx.x; u < P.total_units; u += gridDim.x) {
-            int ot, t, ct, sp, p0, p1;
-            unit_range(u, ot, t, ct, sp, p0, p1);
+            int ot, gi, nb, sp, p0, p1;
+            unit_range(u, ot, gi, nb, sp, p0, p1);
             const bool have = p1 > p0;
             const int buf = lu & 1;
             if (have && !mbar_wait_warp(&sm->acc_full[buf], (lu >> 1) & 1u, abort_flag, P.status, 32)) break;
             tc_fence_after();
             const int o = ot * 128 + q * 32 + lane;
-            const int c_base = ct * (kDwMaxCb * 64);
-            float *dst = P.partial + (long long)sp * P.split_stride + (long long)o * P.K + P.taps[t].koff + c_base;
+            float *row = P.partial + (long long)sp * P.split_stride + (long long)o * P.K;
 #pragma unroll 1
-            for (int c = 0; c < P.ncb * 2; ++c) {
+            for (int c = 0; c < nb * 2; ++c) {
+                // columns [32c, 32c+32) of the accumulator: half of column block c/2
+                const int i = gi * kDwMaxCb + (c >> 1), t = i / P.cblocks, cb = i - t * P.cblocks;
+                const int ch0 = cb * 64 + (c & 1) * 32;          // first input channel of this chunk
+                float *dst = row + P.taps[t].koff + ch0;
                 uint32_t v[32];
                 if (have) {
                     tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + buf * kDwAccCols + c * 32, v);
@@ -168,14 +177,14 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
                 }
                 if (o < P.Cout) {
-                    if (P.vec_ok && c_base + c * 32 + 32 <= P.Cin) {
+                    if (P.vec_ok && ch0 + 32 <= P.Cin) {
 #pragma unroll
                         for (int j = 0; j < 8; ++j)
-                            reinterpret_cast<uint4 *>(dst + c * 32)[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                            reinterpret_cast<uint4 *>(dst)[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
                     } else {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
-                            if (c_base + c * 32 + j < P.Cin) dst[c * 32 + j] = __uint_as_float(v[j]);
+                            if (ch0 + j < P.Cin) dst[j] = __uint_as_float(v[j]);
                     }
                 }
             }
@@ -264,10 +273,10 @@ int dw_plan(const twn_conv_desc_t *d, int sm_count, DwPlan *plan)
     P.pix_tiles = (int)best;
     P.n_otiles = (int)((d->Cout + 127) / 128);
     P.n_taps = d->kh * d->kw;
-    const int cblocks = (int)((d->Cin + 63) / 64);
-    P.n_ctiles = (cblocks + kDwMaxCb - 1) / kDwMaxCb;
-    P.ncb = cblocks < kDwMaxCb ? cblocks : kDwMaxCb;
-    const long long units = (long long)P.n_otiles * P.n_taps * P.n_ctiles;
+    P.cblocks = (int)((d->Cin + 63) / 64);
+    P.n_colblocks = P.n_taps * P.cblocks;
+    P.n_groups = (P.n_colblocks + kDwMaxCb - 1) / kDwMaxCb;
+    const long long units = (long long)P.n_otiles * P.n_groups;
     long long splits = (2LL * sm_count + units - 1) / units;
     if (splits > P.pix_tiles) splits = P.pix_tiles;
     if (splits < 1) splits = 1;

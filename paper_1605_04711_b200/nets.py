@@ -75,7 +75,9 @@ class TernaryNet:
         self.aux: dict[str, torch.Tensor] = {}
         self.grad: dict[str, torch.Tensor] = {}
         self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
-        self.ws_tern = torch.empty(twn.ternarize_workspace_bytes(), dtype=torch.uint8, device="cuda")
+        # the per-layer ternarizations are independent: they run on a few side streams, each layer
+        # with its own scratch
+        self.side_streams = [torch.cuda.Stream() for _ in range(4)]
         self.timed = None          # when a list: (kind, name, flops, start event, end event)
         H, W, C = in_shape
         self.act["input"] = torch.zeros((batch, H, W, C), dtype=torch.bfloat16, device="cuda")
@@ -99,6 +101,7 @@ class TernaryNet:
                 e["ld"] = twn.ld_for(L.K)
                 e["packed"] = torch.zeros((L.Cout, e["ld"] // 16), dtype=torch.int32, device="cuda")
                 e["stats"] = twn.new_stats()
+                e["ws"] = torch.empty(twn.ternarize_workspace_bytes(), dtype=torch.uint8, device="cuda")
                 if L.affine:
                     e["scale"] = _dev(dg.draw(self.seed, f"{self.name}.{L.name}.scale", L.Cout, "normal", 1.0, float(np.sqrt(0.1))))
                     e["shift"] = _dev(dg.draw(self.seed, f"{self.name}.{L.name}.shift", L.Cout, "normal", 0.0, float(np.sqrt(0.1))))
@@ -161,13 +164,19 @@ class TernaryNet:
 
     # ------------------------------------------------------------------ Algorithm 1, first loop
     def ternarize_all(self):
-        for L in self.layers.values():
+        main = torch.cuda.current_stream()
+        for st in self.side_streams:
+            st.wait_stream(main)
+        for i, L in enumerate(self.layers.values()):
             e = L.extra
-            self._call("ternarize", L.name, 0, lambda: twn.ternarize(
-                e["W"], self.delta_factor, e["stats"], e["packed"], e["ld"], None, self.ws_tern,
-                rows=L.Cout, cols=L.K))
-            if self.train and "packed_b" in e:
-                twn.transpose_codes(e["packed"], e["ld"], L.desc, e["packed_b"], e["ld_b"])
+            with torch.cuda.stream(self.side_streams[i % len(self.side_streams)]):
+                self._call("ternarize", L.name, 0, lambda: twn.ternarize(
+                    e["W"], self.delta_factor, e["stats"], e["packed"], e["ld"], None, e["ws"],
+                    rows=L.Cout, cols=L.K))
+                if self.train and "packed_b" in e:
+                    twn.transpose_codes(e["packed"], e["ld"], L.desc, e["packed_b"], e["ld_b"])
+        for st in self.side_streams:
+            main.wait_stream(st)
 
     # ------------------------------------------------------------------ forward
     def forward(self):
