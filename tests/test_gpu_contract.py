@@ -204,3 +204,26 @@ def test_bwd_data_adds_a_second_gradient_branch_through_the_residual():
     dXr, A = oracle.conv2d_bwd_data(oracle.conv_desc(B, H, W, Cin, Cout, k, s, p), dZ,
                                     codes.reshape(Cout, k, k, Cin), alpha)
     assert_within(dX.cpu().numpy(), dXr + other.astype(np.float64), A, alpha)
+
+
+SWEEP = [(K, N, M) for (K, N) in [(512, 512), (1152, 128), (2304, 256), (4608, 512), (4096, 4096)]
+         for M in (128, 1024, 4096, 16384)]
+
+
+@pytest.mark.parametrize("K,N,M", SWEEP)
+def test_gemm_sweep_full_sizes_on_sampled_rows(K, N, M):
+    """The GEMM sweep at its full sizes: the oracle evaluates 64 seeded rows plus every row next
+    to a 128/256-row tile boundary of the first and last tiles."""
+    alpha, codes, packed, ld, stats = ternarized(0, f"sweep{N}x{K}", N, K)
+    X = dg.draw_bf16(1, f"sweepx{M}x{K}", M * K, "normal").reshape(M, K)
+    Y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    twn.gemm(dev_bf16(X), K, packed, ld, stats, M, N, K, None, Y, N, status)
+    rng = np.random.default_rng(M + K)
+    rows = np.concatenate([rng.integers(0, M, 64), [0, 127, 128, 255, 256, M - 257, M - 256, M - 129, M - 128, M - 1]])
+    rows = np.unique(rows[(rows >= 0) & (rows < M)])
+    Yr, A = oracle.gemm(np.ascontiguousarray(X[rows]), codes, alpha)
+    assert twn.read_status(status) == 0
+    Yh = Y.cpu().numpy()
+    assert not np.isnan(Yh).any()
+    assert_within(Yh[rows], Yr, A, alpha)
