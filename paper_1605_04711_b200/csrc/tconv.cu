@@ -39,6 +39,26 @@
 #include "common.cuh"
 #include "tc_ptx.cuh"
 
+// Optional cycle counters per role (compiled in with -DTWN_PROFILE, read back with
+// twn_prof_read; absent from the normal build).
+#ifdef TWN_PROFILE
+__device__ long long g_prof[256 * 16];
+__device__ long long g_tl[4 * 1024];   // block 0: [0] TMA issue, [1] X seen by MMA, [2] A ready seen, [3] commit, per stage
+#define PROF_TL(row, it) do { if (blockIdx.x == 0 && (it) < 1024) g_tl[(row) * 1024 + (it)] = clock64(); } while (0)
+#define PROF_DECL(v) long long v = 0
+#define PROF_NOW() clock64()
+#define PROF_T(v) const long long v = clock64()
+#define PROF_ACC(acc, t0) acc += clock64() - (t0)
+#define PROF_OUT(slot, val) g_prof[blockIdx.x * 16 + (slot)] = (val)
+#else
+#define PROF_TL(row, it)
+#define PROF_DECL(v)
+#define PROF_NOW() 0
+#define PROF_T(v)
+#define PROF_ACC(acc, t0)
+#define PROF_OUT(slot, val)
+#endif
+
 namespace {
 
 constexpr int kChan = 128;          // output channels per tile (UMMA M)
@@ -171,6 +191,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
+            PROF_DECL(w_empty);
             const uint32_t block_bytes = kXBytes;
             for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
                 int pt = tile / P.n_tiles;
@@ -185,7 +206,10 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
                     const int nsb = (kbpt - st * kSub) < kSub ? (kbpt - st * kSub) : kSub;
+                    PROF_T(t_e);
                     if (!mbar_wait(&sm->empty[s], ph ^ 1u, abort_flag, P.status)) { ok = false; break; }
+                    PROF_ACC(w_empty, t_e);
+                    PROF_TL(0, it);
                     mbar_expect_tx(&sm->full[s], nsb * block_bytes);
                     for (int sb = 0; sb < nsb; ++sb) {
                         const Tap tap = P.taps[t];
@@ -194,6 +218,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     }
                 }
             }
+            PROF_OUT(5, w_empty);
         }
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer (whole warp, converged)
@@ -204,17 +229,27 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
             const uint64_t bdesc0 = smem_desc_sw128(smem_u32(sm->x[0][0]));
             uint32_t it = 0, lt = 0;
             bool ok = true;
+            PROF_DECL(w_acc); PROF_DECL(w_ready); PROF_DECL(w_issue);
+            PROF_T(t_start);
             for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x, ++lt) {
                 const int buf = lt % kAccBufs;
                 const uint32_t aph = (lt / kAccBufs) & 1u;
+                PROF_T(t_a);
                 if (!mbar_wait_warp(&sm->acc_empty[buf], aph ^ 1u, abort_flag, P.status, 0)) break;
+                PROF_ACC(w_acc, t_a);
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_acc + buf * PIX;
                 for (int st = 0; st < spt; ++st, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
-                    if (!mbar_wait_warp(&sm->ready_a[s], ph, abort_flag, P.status, 0) ||
-                        !mbar_wait_warp(&sm->full[s], ph, abort_flag, P.status, 0)) { ok = false; break; }
+                    PROF_T(t_r);
+                    if (!mbar_wait_warp(&sm->ready_a[s], ph, abort_flag, P.status, 0)) { ok = false; break; }
+                    PROF_ACC(w_ready, t_r);
+                    if (lane == 0) PROF_TL(2, it);
+                    PROF_T(t_x);
+                    if (!mbar_wait_warp(&sm->full[s], ph, abort_flag, P.status, 0)) { ok = false; break; }
+                    PROF_ACC(w_issue, t_x);
+                    if (lane == 0) PROF_TL(1, it);
                     tc_fence_after();
                     const uint64_t bdesc = bdesc0 + (uint64_t)(s * ((kSub * kXBytes) >> 4));
                     const uint32_t a_tmem = tmem_a + s * kAColsPerStage;
@@ -223,9 +258,11 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     if (kSub > 1 && kbpt - st * kSub > 1)
                         tc_mma_block<false>(d_tmem, a_tmem + kAColsPerBlock, bdesc + (kXBytes >> 4), idesc);
                     tc_commit(&sm->empty[s]);
+                    if (lane == 0) PROF_TL(3, it);
                 }
                 if (ok) tc_commit(&sm->acc_full[buf]);
             }
+            if (lane == 0) { PROF_OUT(0, PROF_NOW() - t_start); PROF_OUT(1, w_acc); PROF_OUT(2, w_issue); PROF_OUT(3, w_ready); PROF_OUT(4, (long long)it); }
         }
     } else if (warp < kFirstEpiWarp) {
         // ------------------------------------------------ decode: codes -> bf16 -> tensor memory
@@ -269,6 +306,8 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
             for (int i = 0; i < steps; ++i)
                 if (++st >= spt) { st = 0; tile += gridDim.x; }
         };
+        PROF_DECL(w_full);
+        PROF_T(t_dec);
         if (spt > 0) {
             int tile0 = blockIdx.x, st0 = 0;
             advance(tile0, st0, set);                       // this group's first stage
@@ -284,7 +323,9 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 const uint32_t ph = (it / kStages) & 1u;
                 const int nsb = (kbpt - st0 * kSub) < kSub ? (kbpt - st0 * kSub) : kSub;
                 // the MMAs that read this slot's previous contents have completed
+                PROF_T(t_f);
                 if (!mbar_wait_warp(&sm->empty[s], ph ^ 1u, abort_flag, P.status, 32)) break;
+                PROF_ACC(w_full, t_f);
                 tc_fence_after();
 #pragma unroll
                 for (int sb = 0; sb < kSub; ++sb) {
@@ -308,6 +349,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 it += kDecodeSets;
             }
         }
+        if (warp == 2 && lane == 0) { PROF_OUT(6, w_full); PROF_OUT(8, PROF_NOW() - t_dec); }
     } else {
         // ------------------------------------------------ epilogue
         const int q = warp & 3;
@@ -317,6 +359,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         const int BWm = (1 << P.lgBW) - 1, BHm = (1 << P.lgBH) - 1;
         const bool out_bf16 = P.out_dtype == TWN_BF16, res_bf16 = P.res_dtype == TWN_BF16;
         uint32_t lt = 0;
+        PROF_DECL(e_wait); PROF_DECL(e_drain);
         for (int tile = blockIdx.x; tile < P.total_tiles; tile += gridDim.x, ++lt) {
             const int nt = tile % P.n_tiles;
             int pt = tile / P.n_tiles;
@@ -341,6 +384,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
             }
             __syncwarp();
             const int buf = lt % kAccBufs;
+            PROF_T(t_w);
             if (kbpt > 0) {
                 // one thread waits for the accumulator; the four warps then decide together, so that
                 // they always execute the same number of named barriers
@@ -349,6 +393,8 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 epi_bar();
                 if (!sm->epi_ok) break;
             }
+            PROF_ACC(e_wait, t_w);
+            PROF_T(t_d);
             tc_fence_after();
             float *const y32 = reinterpret_cast<float *>(P.Y) + n;
             __nv_bfloat16 *const y16 = reinterpret_cast<__nv_bfloat16 *>(P.Y) + n;
@@ -384,6 +430,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&sm->acc_empty[buf]);
+                        PROF_ACC(e_drain, t_d);
                     }
                 } else {
 #pragma unroll
@@ -458,6 +505,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
             }
             __syncwarp();
         }
+        if (ew == 0 && lane == 0) { PROF_OUT(9, e_wait); PROF_OUT(10, e_drain); PROF_OUT(11, (long long)lt); }
         // all bulk stores of this thread have been written before the block may exit
         if (P.tma_store && ew == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
@@ -792,3 +840,15 @@ extern "C" int twn_conv2d_bwd_data(const twn_conv_desc_t *d, const void *dZ, con
         }
     return TWN_OK;
 }
+
+#ifdef TWN_PROFILE
+extern "C" int twn_tl_read(long long *host) { return cudaMemcpyFromSymbol(host, g_tl, sizeof(long long) * 4 * 1024); }
+extern "C" int twn_prof_read(long long *host, int zero)
+{
+    if (zero) {
+        static long long z[256 * 16];
+        return cudaMemcpyToSymbol(g_prof, z, sizeof(z));
+    }
+    return cudaMemcpyFromSymbol(host, g_prof, sizeof(long long) * 256 * 16);
+}
+#endif
