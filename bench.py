@@ -173,7 +173,7 @@ class NetWorkload:
     metric = "images/s"
     unit = "images/s"
     dtype = "bf16"
-    default_steps = 50
+    default_steps = 200
 
     def __init__(self, kind):
         self.kind = kind

@@ -690,10 +690,15 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     P.status = dev_status;
     for (int t = 0; t < g.n_taps; ++t) P.taps[t] = g.taps[t];
 
-    // 256-pixel tiles once they still fill the machine; otherwise 128-pixel tiles
+    // Tile shape by a cost model fitted to measured launches (cycles per round of tiles):
+    //   128 pixels: 2000 + 930 per k-block (epilogue overlapped, 64-cycle MMAs)
+    //   256 pixels: 14000 + 1100 per k-block (epilogue exposed, twice the work per k-block)
     int a, b;
-    const long long tiles256 = pick_tile(g, 256, &a, &b) * P.n_tiles;
-    if (tiles256 >= dev.sm_count) return launch_conv_t<256>(g, P, X, dev, enc, s);
+    const long long kb = (long long)P.n_taps * P.n_cblk;
+    const long long t128 = pick_tile(g, 128, &a, &b) * P.n_tiles, t256 = pick_tile(g, 256, &a, &b) * P.n_tiles;
+    const long long r128 = (t128 + dev.sm_count - 1) / dev.sm_count, r256 = (t256 + dev.sm_count - 1) / dev.sm_count;
+    const long long c128 = r128 * (2000 + 930 * kb), c256 = r256 * (14000 + 1100 * kb);
+    if (c256 < c128) return launch_conv_t<256>(g, P, X, dev, enc, s);
     return launch_conv_t<128>(g, P, X, dev, enc, s);
 }
 
