@@ -109,10 +109,11 @@ size_t twn_ternarize_workspace_bytes(void);
  * packed   uint32 [rows][ld_codes/16].  A field is two bits: 00 = 0, 01 = +1,
  *          11 = -1 (10 is never written).  Code j of a row lives in word j/16;
  *          inside the word the even elements fill the low half-word and the odd
- *          elements the high half-word: element e = j%16 is at bit position
- *          2*(e/2) + 16*(e%2).  (The paper fixes no encoding; this one lets a
- *          shift, one logic op and one bf16x2 subtract turn two fields into a
- *          pair of bf16 tensor-core operands.)
+ *          elements the high half-word, each from its top bits down: element
+ *          e = j%16 is at bit position 14 - 2*(e/2) + 16*(e%2).  (The paper fixes
+ *          no encoding; with this one a left shift by 2*(e/2) and one mask turn
+ *          the fields of elements e, e+1 into the sign and top exponent bit of a
+ *          pair of bf16 tensor-core operands, +-2 or 0.)
  *          ld_codes is a multiple of 64 (rows start 16-byte aligned),
  *          ld_codes >= cols; the padding is written as 00.  16-byte aligned.
  * codes_i8 optional int8 [rows, cols] copy of the codes (16-byte aligned), or NULL.

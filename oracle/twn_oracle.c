@@ -157,11 +157,11 @@ double ref_objective(const float *W, const int8_t *codes, double alpha, int64_t 
  *           (10 is never produced);
  *   word    a row is cut into groups of 16 codes, one 32-bit word per group.
  *           Inside a group the even elements fill the low half-word and the
- *           odd elements the high half-word: element e (0..15) sits at bit
- *           position 2*(e/2) + 16*(e%2);
+ *           odd elements the high half-word, each from its top bits down:
+ *           element e (0..15) sits at bit position 14 - 2*(e/2) + 16*(e%2);
  *   row     ld_codes/16 words (ld_codes a multiple of 16 here), padded with 00.
  * ---------------------------------------------------------------------- */
-static int field_pos(int64_t e) { return (int)(2 * (e / 2) + 16 * (e % 2)); }
+static int field_pos(int64_t e) { return (int)(14 - 2 * (e / 2) + 16 * (e % 2)); }
 
 int ref_pack(const int8_t *codes, int64_t rows, int64_t cols, int64_t ld_codes, uint32_t *packed)
 {

@@ -75,6 +75,8 @@ __device__ __forceinline__ bool mbar_wait(void *bar, uint32_t parity, volatile i
 __device__ __forceinline__ bool mbar_wait_warp(void *bar, uint32_t parity, volatile int *abort_flag, int32_t *status,
                                                uint32_t backoff_ns = 64)
 {
+    // fast path: the phase is already over (one probe by the whole warp, one vote)
+    if (__all_sync(0xffffffffu, mbar_try(bar, parity))) return true;
     int ok = 1;
     if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status, backoff_ns) ? 1 : 0;
     ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -142,6 +144,16 @@ __device__ __forceinline__ void tc_mma_block(uint32_t d_tmem, uint32_t a_tmem, u
     tc_mma_ts<true>(d_tmem, a_tmem + 24, b_desc + 6, idesc);
 }
 
+// Read-only global loads that the compiler neither moves nor wraps in control flow.
+__device__ __forceinline__ void ld_nc_v4(uint4 &v, const uint32_t *p)
+{
+    asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+}
+__device__ __forceinline__ void ld_nc_u32(uint32_t &v, const uint32_t *p)
+{
+    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v) : "l"(p));
+}
+
 // K-major, 128-byte swizzled operand tile: rows of 128 bytes, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr)
 {
@@ -191,15 +203,15 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
         : "memory");
 }
 
-// Two 2-bit fields (bits 1:0 and 17:16 of x) -> two exact bf16 values in {-1, 0, +1}.
-// field ^ 2 is the field's value + 2 (00 -> 2, 01 -> 3, 11 -> 1); or-ing it into the
-// mantissa of 128.0 gives 130 + value, and subtracting 130.0 leaves the value.
-__device__ __forceinline__ uint32_t fields_to_bf16x2(uint32_t x)
+// Element pair j (0..7) of a packed code word -> two bf16 values in {-2, 0, +2}.  The pair's
+// fields sit 2*j bits below the top of the two half-words (bit 0 of a field = non-zero, bit 1 =
+// sign); shifted to the top they are the sign and the high exponent bit of a bf16, and
+// 0x4000 is 2.0.  The factor 2 is taken out again with the scale of the epilogue, so a decoded
+// pair costs one shift and one mask.  (Field 10 would read as -0.)
+constexpr float kDecodedUnit = 2.0f;
+__device__ __forceinline__ uint32_t pair_to_bf16x2(uint32_t w, int j)
 {
-    const uint32_t t = (x & 0x00030003u) ^ 0x43024302u;
-    uint32_t r;
-    asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(t), "r"(0x43024302u));
-    return r;
+    return (w << (2 * j)) & 0xC000C000u;
 }
 
 // ---------------------------------------------------------------- the kernel

@@ -37,21 +37,25 @@
 #include <cstddef>
 
 #include "common.cuh"
+#include <cstdlib>
 #include "tc_ptx.cuh"
 
 // Optional cycle counters per role (compiled in with -DTWN_PROFILE, read back with
 // twn_prof_read; absent from the normal build).
 #ifdef TWN_PROFILE
-__device__ long long g_prof[256 * 16];
+__device__ long long g_prof[256 * 32];
+__device__ long long g_tl2[4 * 1024];  // block 0, first decode warp: [0] slot free seen, [1] stores issued, [2] arrived, [3] next codes fetched
+#define PROF_TL2(row, it) do { if (blockIdx.x == 0 && warp == 2 && lane == 0 && (it) < 1024) g_tl2[(row) * 1024 + (it)] = clock64(); } while (0)
 __device__ long long g_tl[4 * 1024];   // block 0: [0] TMA issue, [1] X seen by MMA, [2] A ready seen, [3] commit, per stage
 #define PROF_TL(row, it) do { if (blockIdx.x == 0 && (it) < 1024) g_tl[(row) * 1024 + (it)] = clock64(); } while (0)
 #define PROF_DECL(v) long long v = 0
 #define PROF_NOW() clock64()
 #define PROF_T(v) const long long v = clock64()
 #define PROF_ACC(acc, t0) acc += clock64() - (t0)
-#define PROF_OUT(slot, val) g_prof[blockIdx.x * 16 + (slot)] = (val)
+#define PROF_OUT(slot, val) g_prof[blockIdx.x * 32 + (slot)] = (val)
 #else
 #define PROF_TL(row, it)
+#define PROF_TL2(row, it)
 #define PROF_DECL(v)
 #define PROF_NOW() 0
 #define PROF_T(v)
@@ -63,10 +67,11 @@ namespace {
 
 constexpr int kChan = 128;          // output channels per tile (UMMA M)
 constexpr int kBlockK = 64;         // reduction elements per k-block (128 bytes of bf16)
-constexpr int kDecodeSets = 2;      // groups of 4 decode warps; a group takes every other stage
+constexpr int kDecodeSets = 1;      // groups of 4 decode warps; a group takes every other stage
 constexpr int kFirstEpiWarp = 2 + 4 * kDecodeSets;
 constexpr int kThreadsConv = 32 * (kFirstEpiWarp + 4);
 constexpr int kMaxTaps = 64;
+constexpr int kWordTab = 512;       // k-blocks per tile whose code offsets are tabulated in shared memory
 constexpr int kAColsPerBlock = kBlockK / 2;    // 32 columns of bf16 pairs per k-block
 constexpr uint32_t kTmemCols = 512;
 
@@ -122,7 +127,7 @@ struct __align__(1024) SmemLayout {
     static constexpr int kXBytes = PIX * kBlockK * 2;
     uint8_t x[kStages][kSub][kXBytes];           // swizzled activation tiles
     unsigned long long full[kStages];      // TMA -> MMA: activation tile landed
-    unsigned long long ready_a[kStages];   // decode -> MMA: weights of the stage are in tensor memory
+    unsigned long long ready_a[8];         // decode -> MMA: weights of the stage / k-block are in tensor memory
     unsigned long long empty[kStages];     // MMA commit -> TMA and decode: both operand slots are free
     unsigned long long acc_full[2];        // MMA commit -> epilogue
     unsigned long long acc_empty[2];       // epilogue -> MMA
@@ -130,6 +135,7 @@ struct __align__(1024) SmemLayout {
     alignas(128) float stage_out[2][32 * kChan];  // output staging for TMA stores: [32 pixels][128 channels]
     alignas(128) __nv_bfloat16 stage_res[3][32 * kChan];  // residual staging, same chunk shape
     unsigned long long res_full[3];
+    uint32_t kword[kWordTab];              // first code word of k-block u in a packed row, u < kWordTab
     uint32_t tmem_base;
     volatile int abort_flag;
     volatile int epi_ok;                   // outcome of the epilogue's wait, shared by its four warps
@@ -164,9 +170,9 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&sm->full[s], 1);
-            mbar_init(&sm->ready_a[s], 4);
             mbar_init(&sm->empty[s], 1);
         }
+        for (int s = 0; s < 8; ++s) mbar_init(&sm->ready_a[s], 4);
         for (int b = 0; b < 2; ++b) {
             mbar_init(&sm->acc_full[b], 1);
             mbar_init(&sm->acc_empty[b], 4);
@@ -174,6 +180,12 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         for (int b = 0; b < 3; ++b) mbar_init(&sm->res_full[b], 1);
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // code-word offset of every k-block, in the order the k-blocks are consumed: taps outer,
+    // channel blocks inner
+    for (int u = threadIdx.x; u < kbpt && u < kWordTab; u += kThreadsConv) {
+        const int t = u / P.n_cblk, cb = u - t * P.n_cblk;
+        sm->kword[u] = (uint32_t)(P.taps[t].koff >> 4) + cb * (kBlockK / 16);
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)), "r"(kTmemCols) : "memory");
@@ -275,57 +287,82 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         const int row = q * 32 + lane;          // channel row inside the tile
         const uint32_t lane_base = tmem_a + ((uint32_t)(q * 32) << 16);
 
+        // Code words are fetched with explicit non-coherent loads straight into the registers that
+        // hold them until they are decoded, from addresses clamped into the packed matrix: no
+        // branch and no register copy stands between a load and its use, so its latency stays
+        // hidden.  What a clamped fetch returns is either never decoded (no such stage) or feeds
+        // channels that are never stored, or multiplies activations that the TMA zero-fills.
         struct Codes { uint4 v[kSub]; };
-        auto fetch = [&](int tile, int st) -> Codes {
-            Codes c;
-#pragma unroll
-            for (int sb = 0; sb < kSub; ++sb) c.v[sb] = make_uint4(0u, 0u, 0u, 0u);
-            if (tile >= P.total_tiles) return c;
-            const long long n = (long long)(tile % P.n_tiles) * kChan + row;
-            if (n >= P.Cout) return c;
-            const uint32_t *rowp = P.T + n * P.wpr;
+        auto fetch = [&](Codes &c, const uint32_t *rowp, int st) {
 #pragma unroll
             for (int sb = 0; sb < kSub; ++sb) {
-                const int u = st * kSub + sb;
-                if (u >= kbpt) break;
-                const int t = u / P.n_cblk, cb = u - t * P.n_cblk;
-                const long long word = (P.taps[t].koff >> 4) + cb * (kBlockK / 16);
-                if (P.codes_aligned) {
-                    c.v[sb] = __ldg(reinterpret_cast<const uint4 *>(rowp + word));
+                int u = st * kSub + sb;
+                u = u < kbpt ? u : kbpt - 1;
+                long long word;
+                if (kbpt <= kWordTab) {
+                    word = sm->kword[u];
                 } else {
-                    uint32_t w4[4];
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) w4[g] = (word + g < P.wpr) ? __ldg(rowp + word + g) : 0u;
-                    c.v[sb] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                    const int t = u / P.n_cblk, cb = u - t * P.n_cblk;
+                    word = (P.taps[t].koff >> 4) + cb * (kBlockK / 16);
+                }
+                if (P.codes_aligned) {
+                    ld_nc_v4(c.v[sb], rowp + word);
+                } else {
+                    const long long last = P.wpr - 1;
+                    ld_nc_u32(c.v[sb].x, rowp + (word + 0 < last ? word + 0 : last));
+                    ld_nc_u32(c.v[sb].y, rowp + (word + 1 < last ? word + 1 : last));
+                    ld_nc_u32(c.v[sb].z, rowp + (word + 2 < last ? word + 2 : last));
+                    ld_nc_u32(c.v[sb].w, rowp + (word + 3 < last ? word + 3 : last));
                 }
             }
-            return c;
         };
         // position of this group's next stages: (tile, st), advanced kDecodeSets stages at a time
         auto advance = [&](int &tile, int &st, int steps) {
             for (int i = 0; i < steps; ++i)
                 if (++st >= spt) { st = 0; tile += gridDim.x; }
         };
-        PROF_DECL(w_full);
+        // the fetch position also carries its row of the packed matrix: the channel tile of
+        // `tile` is tile mod n_tiles, stepped without a division (one sits in the way of every
+        // stage otherwise); rows past Cout read the last row and are never stored
+        const int nt_step = (int)(gridDim.x % (unsigned)P.n_tiles);
+        auto row_ptr = [&](int nt) -> const uint32_t * {
+            long long n = (long long)nt * kChan + row;
+            n = n < P.Cout ? n : P.Cout - 1;
+            return P.T + n * P.wpr;
+        };
+        auto advance_f = [&](int &tile, int &st, int &nt, const uint32_t *&rowp, int steps) {
+            for (int i = 0; i < steps; ++i)
+                if (++st >= spt) {
+                    st = 0; tile += gridDim.x;
+                    nt += nt_step; if (nt >= P.n_tiles) nt -= P.n_tiles;
+                    rowp = row_ptr(nt);
+                }
+        };
+        PROF_DECL(w_full); PROF_DECL(d_alu); PROF_DECL(d_wst); PROF_DECL(d_fetch); PROF_DECL(d_st);
         PROF_T(t_dec);
         if (spt > 0) {
-            int tile0 = blockIdx.x, st0 = 0;
-            advance(tile0, st0, set);                       // this group's first stage
-            int tile1 = tile0, st1 = st0;
-            advance(tile1, st1, kDecodeSets);
-            int tile2 = tile1, st2 = st1;
-            advance(tile2, st2, kDecodeSets);
-            Codes cur = fetch(tile0, st0), nxt = fetch(tile1, st1);
+            // three code buffers in rotation, each refilled right after use for the stage three of
+            // this group's stages ahead: no register is copied while its load is still in flight
+            int tile_c = blockIdx.x, st_c = 0;               // the stage being decoded
+            advance(tile_c, st_c, set);
+            int tile_f = tile_c, st_f = st_c;                // the stage being fetched
+            int nt_f = tile_f % P.n_tiles;
+            const uint32_t *rowp_f = row_ptr(nt_f);
+            Codes c0, c1, c2;
+            fetch(c0, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, kDecodeSets);
+            fetch(c1, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, kDecodeSets);
+            fetch(c2, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, kDecodeSets);
             uint32_t it = set;
-            while (tile0 < P.total_tiles) {
-                const Codes nn = fetch(tile2, st2);         // two stages ahead
+            auto decode_stage = [&](const Codes &cur) -> bool {
                 const int s = it % kStages;
                 const uint32_t ph = (it / kStages) & 1u;
-                const int nsb = (kbpt - st0 * kSub) < kSub ? (kbpt - st0 * kSub) : kSub;
+                const int nsb = (kbpt - st_c * kSub) < kSub ? (kbpt - st_c * kSub) : kSub;
                 // the MMAs that read this slot's previous contents have completed
                 PROF_T(t_f);
-                if (!mbar_wait_warp(&sm->empty[s], ph ^ 1u, abort_flag, P.status, 32)) break;
+                if (!mbar_wait_warp(&sm->empty[s], ph ^ 1u, abort_flag, P.status, 32)) return false;
                 PROF_ACC(w_full, t_f);
+                PROF_TL2(0, it);
+                PROF_T(t_alu);
                 tc_fence_after();
 #pragma unroll
                 for (int sb = 0; sb < kSub; ++sb) {
@@ -335,31 +372,46 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
 #pragma unroll
                         for (int g = 0; g < 4; ++g)
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) out[g * 8 + e] = fields_to_bf16x2(wv[g] >> (2 * e));
+                            for (int e = 0; e < 8; ++e) out[g * 8 + e] = pair_to_bf16x2(wv[g], e);
+                        PROF_T(t_st);
                         tmem_st32(lane_base + s * kAColsPerStage + sb * kAColsPerBlock, out);
+                        PROF_ACC(d_st, t_st);
                     }
                 }
+                PROF_ACC(d_alu, t_alu);
+                PROF_TL2(1, it);
+                PROF_T(t_wst);
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sm->ready_a[s]);
-                cur = nxt; nxt = nn;
-                tile0 = tile1; st0 = st1; tile1 = tile2; st1 = st2;
-                advance(tile2, st2, kDecodeSets);
+                PROF_ACC(d_wst, t_wst);
+                PROF_TL2(2, it);
+                advance(tile_c, st_c, kDecodeSets);
                 it += kDecodeSets;
+                return true;
+            };
+            while (true) {
+                if (tile_c >= P.total_tiles || !decode_stage(c0)) break;
+                { PROF_T(t0); fetch(c0, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, kDecodeSets); PROF_ACC(d_fetch, t0); PROF_TL2(3, it - kDecodeSets); }
+                if (tile_c >= P.total_tiles || !decode_stage(c1)) break;
+                { PROF_T(t1); fetch(c1, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, kDecodeSets); PROF_ACC(d_fetch, t1); }
+                if (tile_c >= P.total_tiles || !decode_stage(c2)) break;
+                { PROF_T(t2); fetch(c2, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, kDecodeSets); PROF_ACC(d_fetch, t2); }
             }
         }
-        if (warp == 2 && lane == 0) { PROF_OUT(6, w_full); PROF_OUT(8, PROF_NOW() - t_dec); }
+        if (warp == 2 && lane == 0) { PROF_OUT(6, w_full); PROF_OUT(8, PROF_NOW() - t_dec); PROF_OUT(12, d_alu); PROF_OUT(13, d_wst); PROF_OUT(14, d_fetch); PROF_OUT(15, d_st); }
     } else {
         // ------------------------------------------------ epilogue
         const int q = warp & 3;
         const int ew = warp - kFirstEpiWarp;
         uint32_t *pix_off = sm->pix_off[ew];
-        const float alpha = P.alpha ? (float)(*P.alpha) : 1.0f;
+        // decoded weights are +-2, so half of alpha scales the accumulators
+        const float alpha = (P.alpha ? (float)(*P.alpha) : 1.0f) * (1.0f / kDecodedUnit);
         const int BWm = (1 << P.lgBW) - 1, BHm = (1 << P.lgBH) - 1;
         const bool out_bf16 = P.out_dtype == TWN_BF16, res_bf16 = P.res_dtype == TWN_BF16;
         uint32_t lt = 0;
-        PROF_DECL(e_wait); PROF_DECL(e_drain);
+        PROF_DECL(e_wait); PROF_DECL(e_drain); PROF_DECL(e_ld); PROF_DECL(e_grp); PROF_DECL(e_math); PROF_DECL(e_st);
         for (int tile = blockIdx.x; tile < P.total_tiles; tile += gridDim.x, ++lt) {
             const int nt = tile % P.n_tiles;
             int pt = tile / P.n_tiles;
@@ -422,6 +474,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     }
                 }
                 uint32_t v[32];
+                PROF_T(t_ld);
                 if (kbpt > 0) {
                     tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + buf * PIX + c * 32, v);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -439,6 +492,8 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 // The inner loops are kept free of conditionals: one warp per scheduler runs this
                 // code, so every instruction fetched and issued here is exposed latency.
                 const float floor_v = P.relu ? 0.0f : -INFINITY;
+                PROF_ACC(e_ld, t_ld);
+                PROF_T(t_grp);
                 if (P.tma_store) {
                     // staging buffer (c & 1) was last read by the store issued two chunks ago; the
                     // residual of this chunk has landed.  One thread waits, all four warps follow.
@@ -454,6 +509,8 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                         if (ew == 0 && lane == 0 && c + 2 < PIX / 32) res_load(c + 2);
                     }
                 }
+                PROF_ACC(e_grp, t_grp);
+                PROF_T(t_math);
                 if (P.res_tma) {
                     const __nv_bfloat16 *rs = sm->stage_res[(g0 + c) % 3] + q * 32 + lane;
 #pragma unroll
@@ -478,14 +535,23 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     if (out_bf16) {
                         __nv_bfloat16 *const st16 = reinterpret_cast<__nv_bfloat16 *>(sm->stage_out[c & 1]) + nl;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) st16[j * kChan] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                        for (int j = 0; j < 32; j += 2) {
+                            // one packed conversion per two pixels (the scalar one runs at a fraction of its rate)
+                            uint32_t pk;
+                            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(__uint_as_float(v[j + 1])), "f"(__uint_as_float(v[j])));
+                            reinterpret_cast<uint16_t *>(st16)[j * kChan] = (uint16_t)pk;
+                            reinterpret_cast<uint16_t *>(st16)[(j + 1) * kChan] = (uint16_t)(pk >> 16);
+                        }
                     } else {
                         uint32_t *const st32 = reinterpret_cast<uint32_t *>(sm->stage_out[c & 1]) + nl;
 #pragma unroll
                         for (int j = 0; j < 32; ++j) st32[j * kChan] = v[j];
                     }
+                    PROF_ACC(e_math, t_math);
+                    PROF_T(t_st);
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     epi_bar();
+                    PROF_ACC(e_st, t_st);
                     if (ew == 0 && lane == 0) {
                         const int p0 = c * 32;
                         tma_store_4d(&map_y, sm->stage_out[c & 1], nt * kChan, (p_w0 + (p0 & BWm)) * P.osw,
@@ -505,7 +571,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
             }
             __syncwarp();
         }
-        if (ew == 0 && lane == 0) { PROF_OUT(9, e_wait); PROF_OUT(10, e_drain); PROF_OUT(11, (long long)lt); }
+        if (ew == 0 && lane == 0) { PROF_OUT(9, e_wait); PROF_OUT(10, e_drain); PROF_OUT(11, (long long)lt); PROF_OUT(16, e_ld); PROF_OUT(17, e_grp); PROF_OUT(18, e_math); PROF_OUT(19, e_st); }
         // all bulk stores of this thread have been written before the block may exit
         if (P.tma_store && ew == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
@@ -690,15 +756,21 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     P.status = dev_status;
     for (int t = 0; t < g.n_taps; ++t) P.taps[t] = g.taps[t];
 
-    // Tile shape by a cost model fitted to measured launches (cycles per round of tiles):
+    // Tile shape and mode by a cost model fitted to measured launches (cycles per round of tiles):
     //   128 pixels: 2000 + 930 per k-block (epilogue overlapped, 64-cycle MMAs)
     //   256 pixels: 14000 + 1100 per k-block (epilogue exposed, twice the work per k-block)
     int a, b;
     const long long kb = (long long)P.n_taps * P.n_cblk;
+    const long long sms = dev.sm_count;
     const long long t128 = pick_tile(g, 128, &a, &b) * P.n_tiles, t256 = pick_tile(g, 256, &a, &b) * P.n_tiles;
-    const long long r128 = (t128 + dev.sm_count - 1) / dev.sm_count, r256 = (t256 + dev.sm_count - 1) / dev.sm_count;
-    const long long c128 = r128 * (2000 + 930 * kb), c256 = r256 * (14000 + 1100 * kb);
-    if (c256 < c128) return launch_conv_t<256>(g, P, X, dev, enc, s);
+    long long best = ((t128 + sms - 1) / sms) * (2000 + 930 * kb);
+    int choice = 0;
+    const long long c256 = ((t256 + sms - 1) / sms) * (14000 + 1100 * kb);
+    if (c256 < best) { best = c256; choice = 1; }
+#ifdef TWN_PROFILE
+    if (const char *force = getenv("TWN_TILE")) choice = atoi(force) & 1;   // profiling builds: pin the variant
+#endif
+    if (choice == 1) return launch_conv_t<256>(g, P, X, dev, enc, s);
     return launch_conv_t<128>(g, P, X, dev, enc, s);
 }
 
@@ -847,13 +919,14 @@ extern "C" int twn_conv2d_bwd_data(const twn_conv_desc_t *d, const void *dZ, con
 }
 
 #ifdef TWN_PROFILE
+extern "C" int twn_tl2_read(long long *host) { return cudaMemcpyFromSymbol(host, g_tl2, sizeof(long long) * 4 * 1024); }
 extern "C" int twn_tl_read(long long *host) { return cudaMemcpyFromSymbol(host, g_tl, sizeof(long long) * 4 * 1024); }
 extern "C" int twn_prof_read(long long *host, int zero)
 {
     if (zero) {
-        static long long z[256 * 16];
+        static long long z[256 * 32];
         return cudaMemcpyToSymbol(g_prof, z, sizeof(z));
     }
-    return cudaMemcpyFromSymbol(host, g_prof, sizeof(long long) * 256 * 16);
+    return cudaMemcpyFromSymbol(host, g_prof, sizeof(long long) * 256 * 32);
 }
 #endif

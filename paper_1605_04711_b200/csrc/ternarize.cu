@@ -146,24 +146,26 @@ __device__ __forceinline__ uint32_t code2(float w, float thr, double &kept_sum)
 }
 
 // Bit position of element e (0..15) inside its word: even elements fill the low
-// half-word, odd elements the high half-word.
-__host__ __device__ __forceinline__ int field_pos(int e) { return 2 * (e >> 1) + 16 * (e & 1); }
+// half-word, odd elements the high half-word, each from the top down, so that a left
+// shift by 2*(e/2) brings the element's field to the top two bits of its half-word.
+__host__ __device__ __forceinline__ int field_pos(int e) { return 14 - 2 * (e >> 1) + 16 * (e & 1); }
 
-// Four consecutive weights -> one byte: low nibble = fields of elements 0 and 2,
-// high nibble = fields of elements 1 and 3.
+// Four consecutive weights -> one byte: low nibble = fields of elements 0 (upper) and 2,
+// high nibble = fields of elements 1 (upper) and 3.
 __device__ __forceinline__ uint32_t code8(const float4 v, float thr, double &k0, double &k1)
 {
-    uint32_t c = code2(v.x, thr, k0);
-    c |= code2(v.z, thr, k0) << 2;
-    c |= code2(v.y, thr, k1) << 4;
-    c |= code2(v.w, thr, k1) << 6;
+    uint32_t c = code2(v.x, thr, k0) << 2;
+    c |= code2(v.z, thr, k0);
+    c |= code2(v.y, thr, k1) << 6;
+    c |= code2(v.w, thr, k1) << 4;
     return c;
 }
 
 // Bytes B0..B3 (as produced by code8 for four consecutive float4) -> the word of
-// those 16 elements: low half = low nibbles, high half = high nibbles.
+// those 16 elements: low half = low nibbles, high half = high nibbles, B0's on top.
 __device__ __forceinline__ uint32_t bytes_to_word(uint32_t r)
 {
+    r = __byte_perm(r, 0u, 0x0123);
     uint32_t lo = r & 0x0F0F0F0Fu, hi = (r >> 4) & 0x0F0F0F0Fu;
     lo = (lo | (lo >> 4)) & 0x00FF00FFu;
     lo = (lo | (lo >> 8)) & 0x0000FFFFu;
@@ -180,7 +182,7 @@ __device__ __forceinline__ uint32_t word_to_bytes(uint32_t w)
     lo = (lo | (lo << 4)) & 0x0F0F0F0Fu;
     hi = (hi | (hi << 8)) & 0x00FF00FFu;
     hi = (hi | (hi << 4)) & 0x0F0F0F0Fu;
-    return lo | (hi << 4);
+    return __byte_perm(lo | (hi << 4), 0u, 0x0123);
 }
 
 // int8 image of the four fields of a code8 byte, in element order:
@@ -190,7 +192,7 @@ __device__ __forceinline__ uint32_t fields_to_i8x4(uint32_t c8)
     uint32_t r = 0;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-        const uint32_t f = (c8 >> (2 * (e >> 1) + 4 * (e & 1))) & 3u;
+        const uint32_t f = (c8 >> (2 - 2 * (e >> 1) + 4 * (e & 1))) & 3u;
         const uint32_t b = (f & 1u) ? ((f & 2u) ? 0xFFu : 0x01u) : 0u;
         r |= b << (8 * e);
     }
@@ -313,9 +315,9 @@ __device__ __forceinline__ uint32_t i8x4_to_fields(uint32_t x, uint32_t &bad)
     const uint32_t inval = __vcmpgtu4(__vadd4(x, 0x01010101u), 0x02020202u);
     bad |= inval;
     x &= ~inval;
-    // low two bits of bytes 0..3 -> fields in code8 order (e0, e2 | e1, e3)
+    // low two bits of bytes 0..3 -> fields in code8 order (low nibble e0, e2; high nibble e1, e3)
     const uint32_t y = x & 0x03030303u;
-    return (y & 3u) | ((y >> 14) & 0xCu) | ((y >> 4) & 0x30u) | ((y >> 18) & 0xC0u);
+    return ((y & 3u) << 2) | ((y >> 16) & 3u) | ((y >> 2) & 0xC0u) | ((y >> 20) & 0x30u);
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -341,7 +343,7 @@ pack_kernel(const int8_t *__restrict__ codes, long long rows, long long cols, lo
                 const long long j = j0 + e;
                 if (j < cols) {
                     const uint32_t b = (uint8_t)codes[r * cols + j];
-                    word |= (i8x4_to_fields(b, bad) & 3u) << field_pos(e);
+                    word |= ((i8x4_to_fields(b, bad) >> 2) & 3u) << field_pos(e);   // byte 0 -> bits 3:2
                 }
             }
         }
@@ -385,10 +387,10 @@ unpack_kernel(const uint32_t *__restrict__ packed, long long rows, long long col
         const uint32_t inval = (word >> 1) & ~word & 0x55555555u;
         const long long j0 = wi << 4;
         const long long valid = cols - j0 >= 16 ? 16 : cols - j0;
-        // fields of elements < valid: ceil(valid/2) in the low half, floor(valid/2) in the high half
+        // fields of elements < valid: the top ceil(valid/2) of the low half, the top floor(valid/2) of the high half
         const uint32_t vmask = valid >= 16 ? 0xFFFFFFFFu
-                                           : (((1u << (2 * ((valid + 1) >> 1))) - 1u) |
-                                              (((1u << (2 * (valid >> 1))) - 1u) << 16));
+                                           : (((0xFFFFu << (16 - 2 * ((valid + 1) >> 1))) & 0xFFFFu) |
+                                              (((0xFFFFu << (16 - 2 * (valid >> 1))) & 0xFFFFu) << 16));
         if (inval & vmask) bad = true;
         const uint32_t clean = word & ~(inval << 1);
         if (vec_ok && valid == 16) {

@@ -205,8 +205,8 @@ def test_pack_flags_codes_outside_the_ternary_set():
 
 
 def test_unpack_flags_the_unused_field():
-    # element 0 (bits 1:0) = +1, element 1 (bits 17:16) = the unused field 10
-    packed = dev_u32(np.array([[0b01 | (0b10 << 16), 0, 0, 0]], dtype=np.uint32))
+    # element 0 (bits 15:14) = +1, element 1 (bits 31:30) = the unused field 10
+    packed = dev_u32(np.array([[(0b01 << 14) | (0b10 << 30), 0, 0, 0]], dtype=np.uint32))
     out = torch.zeros((1, 2), dtype=torch.int8, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     twn.unpack(packed, 1, 2, 64, out, status)

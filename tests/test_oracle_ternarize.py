@@ -218,16 +218,17 @@ def test_golden_closed_forms_file():
 
 # ----------------------------------------------------------- 2-bit storage
 def test_pack_hand_worked_word():
-    # element e of a 16-group -> bit 2*(e//2) + 16*(e%2); 0 -> 00, +1 -> 01, -1 -> 11
-    # e0 = +1 -> bits 1:0 = 01 ; e1 = 0 ; e2 = -1 -> bits 3:2 = 11 ; e3 = +1 -> bits 19:18 = 01
+    # element e of a 16-group -> bit 14 - 2*(e//2) + 16*(e%2); 0 -> 00, +1 -> 01, -1 -> 11
+    # e0 = +1 -> bits 15:14 = 01 ; e1 = 0 ; e2 = -1 -> bits 13:12 = 11 ; e3 = +1 -> bits 29:28 = 01
     codes = np.array([1, 0, -1, 1], dtype=np.int8)
     p = oracle.pack(codes, 16)
-    assert p.shape == (1, 1) and int(p[0, 0]) == (0b1101 | (0b0100 << 16))
-    # e15 (odd, pair 7) -> bits 31:30 ; e16 = element 0 of the next word -> bits 1:0
+    assert p.shape == (1, 1) and int(p[0, 0]) == (0x4000 | 0x3000 | (0x1000 << 16))
+    # e14 (even, pair 7) -> bits 1:0 ; e15 (odd, pair 7) -> bits 17:16 ; e16 = element 0 of the
+    # next word -> bits 15:14
     codes = np.zeros(32, dtype=np.int8); codes[15] = -1; codes[16] = 1; codes[14] = 1
     p = oracle.pack(codes, 64)
     assert p.shape == (1, 4)
-    assert [int(v) for v in p[0]] == [0xC0004000, 0x00000001, 0, 0]
+    assert [int(v) for v in p[0]] == [0x00030001, 0x00004000, 0, 0]
 
 
 def test_pack_round_trip_all_3_pow_16_words():
@@ -266,6 +267,6 @@ def test_pack_ragged_rows_and_size(rows, cols):
 
 def test_unpack_rejects_the_unused_field():
     with pytest.raises(ValueError):
-        oracle.unpack(np.array([[0b10]], dtype=np.uint32), 1, 1, 16)
+        oracle.unpack(np.array([[0b10 << 14]], dtype=np.uint32), 1, 1, 16)
     with pytest.raises(ValueError):
         oracle.pack(np.array([2], dtype=np.int8), 16)
