@@ -100,8 +100,13 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap *map, const void 
         : "memory");
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
-// named barrier of the four epilogue warps
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// named barrier of the four warps of an epilogue group
+__device__ __forceinline__ void epi_bar(int set)
+{
+    // immediate barrier numbers: a register operand would make the compiler reserve all sixteen
+    if (set == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
+    else asm volatile("bar.sync 2, 128;" ::: "memory");
+}
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }

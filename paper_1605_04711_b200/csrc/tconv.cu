@@ -69,9 +69,11 @@ constexpr int kChan = 128;          // output channels per tile (UMMA M)
 constexpr int kBlockK = 64;         // reduction elements per k-block (128 bytes of bf16)
 constexpr int kDecodeSets = 1;      // groups of 4 decode warps; a group takes every other stage
 constexpr int kFirstEpiWarp = 2 + 4 * kDecodeSets;
-constexpr int kThreadsConv = 32 * (kFirstEpiWarp + 4);
+constexpr int kEpiSets = 2;         // groups of 4 epilogue warps; a group drains every other 32-pixel chunk
+constexpr int kThreadsConv = 32 * (kFirstEpiWarp + 4 * kEpiSets);
+constexpr int kStageBytes = 8192;   // one output staging buffer: 32 pixels of bf16 or 16 pixels of fp32, 128 channels
 constexpr int kMaxTaps = 64;
-constexpr int kWordTab = 512;       // k-blocks per tile whose code offsets are tabulated in shared memory
+constexpr int kWordTab = 128;       // k-blocks per tile whose code offsets are tabulated in shared memory
 constexpr int kAColsPerBlock = kBlockK / 2;    // 32 columns of bf16 pairs per k-block
 constexpr uint32_t kTmemCols = 512;
 
@@ -131,14 +133,14 @@ struct __align__(1024) SmemLayout {
     unsigned long long empty[kStages];     // MMA commit -> TMA and decode: both operand slots are free
     unsigned long long acc_full[2];        // MMA commit -> epilogue
     unsigned long long acc_empty[2];       // epilogue -> MMA
-    alignas(16) uint32_t pix_off[4][PIX];  // per epilogue warp: output element offset of a pixel, ~0 = skip
-    alignas(128) float stage_out[2][32 * kChan];  // output staging for TMA stores: [32 pixels][128 channels]
-    alignas(128) __nv_bfloat16 stage_res[3][32 * kChan];  // residual staging, same chunk shape
-    unsigned long long res_full[3];
+    alignas(16) uint32_t pix_off[kEpiSets][PIX / kEpiSets];   // output element offset of the pixels of a group's chunks, ~0 = skip
+    alignas(128) uint8_t stage_out[kEpiSets][2][kStageBytes];   // output staging for TMA stores: [pixels][128 channels]
+    alignas(128) __nv_bfloat16 stage_res[kEpiSets][2][32 * kChan];  // residual staging: [32 pixels][128 channels]
+    unsigned long long res_full[kEpiSets][2];
     uint32_t kword[kWordTab];              // first code word of k-block u in a packed row, u < kWordTab
     uint32_t tmem_base;
     volatile int abort_flag;
-    volatile int epi_ok;                   // outcome of the epilogue's wait, shared by its four warps
+    volatile int epi_ok[kEpiSets][2];      // outcome of a wait of an epilogue group's leader, shared by its four warps
 };
 
 static_assert(offsetof(SmemLayout<128>, stage_res) % 128 == 0 && offsetof(SmemLayout<256>, stage_res) % 128 == 0 &&
@@ -175,9 +177,9 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         for (int s = 0; s < 8; ++s) mbar_init(&sm->ready_a[s], 4);
         for (int b = 0; b < 2; ++b) {
             mbar_init(&sm->acc_full[b], 1);
-            mbar_init(&sm->acc_empty[b], 4);
+            mbar_init(&sm->acc_empty[b], 4 * kEpiSets);
         }
-        for (int b = 0; b < 3; ++b) mbar_init(&sm->res_full[b], 1);
+        for (int b = 0; b < 2 * kEpiSets; ++b) mbar_init(&sm->res_full[0][0] + b, 1);
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -403,14 +405,26 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         if (warp == 2 && lane == 0) { PROF_OUT(6, w_full); PROF_OUT(8, PROF_NOW() - t_dec); PROF_OUT(12, d_alu); PROF_OUT(13, d_wst); PROF_OUT(14, d_fetch); PROF_OUT(15, d_st); }
     } else {
         // ------------------------------------------------ epilogue
+        // Two groups of four warps (one warp per tensor-memory lane quadrant); a group drains
+        // every other 32-pixel chunk of the accumulator: tcgen05.ld -> scale / shift / residual /
+        // ReLU -> its own staging buffers -> TMA store by the group's first thread.  Each group
+        // keeps its own bulk-store accounting, residual buffers and named barrier.
         const int q = warp & 3;
-        const int ew = warp - kFirstEpiWarp;
-        uint32_t *pix_off = sm->pix_off[ew];
+        const int es = (warp - kFirstEpiWarp) >> 2;          // group
+        const int ew = (warp - kFirstEpiWarp) & 3;           // warp inside the group
+        const bool leader = ew == 0 && lane == 0;
         // decoded weights are +-2, so half of alpha scales the accumulators
         const float alpha = (P.alpha ? (float)(*P.alpha) : 1.0f) * (1.0f / kDecodedUnit);
         const int BWm = (1 << P.lgBW) - 1, BHm = (1 << P.lgBH) - 1;
         const bool out_bf16 = P.out_dtype == TWN_BF16, res_bf16 = P.res_dtype == TWN_BF16;
+        const bool need_off = !P.tma_store || (P.residual && !P.res_tma);
+        const float floor_v = P.relu ? 0.0f : -INFINITY;
+        constexpr int kChunks = PIX / 32;
         uint32_t lt = 0;
+        uint32_t nst = 0;      // staging buffers this group has filled so far (selects the buffer)
+        uint32_t nres = 0;     // residual chunks this group has consumed so far (buffer and phase)
+        uint32_t ndec = 0;     // joint decisions taken so far: two flags alternate, so that the leader
+                               // never overwrites one that a slower warp has yet to read
         PROF_DECL(e_wait); PROF_DECL(e_drain); PROF_DECL(e_ld); PROF_DECL(e_grp); PROF_DECL(e_math); PROF_DECL(e_st);
         for (int tile = blockIdx.x; tile < P.total_tiles; tile += gridDim.x, ++lt) {
             const int nt = tile % P.n_tiles;
@@ -420,66 +434,78 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
             const int tbi = pt / P.th;
             const int n = nt * kChan + q * 32 + lane;
             const bool n_ok = n < P.Cout;
+            // a warp whose 32 channels all lie past Cout keeps the barriers and hands the accumulator
+            // back, but loads, computes and stages nothing (its part of the staging buffer is clipped)
+            const bool warp_on = nt * kChan + q * 32 < P.Cout;
             const float sc = ((P.scale && n_ok) ? __ldg(P.scale + n) : 1.0f) * alpha;
             const float sf = (P.shift && n_ok) ? __ldg(P.shift + n) : 0.0f;
-            // output offsets of the tile's pixels (the same for every channel), before the wait
-#pragma unroll
-            for (int j = 0; j < PIX / 32; ++j) {
-                const int p = j * 32 + lane;
-                const int wv = (twi << P.lgBW) + (p & BWm);
-                const int hv = (thi << P.lgBH) + ((p >> P.lgBW) & BHm);
-                const int bv = tbi * (PIX >> (P.lgBW + P.lgBH)) + (p >> (P.lgBW + P.lgBH));
-                uint32_t off = 0xFFFFFFFFu;
-                if (wv < P.Wv && hv < P.Hv && bv < P.Bv)
-                    off = (uint32_t)((((long long)bv * P.OH + (hv * P.osh + P.ooh)) * P.OW + (wv * P.osw + P.oow)) * P.ldy);
-                pix_off[p] = off;
+            const int p_w0 = twi << P.lgBW, p_h0 = thi << P.lgBH, p_b0 = tbi * (PIX >> (P.lgBW + P.lgBH));
+            if (need_off) {
+                // output offsets of the pixels of this group's chunks (the same for every channel),
+                // one per thread; the first barrier keeps the previous tile's readers ahead of the overwrite
+                epi_bar(es);
+                if (ew < kChunks / kEpiSets) {
+                    const int p = (ew * kEpiSets + es) * 32 + lane;
+                    const int wv = p_w0 + (p & BWm);
+                    const int hv = p_h0 + ((p >> P.lgBW) & BHm);
+                    const int bv = p_b0 + (p >> (P.lgBW + P.lgBH));
+                    uint32_t off = 0xFFFFFFFFu;
+                    if (wv < P.Wv && hv < P.Hv && bv < P.Bv)
+                        off = (uint32_t)((((long long)bv * P.OH + (hv * P.osh + P.ooh)) * P.OW + (wv * P.osw + P.oow)) * P.ldy);
+                    sm->pix_off[es][ew * 32 + lane] = off;
+                }
+                epi_bar(es);
             }
-            __syncwarp();
+            // residual chunk `c` of this tile -> the group's buffer `slot` (one thread)
+            auto res_load = [&](int c, uint32_t slot) {
+                const int p0 = c * 32;
+                mbar_expect_tx(&sm->res_full[es][slot], 32 * kChan * 2);
+                tma_load_4d(sm->stage_res[es][slot], &map_r, &sm->res_full[es][slot], nt * kChan,
+                            (p_w0 + (p0 & BWm)) * P.osw, (p_h0 + ((p0 >> P.lgBW) & BHm)) * P.osh,
+                            p_b0 + (p0 >> (P.lgBW + P.lgBH)));
+            };
+            // both buffers are free here: their last readers finished before the group's last barrier
+            if (P.res_tma && leader) {
+                res_load(es, nres & 1u);
+                if (es + kEpiSets < kChunks) res_load(es + kEpiSets, (nres + 1) & 1u);
+            }
             const int buf = lt % kAccBufs;
             PROF_T(t_w);
             if (kbpt > 0) {
-                // one thread waits for the accumulator; the four warps then decide together, so that
-                // they always execute the same number of named barriers
-                if (ew == 0 && lane == 0)
-                    sm->epi_ok = mbar_wait(&sm->acc_full[buf], (lt / kAccBufs) & 1u, abort_flag, P.status, 32) ? 1 : 0;
-                epi_bar();
-                if (!sm->epi_ok) break;
+                // one thread waits for the accumulator; the group's warps then decide together, so
+                // that they always execute the same number of named barriers
+                if (leader)
+                    sm->epi_ok[es][ndec & 1u] = mbar_wait(&sm->acc_full[buf], (lt / kAccBufs) & 1u, abort_flag, P.status, 32) ? 1 : 0;
+                epi_bar(es);
+                if (!sm->epi_ok[es][ndec++ & 1u]) break;
             }
             PROF_ACC(e_wait, t_w);
             PROF_T(t_d);
             tc_fence_after();
             float *const y32 = reinterpret_cast<float *>(P.Y) + n;
             __nv_bfloat16 *const y16 = reinterpret_cast<__nv_bfloat16 *>(P.Y) + n;
-            const int p_w0 = twi << P.lgBW, p_h0 = thi << P.lgBH, p_b0 = tbi * (PIX >> (P.lgBW + P.lgBH));
-            const uint32_t g0 = lt * (PIX / 32);     // running chunk count: selects the residual buffer
-            auto res_load = [&](int c) {             // one thread: stage the residual of chunk c
-                const uint32_t g = g0 + c;
-                const int p0 = c * 32;
-                mbar_expect_tx(&sm->res_full[g % 3], 32 * kChan * 2);
-                tma_load_4d(sm->stage_res[g % 3], &map_r, &sm->res_full[g % 3], nt * kChan,
-                            (p_w0 + (p0 & BWm)) * P.osw, (p_h0 + ((p0 >> P.lgBW) & BHm)) * P.osh,
-                            p_b0 + (p0 >> (P.lgBW + P.lgBH)));
-            };
-            if (P.res_tma && ew == 0 && lane == 0) { res_load(0); res_load(1); }
+            bool alive = true;
 #pragma unroll 1
-            for (int c = 0; c < PIX / 32; ++c) {
+            for (int c = es; c < kChunks && alive; c += kEpiSets) {
                 // the 32 offsets of this chunk: eight 16-byte broadcast loads, issued before the
                 // tensor-memory load is waited for (needed for per-thread stores and for the residual)
                 uint32_t off[32];
-                if (!P.tma_store || (P.residual && !P.res_tma)) {
+                if (need_off) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
-                        const uint4 o = *reinterpret_cast<const uint4 *>(pix_off + c * 32 + i * 4);
+                        const uint4 o = *reinterpret_cast<const uint4 *>(sm->pix_off[es] + (c / kEpiSets) * 32 + i * 4);
                         off[i * 4 + 0] = o.x; off[i * 4 + 1] = o.y; off[i * 4 + 2] = o.z; off[i * 4 + 3] = o.w;
                     }
                 }
                 uint32_t v[32];
                 PROF_T(t_ld);
                 if (kbpt > 0) {
-                    tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + buf * PIX + c * 32, v);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                    if (c == PIX / 32 - 1) {
-                        // the accumulator is in registers: hand it back before the last stores
+                    if (warp_on) {
+                        tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + buf * PIX + c * 32, v);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    }
+                    if (c + kEpiSets >= kChunks) {
+                        // this warp's share of the accumulator is in registers: hand it back
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&sm->acc_empty[buf]);
@@ -489,33 +515,31 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
                 }
-                // The inner loops are kept free of conditionals: one warp per scheduler runs this
-                // code, so every instruction fetched and issued here is exposed latency.
-                const float floor_v = P.relu ? 0.0f : -INFINITY;
                 PROF_ACC(e_ld, t_ld);
                 PROF_T(t_grp);
-                if (P.tma_store) {
-                    // staging buffer (c & 1) was last read by the store issued two chunks ago; the
-                    // residual of this chunk has landed.  One thread waits, all four warps follow.
-                    if (ew == 0 && lane == 0) {
-                        asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                        if (P.res_tma)
-                            sm->epi_ok = mbar_wait(&sm->res_full[(g0 + c) % 3], ((g0 + c) / 3) & 1u, abort_flag, P.status, 32) ? 1 : 0;
-                    }
-                    epi_bar();
-                    if (P.res_tma) {
-                        if (!sm->epi_ok) break;
-                        // the buffer two chunks ahead was last read in the previous chunk
-                        if (ew == 0 && lane == 0 && c + 2 < PIX / 32) res_load(c + 2);
-                    }
+                if (P.res_tma) {
+                    // the residual of this chunk has landed; the buffer of the group's next chunk was
+                    // last read in its previous chunk, which every warp has left by the barrier
+                    if (leader)
+                        sm->epi_ok[es][ndec & 1u] = mbar_wait(&sm->res_full[es][nres & 1u], (nres >> 1) & 1u, abort_flag, P.status, 32) ? 1 : 0;
+                    epi_bar(es);
+                    if (!sm->epi_ok[es][ndec++ & 1u]) { alive = false; break; }
+                    if (leader && c != es && c + kEpiSets < kChunks) res_load(c + kEpiSets, (nres + 1) & 1u);
                 }
                 PROF_ACC(e_grp, t_grp);
                 PROF_T(t_math);
+                // The inner loops are kept free of conditionals: one warp per scheduler runs this
+                // code, so every instruction fetched and issued here is exposed latency.
                 if (P.res_tma) {
-                    const __nv_bfloat16 *rs = sm->stage_res[(g0 + c) % 3] + q * 32 + lane;
+                    const __nv_bfloat16 *rs = sm->stage_res[es][nres & 1u] + q * 32 + lane;
+                    if (warp_on) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        v[j] = __float_as_uint(fmaxf(fmaf(__uint_as_float(v[j]), sc, sf) + __bfloat162float(rs[j * kChan]), floor_v));
+                        for (int j = 0; j < 32; ++j)
+                            v[j] = __float_as_uint(fmaxf(fmaf(__uint_as_float(v[j]), sc, sf) + __bfloat162float(rs[j * kChan]), floor_v));
+                    }
+                    ++nres;
+                } else if (!warp_on) {
+                    // nothing to compute
                 } else if (P.residual) {
                     // y = acc * scale' + shift + residual (residual fetched with the per-pixel offsets)
 #pragma unroll
@@ -530,32 +554,48 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(fmaxf(fmaf(__uint_as_float(v[j]), sc, sf), floor_v));
                 }
+                PROF_ACC(e_math, t_math);
                 if (P.tma_store) {
                     const int nl = q * 32 + lane;
-                    if (out_bf16) {
-                        __nv_bfloat16 *const st16 = reinterpret_cast<__nv_bfloat16 *>(sm->stage_out[c & 1]) + nl;
+                    // a staging buffer holds 32 pixels of bf16 or 16 of fp32: one or two rounds per chunk
+                    const int rounds = out_bf16 ? 1 : 2;
+                    for (int h = 0; h < rounds; ++h) {
+                        // the buffer was last read by the store this group issued two rounds ago
+                        PROF_T(t_st);
+                        if (leader) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                        epi_bar(es);
+                        uint8_t *const sbuf = sm->stage_out[es][nst & 1u];
+                        if (!warp_on) {
+                            // clipped by the store
+                        } else if (out_bf16) {
+                            uint16_t *const st16 = reinterpret_cast<uint16_t *>(sbuf) + nl;
 #pragma unroll
-                        for (int j = 0; j < 32; j += 2) {
-                            // one packed conversion per two pixels (the scalar one runs at a fraction of its rate)
-                            uint32_t pk;
-                            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(__uint_as_float(v[j + 1])), "f"(__uint_as_float(v[j])));
-                            reinterpret_cast<uint16_t *>(st16)[j * kChan] = (uint16_t)pk;
-                            reinterpret_cast<uint16_t *>(st16)[(j + 1) * kChan] = (uint16_t)(pk >> 16);
+                            for (int j = 0; j < 32; j += 2) {
+                                // one packed conversion per two pixels
+                                uint32_t pk;
+                                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(__uint_as_float(v[j + 1])), "f"(__uint_as_float(v[j])));
+                                st16[j * kChan] = (uint16_t)pk;
+                                st16[(j + 1) * kChan] = (uint16_t)(pk >> 16);
+                            }
+                        } else {
+                            uint32_t *const st32 = reinterpret_cast<uint32_t *>(sbuf) + nl;
+                            if (h == 0) {
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) st32[j * kChan] = v[j];
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) st32[j * kChan] = v[16 + j];
+                            }
                         }
-                    } else {
-                        uint32_t *const st32 = reinterpret_cast<uint32_t *>(sm->stage_out[c & 1]) + nl;
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) st32[j * kChan] = v[j];
-                    }
-                    PROF_ACC(e_math, t_math);
-                    PROF_T(t_st);
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    epi_bar();
-                    PROF_ACC(e_st, t_st);
-                    if (ew == 0 && lane == 0) {
-                        const int p0 = c * 32;
-                        tma_store_4d(&map_y, sm->stage_out[c & 1], nt * kChan, (p_w0 + (p0 & BWm)) * P.osw,
-                                     (p_h0 + ((p0 >> P.lgBW) & BHm)) * P.osh, p_b0 + (p0 >> (P.lgBW + P.lgBH)));
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        epi_bar(es);
+                        if (leader) {
+                            const int p0 = c * 32 + h * 16;
+                            tma_store_4d(&map_y, sbuf, nt * kChan, (p_w0 + (p0 & BWm)) * P.osw,
+                                         (p_h0 + ((p0 >> P.lgBW) & BHm)) * P.osh, p_b0 + (p0 >> (P.lgBW + P.lgBH)));
+                        }
+                        ++nst;
+                        PROF_ACC(e_st, t_st);
                     }
                 } else if (n_ok) {
                     if (out_bf16) {
@@ -569,11 +609,12 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     }
                 }
             }
+            if (!alive) break;
             __syncwarp();
         }
-        if (ew == 0 && lane == 0) { PROF_OUT(9, e_wait); PROF_OUT(10, e_drain); PROF_OUT(11, (long long)lt); PROF_OUT(16, e_ld); PROF_OUT(17, e_grp); PROF_OUT(18, e_math); PROF_OUT(19, e_st); }
+        if (ew == 0 && lane == 0 && es == 0) { PROF_OUT(9, e_wait); PROF_OUT(10, e_drain); PROF_OUT(11, (long long)lt); PROF_OUT(16, e_ld); PROF_OUT(17, e_grp); PROF_OUT(18, e_math); PROF_OUT(19, e_st); }
         // all bulk stores of this thread have been written before the block may exit
-        if (P.tma_store && ew == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        if (P.tma_store && leader) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 
     // ---------------------------------------------------- teardown
@@ -686,15 +727,21 @@ int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const twn_dev
     const long long base_pix = (long long)g.ooh * g.OW + g.oow;
     if ((g.ldy * es) % 16 == 0 && ((long long)g.Cout * es) % 16 == 0 && (reinterpret_cast<uintptr_t>(P.Y) % 16) == 0 &&
         g.OW > g.oow && g.OH > g.ooh) {
-        // a chunk of 32 consecutive tile pixels is a sub-box sbw x sbh x sbb of the tile box
-        const int lg_sbw = P.lgBW < 5 ? P.lgBW : 5;
-        const int lg_sbh = P.lgBH < 5 - lg_sbw ? P.lgBH : 5 - lg_sbw;
-        const int lg_sbb = 5 - lg_sbw - lg_sbh;
-        P.lg_sbw = lg_sbw; P.lg_sbh = lg_sbh;
+        // 2^lg consecutive tile pixels are a sub-box sbw x sbh x sbb of the tile box: a staging
+        // buffer holds 32 pixels of bf16 or 16 of fp32, a residual buffer 32 pixels
+        auto sub_box = [&](int lg, cuuint32_t *bx) {
+            const int lg_sbw = P.lgBW < lg ? P.lgBW : lg;
+            const int lg_sbh = P.lgBH < lg - lg_sbw ? P.lgBH : lg - lg_sbw;
+            const int lg_sbb = lg - lg_sbw - lg_sbh;
+            bx[0] = (cuuint32_t)kChan; bx[1] = (cuuint32_t)((1 << lg_sbw) * g.osw);
+            bx[2] = (cuuint32_t)((1 << lg_sbh) * g.osh); bx[3] = 1u << lg_sbb;
+        };
         cuuint64_t dims[4] = {(cuuint64_t)g.Cout, (cuuint64_t)(g.OW - g.oow), (cuuint64_t)(g.OH - g.ooh), (cuuint64_t)g.Bv};
-        cuuint32_t box[4] = {(cuuint32_t)kChan, (cuuint32_t)((1 << lg_sbw) * g.osw), (cuuint32_t)((1 << lg_sbh) * g.osh), 1u << lg_sbb};
+        cuuint32_t box[4], rbox[4];
+        sub_box(es == 2 ? 5 : 4, box);
+        sub_box(5, rbox);
         cuuint32_t estr[4] = {1, (cuuint32_t)g.osw, (cuuint32_t)g.osh, 1};
-        if (box[1] <= 256 && box[2] <= 256) {
+        if (box[1] <= 256 && box[2] <= 256 && rbox[1] <= 256 && rbox[2] <= 256) {
             cuuint64_t strides[3] = {(cuuint64_t)g.ldy * es, (cuuint64_t)g.OW * g.ldy * es, (cuuint64_t)g.OH * g.OW * g.ldy * es};
             void *ybase = static_cast<char *>(P.Y) + base_pix * g.ldy * es;
             if (enc(&map_y, es == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, ybase, dims,
@@ -706,7 +753,7 @@ int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const twn_dev
                 ((long long)g.Cout * 2) % 16 == 0 && (reinterpret_cast<uintptr_t>(P.residual) % 16) == 0) {
                 cuuint64_t rstrides[3] = {(cuuint64_t)g.ldy * 2, (cuuint64_t)g.OW * g.ldy * 2, (cuuint64_t)g.OH * g.OW * g.ldy * 2};
                 void *rbase = const_cast<char *>(static_cast<const char *>(P.residual)) + base_pix * g.ldy * 2;
-                if (enc(&map_r, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, rbase, dims, rstrides, box, estr,
+                if (enc(&map_r, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, rbase, dims, rstrides, rbox, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
                     P.res_tma = 1;
@@ -756,19 +803,20 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     P.status = dev_status;
     for (int t = 0; t < g.n_taps; ++t) P.taps[t] = g.taps[t];
 
-    // Tile shape and mode by a cost model fitted to measured launches (cycles per round of tiles):
-    //   128 pixels: 2000 + 930 per k-block (epilogue overlapped, 64-cycle MMAs)
-    //   256 pixels: 14000 + 1100 per k-block (epilogue exposed, twice the work per k-block)
+    // Tile shape by a cost model fitted to measured launches (cycles per round of tiles, kb = k-blocks
+    // per tile):
+    //   128 pixels: max(2500 + 720 kb, 6500): the epilogue overlaps the next tile and bounds short reductions
+    //   256 pixels: 13500 + 640 kb: one accumulator, so the epilogue is exposed; 8000 when only the
+    //               lower half of the channel tile exists (half of the epilogue warps idle)
     int a, b;
     const long long kb = (long long)P.n_taps * P.n_cblk;
     const long long sms = dev.sm_count;
     const long long t128 = pick_tile(g, 128, &a, &b) * P.n_tiles, t256 = pick_tile(g, 256, &a, &b) * P.n_tiles;
-    long long best = ((t128 + sms - 1) / sms) * (2000 + 930 * kb);
-    int choice = 0;
-    const long long c256 = ((t256 + sms - 1) / sms) * (14000 + 1100 * kb);
-    if (c256 < best) { best = c256; choice = 1; }
-#ifdef TWN_PROFILE
-    if (const char *force = getenv("TWN_TILE")) choice = atoi(force) & 1;   // profiling builds: pin the variant
+    const long long per128 = 2500 + 720 * kb > 6500 ? 2500 + 720 * kb : 6500;
+    const long long per256 = (g.Cout <= kChan / 2 ? 8000 : 13500) + 640 * kb;
+    int choice = ((t256 + sms - 1) / sms) * per256 < ((t128 + sms - 1) / sms) * per128 ? 1 : 0;
+#if defined(TWN_PROFILE) || defined(TWN_TUNE)
+    if (const char *force = getenv("TWN_TILE")) choice = atoi(force) & 1;   // profiling and tuning builds: pin the variant
 #endif
     if (choice == 1) return launch_conv_t<256>(g, P, X, dev, enc, s);
     return launch_conv_t<128>(g, P, X, dev, enc, s);
