@@ -20,9 +20,24 @@
 #include "common.cuh"
 #include "tc_ptx.cuh"
 
+// Optional cycle counters (compiled in with -DTWN_PROFILE, read back with twn_dwprof_read).
+#ifdef TWN_PROFILE
+__device__ long long g_dwprof[256 * 8];
+#define DWPROF_DECL(v) long long v = 0
+#define DWPROF_T(v) const long long v = clock64()
+#define DWPROF_ACC(acc, t0) acc += clock64() - (t0)
+#define DWPROF_OUT(slot, val) g_dwprof[blockIdx.x * 8 + (slot)] = (val)
+#else
+#define DWPROF_DECL(v)
+#define DWPROF_T(v)
+#define DWPROF_ACC(acc, t0)
+#define DWPROF_OUT(slot, val)
+#endif
+
 namespace {
 
-constexpr int kDwStages = 4;
+constexpr int kDwMaxStages = 8;
+constexpr int kDwPoolBytes = 176 * 1024;         // operand ring: stages of 16 KB of dZ plus the X blocks
 constexpr int kDwPix = 64;                       // pixels per k-block
 constexpr int kDwBlockBytes = kDwPix * 128;      // one 64-channel x 64-pixel swizzled block: 8 KB
 constexpr int kDwMaxCb = 4;                      // up to 256 input channels per tile
@@ -43,13 +58,24 @@ struct DwParams {
     float *partial;
     int vec_ok;
     int32_t *status;
+    // row mode (stride-1 layers, 2..4 taps per filter row): a group is one filter row of one
+    // 64-channel block.  Its kw column blocks read ONE activation tile with kw - 1 extra pixel
+    // columns: tap s is the tile one pixel (128 bytes) further, so a single MMA of N = 64 kw
+    // covers the row and the tile is loaded once instead of kw times.
+    int row_mode, kw, x_bytes, k_group_bytes;
+    int mma_off[4];              // byte offset of the 16 pixels of MMA i inside the activation tile
+    int stages, stage_bytes;
     DwTap taps[kDwMaxTaps];
 };
 
 struct __align__(1024) DwSmem {
-    uint8_t a[kDwStages][2][kDwBlockBytes];            // dZ: two 64-channel blocks
-    uint8_t b[kDwStages][kDwMaxCb][kDwBlockBytes];     // X: up to four 64-channel blocks
-    unsigned long long full[kDwStages], empty[kDwStages], acc_full[2], acc_empty[2];
+    // a stage: dZ as two 64-channel blocks (16 KB), then X: up to four 64-channel blocks, or one
+    // tile with its extra columns in row mode
+    uint8_t pool[kDwPoolBytes];
+    // per epilogue warp: 32 rows x 32 fp32 of the accumulator, 16-byte chunks XOR-swizzled by the
+    // row so that row-wise writes and the transposed reads are both free of bank conflicts
+    float4 stg[4][32][8];
+    unsigned long long full[kDwMaxStages], empty[kDwMaxStages], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -64,7 +90,7 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kDwStages; ++s) { mbar_init(&sm->full[s], 1); mbar_init(&sm->empty[s], 1); }
+        for (int s = 0; s < kDwMaxStages; ++s) { mbar_init(&sm->full[s], 1); mbar_init(&sm->empty[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&sm->acc_full[b], 1); mbar_init(&sm->acc_empty[b], 4); }
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -83,8 +109,12 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
         sp = u % P.splits; u /= P.splits;
         gi = u % P.n_groups;
         ot = u / P.n_groups;
-        nb = P.n_colblocks - gi * kDwMaxCb;
-        if (nb > kDwMaxCb) nb = kDwMaxCb;
+        if (P.row_mode) {
+            nb = P.kw;
+        } else {
+            nb = P.n_colblocks - gi * kDwMaxCb;
+            if (nb > kDwMaxCb) nb = kDwMaxCb;
+        }
         p0 = sp * P.tiles_per_split;
         p1 = p0 + P.tiles_per_split;
         if (p1 > P.pix_tiles) p1 = P.pix_tiles;
@@ -98,74 +128,125 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
             for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
                 int ot, gi, nb, sp, p0, p1;
                 unit_range(u, ot, gi, nb, sp, p0, p1);
-                const uint32_t bytes = (2 + nb) * kDwBlockBytes;
-                for (int p = p0; p < p1; ++p, ++it) {
-                    const int s = it % kDwStages;
-                    const uint32_t ph = (it / kDwStages) & 1u;
-                    int q = p;
-                    const int twi = q % P.tw; q /= P.tw;
-                    const int thi = q % P.th;
-                    const int tbi = q / P.th;
-                    const int w0 = twi << P.lgBW, h0 = thi << P.lgBH, b0 = tbi * (kDwPix >> (P.lgBW + P.lgBH));
-                    if (!mbar_wait(&sm->empty[s], ph ^ 1u, abort_flag, P.status, 32)) { ok = false; break; }
-                    mbar_expect_tx(&sm->full[s], bytes);
-                    tma_load_4d(sm->a[s][0], &map_dz, &sm->full[s], ot * 128, w0, h0, b0);
-                    tma_load_4d(sm->a[s][1], &map_dz, &sm->full[s], ot * 128 + 64, w0, h0, b0);
+                const uint32_t bytes = 2 * kDwBlockBytes + (P.row_mode ? P.x_bytes : nb * kDwBlockBytes);
+                // Everything that does not change along the pixel tiles is worked out here: this one
+                // thread paces the pipeline, and an integer division costs it hundreds of cycles.
+                int xc[kDwMaxCb], xdw[kDwMaxCb], xdh[kDwMaxCb];
+                int nx = nb;
+                if (P.row_mode) {
+                    // filter row r = gi / cblocks of channel block gi % cblocks: one box, kw - 1 pixels wider
+                    const int r = gi / P.cblocks, cb = gi - r * P.cblocks;
+                    const DwTap tap = P.taps[r * P.kw];
+                    xc[0] = cb * 64; xdw[0] = tap.dw; xdh[0] = tap.dh;
+                    nx = 1;
+                } else {
                     for (int j = 0; j < nb; ++j) {
                         const int i = gi * kDwMaxCb + j, t = i / P.cblocks, cb = i - t * P.cblocks;
                         const DwTap tap = P.taps[t];
-                        tma_load_4d(sm->b[s][j], &map_x, &sm->full[s], cb * 64, w0 * P.sw + tap.dw,
-                                    h0 * P.sh + tap.dh, b0);
+                        xc[j] = cb * 64; xdw[j] = tap.dw; xdh[j] = tap.dh;
                     }
+                }
+                // pixel tile p0 as (column tile, row tile, image tile), stepped without divisions
+                int twi = p0 % P.tw, thi = (p0 / P.tw) % P.th, tbi = p0 / (P.tw * P.th);
+                const int bstep = kDwPix >> (P.lgBW + P.lgBH);
+                int s = it % P.stages;
+                uint32_t ph = (it / P.stages) & 1u;
+                for (int p = p0; p < p1; ++p, ++it) {
+                    uint8_t *const st = sm->pool + s * P.stage_bytes;
+                    const int w0 = twi << P.lgBW, h0 = thi << P.lgBH, b0 = tbi * bstep;
+                    if (!mbar_wait(&sm->empty[s], ph ^ 1u, abort_flag, P.status, 32)) { ok = false; break; }
+                    mbar_expect_tx(&sm->full[s], bytes);
+                    tma_load_4d(st, &map_dz, &sm->full[s], ot * 128, w0, h0, b0);
+                    tma_load_4d(st + kDwBlockBytes, &map_dz, &sm->full[s], ot * 128 + 64, w0, h0, b0);
+#pragma unroll
+                    for (int j = 0; j < kDwMaxCb; ++j)
+                        if (j < nx)
+                            tma_load_4d(st + (2 + j) * kDwBlockBytes, &map_x, &sm->full[s], xc[j], w0 * P.sw + xdw[j],
+                                        h0 * P.sh + xdh[j], b0);
+                    if (++twi == P.tw) { twi = 0; if (++thi == P.th) { thi = 0; ++tbi; } }
+                    if (++s == P.stages) { s = 0; ph ^= 1u; }
                 }
             }
         }
     } else if (warp == 1) {
         uint32_t it = 0, lu = 0;     // lu counts the units that accumulate something
         bool ok = true;
+        DWPROF_DECL(w_full); DWPROF_DECL(w_acc);
+        DWPROF_T(t_all);
         for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
             int ot, gi, nb, sp, p0, p1;
             unit_range(u, ot, gi, nb, sp, p0, p1);
             if (p1 <= p0) continue;                      // the epilogue writes zeros for an empty split
             const uint32_t idesc = make_idesc_mn(128, 64 * nb);
             const int buf = lu & 1;
+            DWPROF_T(t_a);
             if (!mbar_wait_warp(&sm->acc_empty[buf], ((lu >> 1) & 1u) ^ 1u, abort_flag, P.status, 0)) break;
+            DWPROF_ACC(w_acc, t_a);
             tc_fence_after();
             const uint32_t d_tmem = tmem + buf * kDwAccCols;
+            int s = it % P.stages;
+            uint32_t ph = (it / P.stages) & 1u;
             for (int p = p0; p < p1; ++p, ++it) {
-                const int s = it % kDwStages;
-                const uint32_t ph = (it / kDwStages) & 1u;
+                const uint32_t st = smem_u32(sm->pool) + s * P.stage_bytes;
+                DWPROF_T(t_f);
                 if (!mbar_wait_warp(&sm->full[s], ph, abort_flag, P.status, 0)) { ok = false; break; }
+                DWPROF_ACC(w_full, t_f);
                 tc_fence_after();
-                const uint64_t adesc = smem_desc_mn_sw128(smem_u32(sm->a[s][0]), kDwBlockBytes);
-                const uint64_t bdesc = smem_desc_mn_sw128(smem_u32(sm->b[s][0]), kDwBlockBytes);
+                const uint64_t adesc = smem_desc_mn_sw128(st, kDwBlockBytes);
                 // 16 pixels per MMA = 16 rows of 128 bytes = 2048 bytes
-                if (p == p0) tc_mma_ss<false>(d_tmem, adesc, bdesc, idesc);
-                else tc_mma_ss<true>(d_tmem, adesc, bdesc, idesc);
-                tc_mma_ss<true>(d_tmem, adesc + 128, bdesc + 128, idesc);
-                tc_mma_ss<true>(d_tmem, adesc + 256, bdesc + 256, idesc);
-                tc_mma_ss<true>(d_tmem, adesc + 384, bdesc + 384, idesc);
+                if (P.row_mode) {
+                    const uint32_t xt = st + 2 * kDwBlockBytes;
+                    const uint64_t b0d = smem_desc_mn_sw128_groups(xt + P.mma_off[0], 128, P.k_group_bytes);
+                    const uint64_t b1d = smem_desc_mn_sw128_groups(xt + P.mma_off[1], 128, P.k_group_bytes);
+                    const uint64_t b2d = smem_desc_mn_sw128_groups(xt + P.mma_off[2], 128, P.k_group_bytes);
+                    const uint64_t b3d = smem_desc_mn_sw128_groups(xt + P.mma_off[3], 128, P.k_group_bytes);
+                    if (p == p0) tc_mma_ss<false>(d_tmem, adesc, b0d, idesc);
+                    else tc_mma_ss<true>(d_tmem, adesc, b0d, idesc);
+                    tc_mma_ss<true>(d_tmem, adesc + 128, b1d, idesc);
+                    tc_mma_ss<true>(d_tmem, adesc + 256, b2d, idesc);
+                    tc_mma_ss<true>(d_tmem, adesc + 384, b3d, idesc);
+                } else {
+                    const uint64_t bdesc = smem_desc_mn_sw128(st + 2 * kDwBlockBytes, kDwBlockBytes);
+                    if (p == p0) tc_mma_ss<false>(d_tmem, adesc, bdesc, idesc);
+                    else tc_mma_ss<true>(d_tmem, adesc, bdesc, idesc);
+                    tc_mma_ss<true>(d_tmem, adesc + 128, bdesc + 128, idesc);
+                    tc_mma_ss<true>(d_tmem, adesc + 256, bdesc + 256, idesc);
+                    tc_mma_ss<true>(d_tmem, adesc + 384, bdesc + 384, idesc);
+                }
                 tc_commit(&sm->empty[s]);
+                if (++s == P.stages) { s = 0; ph ^= 1u; }
             }
             if (ok) tc_commit(&sm->acc_full[buf]);
             ++lu;
         }
+        if (lane == 0) { DWPROF_OUT(0, clock64() - t_all); DWPROF_OUT(1, w_full); DWPROF_OUT(2, w_acc); DWPROF_OUT(3, (long long)it); DWPROF_OUT(4, (long long)lu); }
     } else {
         const int q = warp & 3;
         uint32_t lu = 0;
+        DWPROF_DECL(e_busy);
         for (int u = blockIdx.x; u < P.total_units; u += gridDim.x) {
             int ot, gi, nb, sp, p0, p1;
             unit_range(u, ot, gi, nb, sp, p0, p1);
             const bool have = p1 > p0;
             const int buf = lu & 1;
             if (have && !mbar_wait_warp(&sm->acc_full[buf], (lu >> 1) & 1u, abort_flag, P.status, 32)) break;
+            DWPROF_T(t_e);
             tc_fence_after();
             const int o = ot * 128 + q * 32 + lane;
             float *row = P.partial + (long long)sp * P.split_stride + (long long)o * P.K;
 #pragma unroll 1
             for (int c = 0; c < nb * 2; ++c) {
                 // columns [32c, 32c+32) of the accumulator: half of column block c/2
-                const int i = gi * kDwMaxCb + (c >> 1), t = i / P.cblocks, cb = i - t * P.cblocks;
+                int t, cb;
+                if (P.row_mode) {
+                    const int r = gi / P.cblocks;
+                    cb = gi - r * P.cblocks;
+                    t = r * P.kw + (c >> 1);
+                } else {
+                    const int i = gi * kDwMaxCb + (c >> 1);
+                    t = i / P.cblocks;
+                    cb = i - t * P.cblocks;
+                }
                 const int ch0 = cb * 64 + (c & 1) * 32;          // first input channel of this chunk
                 float *dst = row + P.taps[t].koff + ch0;
                 uint32_t v[32];
@@ -176,12 +257,27 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
                 }
-                if (o < P.Cout) {
-                    if (P.vec_ok && ch0 + 32 <= P.Cin) {
+                if (P.vec_ok && ch0 + 32 <= P.Cin) {
+                    // through shared memory, so that a store instruction writes four whole 128-byte
+                    // lines (4 rows x 8 lanes x 16 bytes) instead of 16 bytes in each of 32 rows
+                    float4 (*stg)[8] = sm->stg[q];
 #pragma unroll
-                        for (int j = 0; j < 8; ++j)
-                            reinterpret_cast<uint4 *>(dst)[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-                    } else {
+                    for (int j = 0; j < 8; ++j)
+                        stg[lane][j ^ (lane & 7)] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                                __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                    __syncwarp();
+                    const int rr = lane >> 3, ch = lane & 7;
+                    float *const base = P.partial + (long long)sp * P.split_stride + P.taps[t].koff + ch0 + ch * 4;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int r = i * 4 + rr;
+                        const int orow = ot * 128 + q * 32 + r;
+                        if (orow < P.Cout)
+                            *reinterpret_cast<float4 *>(base + (long long)orow * P.K) = stg[r][ch ^ (r & 7)];
+                    }
+                    __syncwarp();
+                } else if (o < P.Cout) {
+                    {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
                             if (ch0 + j < P.Cin) dst[j] = __uint_as_float(v[j]);
@@ -194,7 +290,9 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
                 if (lane == 0) mbar_arrive(&sm->acc_empty[buf]);
                 ++lu;
             }
+            DWPROF_ACC(e_busy, t_e);
         }
+        if (warp == 2 && lane == 0) DWPROF_OUT(5, e_busy);
     }
 
     tc_fence_before();
@@ -276,8 +374,27 @@ int dw_plan(const twn_conv_desc_t *d, int sm_count, DwPlan *plan)
     P.cblocks = (int)((d->Cin + 63) / 64);
     P.n_colblocks = P.n_taps * P.cblocks;
     P.n_groups = (P.n_colblocks + kDwMaxCb - 1) / kDwMaxCb;
+    P.kw = d->kw;
+    P.stage_bytes = (2 + kDwMaxCb) * kDwBlockBytes;
+    // row mode: stride 1, 2..4 taps per filter row, the tile inside one image and at least 8 pixels wide
+    if (d->stride_h == 1 && d->stride_w == 1 && d->kw >= 2 && d->kw <= kDwMaxCb && BB == 1 && BW >= 8) {
+        P.row_mode = 1;
+        P.n_groups = d->kh * P.cblocks;
+        const int pitch = BW + d->kw - 1;                 // pixels per row of the widened tile
+        P.x_bytes = pitch * BH * 128;
+        P.k_group_bytes = BW == 8 ? pitch * 128 : 1024;   // second 8-pixel run of an MMA: next row, or same row
+        for (int i = 0; i < 4; ++i) {
+            const int h = (16 * i) / BW, w = (16 * i) % BW;
+            P.mma_off[i] = (h * pitch + w) * 128;
+        }
+        P.stage_bytes = 2 * kDwBlockBytes + ((P.x_bytes + 1023) & ~1023);
+    }
+    P.stages = kDwPoolBytes / P.stage_bytes;
+    if (P.stages > kDwMaxStages) P.stages = kDwMaxStages;
     const long long units = (long long)P.n_otiles * P.n_groups;
-    long long splits = (2LL * sm_count + units - 1) / units;
+    // as many splits as keep the unit count within two full rounds of the grid (never a third,
+    // nearly empty round)
+    long long splits = (2LL * sm_count) / units;
     if (splits > P.pix_tiles) splits = P.pix_tiles;
     if (splits < 1) splits = 1;
     P.tiles_per_split = (int)((P.pix_tiles + splits - 1) / splits);
@@ -351,6 +468,7 @@ extern "C" int twn_conv2d_bwd_weight(const twn_conv_desc_t *d, const void *X, co
         cuuint64_t dims[4] = {(cuuint64_t)d->Cin, (cuuint64_t)d->W, (cuuint64_t)d->H, (cuuint64_t)d->B};
         cuuint64_t strides[3] = {(cuuint64_t)d->Cin * 2, (cuuint64_t)d->W * d->Cin * 2, (cuuint64_t)d->H * d->W * d->Cin * 2};
         cuuint32_t box[4] = {64, (cuuint32_t)(BW * d->stride_w), (cuuint32_t)(BH * d->stride_h), (cuuint32_t)BB};
+        if (P.row_mode) box[1] = (cuuint32_t)(BW + d->kw - 1);
         cuuint32_t estr[4] = {1, (cuuint32_t)d->stride_w, (cuuint32_t)d->stride_h, 1};
         if (enc(&map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(X), dims, strides, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -373,3 +491,7 @@ extern "C" int twn_conv2d_bwd_weight(const twn_conv_desc_t *d, const void *X, co
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }
+
+#ifdef TWN_PROFILE
+extern "C" int twn_dwprof_read(long long *host) { return cudaMemcpyFromSymbol(host, g_dwprof, sizeof(long long) * 256 * 8); }
+#endif

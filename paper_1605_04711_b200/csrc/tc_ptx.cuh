@@ -247,6 +247,22 @@ __device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t saddr, uint32_t 
     return d;
 }
 
+// Same, with the distance between consecutive 8-row K groups given as well.  A tile with a halo
+// serves several taps at once: the groups are 8-pixel runs of image rows (`k_group_bytes` = one
+// halo row when a tile row is 8 pixels wide) and the "next MN block" is the same tile one pixel
+// further (128 bytes).  The swizzle is a function of the absolute shared-memory address, so the
+// start may be any 128-byte row of a 1024-byte aligned buffer.
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128_groups(uint32_t saddr, uint32_t mn_block_bytes, uint32_t k_group_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((mn_block_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((k_group_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
 // kind::f16 instruction descriptor, bf16 operands both MN-major, fp32 accumulate.
 __host__ __device__ constexpr uint32_t make_idesc_mn(int M, int N)
 {
