@@ -53,6 +53,64 @@ im2col_kernel(const __nv_bfloat16 *__restrict__ X, twn_conv_desc_t d, I Ho, I Wo
     }
 }
 
+// Patch variant for short rows (small Cin): a block takes 64 consecutive output pixels of one
+// output row.  The input window they read (kh rows of (63*stride_w + kw) pixels) is copied to
+// shared memory with zeros outside the image; the shared-memory offset of every patch column is
+// tabulated once; then each warp writes whole patch rows, one 16-byte chunk per lane, so that a
+// store instruction covers a contiguous run of the output.
+constexpr int kPatchPix = 64;
+constexpr int kPatchMaxElems = 12288;   // window elements (24 KB)
+constexpr int kPatchMaxCols = 1024;     // ldk
+
+__global__ void __launch_bounds__(kT)
+im2col_patch_kernel(const __nv_bfloat16 *__restrict__ X, twn_conv_desc_t d, int Ho, int Wo, int wseg,
+                    __nv_bfloat16 *__restrict__ out, int ldk, int win_w)
+{
+    extern __shared__ __align__(16) unsigned char smem_patch[];
+    __nv_bfloat16 *win = reinterpret_cast<__nv_bfloat16 *>(smem_patch);       // [kh][win_w * Cin] (+1 zero at the end)
+    int *tab = reinterpret_cast<int *>(smem_patch + ((size_t)(d.kh * win_w * (int)d.Cin + 1) * 2 + 15) / 16 * 16);
+    const int Cin = (int)d.Cin, K = d.kh * d.kw * Cin, row_el = win_w * Cin, zero_at = d.kh * row_el;
+    int blk = blockIdx.x;
+    const int seg = blk % wseg; blk /= wseg;
+    const int ho = blk % Ho, b = blk / Ho;
+    const int wo0 = seg * kPatchPix;
+    const int h0 = ho * d.stride_h - d.pad_h, w0 = wo0 * d.stride_w - d.pad_w;
+    const int H = (int)d.H, W = (int)d.W;
+    for (int i = threadIdx.x; i < zero_at + 1; i += kT) {
+        const int r = i / row_el, j = i - r * row_el;
+        const int w = w0 + j / Cin, h = h0 + r;
+        __nv_bfloat16 x = __float2bfloat16_rn(0.0f);
+        if (i < zero_at && h >= 0 && h < H && w >= 0 && w < W)
+            x = X[(((long long)b * H + h) * W + w0) * Cin + j];
+        win[i] = x;
+    }
+    for (int k = threadIdx.x; k < ldk; k += kT) {
+        int off = zero_at;                       // columns K..ldk-1 read the zero
+        if (k < K) {
+            const int t = k / Cin, c = k - t * Cin, r = t / d.kw, sx = t - r * d.kw;
+            off = r * row_el + sx * Cin + c;
+        }
+        tab[k] = off;
+    }
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int chunks = ldk >> 3;
+    const int step = d.stride_w * Cin;           // window elements between neighbouring output pixels
+    const int npix = Wo - wo0 < kPatchPix ? Wo - wo0 : kPatchPix;
+    __nv_bfloat16 *const orow = out + (((long long)b * Ho + ho) * Wo + wo0) * ldk;
+    for (int ch = lane; ch < chunks; ch += 32) {
+        int o[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) o[e] = tab[ch * 8 + e];
+        for (int p = warp; p < npix; p += kT / 32) {
+            __align__(16) __nv_bfloat16 v[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) v[e] = win[o[e] == zero_at ? zero_at : o[e] + p * step];
+            *reinterpret_cast<uint4 *>(orow + (long long)p * ldk + ch * 8) = *reinterpret_cast<const uint4 *>(v);
+        }
+    }
+}
+
 __device__ __forceinline__ void unpack8(const uint4 v, float (&f)[8])
 {
     const __nv_bfloat162 *p = reinterpret_cast<const __nv_bfloat162 *>(&v);
@@ -264,7 +322,14 @@ extern "C" int twn_im2col(const twn_conv_desc_t *d, const void *X, void *Xcol, i
     TWN_REQUIRE(Ho > 0 && Wo > 0, TWN_ERR_INVALID_ARG);
     const long long items = d->B * Ho * Wo * (ldk / 8);
     const bool small = items * 8 < 0x7fffffffLL && d->B * d->H * d->W * d->Cin < 0x7fffffffLL;
-    if (small)
+    const long long win_w = (long long)(kPatchPix - 1) * d->stride_w + d->kw;
+    const long long wseg = (Wo + kPatchPix - 1) / kPatchPix;
+    if (d->kh * win_w * d->Cin <= kPatchMaxElems && ldk <= kPatchMaxCols && d->B * Ho * wseg < 0x7fffffffLL) {
+        const size_t smem = ((size_t)(d->kh * win_w * d->Cin + 1) * 2 + 15) / 16 * 16 + (size_t)ldk * sizeof(int);
+        im2col_patch_kernel<<<(int)(d->B * Ho * wseg), kT, smem, twn_cu(stream)>>>(
+            static_cast<const __nv_bfloat16 *>(X), *d, (int)Ho, (int)Wo, (int)wseg, static_cast<__nv_bfloat16 *>(Xcol),
+            (int)ldk, (int)win_w);
+    } else if (small)
         im2col_kernel<int><<<blocks_for(items, dev.sm_count), kT, 0, twn_cu(stream)>>>(
             static_cast<const __nv_bfloat16 *>(X), *d, (int)Ho, (int)Wo, static_cast<__nv_bfloat16 *>(Xcol), (int)ldk);
     else

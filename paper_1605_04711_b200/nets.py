@@ -163,20 +163,47 @@ class TernaryNet:
         self.timed.append((kind, name, flops, e0, e1))
 
     # ------------------------------------------------------------------ Algorithm 1, first loop
-    def ternarize_all(self):
+    def ternarize_all(self, join: bool = True):
+        """Per-layer ternarization (and the transposed codes for the backward pass) on side streams.
+        Every layer records an event when its codes are ready; forward and backward wait for the
+        event of the layer they are about to run, so the small ternarization kernels of later
+        layers overlap the convolutions of earlier ones."""
         main = torch.cuda.current_stream()
         for st in self.side_streams:
             st.wait_stream(main)
         for i, L in enumerate(self.layers.values()):
             e = L.extra
-            with torch.cuda.stream(self.side_streams[i % len(self.side_streams)]):
+            st = self.side_streams[i % len(self.side_streams)]
+            with torch.cuda.stream(st):
                 self._call("ternarize", L.name, 0, lambda: twn.ternarize(
                     e["W"], self.delta_factor, e["stats"], e["packed"], e["ld"], None, e["ws"],
                     rows=L.Cout, cols=L.K))
+                e["ready"] = torch.cuda.Event()
+                e["ready"].record(st)
                 if self.train and "packed_b" in e:
                     twn.transpose_codes(e["packed"], e["ld"], L.desc, e["packed_b"], e["ld_b"])
-        for st in self.side_streams:
-            main.wait_stream(st)
+                    e["ready_b"] = torch.cuda.Event()
+                    e["ready_b"].record(st)
+        self._pending_join = True
+        if join:
+            self.join_side_streams()
+
+    def _wait_codes(self, L, key="ready"):
+        ev = L.extra.get(key)
+        if ev is not None:
+            torch.cuda.current_stream().wait_event(ev)
+
+    def join_side_streams(self):
+        """All side-stream work rejoins the current stream (required before a graph capture ends
+        and before the master weights change)."""
+        if getattr(self, "_pending_join", False):
+            main = torch.cuda.current_stream()
+            for st in self.side_streams:
+                main.wait_stream(st)
+            self._pending_join = False
+            for L in self.layers.values():      # nothing left to wait for
+                L.extra.pop("ready", None)
+                L.extra.pop("ready_b", None)
 
     # ------------------------------------------------------------------ forward
     def forward(self):
@@ -187,6 +214,7 @@ class TernaryNet:
                 e = L.extra
                 x, y = self.act[L.src], self.act[L.name]
                 fl = 2 * L.macs
+                self._wait_codes(L)
                 if L.small_cin:
                     twn.im2col(L.desc, x, e["xcol"], L.ldk)
                     M = L.B * L.Ho * L.Wo
@@ -251,6 +279,7 @@ class TernaryNet:
                     e["dw_desc"], x, e["dz"], e["dW"], self.ws_dw, self.status))
                 if L.src != "input":
                     def bwd(res, out, L=L, e=e):
+                        self._wait_codes(L, "ready_b")
                         epi = twn.epilogue(residual=res, out_dtype=twn.BF16)
                         self._call("tconv", L.name + ".dX", 2 * L.macs, lambda: twn.conv2d_bwd_data(
                             L.desc, e["dz"], e["packed_b"], e["ld_b"], e["stats"], epi, out, self.status))
@@ -279,9 +308,10 @@ class TernaryNet:
         self.last_grads = acc
 
     def train_step(self, dlogits):
-        self.ternarize_all()
+        self.ternarize_all(join=False)
         self.forward()
         self.backward(dlogits)
+        self.join_side_streams()
 
     def check_status(self):
         s = twn.read_status(self.status)
