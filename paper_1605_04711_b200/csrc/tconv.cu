@@ -38,6 +38,7 @@
 
 #include "common.cuh"
 #include <cstdlib>
+#include <mutex>
 #include "tc_ptx.cuh"
 
 // Optional cycle counters per role (compiled in with -DTWN_PROFILE, read back with
@@ -822,6 +823,34 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     return launch_conv_t<128>(g, P, X, dev, enc, s);
 }
 
+// Helper streams for launches that are independent of one another (the residue classes of a
+// strided backward-for-data pass write disjoint pixels).  They fork from the caller's stream
+// through an event and join it again the same way, so the caller sees one stream-ordered
+// operation; under stream capture the fork and the join become graph edges.  Created once per
+// device; a mutex keeps two host threads from interleaving their use of the shared events.
+struct ForkPool {
+    cudaStream_t side[3];
+    cudaEvent_t fork, join[3];
+    bool ready = false, failed = false;
+};
+std::mutex g_fork_mutex;
+
+ForkPool *fork_pool(int ordinal)
+{
+    static ForkPool pools[64];
+    ForkPool &p = pools[ordinal];
+    if (p.failed) return nullptr;
+    if (!p.ready) {
+        bool ok = cudaEventCreateWithFlags(&p.fork, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; i < 3 && ok; ++i)
+            ok = cudaStreamCreateWithFlags(&p.side[i], cudaStreamNonBlocking) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&p.join[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) { p.failed = true; return nullptr; }
+        p.ready = true;
+    }
+    return &p;
+}
+
 int check_epilogue(const twn_epilogue_t *e)
 {
     if (!e) return TWN_OK;
@@ -932,10 +961,29 @@ extern "C" int twn_conv2d_bwd_data(const twn_conv_desc_t *d, const void *dZ, con
     const long long Wo = (d->W + 2 * d->pad_w - d->kw) / d->stride_w + 1;
     // One launch per residue class (ph, pw) of the input pixel modulo the stride: inside a
     // class the adjoint is a stride-1 sum over the taps r with (ph + pad - r) divisible by
-    // the stride, reading dZ at ho = h' + (ph + pad - r)/stride.
+    // the stride, reading dZ at ho = h' + (ph + pad - r)/stride.  The classes write disjoint
+    // pixels, so with more than one class they run side by side on helper streams.
+    cudaStream_t user = twn_cu(stream);
+    ForkPool *pool = nullptr;
+    std::unique_lock<std::mutex> lock(g_fork_mutex, std::defer_lock);
+    if (d->stride_h * d->stride_w > 1) {
+        twn_device_info dev;
+        rc = twn_current_device(&dev);
+        if (rc != TWN_OK) return rc;
+        lock.lock();
+        pool = fork_pool(dev.ordinal);
+        if (pool) {
+            TWN_CUDA_OK(cudaEventRecord(pool->fork, user));
+            for (int i = 0; i < 3; ++i) TWN_CUDA_OK(cudaStreamWaitEvent(pool->side[i], pool->fork, 0));
+        }
+    }
+    int cls = 0;
+    int first_error = TWN_OK;
     for (int ph = 0; ph < d->stride_h; ++ph)
         for (int pw = 0; pw < d->stride_w; ++pw) {
             if (ph >= d->H || pw >= d->W) continue;
+            cudaStream_t s = (pool && cls % 4 != 0) ? pool->side[cls % 4 - 1] : user;
+            ++cls;
             Geometry g;
             memset(&g, 0, sizeof g);
             g.XB = d->B; g.XH = Ho; g.XW = Wo; g.XC = d->Cout; g.ldx = d->Cout;
@@ -960,10 +1008,17 @@ extern "C" int twn_conv2d_bwd_data(const twn_conv_desc_t *d, const void *dZ, con
                     t.koff = (int32_t)((r * d->kw + s) * d->Cout);
                 }
             }
-            rc = launch_conv(g, dZ, T_bwd, stats, epi, dX, TWN_F32, dev_status, twn_cu(stream));
-            if (rc != TWN_OK) return rc;
+            rc = launch_conv(g, dZ, T_bwd, stats, epi, dX, TWN_F32, dev_status, s);
+            if (rc != TWN_OK && first_error == TWN_OK) first_error = rc;
         }
-    return TWN_OK;
+    if (pool) {
+        // always rejoin, also after a failed launch: the caller's stream must not be left forked
+        for (int i = 0; i < 3; ++i) {
+            TWN_CUDA_OK(cudaEventRecord(pool->join[i], pool->side[i]));
+            TWN_CUDA_OK(cudaStreamWaitEvent(user, pool->join[i], 0));
+        }
+    }
+    return first_error;
 }
 
 #ifdef TWN_PROFILE
