@@ -234,6 +234,103 @@ maxpool_bwd_kernel(const __nv_bfloat16 *__restrict__ dY, const uint8_t *__restri
     }
 }
 
+// Row variants of the two pooling kernels for the common case (8 channels per thread, 32-bit
+// indices): a block walks whole image rows, so a thread needs one integer division instead of
+// ten, and a power-of-two stride turns the window search of the backward pass into shifts.  These
+// sweeps are otherwise bound by their index arithmetic, not by memory.
+__global__ void __launch_bounds__(kT)
+maxpool_fwd_rows_kernel(const __nv_bfloat16 *__restrict__ X, int B, int H, int W, int C, int k, int stride, int pad,
+                        int Ho, int Wo, __nv_bfloat16 *__restrict__ Y, uint8_t *__restrict__ idx)
+{
+    const int Cv = C >> 3, per_row = Wo * Cv;
+    for (int row = blockIdx.x; row < B * Ho; row += gridDim.x) {
+        const int b = row / Ho, ho = row - b * Ho;
+        const int h_lo = ho * stride - pad;
+        for (int i = threadIdx.x; i < per_row; i += kT) {
+            const int wo = i / Cv, cv = i - wo * Cv;
+            const int w_lo = wo * stride - pad;
+            float best[8];
+            int arg[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { best[e] = -INFINITY; arg[e] = 0; }
+            for (int r = 0; r < k; ++r) {
+                const int h = h_lo + r;
+                if (h < 0 || h >= H) continue;
+                const __nv_bfloat16 *rowp = X + ((size_t)(b * H + h) * W) * C + cv * 8;
+                for (int sx = 0; sx < k; ++sx) {
+                    const int w = w_lo + sx;
+                    if (w < 0 || w >= W) continue;
+                    float x[8];
+                    unpack8(__ldg(reinterpret_cast<const uint4 *>(rowp + (size_t)w * C)), x);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        if (x[e] > best[e]) { best[e] = x[e]; arg[e] = r * k + sx; }
+                }
+            }
+            const size_t o = ((size_t)row * Wo + wo) * C + cv * 8;
+            float t8[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) t8[e] = best[e] == -INFINITY ? 0.0f : best[e];
+            *reinterpret_cast<uint4 *>(Y + o) = pack8(t8);     // exact: the values are bf16 already
+            if (idx) {
+                uint2 a;
+                a.x = arg[0] | (arg[1] << 8) | (arg[2] << 16) | (arg[3] << 24);
+                a.y = arg[4] | (arg[5] << 8) | (arg[6] << 16) | (arg[7] << 24);
+                *reinterpret_cast<uint2 *>(idx + o) = a;
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kT)
+maxpool_bwd_rows_kernel(const __nv_bfloat16 *__restrict__ dY, const uint8_t *__restrict__ idx, int B, int H, int W,
+                        int C, int k, int stride, int lg_stride, int pad, int Ho, int Wo,
+                        __nv_bfloat16 *__restrict__ dX)
+{
+    const int Cv = C >> 3, per_row = W * Cv;
+    // window row / column that covers input coordinate x with tap t: (x + pad - t) / stride when divisible
+    auto window = [&](int xn, int limit) -> int {
+        if (xn < 0) return -1;
+        int q;
+        if (lg_stride >= 0) {
+            if (xn & (stride - 1)) return -1;
+            q = xn >> lg_stride;
+        } else {
+            q = xn / stride;
+            if (q * stride != xn) return -1;
+        }
+        return q < limit ? q : -1;
+    };
+    for (int row = blockIdx.x; row < B * H; row += gridDim.x) {
+        const int b = row / H, h = row - b * H;
+        for (int i = threadIdx.x; i < per_row; i += kT) {
+            const int w = i / Cv, cv = i - w * Cv;
+            float g[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) g[e] = 0.0f;
+            for (int r = 0; r < k; ++r) {
+                const int ho = window(h + pad - r, Ho);
+                if (ho < 0) continue;
+                for (int sx = 0; sx < k; ++sx) {
+                    const int wo = window(w + pad - sx, Wo);
+                    if (wo < 0) continue;
+                    const size_t o = ((size_t)(b * Ho + ho) * Wo + wo) * C + cv * 8;
+                    const int want = r * k + sx;
+                    const uint2 a = __ldg(reinterpret_cast<const uint2 *>(idx + o));
+                    float t8[8];
+                    unpack8(__ldg(reinterpret_cast<const uint4 *>(dY + o)), t8);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const int ai = ((e < 4 ? a.x : a.y) >> (8 * (e & 3))) & 0xFF;
+                        if (ai == want) g[e] += t8[e];
+                    }
+                }
+            }
+            *reinterpret_cast<uint4 *>(dX + ((size_t)row * W + w) * C + cv * 8) = pack8(g);
+        }
+    }
+}
+
 // ---- global average pooling [B,H,W,C] -> [B,C] and its backward
 __global__ void __launch_bounds__(kT)
 avgpool_fwd_kernel(const __nv_bfloat16 *__restrict__ X, long long B, long long HW, long long C,
@@ -354,9 +451,12 @@ extern "C" int twn_maxpool2d_fwd(const void *X, int64_t B, int64_t H, int64_t W,
     const bool small = B * H * W * C < 0x7fffffffLL;
     const bool vec = C % 8 == 0 && twn_aligned(X, 16) && twn_aligned(Y, 16) && twn_aligned(argmax, 8);
     cudaStream_t s = twn_cu(stream);
-    if (vec && small)
-        maxpool_fwd_kernel<int, 8><<<blocks_for(B * Ho * Wo * C / 8, dev.sm_count), kT, 0, s>>>(
-            x, (int)B, (int)H, (int)W, (int)C, k, stride, pad, (int)Ho, (int)Wo, y, argmax);
+    if (vec && small) {
+        const long long rows = B * Ho;
+        const int grid = (int)(rows < dev.sm_count * 16LL ? rows : dev.sm_count * 16LL);
+        maxpool_fwd_rows_kernel<<<grid, kT, 0, s>>>(x, (int)B, (int)H, (int)W, (int)C, k, stride, pad, (int)Ho, (int)Wo,
+                                                    y, argmax);
+    }
     else if (vec)
         maxpool_fwd_kernel<long long, 8><<<blocks_for(B * Ho * Wo * C / 8, dev.sm_count), kT, 0, s>>>(
             x, B, H, W, C, k, stride, pad, Ho, Wo, y, argmax);
@@ -382,9 +482,14 @@ extern "C" int twn_maxpool2d_bwd(const void *dY, const uint8_t *argmax, int64_t 
     const bool small = B * H * W * C < 0x7fffffffLL;
     const bool vec = C % 8 == 0 && twn_aligned(dY, 16) && twn_aligned(dX, 16) && twn_aligned(argmax, 8);
     cudaStream_t s = twn_cu(stream);
-    if (vec && small)
-        maxpool_bwd_kernel<int, 8><<<blocks_for(B * H * W * C / 8, dev.sm_count), kT, 0, s>>>(
-            dy, argmax, (int)B, (int)H, (int)W, (int)C, k, stride, pad, (int)Ho, (int)Wo, dx);
+    if (vec && small) {
+        const long long rows = B * H;
+        const int grid = (int)(rows < dev.sm_count * 16LL ? rows : dev.sm_count * 16LL);
+        int lg = -1;
+        for (int i = 0; i < 8; ++i) if ((1 << i) == stride) lg = i;
+        maxpool_bwd_rows_kernel<<<grid, kT, 0, s>>>(dy, argmax, (int)B, (int)H, (int)W, (int)C, k, stride, lg, pad,
+                                                    (int)Ho, (int)Wo, dx);
+    }
     else if (vec)
         maxpool_bwd_kernel<long long, 8><<<blocks_for(B * H * W * C / 8, dev.sm_count), kT, 0, s>>>(
             dy, argmax, B, H, W, C, k, stride, pad, Ho, Wo, dx);
