@@ -286,10 +286,11 @@ class NetWorkload:
         for op in net.ops:
             if op[0] == "layer":
                 L = op[1]
-                n += 1 + (1 if L.small_cin else 0)                       # forward (+ im2col)
+                n += 1 + (1 if L.small_cin else 0)                       # forward (+ im2col or input fold)
                 if self.train:
                     n += 3 + (1 if L.src != "input" else 0)               # memset + 2 ternarize (+ transpose)
-                    n += 1 + 2                                           # act_bwd, dW + reduce
+                    n += 1 if L.fold else 0                              # folded codes
+                    n += 1 + 2 + (1 if L.fold else 0)                    # act_bwd, dW + reduce (+ unfold)
                     if L.src != "input":
                         n += L.stride * L.stride                         # backward for data
             elif op[0] in ("maxpool", "avgpool"):

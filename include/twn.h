@@ -270,6 +270,35 @@ int twn_conv2d_bwd_weight(const twn_conv_desc_t *desc, const void *X, const void
  */
 int twn_im2col(const twn_conv_desc_t *desc, const void *X, void *Xcol, int64_t ldk, twn_stream_t stream);
 
+/*
+ * Folded form of a stride-2 layer with very few input channels (Sec. 3.1: the first layer of
+ * ResNet-18 is a 7x7 stride-2 convolution on 3 channels).  The paper has no counterpart; it
+ * replaces the patch matrix by a tensor barely larger than the input.  Requirements (else
+ * TWN_ERR_INVALID_ARG): stride_h = stride_w = 2, kh <= 8, kw <= 8, 4*Cin <= 16.
+ *   Xf[b, i, j, (dy*2 + dx)*Cin + c] = X[b, 2i + dy - pad_h, 2j + dx - pad_w, c]   (0 outside the
+ *   image; channels 4*Cin..15 are 0), bf16 [B, Hf, Wf, 16], Hf = Ho + ceil(kh/2) - 1, Wf = Wo + 3.
+ * The layer is then the stride-1 sum over folded rows r' < ceil(kh/2) of the 64 consecutive
+ * elements Xf[b, ho + r', wo .. wo+3, 0..15] against folded codes
+ *   Tf[o][r'*64 + s'*16 + (dy*2 + dx)*Cin + c] = T[o][2r' + dy][2s' + dx][c]   (0 where no tap),
+ * uint32 [Cout][ldf/16] in the packed format of twn_ternarize, ldf = 64*ceil(kh/2).
+ * twn_fold_dims writes Hf, Wf, ldf (any may be NULL); twn_fold_input and twn_fold_codes build Xf
+ * (16-byte aligned, overwritten completely) and Tf from X and the packed codes of twn_ternarize
+ * (alpha and the statistics are unchanged).  twn_conv2d_fwd_folded equals twn_im2col + twn_gemm on
+ * the same layer; twn_conv2d_bwd_weight_folded equals the weight gradient of that layer,
+ * dW fp32 [Cout][kh][kw][Cin] overwritten; workspace as in twn_conv2d_bwd_weight (Cout % 8 == 0).
+ */
+int twn_fold_dims(const twn_conv_desc_t *desc, int64_t *Hf, int64_t *Wf, int64_t *ldf);
+int twn_fold_input(const twn_conv_desc_t *desc, const void *X, void *Xf, twn_stream_t stream);
+int twn_fold_codes(const twn_conv_desc_t *desc, const uint32_t *packed, int64_t ld_codes,
+                   uint32_t *packed_folded, int64_t ld_folded, twn_stream_t stream);
+int twn_conv2d_fwd_folded(const twn_conv_desc_t *desc, const void *Xf, const uint32_t *Tf, int64_t ld_folded,
+                          const twn_stats_t *stats, const twn_epilogue_t *epi, void *Y,
+                          int32_t *dev_status, twn_stream_t stream);
+size_t twn_conv2d_bwd_weight_folded_workspace_bytes(const twn_conv_desc_t *desc);
+int twn_conv2d_bwd_weight_folded(const twn_conv_desc_t *desc, const void *Xf, const void *dZ, float *dW,
+                                 void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                 twn_stream_t stream);
+
 /* Max pooling, window k x k (k <= 15), padding with -inf.  X, Y bf16 NHWC; `argmax` (optional,
  * one byte per output element) records the window position r*k+s of the first maximum in
  * scan order, for the backward pass. */

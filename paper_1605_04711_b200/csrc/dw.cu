@@ -431,9 +431,14 @@ extern "C" size_t twn_conv2d_bwd_weight_workspace_bytes(const twn_conv_desc_t *d
     return plan.ws_bytes;
 }
 
-extern "C" int twn_conv2d_bwd_weight(const twn_conv_desc_t *d, const void *X, const void *dZ, float *dW,
-                                     void *workspace, size_t workspace_bytes, int32_t *dev_status,
-                                     twn_stream_t stream)
+namespace {
+
+// dW of layer `d`.  The activation tensor may be laid out with its own pitches (elements between
+// pixels, rows and images; 0 = dense NHWC), which is how the folded first layer presents windows
+// of four 16-channel pixels as 64-channel pixels.
+int dw_run(const twn_conv_desc_t *d, const void *X, long long x_pix, long long x_row, long long x_img,
+           const void *dZ, float *dW, void *workspace, size_t workspace_bytes, int32_t *dev_status,
+           twn_stream_t stream)
 {
     TWN_REQUIRE(X && dZ && dW && workspace, TWN_ERR_INVALID_ARG);
     twn_device_info dev;
@@ -466,7 +471,8 @@ extern "C" int twn_conv2d_bwd_weight(const twn_conv_desc_t *d, const void *X, co
     }
     {
         cuuint64_t dims[4] = {(cuuint64_t)d->Cin, (cuuint64_t)d->W, (cuuint64_t)d->H, (cuuint64_t)d->B};
-        cuuint64_t strides[3] = {(cuuint64_t)d->Cin * 2, (cuuint64_t)d->W * d->Cin * 2, (cuuint64_t)d->H * d->W * d->Cin * 2};
+        const long long pixp = x_pix ? x_pix : d->Cin, rowp = x_row ? x_row : d->W * pixp, imgp = x_img ? x_img : d->H * rowp;
+        cuuint64_t strides[3] = {(cuuint64_t)pixp * 2, (cuuint64_t)rowp * 2, (cuuint64_t)imgp * 2};
         cuuint32_t box[4] = {64, (cuuint32_t)(BW * d->stride_w), (cuuint32_t)(BH * d->stride_h), (cuuint32_t)BB};
         if (P.row_mode) box[1] = (cuuint32_t)(BW + d->kw - 1);
         cuuint32_t estr[4] = {1, (cuuint32_t)d->stride_w, (cuuint32_t)d->stride_h, 1};
@@ -488,6 +494,76 @@ extern "C" int twn_conv2d_bwd_weight(const twn_conv_desc_t *d, const void *X, co
     long long rb = (n + 255) / 256;
     if (rb > dev.sm_count * 8) rb = dev.sm_count * 8;
     dw_reduce_kernel<<<(int)rb, 256, 0, s>>>(P.partial, n, P.splits, dW);
+    TWN_CUDA_OK(cudaGetLastError());
+    return TWN_OK;
+}
+
+// dW[o][r][s][c]  <-  folded gradient dWf[o][(r/2)*64 + (s/2)*16 + ((r%2)*2 + s%2)*Cin + c]
+__global__ void __launch_bounds__(256)
+dw_unfold_kernel(const float *__restrict__ dWf, int Cout, int kh, int kw, int Cin, int ldf, float *__restrict__ dW)
+{
+    const int K = kh * kw * Cin, total = Cout * K;
+    for (int i = blockIdx.x * 256 + threadIdx.x; i < total; i += gridDim.x * 256) {
+        const int o = i / K, k = i - o * K;
+        const int t = k / Cin, c = k - t * Cin, r = t / kw, sx = t - r * kw;
+        dW[i] = dWf[(size_t)o * ldf + (r >> 1) * 64 + (sx >> 1) * 16 + ((r & 1) * 2 + (sx & 1)) * Cin + c];
+    }
+}
+
+// the stride-1 layer that the folded tensors describe: ceil(kh/2) x 1 taps on 64 "channels"
+int folded_desc(const twn_conv_desc_t *d, twn_conv_desc_t *f, int64_t *Hf, int64_t *Wf, int64_t *ldf)
+{
+    const int rc = twn_fold_dims(d, Hf, Wf, ldf);
+    if (rc != TWN_OK) return rc;
+    *f = *d;
+    f->H = *Hf; f->W = *Wf - 3; f->Cin = 64;
+    f->kh = (int)(*ldf / 64); f->kw = 1;
+    f->stride_h = f->stride_w = 1;
+    f->pad_h = f->pad_w = 0;
+    return TWN_OK;
+}
+
+}  // namespace
+
+extern "C" int twn_conv2d_bwd_weight(const twn_conv_desc_t *d, const void *X, const void *dZ, float *dW,
+                                     void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                     twn_stream_t stream)
+{
+    return dw_run(d, X, 0, 0, 0, dZ, dW, workspace, workspace_bytes, dev_status, stream);
+}
+
+extern "C" size_t twn_conv2d_bwd_weight_folded_workspace_bytes(const twn_conv_desc_t *d)
+{
+    twn_conv_desc_t f;
+    int64_t Hf, Wf, ldf;
+    if (folded_desc(d, &f, &Hf, &Wf, &ldf) != TWN_OK) return 0;
+    const size_t inner = twn_conv2d_bwd_weight_workspace_bytes(&f);
+    if (inner == 0) return 0;
+    // the folded gradient [Cout][ldf] first (256-byte multiple), then the partial sums
+    return (((size_t)d->Cout * (size_t)ldf * sizeof(float) + 255) & ~(size_t)255) + inner;
+}
+
+extern "C" int twn_conv2d_bwd_weight_folded(const twn_conv_desc_t *d, const void *Xf, const void *dZ, float *dW,
+                                            void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                            twn_stream_t stream)
+{
+    twn_conv_desc_t f;
+    int64_t Hf, Wf, ldf;
+    int rc = folded_desc(d, &f, &Hf, &Wf, &ldf);
+    if (rc != TWN_OK) return rc;
+    TWN_REQUIRE(Xf && dZ && dW && workspace, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(twn_aligned(workspace, 16) && twn_aligned(dW, 4), TWN_ERR_MISALIGNED);
+    const size_t head = ((size_t)d->Cout * (size_t)ldf * sizeof(float) + 255) & ~(size_t)255;
+    TWN_REQUIRE(workspace_bytes >= twn_conv2d_bwd_weight_folded_workspace_bytes(d) && workspace_bytes > head,
+                TWN_ERR_WORKSPACE);
+    TWN_REQUIRE(d->Cout * (long long)d->kh * d->kw * d->Cin < 0x7fffffffLL, TWN_ERR_INVALID_ARG);
+    float *dWf = static_cast<float *>(workspace);
+    rc = dw_run(&f, Xf, 16, Wf * 16, Hf * Wf * 16, dZ, dWf, static_cast<char *>(workspace) + head,
+                workspace_bytes - head, dev_status, stream);
+    if (rc != TWN_OK) return rc;
+    const int total = (int)(d->Cout * d->kh * d->kw * d->Cin);
+    dw_unfold_kernel<<<(total + 255) / 256, 256, 0, twn_cu(stream)>>>(dWf, (int)d->Cout, d->kh, d->kw, (int)d->Cin,
+                                                                     (int)ldf, dW);
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }

@@ -331,6 +331,36 @@ maxpool_bwd_rows_kernel(const __nv_bfloat16 *__restrict__ dY, const uint8_t *__r
     }
 }
 
+// ---- folded input of a stride-2 layer with very few channels (the first layer of ResNet-18):
+// the 2 x 2 pixel block at (2i - pad_h, 2j - pad_w) becomes the 4*Cin <= 16 channels of folded
+// pixel (i, j), so that the stride-2 k x k layer is a stride-1 ceil(k/2) x ceil(k/2) layer and the
+// four folded pixels a filter row touches are 64 consecutive bf16 (one tensor-core k-block).
+__global__ void __launch_bounds__(kT)
+fold_input_kernel(const __nv_bfloat16 *__restrict__ X, int B, int H, int W, int Cin, int pad_h, int pad_w, int Hf,
+                  int Wf, __nv_bfloat16 *__restrict__ Xf)
+{
+    const int total = B * Hf * Wf;
+    for (int p = blockIdx.x * kT + threadIdx.x; p < total; p += gridDim.x * kT) {
+        const int j = p % Wf, t = p / Wf, i = t % Hf, b = t / Hf;
+        __align__(16) __nv_bfloat16 v[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) v[e] = __float2bfloat16_rn(0.0f);
+        for (int dy = 0; dy < 2; ++dy) {
+            const int h = 2 * i + dy - pad_h;
+            if (h < 0 || h >= H) continue;
+            for (int dx = 0; dx < 2; ++dx) {
+                const int w = 2 * j + dx - pad_w;
+                if (w < 0 || w >= W) continue;
+                const __nv_bfloat16 *src = X + ((size_t)(b * H + h) * W + w) * Cin;
+                for (int c = 0; c < Cin; ++c) v[(dy * 2 + dx) * Cin + c] = src[c];
+            }
+        }
+        uint4 *dst = reinterpret_cast<uint4 *>(Xf + (size_t)p * 16);
+        dst[0] = reinterpret_cast<const uint4 *>(v)[0];
+        dst[1] = reinterpret_cast<const uint4 *>(v)[1];
+    }
+}
+
 // ---- global average pooling [B,H,W,C] -> [B,C] and its backward
 __global__ void __launch_bounds__(kT)
 avgpool_fwd_kernel(const __nv_bfloat16 *__restrict__ X, long long B, long long HW, long long C,
@@ -432,6 +462,41 @@ extern "C" int twn_im2col(const twn_conv_desc_t *d, const void *X, void *Xcol, i
     else
         im2col_kernel<long long><<<blocks_for(items, dev.sm_count), kT, 0, twn_cu(stream)>>>(
             static_cast<const __nv_bfloat16 *>(X), *d, Ho, Wo, static_cast<__nv_bfloat16 *>(Xcol), (long long)ldk);
+    TWN_CUDA_OK(cudaGetLastError());
+    return TWN_OK;
+}
+
+extern "C" int twn_fold_dims(const twn_conv_desc_t *d, int64_t *Hf, int64_t *Wf, int64_t *ldf)
+{
+    TWN_REQUIRE(d != nullptr, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(d->B > 0 && d->H > 0 && d->W > 0 && d->Cin > 0 && d->Cout > 0 && d->kh > 0 && d->kw > 0 &&
+                    d->pad_h >= 0 && d->pad_w >= 0, TWN_ERR_INVALID_ARG);
+    // foldable: stride 2 both ways, at most 8 x 8 taps, the 2 x 2 block fits 16 channels
+    TWN_REQUIRE(d->stride_h == 2 && d->stride_w == 2 && d->kh <= 8 && d->kw <= 8 && 4 * d->Cin <= 16,
+                TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(d->H + 2 * d->pad_h >= d->kh && d->W + 2 * d->pad_w >= d->kw, TWN_ERR_INVALID_ARG);
+    const int64_t Ho = (d->H + 2 * d->pad_h - d->kh) / 2 + 1, Wo = (d->W + 2 * d->pad_w - d->kw) / 2 + 1;
+    const int64_t rf = (d->kh + 1) / 2;
+    if (Hf) *Hf = Ho + rf - 1;
+    if (Wf) *Wf = Wo + 3;         // the 64-element window of the last output pixel ends inside the row
+    if (ldf) *ldf = rf * 64;
+    return TWN_OK;
+}
+
+extern "C" int twn_fold_input(const twn_conv_desc_t *d, const void *X, void *Xf, twn_stream_t stream)
+{
+    int64_t Hf, Wf;
+    int rc = twn_fold_dims(d, &Hf, &Wf, nullptr);
+    if (rc != TWN_OK) return rc;
+    TWN_REQUIRE(X && Xf, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(twn_aligned(X, 2) && twn_aligned(Xf, 16), TWN_ERR_MISALIGNED);
+    TWN_REQUIRE(d->B * Hf * Wf * 16 < 0x7fffffffLL && d->B * d->H * d->W * d->Cin < 0x7fffffffLL, TWN_ERR_INVALID_ARG);
+    twn_device_info dev;
+    rc = twn_current_device(&dev);
+    if (rc != TWN_OK) return rc;
+    fold_input_kernel<<<blocks_for(d->B * Hf * Wf, dev.sm_count), kT, 0, twn_cu(stream)>>>(
+        static_cast<const __nv_bfloat16 *>(X), (int)d->B, (int)d->H, (int)d->W, (int)d->Cin, d->pad_h, d->pad_w, (int)Hf,
+        (int)Wf, static_cast<__nv_bfloat16 *>(Xf));
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }

@@ -655,6 +655,7 @@ EncodeTiledFn encode_fn()
 struct Geometry {
     // input tensor X: NHWC [XB, XH, XW, XC] with pixel pitch ldx (elements)
     long long XB, XH, XW, XC, ldx;
+    long long x_row_pitch, x_img_pitch;   // elements between rows / images; 0 = dense (XW*ldx, XH*XW*ldx)
     // virtual output grid and embedding
     int Bv, Hv, Wv, OH, OW, osh, osw, ooh, oow;
     long long ldy;
@@ -708,7 +709,9 @@ int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const twn_dev
     CUtensorMap map_x;
     {
         cuuint64_t dims[4] = {(cuuint64_t)g.XC, (cuuint64_t)g.XW, (cuuint64_t)g.XH, (cuuint64_t)g.XB};
-        cuuint64_t strides[3] = {(cuuint64_t)g.ldx * 2, (cuuint64_t)g.XW * g.ldx * 2, (cuuint64_t)g.XH * g.XW * g.ldx * 2};
+        const long long rowp = g.x_row_pitch ? g.x_row_pitch : g.XW * g.ldx;
+        const long long imgp = g.x_img_pitch ? g.x_img_pitch : g.XH * rowp;
+        cuuint64_t strides[3] = {(cuuint64_t)g.ldx * 2, (cuuint64_t)rowp * 2, (cuuint64_t)imgp * 2};
         // with a traversal stride the box counts traversed elements: N loaded elements need N * stride
         cuuint32_t box[4] = {(cuuint32_t)kBlockK, (cuuint32_t)(BW * g.sw), (cuuint32_t)(BH * g.sh), (cuuint32_t)BB};
         cuuint32_t estr[4] = {1, (cuuint32_t)g.sw, (cuuint32_t)g.sh, 1};
@@ -941,6 +944,39 @@ extern "C" int twn_conv2d_fwd(const twn_conv_desc_t *d, const void *X, const uin
             t.koff = (int32_t)((r * d->kw + s) * d->Cin);
         }
     return launch_conv(g, X, T_fwd, stats, epi, Y, TWN_F32, dev_status, twn_cu(stream));
+}
+
+extern "C" int twn_conv2d_fwd_folded(const twn_conv_desc_t *d, const void *Xf, const uint32_t *Tf, int64_t ld_folded,
+                                     const twn_stats_t *stats, const twn_epilogue_t *epi, void *Y,
+                                     int32_t *dev_status, twn_stream_t stream)
+{
+    int64_t Hf, Wf, ldf;
+    int rc = twn_fold_dims(d, &Hf, &Wf, &ldf);
+    if (rc != TWN_OK) return rc;
+    TWN_REQUIRE(Xf && Tf && Y && ld_folded == ldf, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(twn_aligned(Xf, 16) && twn_aligned(Tf, 16) && twn_aligned(Y, 4) && twn_aligned(stats, 8) &&
+                    twn_aligned(dev_status, 4), TWN_ERR_MISALIGNED);
+    rc = check_epilogue(epi);
+    if (rc != TWN_OK) return rc;
+    const long long Ho = (d->H + 2 * d->pad_h - d->kh) / 2 + 1, Wo = (d->W + 2 * d->pad_w - d->kw) / 2 + 1;
+    // A 64-"channel" tensor whose pixels are 16 elements apart: window position w reads folded
+    // pixels w..w+3.  One tap per folded filter row, stride 1, no padding.
+    Geometry g;
+    memset(&g, 0, sizeof g);
+    g.XB = d->B; g.XH = Hf; g.XW = Wo; g.XC = 64; g.ldx = 16;
+    g.x_row_pitch = Wf * 16; g.x_img_pitch = Hf * Wf * 16;
+    g.Bv = (int)d->B; g.Hv = (int)Ho; g.Wv = (int)Wo; g.OH = (int)Ho; g.OW = (int)Wo;
+    g.osh = g.osw = 1; g.ooh = g.oow = 0; g.ldy = d->Cout;
+    g.sh = g.sw = 1;
+    g.Cout = (int)d->Cout; g.ld_codes = ldf; g.code_cols = ldf;
+    g.Cin = 64;
+    for (int r = 0; r < (int)(ldf / 64); ++r) {
+        Tap &t = g.taps[g.n_taps++];
+        t.dh = (int16_t)r;
+        t.dw = 0;
+        t.koff = (int32_t)(r * 64);
+    }
+    return launch_conv(g, Xf, Tf, stats, epi, Y, TWN_F32, dev_status, twn_cu(stream));
 }
 
 extern "C" int twn_conv2d_bwd_data(const twn_conv_desc_t *d, const void *dZ, const uint32_t *T_bwd, int64_t ld_codes,

@@ -438,6 +438,33 @@ transpose_codes_kernel(const uint32_t *__restrict__ in, int ld_in, int Cout, int
     }
 }
 
+// Codes of a stride-2 layer re-ordered for the folded input: folded row r' holds 64 columns,
+// column s'*16 + (dy*2 + dx)*Cin + c  <-  tap (2r' + dy, 2s' + dx), channel c; columns without a
+// tap (past kh or kw, or past 4*Cin inside a 16-group) are 0.
+__global__ void __launch_bounds__(kThreads)
+fold_codes_kernel(const uint32_t *__restrict__ in, int ld_in, int Cout, int Cin, int kh, int kw,
+                  uint32_t *__restrict__ out, int ld_out)
+{
+    const int wpr_out = ld_out >> 4, wpr_in = ld_in >> 4;
+    const int total = Cout * wpr_out;
+    for (int w = blockIdx.x * kThreads + threadIdx.x; w < total; w += gridDim.x * kThreads) {
+        const int o = w / wpr_out;
+        const int j0 = (w - o * wpr_out) << 4;      // a word is one (r', s') group of 16 columns
+        const int rf = j0 >> 6, sf = (j0 >> 4) & 3;
+        uint32_t word = 0;
+        for (int e = 0; e < 4 * Cin; ++e) {
+            const int blk = e / Cin, c = e - blk * Cin;
+            const int r = 2 * rf + (blk >> 1), sx = 2 * sf + (blk & 1);
+            if (r < kh && sx < kw) {
+                const int src = (r * kw + sx) * Cin + c;
+                const uint32_t f = (__ldg(in + (size_t)o * wpr_in + (src >> 4)) >> field_pos(src & 15)) & 3u;
+                word |= f << field_pos(e);
+            }
+        }
+        out[w] = word;
+    }
+}
+
 int grid_for(long long items_per_thread_units, int sm_count)
 {
     long long blocks = (items_per_thread_units + kThreads - 1) / kThreads;
@@ -614,6 +641,26 @@ extern "C" int twn_transpose_codes(const uint32_t *packed_fwd, int64_t ld_fwd,
                     ld_bwd < 0x7fffffffLL, TWN_ERR_INVALID_ARG);
     transpose_codes_kernel<<<grid_for(words, dev.sm_count), kThreads, 0, twn_cu(stream)>>>(
         packed_fwd, (int)ld_fwd, (int)d->Cout, (int)d->Cin, (int)taps, packed_bwd, (int)ld_bwd);
+    TWN_CUDA_OK(cudaGetLastError());
+    return TWN_OK;
+}
+
+extern "C" int twn_fold_codes(const twn_conv_desc_t *d, const uint32_t *packed, int64_t ld_codes,
+                              uint32_t *packed_folded, int64_t ld_folded, twn_stream_t stream)
+{
+    int64_t ldf = 0;
+    int rc = twn_fold_dims(d, nullptr, nullptr, &ldf);
+    if (rc != TWN_OK) return rc;
+    TWN_REQUIRE(packed && packed_folded, TWN_ERR_INVALID_ARG);
+    const long long K = (long long)d->kh * d->kw * d->Cin;
+    TWN_REQUIRE(ld_codes % 64 == 0 && ld_codes >= K && ld_folded == ldf, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(twn_aligned(packed, 16) && twn_aligned(packed_folded, 16), TWN_ERR_MISALIGNED);
+    TWN_REQUIRE(d->Cout * (ldf / 16) < 0x7fffffffLL && d->Cout * (ld_codes / 16) < 0x7fffffffLL, TWN_ERR_INVALID_ARG);
+    twn_device_info dev;
+    rc = twn_current_device(&dev);
+    if (rc != TWN_OK) return rc;
+    fold_codes_kernel<<<grid_for(d->Cout * (ldf / 16), dev.sm_count), kThreads, 0, twn_cu(stream)>>>(
+        packed, (int)ld_codes, (int)d->Cout, (int)d->Cin, d->kh, d->kw, packed_folded, (int)ldf);
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }

@@ -47,6 +47,7 @@ class Layer:
     desc: object = None
     K: int = 0
     small_cin: bool = False
+    fold: tuple | None = None      # (Hf, Wf, ldf) when the layer runs in folded form
     ldk: int = 0
     extra: dict = field(default_factory=dict)
 
@@ -108,7 +109,14 @@ class TernaryNet:
                 else:
                     e["scale"] = e["shift"] = None
                 M = B * L.Ho * L.Wo
-                if L.small_cin:
+                # a stride-2 layer on very few channels runs in folded form, other small-Cin layers
+                # through the patch matrix
+                L.fold = twn.fold_dims(L.desc) if L.small_cin else None
+                if L.fold:
+                    Hf, Wf, ldf = L.fold
+                    e["xf"] = torch.zeros((B, Hf, Wf, 16), dtype=torch.bfloat16, device="cuda")
+                    e["packed_f"] = torch.zeros((L.Cout, ldf // 16), dtype=torch.int32, device="cuda")
+                elif L.small_cin:
                     L.ldk = (L.K + 7) // 8 * 8
                     e["xcol"] = torch.zeros((M, L.ldk), dtype=torch.bfloat16, device="cuda")
                 out_dtype = torch.float32 if L.out_f32 else torch.bfloat16
@@ -122,13 +130,18 @@ class TernaryNet:
                         e["ld_b"] = twn.ld_for(L.k * L.k * L.Cout)
                         e["packed_b"] = torch.zeros((L.Cin, e["ld_b"] // 16), dtype=torch.int32, device="cuda")
                     e["dz"] = torch.zeros((B, L.Ho, L.Wo, L.Cout), dtype=torch.bfloat16, device="cuda")
-                    if L.small_cin:
+                    if L.fold:
+                        e["dw_desc"] = L.desc
+                        e["dW"] = torch.zeros((L.Cout, L.K), dtype=torch.float32, device="cuda")
+                        ws_dw = max(ws_dw, twn.conv2d_bwd_weight_folded_workspace_bytes(L.desc))
+                    elif L.small_cin:
                         e["dw_desc"] = twn.conv_desc(1, 1, M, L.ldk, L.Cout, 1, 1, 0)
                         e["dW"] = torch.zeros((L.Cout, L.ldk), dtype=torch.float32, device="cuda")
+                        ws_dw = max(ws_dw, twn.conv2d_bwd_weight_workspace_bytes(e["dw_desc"]))
                     else:
                         e["dw_desc"] = L.desc
                         e["dW"] = torch.zeros((L.Cout, L.K), dtype=torch.float32, device="cuda")
-                    ws_dw = max(ws_dw, twn.conv2d_bwd_weight_workspace_bytes(e["dw_desc"]))
+                        ws_dw = max(ws_dw, twn.conv2d_bwd_weight_workspace_bytes(e["dw_desc"]))
             elif kind == "maxpool":
                 _, name, src, k, s, p = op
                 Bx, H, W, C = self.act[src].shape
@@ -178,6 +191,8 @@ class TernaryNet:
                 self._call("ternarize", L.name, 0, lambda: twn.ternarize(
                     e["W"], self.delta_factor, e["stats"], e["packed"], e["ld"], None, e["ws"],
                     rows=L.Cout, cols=L.K))
+                if L.fold:
+                    twn.fold_codes(L.desc, e["packed"], e["ld"], e["packed_f"], L.fold[2])
                 e["ready"] = torch.cuda.Event()
                 e["ready"].record(st)
                 if self.train and "packed_b" in e:
@@ -215,7 +230,11 @@ class TernaryNet:
                 x, y = self.act[L.src], self.act[L.name]
                 fl = 2 * L.macs
                 self._wait_codes(L)
-                if L.small_cin:
+                if L.fold:
+                    twn.fold_input(L.desc, x, e["xf"])
+                    self._call("tconv", L.name + ".fwd", fl, lambda: twn.conv2d_fwd_folded(
+                        L.desc, e["xf"], e["packed_f"], L.fold[2], e["stats"], e["epi"], y, self.status))
+                elif L.small_cin:
                     twn.im2col(L.desc, x, e["xcol"], L.ldk)
                     M = L.B * L.Ho * L.Wo
                     self._call("tconv", L.name + ".fwd", fl, lambda: twn.gemm(
@@ -274,9 +293,13 @@ class TernaryNet:
                 twn.act_bwd(dY, y, e["scale"], n, L.Cout, e["dz"], dpre)
                 if L.residual:
                     emit_tensor(L.residual, dpre)
-                x = e["xcol"] if L.small_cin else self.act[L.src]
-                self._call("dw", L.name + ".dW", 2 * L.macs, lambda: twn.conv2d_bwd_weight(
-                    e["dw_desc"], x, e["dz"], e["dW"], self.ws_dw, self.status))
+                if L.fold:
+                    self._call("dw", L.name + ".dW", 2 * L.macs, lambda: twn.conv2d_bwd_weight_folded(
+                        L.desc, e["xf"], e["dz"], e["dW"], self.ws_dw, self.status))
+                else:
+                    x = e["xcol"] if L.small_cin else self.act[L.src]
+                    self._call("dw", L.name + ".dW", 2 * L.macs, lambda: twn.conv2d_bwd_weight(
+                        e["dw_desc"], x, e["dz"], e["dW"], self.ws_dw, self.status))
                 if L.src != "input":
                     def bwd(res, out, L=L, e=e):
                         self._wait_codes(L, "ready_b")

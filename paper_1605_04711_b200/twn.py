@@ -66,6 +66,7 @@ def lib() -> C.CDLL:
         l.twn_strerror.restype = C.c_char_p
         l.twn_ternarize_workspace_bytes.restype = C.c_size_t
         l.twn_conv2d_bwd_weight_workspace_bytes.restype = C.c_size_t
+        l.twn_conv2d_bwd_weight_folded_workspace_bytes.restype = C.c_size_t
         _lib = l
     return _lib
 
@@ -207,6 +208,39 @@ def conv2d_bwd_data(desc: ConvDesc, dZ: torch.Tensor, T_bwd: torch.Tensor, ld_co
 
 def im2col(desc: ConvDesc, X: torch.Tensor, Xcol: torch.Tensor, ldk: int, stream=None) -> None:
     _check(lib().twn_im2col(C.byref(desc), _ptr(X), _ptr(Xcol), C.c_int64(ldk), _stream(stream)), "twn_im2col")
+
+
+def fold_dims(desc: ConvDesc):
+    """(Hf, Wf, ldf) of the folded form of a stride-2 layer with few channels, or None if the
+    layer cannot be folded."""
+    hf, wf, ldf = C.c_int64(0), C.c_int64(0), C.c_int64(0)
+    rc = lib().twn_fold_dims(C.byref(desc), C.byref(hf), C.byref(wf), C.byref(ldf))
+    return (hf.value, wf.value, ldf.value) if rc == 0 else None
+
+
+def fold_input(desc: ConvDesc, X, Xf, stream=None) -> None:
+    _check(lib().twn_fold_input(C.byref(desc), _ptr(X), _ptr(Xf), _stream(stream)), "twn_fold_input")
+
+
+def fold_codes(desc: ConvDesc, packed, ld_codes: int, packed_folded, ld_folded: int, stream=None) -> None:
+    _check(lib().twn_fold_codes(C.byref(desc), _ptr(packed), C.c_int64(ld_codes), _ptr(packed_folded),
+                                C.c_int64(ld_folded), _stream(stream)), "twn_fold_codes")
+
+
+def conv2d_fwd_folded(desc: ConvDesc, Xf, Tf, ld_folded: int, stats, epi, Y, dev_status=None, stream=None) -> None:
+    _check(lib().twn_conv2d_fwd_folded(C.byref(desc), _ptr(Xf), _ptr(Tf), C.c_int64(ld_folded), _ptr(stats),
+                                       C.byref(epi) if epi is not None else None, _ptr(Y), _ptr(dev_status),
+                                       _stream(stream)), "twn_conv2d_fwd_folded")
+
+
+def conv2d_bwd_weight_folded_workspace_bytes(desc: ConvDesc) -> int:
+    return int(lib().twn_conv2d_bwd_weight_folded_workspace_bytes(C.byref(desc)))
+
+
+def conv2d_bwd_weight_folded(desc: ConvDesc, Xf, dZ, dW, workspace, dev_status=None, stream=None) -> None:
+    _check(lib().twn_conv2d_bwd_weight_folded(C.byref(desc), _ptr(Xf), _ptr(dZ), _ptr(dW), _ptr(workspace),
+                                              C.c_size_t(workspace.numel() * workspace.element_size()),
+                                              _ptr(dev_status), _stream(stream)), "twn_conv2d_bwd_weight_folded")
 
 
 def maxpool2d_fwd(X, B, H, W, Cc, k, stride, pad, Y, argmax=None, stream=None) -> None:

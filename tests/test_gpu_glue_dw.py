@@ -88,6 +88,85 @@ def test_im2col_then_gemm_is_the_small_channel_conv(case):
     assert np.all(host_bf16_bits(Xcol)[:, K:] == 0)
 
 
+FOLD_CASES = [
+    # B, H, W, Cin, Cout, k, pad  (stride 2)
+    (2, 30, 30, 3, 32, 7, 3),      # the ResNet stem shape in small
+    (3, 17, 23, 3, 64, 7, 3),      # odd extents: ragged last window
+    (2, 20, 20, 1, 16, 5, 2),      # one channel, 5x5
+    (1, 9, 9, 4, 8, 8, 4),         # largest filter and channel count the fold takes
+    (2, 12, 10, 2, 24, 2, 0),      # one folded row, no padding
+    (4, 64, 64, 3, 64, 7, 3),      # several tiles
+]
+
+
+@pytest.mark.parametrize("case", FOLD_CASES)
+def test_folded_layer_is_the_strided_small_channel_conv(case):
+    """twn_fold_input + twn_fold_codes + twn_conv2d_fwd_folded / twn_conv2d_bwd_weight_folded against the
+    oracle's plain convolution and weight gradient of the unfolded layer."""
+    B, H, W, Cin, Cout, k, p = case
+    d = twn.conv_desc(B, H, W, Cin, Cout, k, 2, p)
+    od = oracle.conv_desc(B, H, W, Cin, Cout, k, 2, p)
+    K = k * k * Cin
+    Hf, Wf, ldf = twn.fold_dims(d)
+    assert (Hf, Wf, ldf) == (d.Ho + (k + 1) // 2 - 1, d.Wo + 3, 64 * ((k + 1) // 2))
+    Wm = dg.he_normal(3, f"fold{case}", Cout, K)
+    ref, codes = oracle.ternarize(Wm, 0.7)
+    ld = twn.ld_for(K)
+    stats = twn.new_stats()
+    packed = torch.empty((Cout, ld // 16), dtype=torch.int32, device="cuda")
+    wsb = torch.empty(twn.ternarize_workspace_bytes(), dtype=torch.uint8, device="cuda")
+    twn.ternarize(dev_f32(Wm), 0.7, stats, packed, ld, None, wsb, rows=Cout, cols=K)
+    X = dg.draw_bf16(3, f"foldx{case}", B * H * W * Cin, "normal").reshape(B, H, W, Cin)
+    Xf = torch.full((B, Hf, Wf, 16), 7.0, dtype=torch.bfloat16, device="cuda")
+    twn.fold_input(d, dev_bf16(X), Xf)
+    # the folded tensor, element by element (bit-exact: it only moves values)
+    xf = host_bf16_bits(Xf).reshape(B, Hf, Wf, 16)
+    want = np.zeros_like(xf)
+    for dy in range(2):
+        for dx in range(2):
+            hs = 2 * np.arange(Hf) + dy - p
+            ws_ = 2 * np.arange(Wf) + dx - p
+            hv, wv = (hs >= 0) & (hs < H), (ws_ >= 0) & (ws_ < W)
+            blk = np.zeros((B, Hf, Wf, Cin), dtype=xf.dtype)
+            blk[np.ix_(np.arange(B), np.nonzero(hv)[0], np.nonzero(wv)[0])] = X[np.ix_(np.arange(B), hs[hv], ws_[wv])]
+            want[..., (dy * 2 + dx) * Cin:(dy * 2 + dx + 1) * Cin] = blk
+    assert np.array_equal(xf, want)
+    Tf = torch.full((Cout, ldf // 16), -1, dtype=torch.int32, device="cuda")
+    twn.fold_codes(d, packed, ld, Tf, ldf)
+    cf = oracle.unpack(Tf.cpu().numpy().view(np.uint32), Cout, ldf, ldf).reshape(Cout, ldf // 64, 4, 16)
+    c4 = codes.reshape(Cout, k, k, Cin)
+    for rf in range(ldf // 64):
+        for sf in range(4):
+            for dy in range(2):
+                for dx in range(2):
+                    r, sx = 2 * rf + dy, 2 * sf + dx
+                    got = cf[:, rf, sf, (dy * 2 + dx) * Cin:(dy * 2 + dx + 1) * Cin]
+                    assert np.array_equal(got, c4[:, r, sx, :] if r < k and sx < k else np.zeros_like(got))
+            assert not cf[:, rf, sf, 4 * Cin:].any()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    Y = torch.full((B, d.Ho, d.Wo, Cout), float("nan"), dtype=torch.float32, device="cuda")
+    twn.conv2d_fwd_folded(d, Xf, Tf, ldf, stats, None, Y, status)
+    assert twn.read_status(status) == 0
+    Yr, A = oracle.conv2d_fwd(od, X, c4, ref.alpha)
+    err = np.abs(Y.cpu().numpy().astype(np.float64) - Yr)
+    assert np.all(err <= 1e-4 * ref.alpha * A + 1e-6)
+    # straight-through weight gradient of the same layer
+    dZ = dg.draw_bf16(3, f"foldz{case}", B * d.Ho * d.Wo * Cout, "normal", 0.0, 0.1).reshape(B, d.Ho, d.Wo, Cout)
+    dW = torch.full((Cout, k, k, Cin), float("nan"), dtype=torch.float32, device="cuda")
+    ws = torch.empty(twn.conv2d_bwd_weight_folded_workspace_bytes(d), dtype=torch.uint8, device="cuda")
+    twn.conv2d_bwd_weight_folded(d, Xf, dev_bf16(dZ), dW, ws, status)
+    assert twn.read_status(status) == 0
+    dref, Aw = oracle.conv2d_bwd_weight(od, X, dZ)
+    errw = np.abs(dW.cpu().numpy().astype(np.float64).reshape(dref.shape) - dref)
+    assert np.all(errw <= 1e-4 * Aw + 1e-6), f"worst err/tol {np.max(errw / (1e-4 * Aw + 1e-6)):.3g}"
+
+
+def test_fold_rejects_layers_it_cannot_take():
+    assert twn.fold_dims(twn.conv_desc(1, 8, 8, 3, 8, 3, 1, 1)) is None      # stride 1
+    assert twn.fold_dims(twn.conv_desc(1, 8, 8, 8, 8, 3, 2, 1)) is None      # 4*Cin > 16
+    assert twn.fold_dims(twn.conv_desc(1, 32, 32, 3, 8, 9, 2, 4)) is None    # more than 8 taps per side
+
+
 @pytest.mark.parametrize("k,s,p,H,W,C", [(2, 2, 0, 24, 24, 32), (3, 2, 1, 112, 112, 8), (3, 2, 1, 7, 9, 5), (2, 2, 0, 8, 8, 512)])
 def test_maxpool_forward_and_backward(k, s, p, H, W, C):
     B = 2
