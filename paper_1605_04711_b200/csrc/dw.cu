@@ -128,7 +128,10 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
             for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
                 int ot, gi, nb, sp, p0, p1;
                 unit_range(u, ot, gi, nb, sp, p0, p1);
-                const uint32_t bytes = 2 * kDwBlockBytes + (P.row_mode ? P.x_bytes : nb * kDwBlockBytes);
+                // the second 64-channel block of dZ is not loaded when it lies past Cout: what the MMA
+                // then reads there lands in accumulator rows that are never stored
+                const bool a1 = ot * 128 + 64 < P.Cout;
+                const uint32_t bytes = (a1 ? 2 : 1) * kDwBlockBytes + (P.row_mode ? P.x_bytes : nb * kDwBlockBytes);
                 // Everything that does not change along the pixel tiles is worked out here: this one
                 // thread paces the pipeline, and an integer division costs it hundreds of cycles.
                 int xc[kDwMaxCb], xdw[kDwMaxCb], xdh[kDwMaxCb];
@@ -157,7 +160,7 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
                     if (!mbar_wait(&sm->empty[s], ph ^ 1u, abort_flag, P.status, 32)) { ok = false; break; }
                     mbar_expect_tx(&sm->full[s], bytes);
                     tma_load_4d(st, &map_dz, &sm->full[s], ot * 128, w0, h0, b0);
-                    tma_load_4d(st + kDwBlockBytes, &map_dz, &sm->full[s], ot * 128 + 64, w0, h0, b0);
+                    if (a1) tma_load_4d(st + kDwBlockBytes, &map_dz, &sm->full[s], ot * 128 + 64, w0, h0, b0);
 #pragma unroll
                     for (int j = 0; j < kDwMaxCb; ++j)
                         if (j < nx)
@@ -394,7 +397,7 @@ int dw_plan(const twn_conv_desc_t *d, int sm_count, DwPlan *plan)
     const long long units = (long long)P.n_otiles * P.n_groups;
     // as many splits as keep the unit count within two full rounds of the grid (never a third,
     // nearly empty round)
-    long long splits = (2LL * sm_count) / units;
+    long long splits = (1LL * sm_count) / units;
     if (splits > P.pix_tiles) splits = P.pix_tiles;
     if (splits < 1) splits = 1;
     P.tiles_per_split = (int)((P.pix_tiles + splits - 1) / splits);
