@@ -162,7 +162,10 @@ class TernarizeWorkload:
         return {"bound": "hbm", "kernel": "sum_abs_kernel + code_pack_kernel (one twn_ternarize call)",
                 "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": ach / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                "frac_of_nominal_8TBs": ach / 8000.0, "traffic": None}
+                "frac_of_nominal_8TBs": ach / 8000.0,
+                # dram__bytes_read.sum + dram__bytes_write.sum of the two kernels of one call (ncu capture of
+                # this workload, summarised under profiles/); algorithmic: 8.25e8
+                "traffic": 819.6e6 if self.n == 100_000_000 else None}
 
     def check(self):
         st = self.twn.stats_to_host(self.stats)
@@ -175,6 +178,90 @@ class TernarizeWorkload:
         oracle.pack(codes, self.ld)
         dt = time.perf_counter() - t0
         return self.n * self.bytes_per_unit / dt / 1e9, f"full tensor, n={self.n}", 1
+
+
+class GemmWorkload:
+    """One ternary-weight GEMM (Algorithm 1, forward of a fully connected layer): Y = alpha * X T^T with
+    bf16 X [M, K], 2-bit T [N, K] ternarized from N(0,1) weights, bf16 Y.  2MNK flops per step."""
+    metric = "ternary GEMM TFLOP/s"
+    unit = "TFLOP/s"
+    dtype = "bf16"
+    default_steps = 200
+
+    def __init__(self, M, N=4096, K=4096, seed=0):
+        self.M, self.N, self.K, self.seed = M, N, K, seed
+        self.name = f"ternary_gemm_m{M}_n{N}_k{K}"
+
+    def config(self):
+        mb = (2 * self.M * self.K + 2 * self.M * self.N) / 1e6
+        return {"workload": self.name, "seed": self.seed, "delta_factor": 0.7,
+                "l2": f"X and Y of a step: {mb:.0f} MB" + (" (larger than L2)" if mb > 126 else " (fits L2: weights and X stay resident, as in a served layer)")}
+
+    def host_inputs(self):
+        from paper_1605_04711_b200 import datagen as dg
+        return (dg.draw(self.seed, "gemm.w", self.N * self.K, "normal").reshape(self.N, self.K),
+                dg.draw_bf16(self.seed, "gemm.x", self.M * self.K, "normal").reshape(self.M, self.K))
+
+    def setup(self, torch, twn, host):
+        import numpy as np
+        self.torch, self.twn = torch, twn
+        Wm, X = host
+        self.ld = twn.ld_for(self.K)
+        self.stats = twn.new_stats()
+        self.packed = torch.empty((self.N, self.ld // 16), dtype=torch.int32, device="cuda")
+        ws = torch.empty(twn.ternarize_workspace_bytes(), dtype=torch.uint8, device="cuda")
+        twn.ternarize(torch.from_numpy(Wm).cuda(), 0.7, self.stats, self.packed, self.ld, None, ws,
+                      rows=self.N, cols=self.K)
+        self.host_x = torch.from_numpy(X.view(np.int16)).pin_memory()
+        self.X = self.host_x.cuda().view(torch.bfloat16)
+        self.Y = torch.empty((self.M, self.N), dtype=torch.bfloat16, device="cuda")
+        self.host_y = torch.empty((self.M, self.N), dtype=torch.int16).pin_memory()
+        self.epi = twn.epilogue(out_dtype=twn.BF16)
+        self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def step(self):
+        self.twn.gemm(self.X, self.K, self.packed, self.ld, self.stats, self.M, self.N, self.K, self.epi,
+                      self.Y, self.N, self.status)
+
+    def step_e2e(self):
+        self.X.view(self.torch.int16).copy_(self.host_x, non_blocking=True)
+        self.step()
+        self.host_y.copy_(self.Y.view(self.torch.int16), non_blocking=True)
+
+    def e2e_bytes(self):
+        return self.M * self.K * 2, self.M * self.N * 2
+
+    def launches_per_step(self):
+        return 1
+
+    def units_per_step(self):
+        return 2.0 * self.M * self.N * self.K / 1e12
+
+    def roofline(self, ms_per_step, peaks):
+        ach = self.units_per_step() / (ms_per_step * 1e-3)
+        return {"bound": "tensor", "kernel": "tconv_kernel (one twn_gemm call)", "achieved": ach,
+                "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
+                "peak_source": peaks["source"] + " (bf16 burst: the kernel is timed alone)",
+                # DRAM bytes of one launch from the ncu capture of the M = 4096 case (profiles/)
+                "traffic": 40.1e6 if (self.M, self.N, self.K) == (4096, 4096, 4096) else None}
+
+    def check(self):
+        assert self.twn.read_status(self.status) == 0
+        assert bool(self.torch.isfinite(self.Y[:64].float()).all())
+
+    def cpu_sample(self, host, seconds=10.0):
+        import oracle
+        Wm, X = host
+        st, codes = oracle.ternarize(Wm, 0.7)
+        rows = 8
+        while True:
+            t0 = time.perf_counter()
+            oracle.gemm(X[:rows], codes, st.alpha)
+            dt = time.perf_counter() - t0
+            if dt >= seconds * 0.5 or rows >= self.M:
+                break
+            rows = int(min(self.M, max(rows * 2, rows * seconds / max(dt, 1e-3))))
+        return 2.0 * rows * self.N * self.K / dt / 1e12, f"oracle gemm on {rows} of {self.M} rows ({dt:.1f} s)", oracle.num_threads()
 
 
 class NetWorkload:
@@ -354,6 +441,7 @@ class NetWorkload:
 
 
 WORKLOADS = {"ternarize": lambda: TernarizeWorkload(), "resnet18_train": lambda: NetWorkload("resnet18_train"),
+             "gemm_16384": lambda: GemmWorkload(16384), "gemm_4096": lambda: GemmWorkload(4096),
              "vgg7_fwd": lambda: NetWorkload("vgg7_fwd"), "lenet5_fwd": lambda: NetWorkload("lenet5_fwd")}
 DEFAULT_WORKLOAD = "resnet18_train"
 
@@ -364,7 +452,7 @@ def run_reference(args):
     if rank != 0:
         return
     wl = WORKLOADS[args.workload]()
-    host = wl.host_inputs() if isinstance(wl, TernarizeWorkload) else None
+    host = wl.host_inputs() if isinstance(wl, (TernarizeWorkload, GemmWorkload)) else None
     vals = []
     steps = args.steps if args.steps else 3
     for i in range(args.warmup + steps):
@@ -372,7 +460,7 @@ def run_reference(args):
         if i >= args.warmup:
             vals.append(v)
     value = sum(vals) / len(vals)
-    upstep = wl.units_per_step() if isinstance(wl, TernarizeWorkload) else {"resnet18_train": 64, "vgg7_fwd": 128, "lenet5_fwd": 100}[args.workload]
+    upstep = wl.units_per_step() if isinstance(wl, (TernarizeWorkload, GemmWorkload)) else {"resnet18_train": 64, "vgg7_fwd": 128, "lenet5_fwd": 100}[args.workload]
     line = {"impl": "reference", "metric": wl.metric, "value": value, "unit": wl.unit,
             "n_gpus": args.gpus, "steps": steps, "warmup": args.warmup,
             "ms_per_step": upstep / value * 1e3, "higher_is_better": True,
