@@ -79,6 +79,7 @@ class TernaryNet:
         # the per-layer ternarizations are independent: they run on a few side streams, each layer
         # with its own scratch
         self.side_streams = [torch.cuda.Stream() for _ in range(4)]
+        self.dw_stream = torch.cuda.Stream()     # weight gradients run beside the backward-for-data chain
         self.timed = None          # when a list: (kind, name, flops, start event, end event)
         H, W, C = in_shape
         self.act["input"] = torch.zeros((batch, H, W, C), dtype=torch.bfloat16, device="cuda")
@@ -276,6 +277,8 @@ class TernaryNet:
             fn(acc.get(name), out)
             acc[name] = out
 
+        main = torch.cuda.current_stream()
+        self.dw_stream.wait_stream(main)
         for op in reversed(self.ops):
             kind = op[0]
             if kind == "layer":
@@ -293,13 +296,19 @@ class TernaryNet:
                 twn.act_bwd(dY, y, e["scale"], n, L.Cout, e["dz"], dpre)
                 if L.residual:
                     emit_tensor(L.residual, dpre)
-                if L.fold:
-                    self._call("dw", L.name + ".dW", 2 * L.macs, lambda: twn.conv2d_bwd_weight_folded(
-                        L.desc, e["xf"], e["dz"], e["dW"], self.ws_dw, self.status))
-                else:
-                    x = e["xcol"] if L.small_cin else self.act[L.src]
-                    self._call("dw", L.name + ".dW", 2 * L.macs, lambda: twn.conv2d_bwd_weight(
-                        e["dw_desc"], x, e["dz"], e["dW"], self.ws_dw, self.status))
+                # dW needs only dz and the layer's input: it goes to its own stream (one after the
+                # other there, they share the workspace) and overlaps the dX chain of the layers below
+                dz_ready = torch.cuda.Event()
+                dz_ready.record(main)
+                with torch.cuda.stream(self.dw_stream):
+                    self.dw_stream.wait_event(dz_ready)
+                    if L.fold:
+                        self._call("dw", L.name + ".dW", 2 * L.macs, lambda: twn.conv2d_bwd_weight_folded(
+                            L.desc, e["xf"], e["dz"], e["dW"], self.ws_dw, self.status))
+                    else:
+                        x = e["xcol"] if L.small_cin else self.act[L.src]
+                        self._call("dw", L.name + ".dW", 2 * L.macs, lambda: twn.conv2d_bwd_weight(
+                            e["dw_desc"], x, e["dz"], e["dW"], self.ws_dw, self.status))
                 if L.src != "input":
                     def bwd(res, out, L=L, e=e):
                         self._wait_codes(L, "ready_b")
@@ -328,6 +337,7 @@ class TernaryNet:
             elif kind == "flatten":
                 _, name, src = op
                 emit_tensor(src, acc[name].view(self.act[src].shape))
+        main.wait_stream(self.dw_stream)
         self.last_grads = acc
 
     def train_step(self, dlogits):
