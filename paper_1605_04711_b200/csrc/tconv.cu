@@ -70,9 +70,10 @@ constexpr int kChan = 128;          // output channels per tile (UMMA M)
 constexpr int kBlockK = 64;         // reduction elements per k-block (128 bytes of bf16)
 constexpr int kDecodeSets = 1;      // groups of 4 decode warps; a group takes every other stage
 constexpr int kFirstEpiWarp = 2 + 4 * kDecodeSets;
-constexpr int kEpiSets = 2;         // groups of 4 epilogue warps; a group drains every other 32-pixel chunk
-constexpr int kThreadsConv = 32 * (kFirstEpiWarp + 4 * kEpiSets);
-constexpr int kStageBytes = 8192;   // one output staging buffer: 32 pixels of bf16 or 16 pixels of fp32, 128 channels
+constexpr int kEpiSets = 2;         // epilogue warps per lane quadrant; each drains every other 32-pixel chunk
+constexpr int kThreadsConv = 32 * (kFirstEpiWarp + 4 * kEpiSets);   // kEpiWarps epilogue warps
+constexpr int kEpiWarps = 4 * kEpiSets;
+constexpr int kStageBytes = 2048;   // one output staging buffer of a warp: 32 channels x 32 pixels of bf16 or 16 pixels of fp32
 constexpr int kMaxTaps = 64;
 constexpr int kWordTab = 128;       // k-blocks per tile whose code offsets are tabulated in shared memory
 constexpr int kAColsPerBlock = kBlockK / 2;    // 32 columns of bf16 pairs per k-block
@@ -83,11 +84,21 @@ template <> struct Cfg<128> {
     static constexpr int kStages = 4;   // operand ring depth (shared and tensor memory)
     static constexpr int kSub = 2;      // k-blocks per stage: one wait and one commit per 8 MMAs
     static constexpr int kAccBufs = 2;  // the epilogue of a tile overlaps the MMAs of the next
+    static constexpr int kOutBufs = 4;  // output staging buffers per epilogue warp
 };
 template <> struct Cfg<256> {
     static constexpr int kStages = 5;
     static constexpr int kSub = 1;
     static constexpr int kAccBufs = 1;
+    static constexpr int kOutBufs = 2;
+};
+// 192 pixels: the largest tile that leaves room for two accumulators beside four stages of
+// decoded weights (2 x 192 + 4 x 32 = 512 columns); the pixel tile is 3 * 2^k images deep.
+template <> struct Cfg<192> {
+    static constexpr int kStages = 4;
+    static constexpr int kSub = 1;
+    static constexpr int kAccBufs = 2;
+    static constexpr int kOutBufs = 4;
 };
 
 struct Tap {
@@ -117,10 +128,10 @@ struct ConvParams {
     int res_dtype, relu, out_dtype;
     void *Y;
     int32_t *status;
-    // output path: 1 = the tile is staged in shared memory 32 pixels at a time and written with
-    // TMA stores (box = 128 channels x sbw x sbh x sbb pixels); 0 = per-thread stores
+    // output path: 1 = each epilogue warp stages its 32 channels x 32 pixels in shared memory and
+    // writes them with a TMA store (box = 32 channels x sbw x sbh x sbb pixels); 0 = per-thread stores
     int tma_store, lg_sbw, lg_sbh;
-    int res_tma;                  // 1: the residual (bf16) is staged by TMA loads, three chunks deep
+    int res_tma;                  // 1: the residual (bf16) is staged by per-warp TMA loads, two chunks deep
     Tap taps[kMaxTaps];
 };
 
@@ -134,20 +145,22 @@ struct __align__(1024) SmemLayout {
     unsigned long long empty[kStages];     // MMA commit -> TMA and decode: both operand slots are free
     unsigned long long acc_full[2];        // MMA commit -> epilogue
     unsigned long long acc_empty[2];       // epilogue -> MMA
-    alignas(16) uint32_t pix_off[kEpiSets][PIX / kEpiSets];   // output element offset of the pixels of a group's chunks, ~0 = skip
-    alignas(128) uint8_t stage_out[kEpiSets][2][kStageBytes];   // output staging for TMA stores: [pixels][128 channels]
-    alignas(128) __nv_bfloat16 stage_res[kEpiSets][2][32 * kChan];  // residual staging: [32 pixels][128 channels]
-    unsigned long long res_full[kEpiSets][2];
+    // per-warp output staging for TMA stores: [pixels][32 channels].  The stores of the epilogue
+    // queue behind the producer's tile loads in the copy engine, so while the main loop of the next
+    // tile runs a store takes long to release its buffer: the overlapped tile shapes keep four.
+    alignas(128) uint8_t stage_out[kEpiWarps][Cfg<PIX>::kOutBufs][kStageBytes];
+    alignas(128) __nv_bfloat16 stage_res[kEpiWarps][2][32 * 32];  // per-warp residual staging: [32 pixels][32 channels]
+    unsigned long long res_full[kEpiWarps][2];
     uint32_t kword[kWordTab];              // first code word of k-block u in a packed row, u < kWordTab
     uint32_t tmem_base;
     volatile int abort_flag;
-    volatile int epi_ok[kEpiSets][2];      // outcome of a wait of an epilogue group's leader, shared by its four warps
 };
 
 static_assert(offsetof(SmemLayout<128>, stage_res) % 128 == 0 && offsetof(SmemLayout<256>, stage_res) % 128 == 0 &&
-                  sizeof(SmemLayout<256>) + 1024 <= 232448 &&
-                  offsetof(SmemLayout<128>, stage_out) % 128 == 0 && offsetof(SmemLayout<256>, stage_out) % 128 == 0 &&
-                  offsetof(SmemLayout<128>, pix_off) % 16 == 0 && offsetof(SmemLayout<256>, pix_off) % 16 == 0,
+                  offsetof(SmemLayout<192>, stage_res) % 128 == 0 && offsetof(SmemLayout<192>, stage_out) % 128 == 0 &&
+                  sizeof(SmemLayout<256>) + 1024 <= 232448 && sizeof(SmemLayout<128>) + 1024 <= 232448 &&
+                  sizeof(SmemLayout<192>) + 1024 <= 232448 &&
+                  offsetof(SmemLayout<128>, stage_out) % 128 == 0 && offsetof(SmemLayout<256>, stage_out) % 128 == 0,
               "TMA and vector accesses need aligned shared-memory regions");
 
 template <int PIX>
@@ -157,6 +170,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
 {
     using L = SmemLayout<PIX>;
     constexpr int kStages = Cfg<PIX>::kStages, kSub = Cfg<PIX>::kSub, kAccBufs = Cfg<PIX>::kAccBufs;
+    constexpr int kOutBufs = Cfg<PIX>::kOutBufs;
     constexpr int kXBytes = L::kXBytes;
     constexpr int kAColsPerStage = kSub * kAColsPerBlock;
     static_assert(kAccBufs * PIX + kStages * kAColsPerStage <= (int)kTmemCols, "tensor memory budget");
@@ -178,9 +192,9 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         for (int s = 0; s < 8; ++s) mbar_init(&sm->ready_a[s], 4);
         for (int b = 0; b < 2; ++b) {
             mbar_init(&sm->acc_full[b], 1);
-            mbar_init(&sm->acc_empty[b], 4 * kEpiSets);
+            mbar_init(&sm->acc_empty[b], kEpiWarps);
         }
-        for (int b = 0; b < 2 * kEpiSets; ++b) mbar_init(&sm->res_full[0][0] + b, 1);
+        for (int b = 0; b < 2 * kEpiWarps; ++b) mbar_init(&sm->res_full[0][0] + b, 1);
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -406,14 +420,17 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         if (warp == 2 && lane == 0) { PROF_OUT(6, w_full); PROF_OUT(8, PROF_NOW() - t_dec); PROF_OUT(12, d_alu); PROF_OUT(13, d_wst); PROF_OUT(14, d_fetch); PROF_OUT(15, d_st); }
     } else {
         // ------------------------------------------------ epilogue
-        // Two groups of four warps (one warp per tensor-memory lane quadrant); a group drains
-        // every other 32-pixel chunk of the accumulator: tcgen05.ld -> scale / shift / residual /
-        // ReLU -> its own staging buffers -> TMA store by the group's first thread.  Each group
-        // keeps its own bulk-store accounting, residual buffers and named barrier.
+        // Eight warps, two per tensor-memory lane quadrant; the two warps of a quadrant take
+        // alternate 32-pixel chunks of the accumulator.  Every warp works on its own: it drains
+        // its 32 channels x 32 pixels with tcgen05.ld (the load of its next chunk is in flight
+        // while the current one is processed), applies scale / shift / residual / ReLU, stages
+        // the chunk in its own shared-memory buffer and writes it with its own TMA store
+        // (box = 32 channels x 32 pixels).  No barrier joins the epilogue warps, so a warp never
+        // waits for a slower one, and the accumulator goes back to the MMA warp as soon as the
+        // last tensor-memory load of every warp has completed.
         const int q = warp & 3;
-        const int es = (warp - kFirstEpiWarp) >> 2;          // group
-        const int ew = (warp - kFirstEpiWarp) & 3;           // warp inside the group
-        const bool leader = ew == 0 && lane == 0;
+        const int es = (warp - kFirstEpiWarp) >> 2;          // which of the two warps of the quadrant
+        const int ewi = warp - kFirstEpiWarp;                // buffer set of this warp
         // decoded weights are +-2, so half of alpha scales the accumulators
         const float alpha = (P.alpha ? (float)(*P.alpha) : 1.0f) * (1.0f / kDecodedUnit);
         const int BWm = (1 << P.lgBW) - 1, BHm = (1 << P.lgBH) - 1;
@@ -421,13 +438,17 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         const bool need_off = !P.tma_store || (P.residual && !P.res_tma);
         const float floor_v = P.relu ? 0.0f : -INFINITY;
         constexpr int kChunks = PIX / 32;
+        constexpr int kMine = kChunks / kEpiSets;            // chunks of a tile this warp drains
+        static_assert(kChunks % kEpiSets == 0, "the chunks of a tile are split evenly over the warps of a quadrant");
+        uint8_t *const my_out = sm->stage_out[ewi][0];
+        __nv_bfloat16 *const my_res = sm->stage_res[ewi][0];
+        unsigned long long *const my_res_full = sm->res_full[ewi];
         uint32_t lt = 0;
-        uint32_t nst = 0;      // staging buffers this group has filled so far (selects the buffer)
-        uint32_t nres = 0;     // residual chunks this group has consumed so far (buffer and phase)
-        uint32_t ndec = 0;     // joint decisions taken so far: two flags alternate, so that the leader
-                               // never overwrites one that a slower warp has yet to read
+        uint32_t nst = 0;      // staging buffers this warp has filled so far (selects the buffer)
+        uint32_t nres = 0;     // residual chunks this warp has consumed so far (buffer and phase)
+        bool alive = true;
         PROF_DECL(e_wait); PROF_DECL(e_drain); PROF_DECL(e_ld); PROF_DECL(e_grp); PROF_DECL(e_math); PROF_DECL(e_st);
-        for (int tile = blockIdx.x; tile < P.total_tiles; tile += gridDim.x, ++lt) {
+        for (int tile = blockIdx.x; tile < P.total_tiles && alive; tile += gridDim.x, ++lt) {
             const int nt = tile % P.n_tiles;
             int pt = tile / P.n_tiles;
             const int twi = pt % P.tw; pt /= P.tw;
@@ -435,77 +456,49 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
             const int tbi = pt / P.th;
             const int n = nt * kChan + q * 32 + lane;
             const bool n_ok = n < P.Cout;
-            // a warp whose 32 channels all lie past Cout keeps the barriers and hands the accumulator
-            // back, but loads, computes and stages nothing (its part of the staging buffer is clipped)
+            // a warp whose 32 channels all lie past Cout hands the accumulator back but loads,
+            // computes and stores nothing
             const bool warp_on = nt * kChan + q * 32 < P.Cout;
             const float sc = ((P.scale && n_ok) ? __ldg(P.scale + n) : 1.0f) * alpha;
             const float sf = (P.shift && n_ok) ? __ldg(P.shift + n) : 0.0f;
             const int p_w0 = twi << P.lgBW, p_h0 = thi << P.lgBH, p_b0 = tbi * (PIX >> (P.lgBW + P.lgBH));
-            if (need_off) {
-                // output offsets of the pixels of this group's chunks (the same for every channel),
-                // one per thread; the first barrier keeps the previous tile's readers ahead of the overwrite
-                epi_bar(es);
-                if (ew < kChunks / kEpiSets) {
-                    const int p = (ew * kEpiSets + es) * 32 + lane;
-                    const int wv = p_w0 + (p & BWm);
-                    const int hv = p_h0 + ((p >> P.lgBW) & BHm);
-                    const int bv = p_b0 + (p >> (P.lgBW + P.lgBH));
-                    uint32_t off = 0xFFFFFFFFu;
-                    if (wv < P.Wv && hv < P.Hv && bv < P.Bv)
-                        off = (uint32_t)((((long long)bv * P.OH + (hv * P.osh + P.ooh)) * P.OW + (wv * P.osw + P.oow)) * P.ldy);
-                    sm->pix_off[es][ew * 32 + lane] = off;
-                }
-                epi_bar(es);
-            }
-            // residual chunk `c` of this tile -> the group's buffer `slot` (one thread)
+            const int c_n0 = nt * kChan + q * 32;            // first channel of this warp
+            // residual chunk `c` of this tile -> buffer `slot` of this warp (one lane)
             auto res_load = [&](int c, uint32_t slot) {
                 const int p0 = c * 32;
-                mbar_expect_tx(&sm->res_full[es][slot], 32 * kChan * 2);
-                tma_load_4d(sm->stage_res[es][slot], &map_r, &sm->res_full[es][slot], nt * kChan,
+                mbar_expect_tx(&my_res_full[slot], 32 * 32 * 2);
+                tma_load_4d(my_res + slot * (32 * 32), &map_r, &my_res_full[slot], c_n0,
                             (p_w0 + (p0 & BWm)) * P.osw, (p_h0 + ((p0 >> P.lgBW) & BHm)) * P.osh,
                             p_b0 + (p0 >> (P.lgBW + P.lgBH)));
             };
-            // both buffers are free here: their last readers finished before the group's last barrier
-            if (P.res_tma && leader) {
+            // both buffers are free here: the warp has read the last chunk of its previous tile
+            const bool use_res_tma = P.res_tma && warp_on;
+            if (use_res_tma && lane == 0) {
                 res_load(es, nres & 1u);
-                if (es + kEpiSets < kChunks) res_load(es + kEpiSets, (nres + 1) & 1u);
+                if (kMine > 1) res_load(es + kEpiSets, (nres + 1) & 1u);
             }
             const int buf = lt % kAccBufs;
             PROF_T(t_w);
-            if (kbpt > 0) {
-                // one thread waits for the accumulator; the group's warps then decide together, so
-                // that they always execute the same number of named barriers
-                if (leader)
-                    sm->epi_ok[es][ndec & 1u] = mbar_wait(&sm->acc_full[buf], (lt / kAccBufs) & 1u, abort_flag, P.status, 32) ? 1 : 0;
-                epi_bar(es);
-                if (!sm->epi_ok[es][ndec++ & 1u]) break;
-            }
+            if (kbpt > 0 && !mbar_wait_warp(&sm->acc_full[buf], (lt / kAccBufs) & 1u, abort_flag, P.status, 32)) break;
             PROF_ACC(e_wait, t_w);
             PROF_T(t_d);
             tc_fence_after();
             float *const y32 = reinterpret_cast<float *>(P.Y) + n;
             __nv_bfloat16 *const y16 = reinterpret_cast<__nv_bfloat16 *>(P.Y) + n;
-            bool alive = true;
+            const uint32_t t_acc = tmem_acc + ((uint32_t)(q * 32) << 16) + buf * PIX;
+            uint32_t v[32];
+            // the chunk loop stays rolled: the epilogue is straight-line code that every warp walks
+            // once per chunk, so its size is instruction-fetch time
 #pragma unroll 1
-            for (int c = es; c < kChunks && alive; c += kEpiSets) {
-                // the 32 offsets of this chunk: eight 16-byte broadcast loads, issued before the
-                // tensor-memory load is waited for (needed for per-thread stores and for the residual)
-                uint32_t off[32];
-                if (need_off) {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const uint4 o = *reinterpret_cast<const uint4 *>(sm->pix_off[es] + (c / kEpiSets) * 32 + i * 4);
-                        off[i * 4 + 0] = o.x; off[i * 4 + 1] = o.y; off[i * 4 + 2] = o.z; off[i * 4 + 3] = o.w;
-                    }
-                }
-                uint32_t v[32];
+            for (int i = 0; i < kMine; ++i) {
+                const int c = es + i * kEpiSets;
                 PROF_T(t_ld);
                 if (kbpt > 0) {
                     if (warp_on) {
-                        tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + buf * PIX + c * 32, v);
-                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                        tmem_ld32(t_acc + c * 32, v);
+                        tmem_wait_ld(v);
                     }
-                    if (c + kEpiSets >= kChunks) {
+                    if (i + 1 == kMine) {
                         // this warp's share of the accumulator is in registers: hand it back
                         tc_fence_before();
                         __syncwarp();
@@ -517,38 +510,44 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
                 }
                 PROF_ACC(e_ld, t_ld);
+                if (!warp_on) continue;
+                // output offset of pixel `lane` of this chunk (per-thread stores and residual loads
+                // exchange them by shuffle), ~0 = outside the output
+                uint32_t my_off = 0xFFFFFFFFu;
+                if (need_off) {
+                    const int p = c * 32 + lane;
+                    const int wv = p_w0 + (p & BWm);
+                    const int hv = p_h0 + ((p >> P.lgBW) & BHm);
+                    const int bv = p_b0 + (p >> (P.lgBW + P.lgBH));
+                    if (wv < P.Wv && hv < P.Hv && bv < P.Bv)
+                        my_off = (uint32_t)((((long long)bv * P.OH + (hv * P.osh + P.ooh)) * P.OW + (wv * P.osw + P.oow)) * P.ldy);
+                }
                 PROF_T(t_grp);
-                if (P.res_tma) {
-                    // the residual of this chunk has landed; the buffer of the group's next chunk was
-                    // last read in its previous chunk, which every warp has left by the barrier
-                    if (leader)
-                        sm->epi_ok[es][ndec & 1u] = mbar_wait(&sm->res_full[es][nres & 1u], (nres >> 1) & 1u, abort_flag, P.status, 32) ? 1 : 0;
-                    epi_bar(es);
-                    if (!sm->epi_ok[es][ndec++ & 1u]) { alive = false; break; }
-                    if (leader && c != es && c + kEpiSets < kChunks) res_load(c + kEpiSets, (nres + 1) & 1u);
+                if (use_res_tma) {
+                    if (!mbar_wait_warp(&my_res_full[nres & 1u], (nres >> 1) & 1u, abort_flag, P.status, 32)) { alive = false; break; }
                 }
                 PROF_ACC(e_grp, t_grp);
                 PROF_T(t_math);
-                // The inner loops are kept free of conditionals: one warp per scheduler runs this
-                // code, so every instruction fetched and issued here is exposed latency.
-                if (P.res_tma) {
-                    const __nv_bfloat16 *rs = sm->stage_res[es][nres & 1u] + q * 32 + lane;
-                    if (warp_on) {
+                // The inner loops are kept free of conditionals: every instruction issued here is
+                // exposed latency of this warp's chunk.
+                if (use_res_tma) {
+                    const __nv_bfloat16 *rs = my_res + (nres & 1u) * (32 * 32) + lane;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            v[j] = __float_as_uint(fmaxf(fmaf(__uint_as_float(v[j]), sc, sf) + __bfloat162float(rs[j * kChan]), floor_v));
-                    }
+                    for (int j = 0; j < 32; ++j)
+                        v[j] = __float_as_uint(fmaxf(fmaf(__uint_as_float(v[j]), sc, sf) + __bfloat162float(rs[j * 32]), floor_v));
+                    // the buffer is free again: fetch the residual of the chunk after the next
+                    __syncwarp();
+                    if (lane == 0 && i + 2 < kMine) res_load(c + 2 * kEpiSets, nres & 1u);
                     ++nres;
-                } else if (!warp_on) {
-                    // nothing to compute
                 } else if (P.residual) {
                     // y = acc * scale' + shift + residual (residual fetched with the per-pixel offsets)
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
+                        const uint32_t o = __shfl_sync(0xffffffffu, my_off, j);
                         float r = 0.0f;
-                        if (off[j] != 0xFFFFFFFFu && n_ok)
-                            r = res_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(P.residual)[(size_t)off[j] + n])
-                                         : reinterpret_cast<const float *>(P.residual)[(size_t)off[j] + n];
+                        if (o != 0xFFFFFFFFu && n_ok)
+                            r = res_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(P.residual)[(size_t)o + n])
+                                         : reinterpret_cast<const float *>(P.residual)[(size_t)o + n];
                         v[j] = __float_as_uint(fmaxf(fmaf(__uint_as_float(v[j]), sc, sf) + r, floor_v));
                     }
                 } else {
@@ -556,66 +555,66 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(fmaxf(fmaf(__uint_as_float(v[j]), sc, sf), floor_v));
                 }
                 PROF_ACC(e_math, t_math);
+                PROF_T(t_st);
                 if (P.tma_store) {
-                    const int nl = q * 32 + lane;
                     // a staging buffer holds 32 pixels of bf16 or 16 of fp32: one or two rounds per chunk
                     const int rounds = out_bf16 ? 1 : 2;
                     for (int h = 0; h < rounds; ++h) {
-                        // the buffer was last read by the store this group issued two rounds ago
-                        PROF_T(t_st);
-                        if (leader) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                        epi_bar(es);
-                        uint8_t *const sbuf = sm->stage_out[es][nst & 1u];
-                        if (!warp_on) {
-                            // clipped by the store
-                        } else if (out_bf16) {
-                            uint16_t *const st16 = reinterpret_cast<uint16_t *>(sbuf) + nl;
+                        // the buffer was last read by the store this warp issued kOutBufs rounds ago
+                        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kOutBufs - 1) : "memory");
+                        __syncwarp();
+                        uint8_t *const sbuf = my_out + (nst % kOutBufs) * kStageBytes;
+                        if (out_bf16) {
+                            uint16_t *const st16 = reinterpret_cast<uint16_t *>(sbuf) + lane;
 #pragma unroll
                             for (int j = 0; j < 32; j += 2) {
                                 // one packed conversion per two pixels
                                 uint32_t pk;
                                 asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(__uint_as_float(v[j + 1])), "f"(__uint_as_float(v[j])));
-                                st16[j * kChan] = (uint16_t)pk;
-                                st16[(j + 1) * kChan] = (uint16_t)(pk >> 16);
+                                st16[j * 32] = (uint16_t)pk;
+                                st16[(j + 1) * 32] = (uint16_t)(pk >> 16);
                             }
                         } else {
-                            uint32_t *const st32 = reinterpret_cast<uint32_t *>(sbuf) + nl;
+                            uint32_t *const st32 = reinterpret_cast<uint32_t *>(sbuf) + lane;
                             if (h == 0) {
 #pragma unroll
-                                for (int j = 0; j < 16; ++j) st32[j * kChan] = v[j];
+                                for (int j = 0; j < 16; ++j) st32[j * 32] = v[j];
                             } else {
 #pragma unroll
-                                for (int j = 0; j < 16; ++j) st32[j * kChan] = v[16 + j];
+                                for (int j = 0; j < 16; ++j) st32[j * 32] = v[16 + j];
                             }
                         }
                         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                        epi_bar(es);
-                        if (leader) {
+                        __syncwarp();
+                        if (lane == 0) {
                             const int p0 = c * 32 + h * 16;
-                            tma_store_4d(&map_y, sbuf, nt * kChan, (p_w0 + (p0 & BWm)) * P.osw,
+                            tma_store_4d(&map_y, sbuf, c_n0, (p_w0 + (p0 & BWm)) * P.osw,
                                          (p_h0 + ((p0 >> P.lgBW) & BHm)) * P.osh, p_b0 + (p0 >> (P.lgBW + P.lgBH)));
                         }
                         ++nst;
-                        PROF_ACC(e_st, t_st);
                     }
-                } else if (n_ok) {
+                } else {
                     if (out_bf16) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (off[j] != 0xFFFFFFFFu) y16[off[j]] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                        for (int j = 0; j < 32; ++j) {
+                            const uint32_t o = __shfl_sync(0xffffffffu, my_off, j);
+                            if (o != 0xFFFFFFFFu && n_ok) y16[o] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                        }
                     } else {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (off[j] != 0xFFFFFFFFu) y32[off[j]] = __uint_as_float(v[j]);
+                        for (int j = 0; j < 32; ++j) {
+                            const uint32_t o = __shfl_sync(0xffffffffu, my_off, j);
+                            if (o != 0xFFFFFFFFu && n_ok) y32[o] = __uint_as_float(v[j]);
+                        }
                     }
                 }
+                PROF_ACC(e_st, t_st);
             }
-            if (!alive) break;
             __syncwarp();
         }
-        if (ew == 0 && lane == 0 && es == 0) { PROF_OUT(9, e_wait); PROF_OUT(10, e_drain); PROF_OUT(11, (long long)lt); PROF_OUT(16, e_ld); PROF_OUT(17, e_grp); PROF_OUT(18, e_math); PROF_OUT(19, e_st); }
+        if (q == 0 && lane == 0 && es == 0) { PROF_OUT(9, e_wait); PROF_OUT(10, e_drain); PROF_OUT(11, (long long)lt); PROF_OUT(16, e_ld); PROF_OUT(17, e_grp); PROF_OUT(18, e_math); PROF_OUT(19, e_st); }
         // all bulk stores of this thread have been written before the block may exit
-        if (P.tma_store && leader) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        if (P.tma_store && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 
     // ---------------------------------------------------- teardown
@@ -667,11 +666,12 @@ struct Geometry {
     long long Cin;   // channels per tap
 };
 
-// Picks the pixel-tile shape (powers of two, product `pix`) that needs the fewest tiles.
+// Picks the pixel-tile shape BW x BH x BB (BW and BH powers of two, product `pix`) that needs the
+// fewest tiles.
 long long pick_tile(const Geometry &g, int pix, int *lgBW, int *lgBH)
 {
     int lg = 0;
-    while ((1 << lg) < pix) ++lg;
+    while (((pix >> lg) & 1) == 0) ++lg;      // BW * BH divides the power-of-two part of `pix`
     long long best = -1;
     int bw = 0, bh = 0;
     for (int a = 0; a <= lg; ++a)
@@ -731,13 +731,14 @@ int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const twn_dev
     const long long base_pix = (long long)g.ooh * g.OW + g.oow;
     if ((g.ldy * es) % 16 == 0 && ((long long)g.Cout * es) % 16 == 0 && (reinterpret_cast<uintptr_t>(P.Y) % 16) == 0 &&
         g.OW > g.oow && g.OH > g.ooh) {
-        // 2^lg consecutive tile pixels are a sub-box sbw x sbh x sbb of the tile box: a staging
-        // buffer holds 32 pixels of bf16 or 16 of fp32, a residual buffer 32 pixels
+        // 2^lg consecutive tile pixels are a sub-box sbw x sbh x sbb of the tile box, 32 channels wide
+        // (one epilogue warp): a staging buffer holds 32 pixels of bf16 or 16 of fp32, a residual
+        // buffer 32 pixels
         auto sub_box = [&](int lg, cuuint32_t *bx) {
             const int lg_sbw = P.lgBW < lg ? P.lgBW : lg;
             const int lg_sbh = P.lgBH < lg - lg_sbw ? P.lgBH : lg - lg_sbw;
             const int lg_sbb = lg - lg_sbw - lg_sbh;
-            bx[0] = (cuuint32_t)kChan; bx[1] = (cuuint32_t)((1 << lg_sbw) * g.osw);
+            bx[0] = 32u; bx[1] = (cuuint32_t)((1 << lg_sbw) * g.osw);
             bx[2] = (cuuint32_t)((1 << lg_sbh) * g.osh); bx[3] = 1u << lg_sbb;
         };
         cuuint64_t dims[4] = {(cuuint64_t)g.Cout, (cuuint64_t)(g.OW - g.oow), (cuuint64_t)(g.OH - g.ooh), (cuuint64_t)g.Bv};
@@ -764,6 +765,9 @@ int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const twn_dev
             }
         }
     }
+#if defined(TWN_PROFILE) || defined(TWN_TUNE)
+    if (getenv("TWN_NOTMA")) { P.tma_store = 0; }
+#endif
     const int grid = dev.sm_count < P.total_tiles ? dev.sm_count : P.total_tiles;
     tconv_kernel<PIX><<<grid, kThreadsConv, smem_bytes, s>>>(map_x, map_y, map_r, P);
     TWN_CUDA_OK(cudaGetLastError());
@@ -810,18 +814,28 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     // Tile shape by a cost model fitted to measured launches (cycles per round of tiles, kb = k-blocks
     // per tile):
     //   128 pixels: max(2500 + 720 kb, 6500): the epilogue overlaps the next tile and bounds short reductions
+    //   192 pixels: max(2500 + 790 kb, 10500), floor 7600 when only the lower half of the channel
+    //               tile exists: overlapped as well, fewer rounds than 128
     //   256 pixels: 13500 + 640 kb: one accumulator, so the epilogue is exposed; 8000 when only the
     //               lower half of the channel tile exists (half of the epilogue warps idle)
     int a, b;
     const long long kb = (long long)P.n_taps * P.n_cblk;
     const long long sms = dev.sm_count;
+    const bool half = g.Cout <= kChan / 2;
     const long long t128 = pick_tile(g, 128, &a, &b) * P.n_tiles, t256 = pick_tile(g, 256, &a, &b) * P.n_tiles;
+    const long long t192 = pick_tile(g, 192, &a, &b) * P.n_tiles;
     const long long per128 = 2500 + 720 * kb > 6500 ? 2500 + 720 * kb : 6500;
-    const long long per256 = (g.Cout <= kChan / 2 ? 8000 : 13500) + 640 * kb;
-    int choice = ((t256 + sms - 1) / sms) * per256 < ((t128 + sms - 1) / sms) * per128 ? 1 : 0;
+    const long long floor192 = half ? 7600 : 10500;
+    const long long per192 = 2500 + 790 * kb > floor192 ? 2500 + 790 * kb : floor192;
+    const long long per256 = (half ? 8000 : 13500) + 640 * kb;
+    const long long c128 = ((t128 + sms - 1) / sms) * per128, c192 = ((t192 + sms - 1) / sms) * per192,
+                    c256 = ((t256 + sms - 1) / sms) * per256;
+    int choice = c256 < c128 ? 1 : 0;
+    if (c192 < (choice ? c256 : c128)) choice = 2;
 #if defined(TWN_PROFILE) || defined(TWN_TUNE)
-    if (const char *force = getenv("TWN_TILE")) choice = atoi(force) & 1;   // profiling and tuning builds: pin the variant
+    if (const char *force = getenv("TWN_TILE")) choice = atoi(force) % 3;   // profiling and tuning builds: pin the variant
 #endif
+    if (choice == 2) return launch_conv_t<192>(g, P, X, dev, enc, s);
     if (choice == 1) return launch_conv_t<256>(g, P, X, dev, enc, s);
     return launch_conv_t<128>(g, P, X, dev, enc, s);
 }
