@@ -134,6 +134,20 @@ def ternarize(W, delta_factor: float = 0.7, want_codes: bool = True):
                  st.n_boundary, bool(st.nonfinite)), codes
 
 
+def ternarize_rows(W, delta_factor: float = 0.7):
+    """Algorithm 1 as printed: one threshold and one scale per filter (row of the 2-D fp32
+    matrix W).  Returns (list of Stats, one per row; int8 codes shaped like W)."""
+    w = _f32(W)
+    assert w.ndim == 2
+    rows, cols = w.shape
+    st = (_Stats * max(rows, 1))()
+    codes = np.empty(w.shape, dtype=np.int8)
+    lib().ref_ternarize_rows(_p(w), C.c_int64(rows), C.c_int64(cols), C.c_double(delta_factor), st, _p(codes))
+    out = [Stats(s.delta, s.alpha, s.sum_abs, s.sum_abs_kept, s.n_neg, s.n_zero, s.n_pos,
+                 s.n_boundary, bool(s.nonfinite)) for s in st[:rows]]
+    return out, codes
+
+
 def alpha_alg1(W, codes) -> float:
     w, c = _f32(W), _i8(codes)
     return float(lib().ref_alpha_alg1(_p(w), _p(c), C.c_int64(w.size)))

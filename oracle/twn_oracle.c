@@ -15,7 +15,7 @@
  *     epilogue), the quantity the parity tolerance is stated in.
  *
  * Pins (tests/test_oracle_*.py): closed form of alpha vs. Algorithm 1's
- * quotient, 3^n enumeration of Eq. 1, threshold sweeps vs. the paper's
+ * quotient (per layer and per filter), a hand-worked per-filter example, 3^n enumeration of Eq. 1, threshold sweeps vs. the paper's
  * closed forms for uniform / normal weights, pack round trip over all 3^16
  * words, numpy/torch fp64 matmul and conv2d, adjoint identities.
  * Parity unpinned: none of the functions below.
@@ -118,6 +118,23 @@ int ref_ternarize(const float *W, int64_t n, double c, ref_stats *st, int8_t *co
     int64_t kept = st->n_pos + st->n_neg;
     st->alpha = kept > 0 ? st->sum_abs_kept / (double)kept : 0.0;
     return 0;
+}
+
+/* ------------------------------------------------------------------------
+ * Per-filter ternarization: Algorithm 1 as printed, whose first loop runs over
+ * the filters of a layer.  Filter r (row r of W[rows][cols]) gets its own
+ *   delta_r = c/cols * ||W_r||_1,   codes by Eq. 3 against delta_r,
+ *   alpha_r = mean of |W_r,i| over |W_r,i| > delta_r            (Eq. 5)
+ * n in the threshold rule is the element count of the filter.  st has `rows`
+ * entries, codes (optional) rows*cols.  Returns the number of rows that hold
+ * a non-finite weight.
+ * ---------------------------------------------------------------------- */
+int ref_ternarize_rows(const float *W, int64_t rows, int64_t cols, double c, ref_stats *st, int8_t *codes)
+{
+    int bad = 0;
+    for (int64_t r = 0; r < rows; ++r)
+        bad += ref_ternarize(W + r * cols, cols, c, st + r, codes ? codes + r * cols : NULL);
+    return bad;
 }
 
 /* Algorithm 1's form of the scale: alpha = (W . W~) / (W~ . W~), in long double. */
