@@ -180,6 +180,62 @@ class TernarizeWorkload:
         return self.n * self.bytes_per_unit / dt / 1e9, f"full tensor, n={self.n}", 1
 
 
+class TernarizeRowsWorkload(TernarizeWorkload):
+    """Per-filter ternarize + pack (Algorithm 1 as printed: one threshold and one scale per filter)
+    of a [rows, cols] fp32 matrix drawn N(0,1).  A filter stays on chip between the threshold
+    reduction and the coding, so the algorithmic traffic is 4.25 bytes per weight (one read,
+    0.25 B written)."""
+    name = "ternarize_rows_pack_12288x8192_normal"
+    bytes_per_unit = 4.25
+
+    def __init__(self, rows=12288, cols=8192, seed=0):
+        super().__init__(rows * cols, seed)
+        self.rows, self.cols = rows, cols
+
+    def config(self):
+        return {"workload": self.name, "rows": self.rows, "cols": self.cols, "dist": "normal", "seed": self.seed,
+                "delta_factor": 0.7, "l2": "input (403 MB) larger than L2 (126 MB)"}
+
+    def setup(self, torch, twn, host_W):
+        self.torch, self.twn = torch, twn
+        self.ld = twn.ld_for(self.cols)
+        self.W = torch.from_numpy(host_W).cuda().view(self.rows, self.cols)
+        self.stats = twn.new_stats_rows(self.rows)
+        self.packed = torch.empty((self.rows, self.ld // 16), dtype=torch.int32, device="cuda")
+        self.host_W = torch.from_numpy(host_W).pin_memory().view(self.rows, self.cols)
+        self.host_packed = torch.empty((self.rows, self.ld // 16), dtype=torch.int32).pin_memory()
+        self.host_stats = torch.empty((self.rows, 8), dtype=torch.int64).pin_memory()
+
+    def step(self):
+        self.twn.ternarize_rows(self.W, 0.7, self.stats, self.packed, self.ld)
+
+    def e2e_bytes(self):
+        return self.n * 4, self.rows * (self.ld // 4 + 64)
+
+    def launches_per_step(self):
+        return 1
+
+    def roofline(self, ms_per_step, peaks):
+        r = super().roofline(ms_per_step, peaks)
+        r["kernel"] = "ternarize_rows_kernel (one twn_ternarize_rows call)"
+        r["traffic"] = None
+        return r
+
+    def check(self):
+        st = self.twn.stats_rows_to_host(self.stats[:4])
+        assert all(s["status"] == 0 and s["n_neg"] + s["n_zero"] + s["n_pos"] == self.cols for s in st), st
+
+    def cpu_sample(self, host_W):
+        import oracle
+        rows = 1536          # a bounded sample of the filters (about 10 s of the oracle)
+        W = host_W.reshape(self.rows, self.cols)[:rows]
+        t0 = time.perf_counter()
+        st, codes = oracle.ternarize_rows(W, 0.7)
+        oracle.pack(codes, self.ld)
+        dt = time.perf_counter() - t0
+        return rows * self.cols * self.bytes_per_unit / dt / 1e9, f"oracle on {rows} of {self.rows} filters ({dt:.1f} s)", 1
+
+
 class GemmWorkload:
     """One ternary-weight GEMM (Algorithm 1, forward of a fully connected layer): Y = alpha * X T^T with
     bf16 X [M, K], 2-bit T [N, K] ternarized from N(0,1) weights, bf16 Y.  2MNK flops per step."""
@@ -440,7 +496,7 @@ class NetWorkload:
         return {"resnet18_train": 340.7e9 / 64 * 1.0, "vgg7_fwd": 615.9e6, "lenet5_fwd": 4.27e6}[self.kind]
 
 
-WORKLOADS = {"ternarize": lambda: TernarizeWorkload(), "resnet18_train": lambda: NetWorkload("resnet18_train"),
+WORKLOADS = {"ternarize": lambda: TernarizeWorkload(), "ternarize_rows": lambda: TernarizeRowsWorkload(), "resnet18_train": lambda: NetWorkload("resnet18_train"),
              "gemm_16384": lambda: GemmWorkload(16384), "gemm_4096": lambda: GemmWorkload(4096),
              "vgg7_fwd": lambda: NetWorkload("vgg7_fwd"), "lenet5_fwd": lambda: NetWorkload("lenet5_fwd")}
 DEFAULT_WORKLOAD = "resnet18_train"
@@ -452,7 +508,7 @@ def run_reference(args):
     if rank != 0:
         return
     wl = WORKLOADS[args.workload]()
-    host = wl.host_inputs() if isinstance(wl, (TernarizeWorkload, GemmWorkload)) else None
+    host = wl.host_inputs() if isinstance(wl, (TernarizeWorkload, GemmWorkload)) else None   # (covers the per-filter workload)
     vals = []
     steps = args.steps if args.steps else 3
     for i in range(args.warmup + steps):

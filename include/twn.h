@@ -163,6 +163,34 @@ int twn_ternarize_static(const float *W, int64_t rows, int64_t cols, double delt
                          twn_stats_t *stats, uint32_t *packed, int64_t ld_codes,
                          int8_t *codes_i8, twn_stream_t stream);
 
+/*
+ * Per-filter threshold ternarization fused with 2-bit packing: Algorithm 1 as printed,
+ * whose first loop runs over the filters of a layer.  Row r of W is one filter and gets
+ *   delta_r = delta_factor * (1/cols) * sum_i |W_r,i|          (Sec. 2.3, n = cols)
+ *   codes by Eq. 3 against delta_r
+ *   alpha_r = mean of |W_r,i| over { i : |W_r,i| > delta_r }   (Eq. 5)
+ * W        fp32 [rows, cols], contiguous, 4-byte aligned (a 16-byte aligned matrix with
+ *          cols % 4 == 0 takes the fast path: filters of up to 16384 weights cross HBM once).
+ * stats    twn_stats_t [rows], 8-byte aligned; entry r is written completely (status
+ *          TWN_ERR_NONFINITE when filter r holds a NaN/Inf; the other filters are unaffected).
+ * packed   uint32 [rows][ld_codes/16], layout and padding as for twn_ternarize; 16-byte aligned.
+ * codes_i8 optional int8 [rows, cols] copy of the codes, or NULL.
+ * Needs no scratch memory.  Deterministic; the comparison is done as in twn_ternarize.
+ * The contraction kernels take one alpha per call, so for per-filter scales pass stats = NULL
+ * to them and fold the alphas into the epilogue's per-channel scale with twn_rows_scale
+ * (forward), or into the scale of twn_act_bwd (backward: the gradient with respect to the
+ * ternary weights' output carries alpha_r on the reduction index of the backward-for-data pass).
+ */
+int twn_ternarize_rows(const float *W, int64_t rows, int64_t cols, double delta_factor,
+                       twn_stats_t *stats, uint32_t *packed, int64_t ld_codes,
+                       int8_t *codes_i8, twn_stream_t stream);
+
+/* scale_out[r] = alpha_r * scale_in[r] (scale_in NULL: 1), r < rows, fp32: the per-filter scales
+ * of Algorithm 1 as the per-channel scale of twn_epilogue_t.  The most severe status of the
+ * `rows` entries is merged into *dev_status (optional). */
+int twn_rows_scale(const twn_stats_t *stats, int64_t rows, const float *scale_in, float *scale_out,
+                   int32_t *dev_status, twn_stream_t stream);
+
 /* ---- 2-bit storage (Sec. 2.1, model compression) ------------------------- */
 
 /*

@@ -133,6 +133,38 @@ def ternarize(W: torch.Tensor, delta_factor: float, stats: torch.Tensor, packed:
                                _stream(stream)), "twn_ternarize")
 
 
+def ternarize_rows(W: torch.Tensor, delta_factor: float, stats: torch.Tensor, packed: torch.Tensor,
+                   ld_codes: int, codes_i8=None, stream=None) -> None:
+    """twn_ternarize_rows: one threshold and one scale per filter.  W fp32 [rows, cols];
+    stats int64 [rows, 8] (one twn_stats_t per row)."""
+    rows, cols = W.shape[0], W.numel() // max(W.shape[0], 1)
+    assert stats.numel() * stats.element_size() >= 64 * rows
+    _check(lib().twn_ternarize_rows(_ptr(W), C.c_int64(rows), C.c_int64(cols), C.c_double(delta_factor),
+                                    _ptr(stats), _ptr(packed), C.c_int64(ld_codes), _ptr(codes_i8),
+                                    _stream(stream)), "twn_ternarize_rows")
+
+
+def rows_scale(stats: torch.Tensor, rows: int, scale_in, scale_out: torch.Tensor, dev_status=None,
+               stream=None) -> None:
+    """twn_rows_scale: scale_out[r] = alpha_r * scale_in[r]."""
+    _check(lib().twn_rows_scale(_ptr(stats), C.c_int64(rows), _ptr(scale_in), _ptr(scale_out),
+                                _ptr(dev_status), _stream(stream)), "twn_rows_scale")
+
+
+def new_stats_rows(rows: int, device="cuda") -> torch.Tensor:
+    """Zeroed device array of `rows` twn_stats_t."""
+    return torch.zeros((rows, 8), dtype=torch.int64, device=device)
+
+
+def stats_rows_to_host(stats: torch.Tensor) -> list:
+    h = stats.cpu().contiguous()
+    d = h.view(torch.float64)
+    i32 = h.view(torch.int32)
+    return [{"delta": float(d[r, 0]), "alpha": float(d[r, 1]), "sum_abs": float(d[r, 2]),
+             "sum_abs_kept": float(d[r, 3]), "n_neg": int(h[r, 4]), "n_zero": int(h[r, 5]),
+             "n_pos": int(h[r, 6]), "status": int(i32[r, 14])} for r in range(h.shape[0])]
+
+
 TERNARIZE_STATIC_MAX_WEIGHTS = 1 << 31
 
 
