@@ -218,7 +218,8 @@ class TernarizeRowsWorkload(TernarizeWorkload):
     def roofline(self, ms_per_step, peaks):
         r = super().roofline(ms_per_step, peaks)
         r["kernel"] = "ternarize_rows_kernel (one twn_ternarize_rows call)"
-        r["traffic"] = None
+        # dram bytes of one launch from the ncu capture of this workload (profiles/); algorithmic: 4.28e8
+        r["traffic"] = 426.0e6 if (self.rows, self.cols) == (12288, 8192) else None
         return r
 
     def check(self):
@@ -299,7 +300,7 @@ class GemmWorkload:
                 "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
                 "peak_source": peaks["source"] + " (bf16 burst: the kernel is timed alone)",
                 # DRAM bytes of one launch from the ncu capture of the M = 4096 case (profiles/)
-                "traffic": 40.1e6 if (self.M, self.N, self.K) == (4096, 4096, 4096) else None}
+                "traffic": 40.6e6 if (self.M, self.N, self.K) == (4096, 4096, 4096) else None}
 
     def check(self):
         assert self.twn.read_status(self.status) == 0
@@ -528,6 +529,40 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def ternarize_leg(torch, twn, peaks, steps=300):
+    """GB/s of twn_ternarize (per layer) and twn_ternarize_rows (per filter) on 1e8 seeded N(0,1)
+    weights, timed with CUDA events after warm-up; the 400 MB input exceeds L2."""
+    wl = TernarizeWorkload()
+    W = wl.host_inputs()
+    wl.setup(torch, twn, W)
+    out = {}
+    rows_wl = TernarizeRowsWorkload(rows=wl.n // 8192)      # the same weights as 12207 filters of 8192
+    legs = [("per_layer", wl, wl.step)]
+    if wl.n >= rows_wl.n:
+        rows_wl.torch, rows_wl.twn = torch, twn
+        rows_wl.ld = twn.ld_for(rows_wl.cols)
+        rows_wl.W = wl.W[:rows_wl.n].view(rows_wl.rows, rows_wl.cols)
+        rows_wl.stats = twn.new_stats_rows(rows_wl.rows)
+        rows_wl.packed = torch.empty((rows_wl.rows, rows_wl.ld // 16), dtype=torch.int32, device="cuda")
+        legs.append(("per_filter", rows_wl, rows_wl.step))
+    for name, w, fn in legs:
+        for _ in range(5):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        w.check()
+        ms = e0.elapsed_time(e1) / steps
+        gbs = w.n * w.bytes_per_unit / (ms * 1e-3) / 1e9
+        out[name] = {"value": gbs, "unit": "GB/s", "n": w.n, "bytes_per_weight": w.bytes_per_unit, "ms": ms,
+                     "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"]}
+    return out
+
+
 def run_ours(args):
     import torch
     from paper_1605_04711_b200 import twn
@@ -582,6 +617,10 @@ def run_ours(args):
                         "ms_per_step": ms_e2e, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
                 "gpu_launches": wl.launches_per_step() * steps,
                 "roofline": wl.roofline(ms, peaks)}
+        if args.workload == DEFAULT_WORKLOAD and not args.no_ternarize_leg:
+            # the second half of the headline metric, measured in the same run: ternarize + pack of
+            # one 1e8-weight tensor (larger than L2), in GB/s of algorithmic traffic
+            line["ternarize_pack"] = ternarize_leg(torch, twn, peaks)
         if world == 1 and not args.no_cpu:
             v, sample, cores = wl.cpu_sample(host)
             line["cpu_baseline"] = {"value": v, "unit": wl.unit, "cores": cores, "kind": "oracle",
@@ -599,6 +638,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--no-ternarize-leg", action="store_true",
+                    help="default workload only: skip the ternarize+pack GB/s measurement added to the line")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
