@@ -344,7 +344,8 @@ class NetWorkload:
     def config(self):
         c = {"workload": self.name, "seed": 0, "delta_factor": 0.7,
              "l2": "activations of a step (> 1 GB for ResNet-18) exceed L2 (126 MB)",
-             "launch": "one CUDA graph replay per step"}
+             "launch": "one CUDA graph replay per step",
+             "e2e": "pipelined: the pinned-host copy of batch i+1 runs on a copy stream while step i computes"}
         if self.kind == "resnet18_train":
             c["step"] = ("ternarize+pack 21 tensors, transpose codes, forward, backward for data, "
                          "straight-through dW; synthetic dY N(0,1e-2) at the logits")
@@ -412,11 +413,36 @@ class NetWorkload:
     def step(self):
         self.graph.replay()
 
-    def step_e2e(self):
+    def _prefetch(self):
+        """Enqueues, on the copy stream, the host-to-device copy of the next step's inputs into the
+        staging buffers (once the previous contents have been consumed)."""
         t = self.torch
-        self.net.act["input"].view(t.int16).view(-1).copy_(self.host_x, non_blocking=True)
+        with t.cuda.stream(self.copy_stream):
+            self.copy_stream.wait_event(self.ev_free)
+            self.stage_x.view(t.int16).view(-1).copy_(self.host_x, non_blocking=True)
+            if self.train:
+                self.stage_dy.view(t.int16).view(-1).copy_(self.host_dy, non_blocking=True)
+            self.ev_h2d.record(self.copy_stream)
+
+    def step_e2e(self):
+        """One step as an input pipeline runs it: every step copies one batch from pinned host memory
+        (on a copy stream, so the batch of step i+1 travels while step i computes), moves it into the
+        network's input buffer, replays the step and reads the logits back."""
+        t = self.torch
+        main = t.cuda.current_stream()
+        if not hasattr(self, "copy_stream"):
+            self.copy_stream = t.cuda.Stream()
+            self.stage_x = t.empty_like(self.net.act["input"])
+            self.stage_dy = t.empty_like(self.dY) if self.train else None
+            self.ev_h2d, self.ev_free = t.cuda.Event(), t.cuda.Event()
+            self.ev_free.record(main)
+            self._prefetch()
+        main.wait_event(self.ev_h2d)
+        self.net.act["input"].copy_(self.stage_x, non_blocking=True)
         if self.train:
-            self.dY.view(t.int16).view(-1).copy_(self.host_dy, non_blocking=True)
+            self.dY.copy_(self.stage_dy, non_blocking=True)
+        self.ev_free.record(main)
+        self._prefetch()
         self.graph.replay()
         self.host_logits.copy_(self.logits, non_blocking=True)
 
@@ -432,13 +458,15 @@ class NetWorkload:
                 L = op[1]
                 n += 1 + (1 if L.small_cin else 0)                       # forward (+ im2col or input fold)
                 if self.train:
-                    n += 3 + (1 if L.src != "input" else 0)               # memset + 2 ternarize (+ transpose)
+                    n += 1 if L.src != "input" else 0                    # transposed codes for the backward pass
                     n += 1 if L.fold else 0                              # folded codes
                     n += 1 + 2 + (1 if L.fold else 0)                    # act_bwd, dW + reduce (+ unfold)
                     if L.src != "input":
                         n += L.stride * L.stride                         # backward for data
             elif op[0] in ("maxpool", "avgpool"):
                 n += 2 if self.train else 1
+        if self.train:
+            n += 2 * ((len(net.layers) + 31) // 32)                      # the two sweeps of the batched ternarization
         return n
 
     def units_per_step(self):

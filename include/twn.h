@@ -132,6 +132,29 @@ int twn_ternarize(const float *W, int64_t rows, int64_t cols, double delta_facto
                   twn_stream_t stream);
 
 /*
+ * The first loop of Algorithm 1 for a whole network: ternarizes up to 32 tensors (layers) with one
+ * launch per sweep instead of one per tensor.  Every tensor gets its own per-layer threshold,
+ * codes and scale exactly as from a twn_ternarize call of its own (same reduction order, same bits).
+ *   items     HOST array of `count` descriptors; the fields have the meaning and the alignment
+ *             rules of the twn_ternarize arguments of the same name (device pointers inside).
+ *             Read during the call only.
+ *   workspace device scratch of at least twn_ternarize_batch_workspace_bytes(count), 256-byte
+ *             aligned; contents need not be preserved or initialised.
+ * Errors: TWN_ERR_INVALID_ARG for count > 32 or a bad descriptor (nothing is launched).
+ */
+typedef struct {
+    const float *W;
+    int64_t rows, cols;
+    twn_stats_t *stats;
+    uint32_t *packed;
+    int64_t ld_codes;
+    int8_t *codes_i8;     /* optional */
+} twn_ternarize_item_t;
+size_t twn_ternarize_batch_workspace_bytes(int count);
+int twn_ternarize_batch(const twn_ternarize_item_t *items, int count, double delta_factor,
+                        void *workspace, size_t workspace_bytes, twn_stream_t stream);
+
+/*
  * twn_ternarize for callers that may not allocate.  (The paper has no counterpart;
  * this is a packaging variant of the call above, same arithmetic, same results.)
  *

@@ -303,6 +303,50 @@ maxpool_bwd_rows_kernel(const __nv_bfloat16 *__restrict__ dY, const uint8_t *__r
     };
     for (int row = blockIdx.x; row < B * H; row += gridDim.x) {
         const int b = row / H, h = row - b * H;
+        if (k <= 2 * stride) {
+            // At most two windows per dimension cover a pixel: their argmax bytes and gradients
+            // (up to four of each) are loaded before any of them is used, so the loads overlap.
+            int hos[2] = {0, 0}, rs[2] = {0, 0}, nh = 0;
+            for (int r = 0; r < k; ++r) {
+                const int ho = window(h + pad - r, Ho);
+                if (ho >= 0 && nh < 2) { hos[nh] = ho; rs[nh] = r; ++nh; }
+            }
+            for (int i = threadIdx.x; i < per_row; i += kT) {
+                const int w = i / Cv, cv = i - w * Cv;
+                int wos[2] = {0, 0}, sxs[2] = {0, 0}, nw = 0;
+                for (int sx = 0; sx < k; ++sx) {
+                    const int wo = window(w + pad - sx, Wo);
+                    if (wo >= 0 && nw < 2) { wos[nw] = wo; sxs[nw] = sx; ++nw; }
+                }
+                uint2 a[4];
+                uint4 d[4];
+                int want[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int ih = q >> 1, iw = q & 1;
+                    const bool ok = ih < nh && iw < nw;
+                    const size_t o = ((size_t)(b * Ho + hos[ih]) * Wo + wos[iw]) * C + cv * 8;   // in range also when !ok
+                    a[q] = ok ? __ldg(reinterpret_cast<const uint2 *>(idx + o)) : make_uint2(0xFFFFFFFFu, 0xFFFFFFFFu);
+                    d[q] = ok ? __ldg(reinterpret_cast<const uint4 *>(dY + o)) : make_uint4(0u, 0u, 0u, 0u);
+                    want[q] = rs[ih] * k + sxs[iw];     // < 255: an absent window's 0xFF bytes never match
+                }
+                float g[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) g[e] = 0.0f;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    float t8[8];
+                    unpack8(d[q], t8);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const int ai = ((e < 4 ? a[q].x : a[q].y) >> (8 * (e & 3))) & 0xFF;
+                        if (ai == want[q]) g[e] += t8[e];
+                    }
+                }
+                *reinterpret_cast<uint4 *>(dX + ((size_t)row * W + w) * C + cv * 8) = pack8(g);
+            }
+            continue;
+        }
         for (int i = threadIdx.x; i < per_row; i += kT) {
             const int w = i / Cv, cv = i - w * Cv;
             float g[8];

@@ -74,28 +74,28 @@ __device__ __forceinline__ T block_sum(T v, T *smem /* kWarps entries */)
     return r;
 }
 
-// Returns true in every thread of the block that took the last ticket.
-__device__ __forceinline__ bool last_block(unsigned int *ticket)
+// Returns true in every thread of the block that took the last of `grid` tickets.
+__device__ __forceinline__ bool last_block(unsigned int *ticket, unsigned int grid)
 {
     __shared__ bool is_last;
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) is_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+    if (threadIdx.x == 0) is_last = (atomicAdd(ticket, 1u) == grid - 1);
     __syncthreads();
     return is_last;
 }
 
 // ---- sweep 1 -------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads)
-sum_abs_kernel(const float *__restrict__ W, long long n, double factor, void *ws_raw,
-               twn_stats_t *__restrict__ stats)
+// `vb` of `vg`: this block's index and the number of blocks that work on this tensor (the whole
+// grid for a single tensor, a slice of it when several tensors share one launch).
+__device__ __forceinline__ void sum_abs_body(const float *__restrict__ W, long long n, double factor, const Workspace ws,
+                                             twn_stats_t *__restrict__ stats, unsigned int vb, unsigned int vg)
 {
     __shared__ double red[kWarps];
-    const Workspace ws = carve(ws_raw);
     const long long n4 = n >> 2;
     const float4 *W4 = reinterpret_cast<const float4 *>(W);
-    const long long stride = (long long)gridDim.x * kThreads;
-    long long i = (long long)blockIdx.x * kThreads + threadIdx.x;
+    const long long stride = (long long)vg * kThreads;
+    long long i = (long long)vb * kThreads + threadIdx.x;
 
     double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
     for (; i + 3 * stride < n4; i += 4 * stride) {
@@ -113,16 +113,16 @@ sum_abs_kernel(const float *__restrict__ W, long long n, double factor, void *ws
         a0 += (double)fabsf(v.x); a1 += (double)fabsf(v.y); a2 += (double)fabsf(v.z); a3 += (double)fabsf(v.w);
     }
     // scalar tail (n % 4 elements), by the first threads of block 0
-    if (blockIdx.x == 0) {
+    if (vb == 0) {
         const long long t = (n4 << 2) + threadIdx.x;
         if (t < n) a0 += (double)fabsf(__ldg(W + t));
     }
     const double bsum = block_sum((a0 + a1) + (a2 + a3), red);
-    if (threadIdx.x == 0) ws.part_sum[blockIdx.x] = bsum;
+    if (threadIdx.x == 0) ws.part_sum[vb] = bsum;
 
-    if (last_block(ws.ticket1)) {
+    if (last_block(ws.ticket1, vg)) {
         double s = 0.0;
-        for (int b = threadIdx.x; b < (int)gridDim.x; b += kThreads) s += __ldcg(ws.part_sum + b);
+        for (int b = threadIdx.x; b < (int)vg; b += kThreads) s += __ldcg(ws.part_sum + b);
         s = block_sum(s, red);
         if (threadIdx.x == 0) {
             const double delta = n > 0 ? factor * (s / (double)n) : 0.0;
@@ -133,6 +133,13 @@ sum_abs_kernel(const float *__restrict__ W, long long n, double factor, void *ws
             *ws.ticket1 = 0u;
         }
     }
+}
+
+__global__ void __launch_bounds__(kThreads)
+sum_abs_kernel(const float *__restrict__ W, long long n, double factor, void *ws_raw,
+               twn_stats_t *__restrict__ stats)
+{
+    sum_abs_body(W, n, factor, carve(ws_raw), stats, blockIdx.x, gridDim.x);
 }
 
 // ---- sweep 2 -------------------------------------------------------------
@@ -204,14 +211,13 @@ __device__ __forceinline__ uint32_t fields_to_i8x4(uint32_t c8)
 // every load instruction covers 512 contiguous bytes.  A 4x4 byte transpose inside
 // each group of four lanes then leaves lane l with the four bytes of word
 // unit*32 + (l%4)*8 + l/4, and the warp stores one contiguous 128-byte line.
-__global__ void __launch_bounds__(kThreads)
-code_pack_kernel(const float *__restrict__ W, long long rows, long long cols, long long ld_codes,
-                 long long fast_units, uint32_t *__restrict__ packed, int8_t *__restrict__ codes_i8,
-                 void *ws_raw, twn_stats_t *__restrict__ stats)
+__device__ __forceinline__ void code_pack_body(const float *__restrict__ W, long long rows, long long cols,
+                                               long long ld_codes, long long fast_units, uint32_t *__restrict__ packed,
+                                               int8_t *__restrict__ codes_i8, const Workspace ws,
+                                               twn_stats_t *__restrict__ stats, unsigned int vb, unsigned int vg)
 {
     __shared__ double red[kWarps];
     __shared__ unsigned long long redu[kWarps];
-    const Workspace ws = carve(ws_raw);
     const long long n = rows * cols;
     // delta rounded toward -inf: for any float w,  w > delta  <=>  w > thr
     const float thr = __double2float_rd(stats->delta);
@@ -221,9 +227,9 @@ code_pack_kernel(const float *__restrict__ W, long long rows, long long cols, lo
     unsigned long long npos = 0, nneg = 0;
 
     // -- fast units, back to front
-    const long long gwarps = (long long)gridDim.x * kWarps;
+    const long long gwarps = (long long)vg * kWarps;
     const float4 *W4 = reinterpret_cast<const float4 *>(W);
-    for (long long u = fast_units - 1 - ((long long)blockIdx.x * kWarps + warp); u >= 0; u -= gwarps) {
+    for (long long u = fast_units - 1 - ((long long)vb * kWarps + warp); u >= 0; u -= gwarps) {
         const long long f0 = u * 128 + lane;
         const float4 v0 = __ldg(W4 + f0);
         const float4 v1 = __ldg(W4 + f0 + 32);
@@ -256,8 +262,8 @@ code_pack_kernel(const float *__restrict__ W, long long rows, long long cols, lo
     const long long wpr = ld_codes >> 4;
     const long long total_words = rows * wpr;
     const long long first_word = fast_units * 32;
-    for (long long w = first_word + (long long)blockIdx.x * kThreads + threadIdx.x; w < total_words;
-         w += (long long)gridDim.x * kThreads) {
+    for (long long w = first_word + (long long)vb * kThreads + threadIdx.x; w < total_words;
+         w += (long long)vg * kThreads) {
         const long long r = w / wpr;
         const long long j0 = (w - r * wpr) << 4;
         uint32_t word = 0;
@@ -281,14 +287,14 @@ code_pack_kernel(const float *__restrict__ W, long long rows, long long cols, lo
     const unsigned long long bp = block_sum(npos, redu);
     const unsigned long long bn = block_sum(nneg, redu);
     if (threadIdx.x == 0) {
-        ws.part_kept[blockIdx.x] = bk;
-        ws.part_pos[blockIdx.x] = bp;
-        ws.part_neg[blockIdx.x] = bn;
+        ws.part_kept[vb] = bk;
+        ws.part_pos[vb] = bp;
+        ws.part_neg[vb] = bn;
     }
-    if (last_block(ws.ticket2)) {
+    if (last_block(ws.ticket2, vg)) {
         double s = 0.0;
         unsigned long long p = 0, q = 0;
-        for (int b = threadIdx.x; b < (int)gridDim.x; b += kThreads) {
+        for (int b = threadIdx.x; b < (int)vg; b += kThreads) {
             s += __ldcg(ws.part_kept + b);
             p += __ldcg(ws.part_pos + b);
             q += __ldcg(ws.part_neg + b);
@@ -306,6 +312,75 @@ code_pack_kernel(const float *__restrict__ W, long long rows, long long cols, lo
             *ws.ticket2 = 0u;
         }
     }
+}
+
+__global__ void __launch_bounds__(kThreads)
+code_pack_kernel(const float *__restrict__ W, long long rows, long long cols, long long ld_codes,
+                 long long fast_units, uint32_t *__restrict__ packed, int8_t *__restrict__ codes_i8,
+                 void *ws_raw, twn_stats_t *__restrict__ stats)
+{
+    code_pack_body(W, rows, cols, ld_codes, fast_units, packed, codes_i8, carve(ws_raw), stats, blockIdx.x, gridDim.x);
+}
+
+// ---- several tensors in one launch ------------------------------------------
+// A training step ternarizes every layer (Algorithm 1, first loop).  One launch per sweep for
+// all of them: the blocks of the grid are dealt out to the tensors in proportion to their size,
+// and each tensor keeps its own tickets and partials, so its results are bit-identical to those
+// of a call of its own.
+constexpr int kMaxBatch = 32;
+struct BatchItem {
+    const float *W;
+    long long rows, cols, ld_codes, fast_units;
+    uint32_t *packed;
+    int8_t *codes_i8;
+    twn_stats_t *stats;
+};
+struct BatchParams {
+    int count;
+    unsigned int first_block[kMaxBatch + 1];   // blocks [first_block[t], first_block[t+1]) work on tensor t
+    BatchItem item[kMaxBatch];
+};
+
+// Slice t of a batch workspace: the tickets of all tensors come first (256 bytes each, so that one
+// small memset clears them), then the partials.
+__host__ __device__ inline Workspace carve_batch(void *ws, int t, int count)
+{
+    char *b = static_cast<char *>(ws);
+    Workspace w;
+    w.ticket1 = reinterpret_cast<unsigned int *>(b + (size_t)t * 256);
+    w.ticket2 = reinterpret_cast<unsigned int *>(b + (size_t)t * 256 + 64);
+    char *p = b + (size_t)count * 256 + (size_t)t * (4 * size_t(kMaxBlocks) * 8);
+    w.part_sum = reinterpret_cast<double *>(p);
+    w.part_kept = w.part_sum + kMaxBlocks;
+    w.part_pos = reinterpret_cast<unsigned long long *>(w.part_kept + kMaxBlocks);
+    w.part_neg = w.part_pos + kMaxBlocks;
+    return w;
+}
+
+__device__ __forceinline__ int batch_tensor_of(const BatchParams &P, unsigned int block)
+{
+    int t = 0;
+    while (t + 1 < P.count && block >= P.first_block[t + 1]) ++t;
+    return t;
+}
+
+__global__ void __launch_bounds__(kThreads)
+sum_abs_batch_kernel(const __grid_constant__ BatchParams P, double factor, void *ws_raw)
+{
+    const int t = batch_tensor_of(P, blockIdx.x);
+    const BatchItem &it = P.item[t];
+    sum_abs_body(it.W, it.rows * it.cols, factor, carve_batch(ws_raw, t, P.count), it.stats,
+                 blockIdx.x - P.first_block[t], P.first_block[t + 1] - P.first_block[t]);
+}
+
+__global__ void __launch_bounds__(kThreads)
+code_pack_batch_kernel(const __grid_constant__ BatchParams P, void *ws_raw)
+{
+    const int t = batch_tensor_of(P, blockIdx.x);
+    const BatchItem &it = P.item[t];
+    code_pack_body(it.W, it.rows, it.cols, it.ld_codes, it.fast_units, it.packed, it.codes_i8,
+                   carve_batch(ws_raw, t, P.count), it.stats, blockIdx.x - P.first_block[t],
+                   P.first_block[t + 1] - P.first_block[t]);
 }
 
 // ---- standalone pack / unpack / re-layout ----------------------------------
@@ -512,6 +587,60 @@ extern "C" int twn_ternarize(const float *W, int64_t rows, int64_t cols, double 
     const int g2 = grid_for(work, dev.sm_count);
     code_pack_kernel<<<g2, kThreads, 0, s>>>(W, rows, cols, ld_codes, fast_units, packed, codes_i8,
                                              workspace, stats);
+    TWN_CUDA_OK(cudaGetLastError());
+    return TWN_OK;
+}
+
+extern "C" size_t twn_ternarize_batch_workspace_bytes(int count)
+{
+    return count > 0 ? (size_t)count * (256 + 4 * size_t(kMaxBlocks) * 8) : 0;
+}
+
+extern "C" int twn_ternarize_batch(const twn_ternarize_item_t *items, int count, double delta_factor,
+                                   void *workspace, size_t workspace_bytes, twn_stream_t stream)
+{
+    TWN_REQUIRE(count >= 0 && count <= kMaxBatch, TWN_ERR_INVALID_ARG);
+    if (count == 0) return TWN_OK;
+    TWN_REQUIRE(items != nullptr && workspace != nullptr, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(delta_factor >= 0.0 && delta_factor == delta_factor, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(workspace_bytes >= twn_ternarize_batch_workspace_bytes(count), TWN_ERR_WORKSPACE);
+    TWN_REQUIRE(twn_aligned(workspace, 256), TWN_ERR_MISALIGNED);
+    twn_device_info dev;
+    const int rc = twn_current_device(&dev);
+    if (rc != TWN_OK) return rc;
+
+    BatchParams A, B;
+    A.count = B.count = count;
+    unsigned int ga = 0, gb = 0;
+    for (int t = 0; t < count; ++t) {
+        const twn_ternarize_item_t &it = items[t];
+        TWN_REQUIRE(it.rows >= 0 && it.cols >= 0 && it.stats != nullptr, TWN_ERR_INVALID_ARG);
+        TWN_REQUIRE(it.ld_codes >= it.cols && it.ld_codes % 64 == 0, TWN_ERR_INVALID_ARG);
+        const long long n = (long long)it.rows * it.cols;
+        TWN_REQUIRE(n == 0 || (it.W != nullptr && it.packed != nullptr), TWN_ERR_INVALID_ARG);
+        TWN_REQUIRE(twn_aligned(it.W, 16) && twn_aligned(it.packed, 16) && twn_aligned(it.stats, 8) &&
+                        twn_aligned(it.codes_i8, 16), TWN_ERR_MISALIGNED);
+        // the same grids and the same split into fast units and rest as a call of its own
+        const bool flat = (it.rows <= 1) || (it.ld_codes == it.cols);
+        const long long fast_units = flat ? n / 512 : 0;
+        const long long rest_words = (long long)it.rows * (it.ld_codes / 16) - fast_units * 32;
+        long long work = fast_units * 32 / 4;
+        if (rest_words > work) work = rest_words;
+        BatchItem bi;
+        bi.W = it.W; bi.rows = it.rows; bi.cols = it.cols; bi.ld_codes = it.ld_codes; bi.fast_units = fast_units;
+        bi.packed = it.packed; bi.codes_i8 = it.codes_i8; bi.stats = it.stats;
+        A.item[t] = B.item[t] = bi;
+        A.first_block[t] = ga;
+        B.first_block[t] = gb;
+        ga += (unsigned int)grid_for((n / 4 + 3) / 4, dev.sm_count);
+        gb += (unsigned int)grid_for(work, dev.sm_count);
+    }
+    A.first_block[count] = ga;
+    B.first_block[count] = gb;
+    cudaStream_t s = twn_cu(stream);
+    TWN_CUDA_OK(cudaMemsetAsync(workspace, 0, (size_t)count * 256, s));     // the tickets start at zero
+    sum_abs_batch_kernel<<<ga, kThreads, 0, s>>>(A, delta_factor, workspace);
+    code_pack_batch_kernel<<<gb, kThreads, 0, s>>>(B, workspace);
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }

@@ -103,7 +103,6 @@ class TernaryNet:
                 e["ld"] = twn.ld_for(L.K)
                 e["packed"] = torch.zeros((L.Cout, e["ld"] // 16), dtype=torch.int32, device="cuda")
                 e["stats"] = twn.new_stats()
-                e["ws"] = torch.empty(twn.ternarize_workspace_bytes(), dtype=torch.uint8, device="cuda")
                 if L.affine:
                     e["scale"] = _dev(dg.draw(self.seed, f"{self.name}.{L.name}.scale", L.Cout, "normal", 1.0, float(np.sqrt(0.1))))
                     e["shift"] = _dev(dg.draw(self.seed, f"{self.name}.{L.name}.shift", L.Cout, "normal", 0.0, float(np.sqrt(0.1))))
@@ -158,6 +157,8 @@ class TernaryNet:
                 _, name, src = op
                 a = self.act[src]
                 self.act[name] = a.view(a.shape[0], 1, 1, -1)
+        self.ws_tern = torch.empty(twn.ternarize_batch_workspace_bytes(min(len(self.layers), 32)),
+                                   dtype=torch.uint8, device="cuda")
         if self.train:
             for name, a in self.act.items():
                 if name != "input" and a.dtype == torch.bfloat16:
@@ -178,29 +179,36 @@ class TernaryNet:
 
     # ------------------------------------------------------------------ Algorithm 1, first loop
     def ternarize_all(self, join: bool = True):
-        """Per-layer ternarization (and the transposed codes for the backward pass) on side streams.
-        Every layer records an event when its codes are ready; forward and backward wait for the
-        event of the layer they are about to run, so the small ternarization kernels of later
-        layers overlap the convolutions of earlier ones."""
+        """Algorithm 1, first loop: every layer's threshold, codes and scale, all layers in one
+        batched call (two launches per 32 layers) on the current stream.  The re-layouts of the codes
+        for the backward pass follow on side streams; each records an event when its codes are ready,
+        and the backward pass waits for the event of the layer it is about to run."""
         main = torch.cuda.current_stream()
-        for st in self.side_streams:
-            st.wait_stream(main)
-        for i, L in enumerate(self.layers.values()):
-            e = L.extra
-            st = self.side_streams[i % len(self.side_streams)]
-            with torch.cuda.stream(st):
-                self._call("ternarize", L.name, 0, lambda: twn.ternarize(
-                    e["W"], self.delta_factor, e["stats"], e["packed"], e["ld"], None, e["ws"],
-                    rows=L.Cout, cols=L.K))
-                if L.fold:
-                    twn.fold_codes(L.desc, e["packed"], e["ld"], e["packed_f"], L.fold[2])
-                e["ready"] = torch.cuda.Event()
-                e["ready"].record(st)
-                if self.train and "packed_b" in e:
+        layers = list(self.layers.values())
+        for i in range(0, len(layers), 32):
+            group = layers[i:i + 32]
+            items = [(L.extra["W"], L.Cout, L.K, L.extra["stats"], L.extra["packed"], L.extra["ld"], None)
+                     for L in group]
+            self._call("ternarize", f"layers {i}..{i + len(group) - 1}", 0,
+                       lambda: twn.ternarize_batch(items, self.delta_factor, self.ws_tern))
+        for L in layers:
+            if L.fold:
+                twn.fold_codes(L.desc, L.extra["packed"], L.extra["ld"], L.extra["packed_f"], L.fold[2])
+        if self.train:
+            for st in self.side_streams:
+                st.wait_stream(main)
+            j = 0
+            for L in layers:
+                e = L.extra
+                if "packed_b" not in e:
+                    continue
+                st = self.side_streams[j % len(self.side_streams)]
+                j += 1
+                with torch.cuda.stream(st):
                     twn.transpose_codes(e["packed"], e["ld"], L.desc, e["packed_b"], e["ld_b"])
                     e["ready_b"] = torch.cuda.Event()
                     e["ready_b"].record(st)
-        self._pending_join = True
+            self._pending_join = True
         if join:
             self.join_side_streams()
 

@@ -65,6 +65,7 @@ def lib() -> C.CDLL:
         l = C.CDLL(LIB_PATH)
         l.twn_strerror.restype = C.c_char_p
         l.twn_ternarize_workspace_bytes.restype = C.c_size_t
+        l.twn_ternarize_batch_workspace_bytes.restype = C.c_size_t
         l.twn_conv2d_bwd_weight_workspace_bytes.restype = C.c_size_t
         l.twn_conv2d_bwd_weight_folded_workspace_bytes.restype = C.c_size_t
         _lib = l
@@ -131,6 +132,26 @@ def ternarize(W: torch.Tensor, delta_factor: float, stats: torch.Tensor, packed:
                                _ptr(stats), _ptr(packed), C.c_int64(ld_codes), _ptr(codes_i8),
                                _ptr(workspace), C.c_size_t(workspace.numel() * workspace.element_size()),
                                _stream(stream)), "twn_ternarize")
+
+
+class TernarizeItem(C.Structure):
+    _fields_ = [("W", C.c_void_p), ("rows", C.c_int64), ("cols", C.c_int64), ("stats", C.c_void_p),
+                ("packed", C.c_void_p), ("ld_codes", C.c_int64), ("codes_i8", C.c_void_p)]
+
+
+def ternarize_batch_workspace_bytes(count: int) -> int:
+    return int(lib().twn_ternarize_batch_workspace_bytes(C.c_int(count)))
+
+
+def ternarize_batch(items, delta_factor: float, workspace: torch.Tensor, stream=None) -> None:
+    """twn_ternarize_batch.  items: list of (W, rows, cols, stats, packed, ld_codes, codes_i8 or None)."""
+    arr = (TernarizeItem * max(len(items), 1))()
+    for i, (W, rows, cols, stats, packed, ld, codes) in enumerate(items):
+        arr[i] = TernarizeItem(_ptr(W).value, rows, cols, _ptr(stats).value, _ptr(packed).value, ld,
+                               _ptr(codes).value)
+    _check(lib().twn_ternarize_batch(arr, C.c_int(len(items)), C.c_double(delta_factor), _ptr(workspace),
+                                     C.c_size_t(workspace.numel() * workspace.element_size()),
+                                     _stream(stream)), "twn_ternarize_batch")
 
 
 def ternarize_rows(W: torch.Tensor, delta_factor: float, stats: torch.Tensor, packed: torch.Tensor,

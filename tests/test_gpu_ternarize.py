@@ -224,3 +224,55 @@ def test_transpose_codes(Cout, Cin, k):
     twn.transpose_codes(pf, ld_f, twn.conv_desc(1, 8, 8, Cin, Cout, k), pb, ld_b)
     want = oracle.pack(np.ascontiguousarray(codes.transpose(3, 1, 2, 0)).reshape(Cin, -1), ld_b)
     assert np.array_equal(host_u32(pb), want)
+
+
+def test_batched_call_equals_one_call_per_tensor():
+    """twn_ternarize_batch (the first loop of Algorithm 1 for a whole network in one launch per
+    sweep) gives every tensor the bits of a twn_ternarize call of its own, and those match the oracle."""
+    shapes = [(64, 147), (64, 576), (128, 1152), (256, 2304), (1000, 512), (10, 1024), (32, 25), (3, 5),
+              (1, 1), (512, 4608), (1, 70000), (7, 0)]
+    Ws = [dg.he_normal(31, f"batch{i}", r, max(c, 1))[:, :c] * np.float32(0.3 + i) for i, (r, c) in enumerate(shapes)]
+    Ws = [np.ascontiguousarray(w) for w in Ws]
+    dev, items, outs = [], [], []
+    for w in Ws:
+        rows, cols = w.shape
+        ld = twn.ld_for(max(cols, 1))
+        Wd = dev_f32(w) if w.size else torch.zeros(4, dtype=torch.float32, device="cuda")
+        stats = twn.new_stats()
+        packed = torch.full((rows, ld // 16), -1, dtype=torch.int32, device="cuda")
+        codes = torch.full((rows, max(cols, 1)), 7, dtype=torch.int8, device="cuda")[:, :cols].contiguous() if cols else None
+        dev.append(Wd)
+        items.append((Wd, rows, cols, stats, packed, ld, codes))
+        outs.append((stats, packed, codes))
+    ws = workspace(twn.ternarize_batch_workspace_bytes(len(items)))
+    twn.ternarize_batch(items, 0.7, ws)
+    torch.cuda.synchronize()
+    for w, (stats, packed, codes) in zip(Ws, outs):
+        rows, cols = w.shape
+        ld = twn.ld_for(max(cols, 1))
+        st1, packed1, codes1 = run_ternarize(w, 0.7, ld) if w.size else (None, None, None)
+        st = twn.stats_to_host(stats)
+        if w.size == 0:
+            assert st["status"] == 0 and st["delta"] == 0.0 and st["alpha"] == 0.0
+            assert not host_u32(packed).any()
+            continue
+        assert st == st1                                   # same reduction order: same bits
+        assert np.array_equal(host_u32(packed), packed1)
+        assert np.array_equal(codes.cpu().numpy(), codes1)
+        ref, ref_codes = oracle.ternarize(w, 0.7)
+        assert abs(st["delta"] - ref.delta) <= REL * ref.delta and abs(st["alpha"] - ref.alpha) <= REL * ref.alpha
+        assert np.array_equal(host_u32(packed), oracle.pack(ref_codes.reshape(rows, cols), ld))
+
+
+def test_batched_call_argument_checks():
+    ws = workspace(twn.ternarize_batch_workspace_bytes(2))
+    W = torch.zeros((1, 64), dtype=torch.float32, device="cuda")
+    item = (W, 1, 64, twn.new_stats(), torch.zeros((1, 4), dtype=torch.int32, device="cuda"), 64, None)
+    twn.ternarize_batch([], 0.7, ws)
+    with pytest.raises(twn.TwnError):
+        twn.ternarize_batch([item] * 33, 0.7, ws)               # more than 32 tensors
+    with pytest.raises(twn.TwnError):
+        twn.ternarize_batch([item] * 3, 0.7, ws)                # workspace sized for two
+    bad = (W, 1, 64, twn.new_stats(), torch.zeros((1, 4), dtype=torch.int32, device="cuda"), 32, None)
+    with pytest.raises(twn.TwnError):
+        twn.ternarize_batch([bad], 0.7, ws)                     # pitch shorter than the row
