@@ -458,7 +458,6 @@ class NetWorkload:
                 L = op[1]
                 n += 1 + (1 if L.small_cin else 0)                       # forward (+ im2col or input fold)
                 if self.train:
-                    n += 1 if L.src != "input" else 0                    # transposed codes for the backward pass
                     n += 1 if L.fold else 0                              # folded codes
                     n += 1 + 2 + (1 if L.fold else 0)                    # act_bwd, dW + reduce (+ unfold)
                     if L.src != "input":
@@ -466,7 +465,7 @@ class NetWorkload:
             elif op[0] in ("maxpool", "avgpool"):
                 n += 2 if self.train else 1
         if self.train:
-            n += 2 * ((len(net.layers) + 31) // 32)                      # the two sweeps of the batched ternarization
+            n += 3 * ((len(net.layers) + 31) // 32)     # batched ternarization (two sweeps) and code transposes
         return n
 
     def units_per_step(self):

@@ -239,6 +239,17 @@ int twn_unpack(const uint32_t *packed, int64_t rows, int64_t cols, int64_t ld_co
 int twn_transpose_codes(const uint32_t *packed_fwd, int64_t ld_fwd, const twn_conv_desc_t *desc,
                         uint32_t *packed_bwd, int64_t ld_bwd, twn_stream_t stream);
 
+/* twn_transpose_codes for up to 32 filter banks in one launch (all layers of a training step).
+ * items: HOST array, read during the call only; fields as the arguments of twn_transpose_codes. */
+typedef struct {
+    const uint32_t *packed_fwd;
+    int64_t ld_fwd;
+    twn_conv_desc_t desc;
+    uint32_t *packed_bwd;
+    int64_t ld_bwd;
+} twn_transpose_item_t;
+int twn_transpose_codes_batch(const twn_transpose_item_t *items, int count, twn_stream_t stream);
+
 /* ---- ternary-weight contractions (Eq. 2; Algorithm 1, TernaryForward/Backward) ---- */
 
 /*

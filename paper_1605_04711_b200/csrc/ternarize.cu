@@ -488,14 +488,15 @@ unpack_kernel(const uint32_t *__restrict__ packed, long long rows, long long col
 
 // out row c, column t*Cout + o  <-  in row o, column t*Cin + c   (t = tap index)
 // (32-bit index arithmetic: a filter bank has far fewer than 2^31 codes)
-__global__ void __launch_bounds__(kThreads)
-transpose_codes_kernel(const uint32_t *__restrict__ in, int ld_in, int Cout, int Cin,
-                       int taps, uint32_t *__restrict__ out, int ld_out)
+// `vb` of `vg`: this block's index among the blocks that work on this filter bank.
+__device__ __forceinline__ void transpose_codes_body(const uint32_t *__restrict__ in, int ld_in, int Cout, int Cin,
+                                                     int taps, uint32_t *__restrict__ out, int ld_out,
+                                                     unsigned int vb, unsigned int vg)
 {
     const int wpr_out = ld_out >> 4, wpr_in = ld_in >> 4;
     const int total = Cin * wpr_out;
     const int cols_out = taps * Cout;
-    for (int w = blockIdx.x * kThreads + threadIdx.x; w < total; w += gridDim.x * kThreads) {
+    for (int w = vb * kThreads + threadIdx.x; w < total; w += vg * kThreads) {
         const int c = w / wpr_out;
         const int j0 = (w - c * wpr_out) << 4;
         int t = j0 / Cout, o = j0 - t * Cout;
@@ -511,6 +512,35 @@ transpose_codes_kernel(const uint32_t *__restrict__ in, int ld_in, int Cout, int
         }
         out[w] = word;
     }
+}
+
+__global__ void __launch_bounds__(kThreads)
+transpose_codes_kernel(const uint32_t *__restrict__ in, int ld_in, int Cout, int Cin,
+                       int taps, uint32_t *__restrict__ out, int ld_out)
+{
+    transpose_codes_body(in, ld_in, Cout, Cin, taps, out, ld_out, blockIdx.x, gridDim.x);
+}
+
+// The filter banks of a whole network in one launch (the backward pass of a step needs them all).
+struct TransposeItem {
+    const uint32_t *in;
+    uint32_t *out;
+    int ld_in, ld_out, Cout, Cin, taps;
+};
+struct TransposeBatch {
+    int count;
+    unsigned int first_block[kMaxBatch + 1];
+    TransposeItem item[kMaxBatch];
+};
+
+__global__ void __launch_bounds__(kThreads)
+transpose_codes_batch_kernel(const __grid_constant__ TransposeBatch P)
+{
+    int t = 0;
+    while (t + 1 < P.count && blockIdx.x >= P.first_block[t + 1]) ++t;
+    const TransposeItem &it = P.item[t];
+    transpose_codes_body(it.in, it.ld_in, it.Cout, it.Cin, it.taps, it.out, it.ld_out,
+                         blockIdx.x - P.first_block[t], P.first_block[t + 1] - P.first_block[t]);
 }
 
 // Codes of a stride-2 layer re-ordered for the folded input: folded row r' holds 64 columns,
@@ -770,6 +800,42 @@ extern "C" int twn_transpose_codes(const uint32_t *packed_fwd, int64_t ld_fwd,
                     ld_bwd < 0x7fffffffLL, TWN_ERR_INVALID_ARG);
     transpose_codes_kernel<<<grid_for(words, dev.sm_count), kThreads, 0, twn_cu(stream)>>>(
         packed_fwd, (int)ld_fwd, (int)d->Cout, (int)d->Cin, (int)taps, packed_bwd, (int)ld_bwd);
+    TWN_CUDA_OK(cudaGetLastError());
+    return TWN_OK;
+}
+
+extern "C" int twn_transpose_codes_batch(const twn_transpose_item_t *items, int count, twn_stream_t stream)
+{
+    TWN_REQUIRE(count >= 0 && count <= kMaxBatch, TWN_ERR_INVALID_ARG);
+    if (count == 0) return TWN_OK;
+    TWN_REQUIRE(items != nullptr, TWN_ERR_INVALID_ARG);
+    twn_device_info dev;
+    const int rc = twn_current_device(&dev);
+    if (rc != TWN_OK) return rc;
+    TransposeBatch P;
+    P.count = count;
+    unsigned int g = 0;
+    for (int t = 0; t < count; ++t) {
+        const twn_transpose_item_t &it = items[t];
+        const twn_conv_desc_t *d = &it.desc;
+        TWN_REQUIRE(it.packed_fwd && it.packed_bwd, TWN_ERR_INVALID_ARG);
+        TWN_REQUIRE(d->Cin > 0 && d->Cout > 0 && d->kh > 0 && d->kw > 0, TWN_ERR_INVALID_ARG);
+        const long long taps = (long long)d->kh * d->kw;
+        TWN_REQUIRE(it.ld_fwd % 64 == 0 && it.ld_bwd % 64 == 0 && it.ld_fwd >= taps * d->Cin && it.ld_bwd >= taps * d->Cout,
+                    TWN_ERR_INVALID_ARG);
+        TWN_REQUIRE(twn_aligned(it.packed_fwd, 16) && twn_aligned(it.packed_bwd, 16), TWN_ERR_MISALIGNED);
+        const long long words = d->Cin * (it.ld_bwd / 16);
+        TWN_REQUIRE(words < 0x7fffffffLL && d->Cout * (it.ld_fwd / 16) < 0x7fffffffLL && it.ld_fwd < 0x7fffffffLL &&
+                        it.ld_bwd < 0x7fffffffLL, TWN_ERR_INVALID_ARG);
+        TransposeItem ti;
+        ti.in = it.packed_fwd; ti.out = it.packed_bwd; ti.ld_in = (int)it.ld_fwd; ti.ld_out = (int)it.ld_bwd;
+        ti.Cout = (int)d->Cout; ti.Cin = (int)d->Cin; ti.taps = (int)taps;
+        P.item[t] = ti;
+        P.first_block[t] = g;
+        g += (unsigned int)grid_for(words, dev.sm_count);
+    }
+    P.first_block[count] = g;
+    transpose_codes_batch_kernel<<<g, kThreads, 0, twn_cu(stream)>>>(P);
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }

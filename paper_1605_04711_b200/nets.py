@@ -76,9 +76,8 @@ class TernaryNet:
         self.aux: dict[str, torch.Tensor] = {}
         self.grad: dict[str, torch.Tensor] = {}
         self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
-        # the per-layer ternarizations are independent: they run on a few side streams, each layer
-        # with its own scratch
-        self.side_streams = [torch.cuda.Stream() for _ in range(4)]
+        # the code re-layouts for the backward pass run on a side stream beside the forward pass
+        self.side_streams = [torch.cuda.Stream()]
         self.dw_stream = torch.cuda.Stream()     # weight gradients run beside the backward-for-data chain
         self.timed = None          # when a list: (kind, name, flops, start event, end event)
         H, W, C = in_shape
@@ -181,8 +180,8 @@ class TernaryNet:
     def ternarize_all(self, join: bool = True):
         """Algorithm 1, first loop: every layer's threshold, codes and scale, all layers in one
         batched call (two launches per 32 layers) on the current stream.  The re-layouts of the codes
-        for the backward pass follow on side streams; each records an event when its codes are ready,
-        and the backward pass waits for the event of the layer it is about to run."""
+        for the backward pass follow as one batched launch on a side stream, beside the forward pass;
+        the backward pass waits for its event."""
         main = torch.cuda.current_stream()
         layers = list(self.layers.values())
         for i in range(0, len(layers), 32):
@@ -195,19 +194,18 @@ class TernaryNet:
             if L.fold:
                 twn.fold_codes(L.desc, L.extra["packed"], L.extra["ld"], L.extra["packed_f"], L.fold[2])
         if self.train:
-            for st in self.side_streams:
-                st.wait_stream(main)
-            j = 0
-            for L in layers:
-                e = L.extra
-                if "packed_b" not in e:
-                    continue
-                st = self.side_streams[j % len(self.side_streams)]
-                j += 1
-                with torch.cuda.stream(st):
-                    twn.transpose_codes(e["packed"], e["ld"], L.desc, e["packed_b"], e["ld_b"])
-                    e["ready_b"] = torch.cuda.Event()
-                    e["ready_b"].record(st)
+            # the re-layouts for the backward pass: one batched launch beside the forward pass
+            st = self.side_streams[0]
+            st.wait_stream(main)
+            todo = [L for L in layers if "packed_b" in L.extra]
+            with torch.cuda.stream(st):
+                for i in range(0, len(todo), 32):
+                    twn.transpose_codes_batch([(L.extra["packed"], L.extra["ld"], L.desc, L.extra["packed_b"],
+                                                L.extra["ld_b"]) for L in todo[i:i + 32]])
+                ev = torch.cuda.Event()
+                ev.record(st)
+            for L in todo:
+                L.extra["ready_b"] = ev
             self._pending_join = True
         if join:
             self.join_side_streams()
@@ -222,8 +220,7 @@ class TernaryNet:
         and before the master weights change)."""
         if getattr(self, "_pending_join", False):
             main = torch.cuda.current_stream()
-            for st in self.side_streams:
-                main.wait_stream(st)
+            main.wait_stream(self.side_streams[0])      # the only side stream ternarize_all forks
             self._pending_join = False
             for L in self.layers.values():      # nothing left to wait for
                 L.extra.pop("ready", None)

@@ -154,6 +154,19 @@ def ternarize_batch(items, delta_factor: float, workspace: torch.Tensor, stream=
                                      _stream(stream)), "twn_ternarize_batch")
 
 
+class TransposeItem(C.Structure):
+    _fields_ = [("packed_fwd", C.c_void_p), ("ld_fwd", C.c_int64), ("desc", ConvDesc), ("packed_bwd", C.c_void_p),
+                ("ld_bwd", C.c_int64)]
+
+
+def transpose_codes_batch(items, stream=None) -> None:
+    """twn_transpose_codes_batch.  items: list of (packed_fwd, ld_fwd, desc, packed_bwd, ld_bwd)."""
+    arr = (TransposeItem * max(len(items), 1))()
+    for i, (pf, ldf, desc, pb, ldb) in enumerate(items):
+        arr[i] = TransposeItem(_ptr(pf).value, ldf, desc, _ptr(pb).value, ldb)
+    _check(lib().twn_transpose_codes_batch(arr, C.c_int(len(items)), _stream(stream)), "twn_transpose_codes_batch")
+
+
 def ternarize_rows(W: torch.Tensor, delta_factor: float, stats: torch.Tensor, packed: torch.Tensor,
                    ld_codes: int, codes_i8=None, stream=None) -> None:
     """twn_ternarize_rows: one threshold and one scale per filter.  W fp32 [rows, cols];

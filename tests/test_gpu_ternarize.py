@@ -276,3 +276,27 @@ def test_batched_call_argument_checks():
     bad = (W, 1, 64, twn.new_stats(), torch.zeros((1, 4), dtype=torch.int32, device="cuda"), 32, None)
     with pytest.raises(twn.TwnError):
         twn.ternarize_batch([bad], 0.7, ws)                     # pitch shorter than the row
+
+
+def test_batched_transpose_equals_one_call_per_filter_bank():
+    cases = [(64, 64, 3), (64, 128, 3), (128, 256, 1), (512, 1000, 1), (16, 24, 5)]
+    items, want = [], []
+    for i, (cin, cout, k) in enumerate(cases):
+        K = k * k * cin
+        codes = np.sign(dg.draw(41, f"tb{i}", cout * K, "normal")).astype(np.int8).reshape(cout, K)
+        codes[np.abs(dg.draw(42, f"tbz{i}", cout * K, "normal").reshape(cout, K)) < 0.5] = 0
+        ld, ld_b = twn.ld_for(K), twn.ld_for(k * k * cout)
+        pf = dev_u32(oracle.pack(codes, ld))
+        d = twn.conv_desc(1, 8, 8, cin, cout, k, 1, k // 2)
+        one = torch.full((cin, ld_b // 16), -1, dtype=torch.int32, device="cuda")
+        twn.transpose_codes(pf, ld, d, one, ld_b)
+        out = torch.full((cin, ld_b // 16), -1, dtype=torch.int32, device="cuda")
+        items.append((pf, ld, d, out, ld_b))
+        # [Cout][taps][Cin] -> [Cin][taps][Cout]
+        t = codes.reshape(cout, k * k, cin).transpose(2, 1, 0).reshape(cin, k * k * cout)
+        want.append((one, oracle.pack(np.ascontiguousarray(t), ld_b)))
+    twn.transpose_codes_batch(items)
+    torch.cuda.synchronize()
+    for (pf, ld, d, out, ld_b), (one, ref) in zip(items, want):
+        assert torch.equal(out, one)
+        assert np.array_equal(host_u32(out), ref)
