@@ -71,7 +71,14 @@ typedef struct {
 /* What follows the contraction, per output element with channel n:
  *   y = acc * alpha;  y = y * scale[n] + shift[n];  y += residual;  y = max(y, 0)
  * each step only if its field is set.  (Eq. 2 puts alpha on the input; a scalar
- * commutes with the sum, so it is applied once per output here.) */
+ * commutes with the sum, so it is applied once per output here.)
+ * With residual_op = TWN_RESIDUAL_GATE the tensor given as `residual` is not added but gates
+ * the result: y is kept where residual > 0 and is 0 elsewhere.  This is the backward pass of
+ * a ReLU fused into the backward-for-data pass of the layer above it: with `residual` = the
+ * lower layer's output and `scale` = its folded batch-norm scale, twn_conv2d_bwd_data writes
+ * the lower layer's dZ directly (Algorithm 1, TernaryBackward, followed by the chain rule
+ * through y = relu(z * scale + shift)). */
+enum { TWN_RESIDUAL_ADD = 0, TWN_RESIDUAL_GATE = 1 };
 typedef struct {
     const float *scale;    /* fp32 [N] or NULL (folded batch-norm scale)            */
     const float *shift;    /* fp32 [N] or NULL                                      */
@@ -79,7 +86,7 @@ typedef struct {
     int32_t residual_dtype;/* TWN_F32 | TWN_BF16                                    */
     int32_t relu;          /* 0 | 1                                                 */
     int32_t out_dtype;     /* TWN_F32 | TWN_BF16 (round to nearest even)            */
-    int32_t reserved;
+    int32_t residual_op;   /* TWN_RESIDUAL_ADD (0) | TWN_RESIDUAL_GATE              */
 } twn_epilogue_t;
 
 /* ---- library ---------------------------------------------------------- */

@@ -126,6 +126,7 @@ struct ConvParams {
     const float *scale, *shift;
     const void *residual;
     int res_dtype, relu, out_dtype;
+    int res_gate;                 // 0: the residual is added; 1: it gates the result (kept where residual > 0)
     void *Y;
     int32_t *status;
     // output path: 1 = each epilogue warp stages its 32 channels x 32 pixels in shared memory and
@@ -532,9 +533,17 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 // exposed latency of this warp's chunk.
                 if (use_res_tma) {
                     const __nv_bfloat16 *rs = my_res + (nres & 1u) * (32 * 32) + lane;
+                    if (P.res_gate) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        v[j] = __float_as_uint(fmaxf(fmaf(__uint_as_float(v[j]), sc, sf) + __bfloat162float(rs[j * 32]), floor_v));
+                        for (int j = 0; j < 32; ++j) {
+                            const float y = fmaxf(fmaf(__uint_as_float(v[j]), sc, sf), floor_v);
+                            v[j] = __float_as_uint(__bfloat162float(rs[j * 32]) > 0.0f ? y : 0.0f);
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            v[j] = __float_as_uint(fmaxf(fmaf(__uint_as_float(v[j]), sc, sf) + __bfloat162float(rs[j * 32]), floor_v));
+                    }
                     // the buffer is free again: fetch the residual of the chunk after the next
                     __syncwarp();
                     if (lane == 0 && i + 2 < kMine) res_load(c + 2 * kEpiSets, nres & 1u);
@@ -548,7 +557,8 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                         if (o != 0xFFFFFFFFu && n_ok)
                             r = res_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(P.residual)[(size_t)o + n])
                                          : reinterpret_cast<const float *>(P.residual)[(size_t)o + n];
-                        v[j] = __float_as_uint(fmaxf(fmaf(__uint_as_float(v[j]), sc, sf) + r, floor_v));
+                        const float y = fmaf(__uint_as_float(v[j]), sc, sf);
+                        v[j] = __float_as_uint(P.res_gate ? (r > 0.0f ? fmaxf(y, floor_v) : 0.0f) : fmaxf(y + r, floor_v));
                     }
                 } else {
 #pragma unroll
@@ -805,6 +815,7 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     P.shift = epi ? epi->shift : nullptr;
     P.residual = epi ? epi->residual : nullptr;
     P.res_dtype = epi ? epi->residual_dtype : TWN_F32;
+    P.res_gate = (epi && epi->residual) ? epi->residual_op : 0;
     P.relu = epi ? epi->relu : 0;
     P.out_dtype = epi ? epi->out_dtype : out_dtype_default;
     P.Y = Y;
@@ -874,6 +885,7 @@ int check_epilogue(const twn_epilogue_t *e)
     TWN_REQUIRE(e->out_dtype == TWN_F32 || e->out_dtype == TWN_BF16, TWN_ERR_INVALID_ARG);
     TWN_REQUIRE(e->residual_dtype == TWN_F32 || e->residual_dtype == TWN_BF16, TWN_ERR_INVALID_ARG);
     TWN_REQUIRE(e->relu == 0 || e->relu == 1, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(e->residual_op == TWN_RESIDUAL_ADD || e->residual_op == TWN_RESIDUAL_GATE, TWN_ERR_INVALID_ARG);
     TWN_REQUIRE(twn_aligned(e->scale, 4) && twn_aligned(e->shift, 4) && twn_aligned(e->residual, 4), TWN_ERR_MISALIGNED);
     return TWN_OK;
 }

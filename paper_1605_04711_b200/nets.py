@@ -282,6 +282,25 @@ class TernaryNet:
             fn(acc.get(name), out)
             acc[name] = out
 
+        # A layer P = relu(z * scale + shift) whose output feeds exactly one convolution gets its
+        # dZ straight from that convolution's backward-for-data pass (the ReLU gate and the scale
+        # applied in its epilogue) instead of from an activation-backward sweep of its own.
+        consumers: dict[str, list] = {}
+        for op in self.ops:
+            if op[0] == "layer":
+                consumers.setdefault(op[1].src, []).append(op[1])
+                if op[1].residual:
+                    consumers.setdefault(op[1].residual, []).append(None)
+            elif op[0] in ("maxpool", "avgpool", "flatten"):
+                consumers.setdefault(op[2], []).append(None)
+        FUSED = object()
+
+        def fused_producer(L):
+            P = self.layers.get(L.src)
+            if P is None or not P.relu or P.residual or P.out_f32 or L.fold or L.small_cin:
+                return None
+            return P if consumers.get(P.name) == [L] else None
+
         main = torch.cuda.current_stream()
         self.dw_stream.wait_stream(main)
         for op in reversed(self.ops):
@@ -290,17 +309,18 @@ class TernaryNet:
                 L: Layer = op[1]
                 e = L.extra
                 dY = acc[L.name]
-                n = dY.numel()
-                y = self.act[L.name] if L.relu else None
-                dpre = None
-                if L.residual:
-                    # the gradient before the ReLU also flows, unscaled, into the shortcut branch
-                    dpre = e.get("dpre")
-                    if dpre is None:
-                        dpre = e["dpre"] = torch.zeros_like(e["dz"])
-                twn.act_bwd(dY, y, e["scale"], n, L.Cout, e["dz"], dpre)
-                if L.residual:
-                    emit_tensor(L.residual, dpre)
+                if dY is not FUSED:
+                    n = dY.numel()
+                    y = self.act[L.name] if L.relu else None
+                    dpre = None
+                    if L.residual:
+                        # the gradient before the ReLU also flows, unscaled, into the shortcut branch
+                        dpre = e.get("dpre")
+                        if dpre is None:
+                            dpre = e["dpre"] = torch.zeros_like(e["dz"])
+                    twn.act_bwd(dY, y, e["scale"], n, L.Cout, e["dz"], dpre)
+                    if L.residual:
+                        emit_tensor(L.residual, dpre)
                 # dW needs only dz and the layer's input: it goes to its own stream (one after the
                 # other there, they share the workspace) and overlaps the dX chain of the layers below
                 dz_ready = torch.cuda.Event()
@@ -314,7 +334,16 @@ class TernaryNet:
                         x = e["xcol"] if L.small_cin else self.act[L.src]
                         self._call("dw", L.name + ".dW", 2 * L.macs, lambda: twn.conv2d_bwd_weight(
                             e["dw_desc"], x, e["dz"], e["dW"], self.ws_dw, self.status))
-                if L.src != "input":
+                P = fused_producer(L) if L.src != "input" else None
+                if P is not None:
+                    self._wait_codes(L, "ready_b")
+                    epi = twn.epilogue(scale=P.extra["scale"], residual=self.act[P.name], out_dtype=twn.BF16,
+                                       residual_op=twn.RESIDUAL_GATE)
+                    self._call("tconv", L.name + ".dX", 2 * L.macs, lambda: twn.conv2d_bwd_data(
+                        L.desc, e["dz"], e["packed_b"], e["ld_b"], e["stats"], epi, P.extra["dz"], self.status))
+                    assert P.name not in acc
+                    acc[P.name] = FUSED
+                elif L.src != "input":
                     def bwd(res, out, L=L, e=e):
                         self._wait_codes(L, "ready_b")
                         epi = twn.epilogue(residual=res, out_dtype=twn.BF16)

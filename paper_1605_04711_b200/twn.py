@@ -49,7 +49,7 @@ def conv_desc(B, H, W, Cin, Cout, k, stride=1, pad=0) -> ConvDesc:
 class Epilogue(C.Structure):
     _fields_ = [("scale", C.c_void_p), ("shift", C.c_void_p), ("residual", C.c_void_p),
                 ("residual_dtype", C.c_int32), ("relu", C.c_int32), ("out_dtype", C.c_int32),
-                ("reserved", C.c_int32)]
+                ("residual_op", C.c_int32)]
 
 
 _lib = None
@@ -234,7 +234,10 @@ def transpose_codes(packed_fwd: torch.Tensor, ld_fwd: int, desc: ConvDesc, packe
            "twn_transpose_codes")
 
 
-def epilogue(scale=None, shift=None, residual=None, relu=False, out_dtype=F32):
+RESIDUAL_ADD, RESIDUAL_GATE = 0, 1
+
+
+def epilogue(scale=None, shift=None, residual=None, relu=False, out_dtype=F32, residual_op=RESIDUAL_ADD):
     """Builds a twn_epilogue_t; keeps no reference, the caller keeps the tensors alive."""
     e = Epilogue()
     e.scale = _ptr(scale).value or None
@@ -243,6 +246,7 @@ def epilogue(scale=None, shift=None, residual=None, relu=False, out_dtype=F32):
     e.residual_dtype = BF16 if (residual is not None and residual.dtype == torch.bfloat16) else F32
     e.relu = int(bool(relu))
     e.out_dtype = out_dtype
+    e.residual_op = residual_op
     return e
 
 

@@ -206,6 +206,50 @@ def test_bwd_data_adds_a_second_gradient_branch_through_the_residual():
     assert_within(dX.cpu().numpy(), dXr + other.astype(np.float64), A, alpha)
 
 
+@pytest.mark.parametrize("gate_dtype,out_dtype", [("bf16", "bf16"), ("f32", "f32"), ("bf16", "f32")])
+@pytest.mark.parametrize("stride", [1, 2])
+def test_bwd_data_gated_by_the_lower_layers_output(gate_dtype, out_dtype, stride):
+    """TWN_RESIDUAL_GATE: the backward-for-data pass writes the lower layer's dZ, i.e. the gradient
+    times that layer's scale where its (ReLU) output is positive and 0 elsewhere."""
+    B, H, W, Cin, Cout, k, p = 3, 10, 10, 96, 64, 3, 1
+    alpha, codes, packed, ld, stats = ternarized(9, f"gw{stride}", Cout, k * k * Cin)
+    d = twn.conv_desc(B, H, W, Cin, Cout, k, stride, p)
+    ld_b = twn.ld_for(k * k * Cout)
+    packed_b = torch.empty((Cin, ld_b // 16), dtype=torch.int32, device="cuda")
+    twn.transpose_codes(packed, ld, d, packed_b, ld_b)
+    dZ = dg.draw_bf16(9, f"gz{stride}", B * d.Ho * d.Wo * Cout, "normal").reshape(B, d.Ho, d.Wo, Cout)
+    ybits = dg.draw_bf16(9, "gy", B * H * W * Cin, "normal").reshape(B, H, W, Cin)
+    y = np.maximum(dg.bf16_bits_to_f64(ybits), 0.0)                  # a ReLU output: about half zeros
+    scale = dg.draw(9, "gs", Cin, "normal", 1.0, 0.3)
+    yd = dev_bf16(dg.f32_to_bf16_bits(y.astype(np.float32))) if gate_dtype == "bf16" else dev_f32(y)
+    sd = dev_f32(scale)
+    tdt = torch.bfloat16 if out_dtype == "bf16" else torch.float32
+    dX = torch.full((B, H, W, Cin), float("nan"), dtype=tdt, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    epi = twn.epilogue(scale=sd, residual=yd, out_dtype=twn.BF16 if out_dtype == "bf16" else twn.F32,
+                       residual_op=twn.RESIDUAL_GATE)
+    twn.conv2d_bwd_data(d, dev_bf16(dZ), packed_b, ld_b, stats, epi, dX, status)
+    dXr, A = oracle.conv2d_bwd_data(oracle.conv_desc(B, H, W, Cin, Cout, k, stride, p), dZ,
+                                    codes.reshape(Cout, k, k, Cin), alpha)
+    want = np.where(y > 0, dXr * scale.astype(np.float64), 0.0)
+    tol = 1e-4 * alpha * np.abs(scale.astype(np.float64)) * A + 1e-6
+    assert twn.read_status(status) == 0
+    got = dX.float().cpu().numpy().astype(np.float64)
+    if out_dtype == "bf16":
+        tol = tol + 2.0 ** -8 * (np.abs(want) + tol)
+    assert np.all(np.abs(got - want) <= tol)
+    assert np.all(got[y <= 0] == 0.0)
+
+
+def test_epilogue_rejects_an_unknown_residual_op():
+    alpha, codes, packed, ld, stats = ternarized(9, "gbad", 64, 64)
+    X = torch.zeros((8, 64), dtype=torch.bfloat16, device="cuda")
+    Y = torch.zeros((8, 64), dtype=torch.float32, device="cuda")
+    epi = twn.epilogue(residual=Y, residual_op=7)
+    with pytest.raises(twn.TwnError):
+        twn.gemm(X, 64, packed, ld, stats, 8, 64, 64, epi, Y, 64)
+
+
 SWEEP = [(K, N, M) for (K, N) in [(512, 512), (1152, 128), (2304, 256), (4608, 512), (4096, 4096)]
          for M in (128, 1024, 4096, 16384)]
 

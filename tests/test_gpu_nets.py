@@ -103,7 +103,15 @@ def check_backward(net, npix=96, nent=200):
         tol = 1e-4 * alpha * A + 1e-6
         got = f64(net.grad_of_input[L.name]).reshape(-1, L.Cin)[pix]
         prior = net.prior_of_input[L.name]
-        if prior is not None:
+        if net.gated_input.get(L.name):
+            # the pass wrote the lower layer's dZ: its ReLU gate and folded batch-norm scale are
+            # applied to the gradient in the epilogue (`prior` is that layer's output)
+            P = net.layers[L.src]
+            sc = P.extra["scale"].cpu().numpy().astype(np.float64) if P.extra["scale"] is not None else np.ones(L.Cin)
+            gate = f64(prior).reshape(-1, L.Cin)[pix] > 0
+            ref = np.where(gate, ref * sc, 0.0)
+            tol = tol * np.abs(sc)
+        elif prior is not None:
             ref = ref + f64(prior).reshape(-1, L.Cin)[pix]
         within(got, ref, tol, True)
 
@@ -111,7 +119,7 @@ def check_backward(net, npix=96, nent=200):
 def record_dx(net):
     """Wraps conv2d_bwd_data to keep, per layer, a copy of what was in the output buffer before
     (the other branch's gradient) and of the result."""
-    net.grad_of_input, net.prior_of_input = {}, {}
+    net.grad_of_input, net.prior_of_input, net.gated_input = {}, {}, {}
     orig = twn.conv2d_bwd_data
     by_desc = {id(L.desc): L for L in net.layers.values()}
 
@@ -124,6 +132,7 @@ def record_dx(net):
         orig(desc, dZ, T_bwd, ld, stats, epi, dX, status, stream)
         net.grad_of_input[L.name] = dX.clone()
         net.prior_of_input[L.name] = prior
+        net.gated_input[L.name] = epi is not None and epi.residual_op == twn.RESIDUAL_GATE
     return orig, wrapped
 
 
@@ -136,9 +145,9 @@ def run_train_step(net, monkeypatch):
     # keep copies of every backward-for-data result and of the residual it was added to
     orig_epi = twn.epilogue
 
-    def epi_spy(scale=None, shift=None, residual=None, relu=False, out_dtype=twn.F32):
+    def epi_spy(scale=None, shift=None, residual=None, relu=False, out_dtype=twn.F32, residual_op=twn.RESIDUAL_ADD):
         net.last_res = residual
-        return orig_epi(scale, shift, residual, relu, out_dtype)
+        return orig_epi(scale, shift, residual, relu, out_dtype, residual_op)
     orig, wrapped = record_dx(net)
     monkeypatch.setattr(twn, "epilogue", epi_spy)
     monkeypatch.setattr(twn, "conv2d_bwd_data", wrapped)
