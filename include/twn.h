@@ -377,6 +377,18 @@ int twn_maxpool2d_fwd(const void *X, int64_t B, int64_t H, int64_t W, int64_t C,
 int twn_maxpool2d_bwd(const void *dY, const uint8_t *argmax, int64_t B, int64_t H, int64_t W, int64_t C,
                       int k, int stride, int pad, void *dX, twn_stream_t stream);
 
+/* Backward through a max-pool that directly follows a layer y = relu(z * scale[c] + shift[c]),
+ * fused with the backward through that ReLU and scale:
+ *   dZ[b,h,w,c] = scale[c] * sum of dY over the windows whose recorded maximum is (h,w) and whose
+ *                 pooled value is positive
+ * (the pooled value is the layer's output at the window's arg-max, so "pooled > 0" is the ReLU gate
+ * there; everywhere else the gradient is 0 anyway).  pooled: the bf16 output of twn_maxpool2d_fwd,
+ * same shape as dY.  scale fp32 [C] or NULL (1).  Equals twn_maxpool2d_bwd followed by twn_act_bwd
+ * up to one rounding to bf16 instead of two.  Deterministic. */
+int twn_maxpool2d_bwd_act(const void *dY, const uint8_t *argmax, const void *pooled, const float *scale,
+                          int64_t B, int64_t H, int64_t W, int64_t C, int k, int stride, int pad,
+                          void *dZ, twn_stream_t stream);
+
 /* Global average pooling: X bf16 [B, HW, C] -> Y bf16 [B, C]; backward dX = dY / HW. */
 int twn_avgpool_fwd(const void *X, int64_t B, int64_t HW, int64_t C, void *Y, twn_stream_t stream);
 int twn_avgpool_bwd(const void *dY, int64_t B, int64_t HW, int64_t C, void *dX, twn_stream_t stream);

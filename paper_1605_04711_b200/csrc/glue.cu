@@ -182,12 +182,22 @@ maxpool_fwd_kernel(const __nv_bfloat16 *__restrict__ X, I B, I H, I W, I C,
     }
 }
 
+// t[e] = 0 where the pooled value (the window's maximum, i.e. the ReLU output at the arg-max) is not positive
+__device__ __forceinline__ void gate8(float (&t)[8], const uint4 pooled)
+{
+    float p[8];
+    unpack8(pooled, p);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) t[e] = p[e] > 0.0f ? t[e] : 0.0f;
+}
+
 // gather form: an input pixel collects the gradient of every window whose maximum it was
 template <typename I, int V>
 __global__ void __launch_bounds__(kT)
 maxpool_bwd_kernel(const __nv_bfloat16 *__restrict__ dY, const uint8_t *__restrict__ idx, I B, I H,
                    I W, I C, int k, int stride, int pad, I Ho, I Wo,
-                   __nv_bfloat16 *__restrict__ dX)
+                   __nv_bfloat16 *__restrict__ dX, const __nv_bfloat16 *__restrict__ pooled,
+                   const float *__restrict__ scale)
 {
     const I Cv = C / V;
     const I total = B * H * W * Cv;
@@ -212,17 +222,22 @@ maxpool_bwd_kernel(const __nv_bfloat16 *__restrict__ dY, const uint8_t *__restri
                     const uint2 a = __ldg(reinterpret_cast<const uint2 *>(idx + o));
                     float t8[8];
                     unpack8(__ldg(reinterpret_cast<const uint4 *>(dY + o)), t8);
+                    if (pooled) gate8(t8, __ldg(reinterpret_cast<const uint4 *>(pooled + o)));
 #pragma unroll
                     for (int e = 0; e < V; ++e) {
                         const int ai = ((e < 4 ? a.x : a.y) >> (8 * (e & 3))) & 0xFF;
                         if (ai == want) g[e] += t8[e];
                     }
                 } else {
-                    if (idx[o] == want) g[0] += __bfloat162float(dY[o]);
+                    if (idx[o] == want && (!pooled || __bfloat162float(pooled[o]) > 0.0f)) g[0] += __bfloat162float(dY[o]);
                 }
             }
         }
         const I o = ((b * H + h) * W + w) * C + cv * V;
+        if (scale) {
+#pragma unroll
+            for (int e = 0; e < V; ++e) g[e] *= __ldg(scale + cv * V + e);
+        }
         if (V == 8) {
             float t8[8];
 #pragma unroll
@@ -285,7 +300,8 @@ maxpool_fwd_rows_kernel(const __nv_bfloat16 *__restrict__ X, int B, int H, int W
 __global__ void __launch_bounds__(kT)
 maxpool_bwd_rows_kernel(const __nv_bfloat16 *__restrict__ dY, const uint8_t *__restrict__ idx, int B, int H, int W,
                         int C, int k, int stride, int lg_stride, int pad, int Ho, int Wo,
-                        __nv_bfloat16 *__restrict__ dX)
+                        __nv_bfloat16 *__restrict__ dX, const __nv_bfloat16 *__restrict__ pooled,
+                        const float *__restrict__ scale)
 {
     const int Cv = C >> 3, per_row = W * Cv;
     // window row / column that covers input coordinate x with tap t: (x + pad - t) / stride when divisible
@@ -319,7 +335,7 @@ maxpool_bwd_rows_kernel(const __nv_bfloat16 *__restrict__ dY, const uint8_t *__r
                     if (wo >= 0 && nw < 2) { wos[nw] = wo; sxs[nw] = sx; ++nw; }
                 }
                 uint2 a[4];
-                uint4 d[4];
+                uint4 d[4], pl[4];
                 int want[4];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
@@ -328,6 +344,7 @@ maxpool_bwd_rows_kernel(const __nv_bfloat16 *__restrict__ dY, const uint8_t *__r
                     const size_t o = ((size_t)(b * Ho + hos[ih]) * Wo + wos[iw]) * C + cv * 8;   // in range also when !ok
                     a[q] = ok ? __ldg(reinterpret_cast<const uint2 *>(idx + o)) : make_uint2(0xFFFFFFFFu, 0xFFFFFFFFu);
                     d[q] = ok ? __ldg(reinterpret_cast<const uint4 *>(dY + o)) : make_uint4(0u, 0u, 0u, 0u);
+                    if (pooled) pl[q] = ok ? __ldg(reinterpret_cast<const uint4 *>(pooled + o)) : make_uint4(0u, 0u, 0u, 0u);
                     want[q] = rs[ih] * k + sxs[iw];     // < 255: an absent window's 0xFF bytes never match
                 }
                 float g[8];
@@ -337,11 +354,18 @@ maxpool_bwd_rows_kernel(const __nv_bfloat16 *__restrict__ dY, const uint8_t *__r
                 for (int q = 0; q < 4; ++q) {
                     float t8[8];
                     unpack8(d[q], t8);
+                    if (pooled) gate8(t8, pl[q]);
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
                         const int ai = ((e < 4 ? a[q].x : a[q].y) >> (8 * (e & 3))) & 0xFF;
                         if (ai == want[q]) g[e] += t8[e];
                     }
+                }
+                if (scale) {
+                    const float4 s0 = __ldg(reinterpret_cast<const float4 *>(scale + cv * 8));
+                    const float4 s1 = __ldg(reinterpret_cast<const float4 *>(scale + cv * 8 + 4));
+                    g[0] *= s0.x; g[1] *= s0.y; g[2] *= s0.z; g[3] *= s0.w;
+                    g[4] *= s1.x; g[5] *= s1.y; g[6] *= s1.z; g[7] *= s1.w;
                 }
                 *reinterpret_cast<uint4 *>(dX + ((size_t)row * W + w) * C + cv * 8) = pack8(g);
             }
@@ -363,12 +387,17 @@ maxpool_bwd_rows_kernel(const __nv_bfloat16 *__restrict__ dY, const uint8_t *__r
                     const uint2 a = __ldg(reinterpret_cast<const uint2 *>(idx + o));
                     float t8[8];
                     unpack8(__ldg(reinterpret_cast<const uint4 *>(dY + o)), t8);
+                    if (pooled) gate8(t8, __ldg(reinterpret_cast<const uint4 *>(pooled + o)));
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
                         const int ai = ((e < 4 ? a.x : a.y) >> (8 * (e & 3))) & 0xFF;
                         if (ai == want) g[e] += t8[e];
                     }
                 }
+            }
+            if (scale) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) g[e] *= __ldg(scale + cv * 8 + e);
             }
             *reinterpret_cast<uint4 *>(dX + ((size_t)row * W + w) * C + cv * 8) = pack8(g);
         }
@@ -576,8 +605,10 @@ extern "C" int twn_maxpool2d_fwd(const void *X, int64_t B, int64_t H, int64_t W,
     return TWN_OK;
 }
 
-extern "C" int twn_maxpool2d_bwd(const void *dY, const uint8_t *argmax, int64_t B, int64_t H, int64_t W, int64_t C,
-                                 int k, int stride, int pad, void *dX, twn_stream_t stream)
+namespace {
+
+int maxpool_bwd_launch(const void *dY, const uint8_t *argmax, const void *pooled_v, const float *scale, int64_t B,
+                       int64_t H, int64_t W, int64_t C, int k, int stride, int pad, void *dX, twn_stream_t stream)
 {
     TWN_REQUIRE(dY && argmax && dX && B > 0 && H > 0 && W > 0 && C > 0 && k > 0 && k <= 15 && stride > 0 &&
                     pad >= 0 && pad < k, TWN_ERR_INVALID_ARG);
@@ -587,9 +618,11 @@ extern "C" int twn_maxpool2d_bwd(const void *dY, const uint8_t *argmax, int64_t 
     const long long Ho = pool_extent(H, k, stride, pad), Wo = pool_extent(W, k, stride, pad);
     TWN_REQUIRE(Ho > 0 && Wo > 0, TWN_ERR_INVALID_ARG);
     const __nv_bfloat16 *dy = static_cast<const __nv_bfloat16 *>(dY);
+    const __nv_bfloat16 *pooled = static_cast<const __nv_bfloat16 *>(pooled_v);
     __nv_bfloat16 *dx = static_cast<__nv_bfloat16 *>(dX);
     const bool small = B * H * W * C < 0x7fffffffLL;
-    const bool vec = C % 8 == 0 && twn_aligned(dY, 16) && twn_aligned(dX, 16) && twn_aligned(argmax, 8);
+    const bool vec = C % 8 == 0 && twn_aligned(dY, 16) && twn_aligned(dX, 16) && twn_aligned(argmax, 8) &&
+                     twn_aligned(pooled_v, 16) && twn_aligned(scale, 16);
     cudaStream_t s = twn_cu(stream);
     if (vec && small) {
         const long long rows = B * H;
@@ -597,16 +630,33 @@ extern "C" int twn_maxpool2d_bwd(const void *dY, const uint8_t *argmax, int64_t 
         int lg = -1;
         for (int i = 0; i < 8; ++i) if ((1 << i) == stride) lg = i;
         maxpool_bwd_rows_kernel<<<grid, kT, 0, s>>>(dy, argmax, (int)B, (int)H, (int)W, (int)C, k, stride, lg, pad,
-                                                    (int)Ho, (int)Wo, dx);
+                                                    (int)Ho, (int)Wo, dx, pooled, scale);
     }
     else if (vec)
         maxpool_bwd_kernel<long long, 8><<<blocks_for(B * H * W * C / 8, dev.sm_count), kT, 0, s>>>(
-            dy, argmax, B, H, W, C, k, stride, pad, Ho, Wo, dx);
+            dy, argmax, B, H, W, C, k, stride, pad, Ho, Wo, dx, pooled, scale);
     else
         maxpool_bwd_kernel<long long, 1><<<blocks_for(B * H * W * C, dev.sm_count), kT, 0, s>>>(
-            dy, argmax, B, H, W, C, k, stride, pad, Ho, Wo, dx);
+            dy, argmax, B, H, W, C, k, stride, pad, Ho, Wo, dx, pooled, scale);
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
+}
+
+}  // namespace
+
+extern "C" int twn_maxpool2d_bwd(const void *dY, const uint8_t *argmax, int64_t B, int64_t H, int64_t W, int64_t C,
+                                 int k, int stride, int pad, void *dX, twn_stream_t stream)
+{
+    return maxpool_bwd_launch(dY, argmax, nullptr, nullptr, B, H, W, C, k, stride, pad, dX, stream);
+}
+
+extern "C" int twn_maxpool2d_bwd_act(const void *dY, const uint8_t *argmax, const void *pooled, const float *scale,
+                                     int64_t B, int64_t H, int64_t W, int64_t C, int k, int stride, int pad,
+                                     void *dZ, twn_stream_t stream)
+{
+    TWN_REQUIRE(pooled != nullptr, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(twn_aligned(pooled, 2) && twn_aligned(scale, 4), TWN_ERR_MISALIGNED);
+    return maxpool_bwd_launch(dY, argmax, pooled, scale, B, H, W, C, k, stride, pad, dZ, stream);
 }
 
 extern "C" int twn_avgpool_fwd(const void *X, int64_t B, int64_t HW, int64_t C, void *Y, twn_stream_t stream)

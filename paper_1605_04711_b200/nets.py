@@ -292,7 +292,7 @@ class TernaryNet:
                 if op[1].residual:
                     consumers.setdefault(op[1].residual, []).append(None)
             elif op[0] in ("maxpool", "avgpool", "flatten"):
-                consumers.setdefault(op[2], []).append(None)
+                consumers.setdefault(op[2], []).append(op[1])
         FUSED = object()
 
         def fused_producer(L):
@@ -354,6 +354,15 @@ class TernaryNet:
                 _, name, src, k, s, p = op
                 Bx, H, W, C = self.act[src].shape
                 dY = acc[name]
+
+                P = self.layers.get(src)
+                if P is not None and P.relu and not P.residual and consumers.get(src) == [name]:
+                    # the pool is the only reader of a ReLU layer: its backward pass writes that
+                    # layer's dZ (gate by the pooled value, folded batch-norm scale) in one sweep
+                    twn.maxpool2d_bwd_act(dY, self.aux[name], self.act[name], P.extra["scale"], Bx, H, W, C, k, s, p,
+                                          P.extra["dz"])
+                    acc[src] = FUSED
+                    continue
 
                 def mp(res, out, dY=dY, name=name, Bx=Bx, H=H, W=W, C=C, k=k, s=s, p=p):
                     assert res is None

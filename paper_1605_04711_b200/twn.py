@@ -325,6 +325,12 @@ def maxpool2d_bwd(dY, argmax, B, H, W, Cc, k, stride, pad, dX, stream=None) -> N
                                    _stream(stream)), "twn_maxpool2d_bwd")
 
 
+def maxpool2d_bwd_act(dY, argmax, pooled, scale, B, H, W, Cc, k, stride, pad, dZ, stream=None) -> None:
+    _check(lib().twn_maxpool2d_bwd_act(_ptr(dY), _ptr(argmax), _ptr(pooled), _ptr(scale), C.c_int64(B),
+                                       C.c_int64(H), C.c_int64(W), C.c_int64(Cc), C.c_int(k), C.c_int(stride),
+                                       C.c_int(pad), _ptr(dZ), _stream(stream)), "twn_maxpool2d_bwd_act")
+
+
 def avgpool_fwd(X, B, HW, Cc, Y, stream=None) -> None:
     _check(lib().twn_avgpool_fwd(_ptr(X), C.c_int64(B), C.c_int64(HW), C.c_int64(Cc), _ptr(Y),
                                  _stream(stream)), "twn_avgpool_fwd")

@@ -184,6 +184,16 @@ def test_maxpool_forward_and_backward(k, s, p, H, W, C):
     got = dg.bf16_bits_to_f64(host_bf16_bits(dX))
     # up to four window gradients are added in fp32 and rounded once to bf16
     assert np.all(np.abs(got - dxr) <= 2.0 ** -8 * np.abs(dxr) + 1e-30)
+    # fused with the backward through y = relu(z * scale + shift) of the layer below the pool:
+    # windows whose pooled value is not positive pass nothing, the sum is scaled per channel
+    scale = dg.draw(3, f"mps{H}{C}", C, "normal", 1.0, 0.3)
+    dZ = torch.full((B, H, W, C), float("nan"), dtype=torch.bfloat16, device="cuda")
+    sd = dev_f32(scale)
+    twn.maxpool2d_bwd_act(dev_bf16(dyb), arg, Y, sd, B, H, W, C, k, s, p, dZ)
+    gated = np.where(yr > 0, dg.bf16_bits_to_f64(dyb), 0.0)
+    dzr = oracle.maxpool_bwd(gated, argr, H, W) * scale.astype(np.float64)
+    gotz = dg.bf16_bits_to_f64(host_bf16_bits(dZ))
+    assert np.all(np.abs(gotz - dzr) <= 2.0 ** -8 * np.abs(dzr) + 1e-30)
 
 
 def test_avgpool_and_activation_backward():
