@@ -332,11 +332,16 @@ class NetWorkload:
     def __init__(self, kind):
         self.kind = kind
         self.name = {"resnet18_train": "resnet18_train_step_b64_224", "vgg7_fwd": "vgg7_forward_b128",
-                     "lenet5_fwd": "lenet5_forward_b100"}[kind]
+                     "lenet5_fwd": "lenet5_forward_b100", "resnet18b_train": "resnet18b_train_step_b64_224"}[kind]
+
+    def train_kind(self):
+        return self.kind in ("resnet18_train", "resnet18b_train")
 
     def make(self, nets):
         if self.kind == "resnet18_train":
             return nets.resnet18(64, train=True)
+        if self.kind == "resnet18b_train":
+            return nets.resnet18b(64, train=True)
         if self.kind == "vgg7_fwd":
             return nets.vgg7(128)
         return nets.lenet5(100)
@@ -346,7 +351,7 @@ class NetWorkload:
              "l2": "activations of a step (> 1 GB for ResNet-18) exceed L2 (126 MB)",
              "launch": "one CUDA graph replay per step",
              "e2e": "pipelined: the pinned-host copy of batch i+1 runs on a copy stream while step i computes"}
-        if self.kind == "resnet18_train":
+        if self.train_kind():
             c["step"] = ("ternarize+pack 21 tensors, transpose codes, forward, backward for data, "
                          "straight-through dW; synthetic dY N(0,1e-2) at the logits")
         else:
@@ -356,13 +361,14 @@ class NetWorkload:
 
     def host_inputs(self):
         from paper_1605_04711_b200 import datagen as dg
-        shape = {"resnet18_train": (64, 224, 224, 3), "vgg7_fwd": (128, 32, 32, 3), "lenet5_fwd": (100, 28, 28, 1)}[self.kind]
+        shape = {"resnet18_train": (64, 224, 224, 3), "resnet18b_train": (64, 224, 224, 3), "vgg7_fwd": (128, 32, 32, 3),
+                 "lenet5_fwd": (100, 28, 28, 1)}[self.kind]
         n = 1
         for s in shape:
             n *= s
         dist = "uniform01" if self.kind == "lenet5_fwd" else "normal"
         x = dg.draw_bf16(0, f"{self.name}.input", n, dist)
-        dy = dg.draw_bf16(0, f"{self.name}.dlogits", 64 * 1000, "normal", 0.0, 0.1) if self.kind == "resnet18_train" else None
+        dy = dg.draw_bf16(0, f"{self.name}.dlogits", 64 * 1000, "normal", 0.0, 0.1) if self.train_kind() else None
         return x, dy
 
     def setup(self, torch, twn, host):
@@ -371,7 +377,7 @@ class NetWorkload:
         self.torch, self.twn = torch, twn
         x, dy = host
         self.net = net = self.make(nets)
-        self.train = self.kind == "resnet18_train"
+        self.train = self.train_kind()
         self.host_x = torch.from_numpy(x.view(np.int16)).pin_memory()
         net.act["input"].view(torch.int16).view(-1).copy_(self.host_x)
         last = net.ops[-1][1]
@@ -521,12 +527,14 @@ class NetWorkload:
     def _macs_per_image(self):
         if hasattr(self, "net"):
             return self.net.total_macs() / self.net.B
-        return {"resnet18_train": 340.7e9 / 64 * 1.0, "vgg7_fwd": 615.9e6, "lenet5_fwd": 4.27e6}[self.kind]
+        return {"resnet18_train": 340.7e9 / 64, "resnet18b_train": 755.3e9 / 64, "vgg7_fwd": 615.9e6,
+                "lenet5_fwd": 4.27e6}[self.kind]
 
 
 WORKLOADS = {"ternarize": lambda: TernarizeWorkload(), "ternarize_rows": lambda: TernarizeRowsWorkload(), "resnet18_train": lambda: NetWorkload("resnet18_train"),
              "gemm_16384": lambda: GemmWorkload(16384), "gemm_4096": lambda: GemmWorkload(4096),
-             "vgg7_fwd": lambda: NetWorkload("vgg7_fwd"), "lenet5_fwd": lambda: NetWorkload("lenet5_fwd")}
+             "vgg7_fwd": lambda: NetWorkload("vgg7_fwd"), "lenet5_fwd": lambda: NetWorkload("lenet5_fwd"),
+             "resnet18b_train": lambda: NetWorkload("resnet18b_train")}
 DEFAULT_WORKLOAD = "resnet18_train"
 
 
@@ -544,7 +552,7 @@ def run_reference(args):
         if i >= args.warmup:
             vals.append(v)
     value = sum(vals) / len(vals)
-    upstep = wl.units_per_step() if isinstance(wl, (TernarizeWorkload, GemmWorkload)) else {"resnet18_train": 64, "vgg7_fwd": 128, "lenet5_fwd": 100}[args.workload]
+    upstep = wl.units_per_step() if isinstance(wl, (TernarizeWorkload, GemmWorkload)) else {"resnet18_train": 64, "resnet18b_train": 64, "vgg7_fwd": 128, "lenet5_fwd": 100}[args.workload]
     line = {"impl": "reference", "metric": wl.metric, "value": value, "unit": wl.unit,
             "n_gpus": args.gpus, "steps": steps, "warmup": args.warmup,
             "ms_per_step": upstep / value * 1e3, "higher_is_better": True,

@@ -432,13 +432,16 @@ def vgg7(batch=128, train=False, seed=0):
     return TernaryNet("vgg7", batch, (32, 32, 3), ops, seed, train=train)
 
 
-def resnet18(batch=64, train=True, seed=0, image=224, classes=1000):
-    ops = [("layer", Layer("stem", 3, 64, 7, 2, 3, image, image, affine=True, src="input"))]
+def resnet18(batch=64, train=True, seed=0, image=224, classes=1000, widths=(64, 128, 256, 512), name="resnet18"):
+    """BasicBlock layout [2, 2, 2, 2] with a 7x7/2 first layer.  `widths` are the channels of the four
+    stages; (96, 192, 384, 768) is the 1.5x wider "ResNet-18B" of the paper's ImageNet experiments."""
+    w0 = widths[0]
+    ops = [("layer", Layer("stem", 3, w0, 7, 2, 3, image, image, affine=True, src="input"))]
     H = (image + 6 - 7) // 2 + 1
     ops.append(("maxpool", "pool0", "stem", 3, 2, 1))
     H = (H + 2 - 3) // 2 + 1
-    src, cin = "pool0", 64
-    for li, c in enumerate([64, 128, 256, 512], 1):
+    src, cin = "pool0", w0
+    for li, c in enumerate(widths, 1):
         for b in range(2):
             stride = 2 if (li > 1 and b == 0) else 1
             p = f"l{li}.b{b}"
@@ -452,5 +455,9 @@ def resnet18(batch=64, train=True, seed=0, image=224, classes=1000):
                                        src=p + ".conv1")))
             src, cin, H = p + ".conv2", c, Ho
     ops.append(("avgpool", "gap", src))
-    ops.append(("layer", Layer("fc", 512, classes, relu=False, src="gap", out_f32=True)))
-    return TernaryNet("resnet18", batch, (image, image, 3), ops, seed, train=train)
+    ops.append(("layer", Layer("fc", widths[-1], classes, relu=False, src="gap", out_f32=True)))
+    return TernaryNet(name, batch, (image, image, 3), ops, seed, train=train)
+
+
+def resnet18b(batch=64, train=True, seed=0, image=224, classes=1000):
+    return resnet18(batch, train, seed, image, classes, widths=(96, 192, 384, 768), name="resnet18b")

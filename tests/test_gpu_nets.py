@@ -190,6 +190,17 @@ def test_resnet18_small_train_step(monkeypatch):
     check_backward(net, npix=300, nent=300)
 
 
+def test_resnet18b_wider_stages_small_train_step(monkeypatch):
+    """The 1.5x wider variant of the paper's ImageNet experiments: 96/192/384/768 channels, i.e.
+    reductions that are not multiples of 64 per tap (the last 64-channel block of a tap is half
+    empty and the code columns of a tap do not start on 16-byte boundaries)."""
+    net = nets.resnet18b(batch=2, train=True, image=64, classes=24)
+    run_train_step(net, monkeypatch)
+    check_forward(net, npix=300)
+    check_pools(net)
+    check_backward(net, npix=200, nent=200)
+
+
 def test_resnet18_train_step_batch64(monkeypatch):
     net = nets.resnet18(batch=64, train=True)
     run_train_step(net, monkeypatch)
