@@ -148,6 +148,21 @@ def ternarize_rows(W, delta_factor: float = 0.7):
     return out, codes
 
 
+def sgd_update(W, dW, V, lr: float, momentum: float, weight_decay: float):
+    """Last step of Algorithm 1 (UpdateParameters; the paper uses SGD with momentum and an L2 weight
+    decay, Sec. 3) on the fp32 master weights:
+        g = dW + weight_decay * W;   V' = momentum * V + g;   W' = W - lr * V'
+    The master weights are fp32, so every operation is an fp32 operation rounded to nearest, in
+    exactly this order and without fused multiply-adds (numpy float32 arithmetic).  Returns (W', V')."""
+    w, g, v = _f32(W), _f32(dW), _f32(V)
+    lr32, mu32, wd32 = np.float32(lr), np.float32(momentum), np.float32(weight_decay)
+    grad = g + wd32 * w
+    v_new = mu32 * v + grad
+    w_new = w - lr32 * v_new
+    assert grad.dtype == np.float32 and v_new.dtype == np.float32 and w_new.dtype == np.float32
+    return w_new, v_new
+
+
 def alpha_alg1(W, codes) -> float:
     w, c = _f32(W), _i8(codes)
     return float(lib().ref_alpha_alg1(_p(w), _p(c), C.c_int64(w.size)))
