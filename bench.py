@@ -237,6 +237,57 @@ class TernarizeRowsWorkload(TernarizeWorkload):
         return rows * self.cols * self.bytes_per_unit / dt / 1e9, f"oracle on {rows} of {self.rows} filters ({dt:.1f} s)", 1
 
 
+class SgdTernarizeWorkload(TernarizeWorkload):
+    """End of one iteration and start of the next (Algorithm 1): SGD-with-momentum update of 1e8 fp32
+    master weights fused with the threshold reduction of the updated weights, then the coding sweep
+    (codes, 2-bit packing, scale).  Algorithmic bytes per weight: update 12 read (W, dW, V) + 8 written
+    (W, V), coding 4 read + 0.25 written = 24.25; the unfused sequence reads the weights once more."""
+    name = "sgd_update_ternarize_n1e8_normal"
+    metric = "sgd update + ternarize+pack GB/s"
+    bytes_per_unit = 24.25
+
+    def config(self):
+        c = super().config()
+        c.update({"workload": self.name, "lr": 0.01, "momentum": 0.9, "weight_decay": 1e-4,
+                  "l2": "W, dW, V (1.2 GB) larger than L2 (126 MB)"})
+        return c
+
+    def setup(self, torch, twn, host_W):
+        from paper_1605_04711_b200 import datagen as dg
+        super().setup(torch, twn, host_W)
+        self.dW = torch.from_numpy(dg.draw(self.seed, "sweep-grad", self.n, "normal", 0.0, 0.01)).cuda()
+        self.V = torch.zeros(self.n, dtype=torch.float32, device="cuda")
+
+    def step(self):
+        self.twn.sgd_update(self.W, self.dW, self.V, 0.01, 0.9, 1e-4, 0.7, self.stats, self.ws)
+        self.twn.ternarize_codes(self.W, 1, self.n, self.stats, self.packed, self.ld, None, self.ws)
+
+    def step_e2e(self):
+        self.dW.copy_(self.host_W, non_blocking=True)       # a gradient-sized tensor arrives from the host
+        self.step()
+        self.host_packed.copy_(self.packed, non_blocking=True)
+        self.host_stats.copy_(self.stats, non_blocking=True)
+
+    def roofline(self, ms_per_step, peaks):
+        r = super().roofline(ms_per_step, peaks)
+        r["kernel"] = "sgd_update_kernel + code_pack_kernel (twn_sgd_update, twn_ternarize_codes)"
+        r["traffic"] = None
+        return r
+
+    def cpu_sample(self, host_W):
+        import oracle
+        import numpy as np
+        n = self.n
+        W = host_W[:n]
+        g = np.full(n, 0.01, np.float32)
+        t0 = time.perf_counter()
+        w1, v1 = oracle.sgd_update(W, g, np.zeros(n, np.float32), 0.01, 0.9, 1e-4)
+        st, codes = oracle.ternarize(w1, 0.7)
+        oracle.pack(codes, oracle.ld_for(n))
+        dt = time.perf_counter() - t0
+        return n * self.bytes_per_unit / dt / 1e9, f"oracle on all {n} weights ({dt:.1f} s)", 1
+
+
 class GemmWorkload:
     """One ternary-weight GEMM (Algorithm 1, forward of a fully connected layer): Y = alpha * X T^T with
     bf16 X [M, K], 2-bit T [N, K] ternarized from N(0,1) weights, bf16 Y.  2MNK flops per step."""
@@ -531,7 +582,7 @@ class NetWorkload:
                 "lenet5_fwd": 4.27e6}[self.kind]
 
 
-WORKLOADS = {"ternarize": lambda: TernarizeWorkload(), "ternarize_rows": lambda: TernarizeRowsWorkload(), "resnet18_train": lambda: NetWorkload("resnet18_train"),
+WORKLOADS = {"ternarize": lambda: TernarizeWorkload(), "sgd_ternarize": lambda: SgdTernarizeWorkload(), "ternarize_rows": lambda: TernarizeRowsWorkload(), "resnet18_train": lambda: NetWorkload("resnet18_train"),
              "gemm_16384": lambda: GemmWorkload(16384), "gemm_4096": lambda: GemmWorkload(4096),
              "vgg7_fwd": lambda: NetWorkload("vgg7_fwd"), "lenet5_fwd": lambda: NetWorkload("lenet5_fwd"),
              "resnet18b_train": lambda: NetWorkload("resnet18b_train")}

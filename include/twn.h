@@ -194,6 +194,34 @@ int twn_ternarize_static(const float *W, int64_t rows, int64_t cols, double delt
                          int8_t *codes_i8, twn_stream_t stream);
 
 /*
+ * Parameter update of Algorithm 1 (UpdateParameters; the paper trains with SGD with momentum and
+ * an L2 weight decay, Sec. 3) on the fp32 master weights, in place:
+ *     g = dW + weight_decay * W;   V = momentum * V + g;   W = W - lr * V
+ * Every operation is a separately rounded fp32 operation in exactly this order (no fused
+ * multiply-add): the result is defined to the bit.  dW is the straight-through gradient of
+ * twn_conv2d_bwd_weight (or any fp32 gradient of the same shape), V the momentum buffer.
+ * The next iteration begins by ternarizing the updated weights; its threshold needs
+ * sum |W|, which this call accumulates while the updated weights are still in registers:
+ *   stats_next (optional) receives sum_abs, delta = delta_factor * sum_abs / n and status
+ *              (TWN_ERR_NONFINITE if an updated weight is NaN/Inf) of the updated tensor,
+ * so that twn_ternarize_codes can write the codes and the scale without the first sweep.
+ * W, dW, V: fp32 [n], 16-byte aligned.  workspace as for twn_ternarize.  Deterministic.
+ */
+int twn_sgd_update(float *W, const float *dW, float *V, int64_t n, float lr, float momentum,
+                   float weight_decay, double delta_factor, twn_stats_t *stats_next,
+                   void *workspace, size_t workspace_bytes, twn_stream_t stream);
+
+/*
+ * Second sweep of twn_ternarize alone: codes by Eq. 3 against the threshold already in
+ * stats->delta (written by twn_sgd_update or by an earlier twn_ternarize of the same weights),
+ * 2-bit packing, alpha by Eq. 5 and the counts.  Arguments as for twn_ternarize; stats->delta,
+ * sum_abs and status are read and kept, the other fields are written.
+ */
+int twn_ternarize_codes(const float *W, int64_t rows, int64_t cols, twn_stats_t *stats,
+                        uint32_t *packed, int64_t ld_codes, int8_t *codes_i8,
+                        void *workspace, size_t workspace_bytes, twn_stream_t stream);
+
+/*
  * Per-filter threshold ternarization fused with 2-bit packing: Algorithm 1 as printed,
  * whose first loop runs over the filters of a layer.  Row r of W is one filter and gets
  *   delta_r = delta_factor * (1/cols) * sum_i |W_r,i|          (Sec. 2.3, n = cols)

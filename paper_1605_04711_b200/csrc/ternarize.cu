@@ -142,6 +142,73 @@ sum_abs_kernel(const float *__restrict__ W, long long n, double factor, void *ws
     sum_abs_body(W, n, factor, carve(ws_raw), stats, blockIdx.x, gridDim.x);
 }
 
+// ---- parameter update fused with sweep 1 of the next iteration -------------
+// Last step of Algorithm 1 (UpdateParameters: SGD with momentum and L2 weight decay on the fp32
+// master weights, Sec. 3):
+//     g = dW + wd * W;   V' = mu * V + g;   W' = W - lr * V'
+// every operation a separately rounded fp32 operation in this order (no fused multiply-add), so
+// the result is defined to the bit.  The next iteration starts by ternarizing W', whose
+// threshold needs sum |W'|: it is accumulated here while W' is still in registers, which saves
+// the first sweep of that ternarization (one read of the weights).
+__device__ __forceinline__ float sgd_one(float w, float g, float &v, float lr, float mu, float wd)
+{
+    const float grad = __fadd_rn(g, __fmul_rn(wd, w));
+    v = __fadd_rn(__fmul_rn(mu, v), grad);
+    return __fsub_rn(w, __fmul_rn(lr, v));
+}
+
+__global__ void __launch_bounds__(kThreads)
+sgd_update_kernel(float *__restrict__ W, const float *__restrict__ dW, float *__restrict__ V, long long n,
+                  float lr, float mu, float wd, double factor, void *ws_raw, twn_stats_t *__restrict__ stats)
+{
+    __shared__ double red[kWarps];
+    const Workspace ws = carve(ws_raw);
+    const long long n4 = n >> 2;
+    float4 *W4 = reinterpret_cast<float4 *>(W);
+    float4 *V4 = reinterpret_cast<float4 *>(V);
+    const float4 *G4 = reinterpret_cast<const float4 *>(dW);
+    const long long stride = (long long)gridDim.x * kThreads;
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+#pragma unroll 2
+    for (long long i = (long long)blockIdx.x * kThreads + threadIdx.x; i < n4; i += stride) {
+        float4 w = W4[i], v = V4[i];
+        const float4 g = __ldg(G4 + i);
+        w.x = sgd_one(w.x, g.x, v.x, lr, mu, wd);
+        w.y = sgd_one(w.y, g.y, v.y, lr, mu, wd);
+        w.z = sgd_one(w.z, g.z, v.z, lr, mu, wd);
+        w.w = sgd_one(w.w, g.w, v.w, lr, mu, wd);
+        W4[i] = w;
+        V4[i] = v;
+        a0 += (double)fabsf(w.x); a1 += (double)fabsf(w.y); a2 += (double)fabsf(w.z); a3 += (double)fabsf(w.w);
+    }
+    if (blockIdx.x == 0) {
+        const long long t = (n4 << 2) + threadIdx.x;
+        if (t < n) {
+            float v = V[t];
+            const float w = sgd_one(W[t], __ldg(dW + t), v, lr, mu, wd);
+            W[t] = w;
+            V[t] = v;
+            a0 += (double)fabsf(w);
+        }
+    }
+    const double bsum = block_sum((a0 + a1) + (a2 + a3), red);
+    if (threadIdx.x == 0) ws.part_sum[blockIdx.x] = bsum;
+    if (last_block(ws.ticket1, gridDim.x)) {
+        double s = 0.0;
+        for (int b = threadIdx.x; b < (int)gridDim.x; b += kThreads) s += __ldcg(ws.part_sum + b);
+        s = block_sum(s, red);
+        if (threadIdx.x == 0) {
+            if (stats) {
+                stats->sum_abs = s;
+                stats->delta = n > 0 ? factor * (s / (double)n) : 0.0;
+                stats->status = isfinite(s) ? TWN_OK : TWN_ERR_NONFINITE;
+                stats->reserved = 0;
+            }
+            *ws.ticket1 = 0u;
+        }
+    }
+}
+
 // ---- sweep 2 -------------------------------------------------------------
 // 2-bit field of one weight: bit 0 = kept, bit 1 = negative  (00 / 01 / 11).
 __device__ __forceinline__ uint32_t code2(float w, float thr, double &kept_sum)
@@ -617,6 +684,57 @@ extern "C" int twn_ternarize(const float *W, int64_t rows, int64_t cols, double 
     const int g2 = grid_for(work, dev.sm_count);
     code_pack_kernel<<<g2, kThreads, 0, s>>>(W, rows, cols, ld_codes, fast_units, packed, codes_i8,
                                              workspace, stats);
+    TWN_CUDA_OK(cudaGetLastError());
+    return TWN_OK;
+}
+
+extern "C" int twn_sgd_update(float *W, const float *dW, float *V, int64_t n, float lr, float momentum,
+                              float weight_decay, double delta_factor, twn_stats_t *stats_next, void *workspace,
+                              size_t workspace_bytes, twn_stream_t stream)
+{
+    TWN_REQUIRE(n >= 0, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(workspace != nullptr, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(n == 0 || (W != nullptr && dW != nullptr && V != nullptr), TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(lr == lr && momentum == momentum && weight_decay == weight_decay, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(delta_factor >= 0.0 && delta_factor == delta_factor, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(workspace_bytes >= kWorkspaceBytes, TWN_ERR_WORKSPACE);
+    TWN_REQUIRE(twn_aligned(W, 16) && twn_aligned(dW, 16) && twn_aligned(V, 16) && twn_aligned(stats_next, 8) &&
+                    twn_aligned(workspace, 256), TWN_ERR_MISALIGNED);
+    twn_device_info dev;
+    const int rc = twn_current_device(&dev);
+    if (rc != TWN_OK) return rc;
+    cudaStream_t s = twn_cu(stream);
+    TWN_CUDA_OK(cudaMemsetAsync(workspace, 0, 128, s));
+    const int g = grid_for((n / 4 + 1) / 2, dev.sm_count);
+    sgd_update_kernel<<<g, kThreads, 0, s>>>(W, dW, V, n, lr, momentum, weight_decay, delta_factor, workspace, stats_next);
+    TWN_CUDA_OK(cudaGetLastError());
+    return TWN_OK;
+}
+
+extern "C" int twn_ternarize_codes(const float *W, int64_t rows, int64_t cols, twn_stats_t *stats, uint32_t *packed,
+                                   int64_t ld_codes, int8_t *codes_i8, void *workspace, size_t workspace_bytes,
+                                   twn_stream_t stream)
+{
+    TWN_REQUIRE(rows >= 0 && cols >= 0, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(stats != nullptr && workspace != nullptr, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(ld_codes >= cols && ld_codes % 64 == 0, TWN_ERR_INVALID_ARG);
+    const long long n = (long long)rows * cols;
+    TWN_REQUIRE(n == 0 || (W != nullptr && packed != nullptr), TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(workspace_bytes >= kWorkspaceBytes, TWN_ERR_WORKSPACE);
+    TWN_REQUIRE(twn_aligned(W, 16) && twn_aligned(packed, 16) && twn_aligned(stats, 8) &&
+                    twn_aligned(workspace, 256) && twn_aligned(codes_i8, 16), TWN_ERR_MISALIGNED);
+    twn_device_info dev;
+    const int rc = twn_current_device(&dev);
+    if (rc != TWN_OK) return rc;
+    cudaStream_t s = twn_cu(stream);
+    TWN_CUDA_OK(cudaMemsetAsync(workspace, 0, 128, s));
+    const bool flat = (rows <= 1) || (ld_codes == cols);
+    const long long fast_units = flat ? n / 512 : 0;
+    const long long rest_words = (long long)rows * (ld_codes / 16) - fast_units * 32;
+    long long work = fast_units * 32 / 4;
+    if (rest_words > work) work = rest_words;
+    code_pack_kernel<<<grid_for(work, dev.sm_count), kThreads, 0, s>>>(W, rows, cols, ld_codes, fast_units, packed,
+                                                                       codes_i8, workspace, stats);
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }

@@ -134,6 +134,26 @@ def ternarize(W: torch.Tensor, delta_factor: float, stats: torch.Tensor, packed:
                                _stream(stream)), "twn_ternarize")
 
 
+def sgd_update(W: torch.Tensor, dW: torch.Tensor, V: torch.Tensor, lr: float, momentum: float,
+               weight_decay: float, delta_factor: float, stats_next, workspace: torch.Tensor, stream=None) -> None:
+    """twn_sgd_update: in-place SGD step on the fp32 master weights; stats_next (optional) receives
+    the threshold of the updated weights."""
+    _check(lib().twn_sgd_update(_ptr(W), _ptr(dW), _ptr(V), C.c_int64(W.numel()), C.c_float(lr),
+                                C.c_float(momentum), C.c_float(weight_decay), C.c_double(delta_factor),
+                                _ptr(stats_next), _ptr(workspace),
+                                C.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream)),
+           "twn_sgd_update")
+
+
+def ternarize_codes(W: torch.Tensor, rows: int, cols: int, stats: torch.Tensor, packed: torch.Tensor,
+                    ld_codes: int, codes_i8, workspace: torch.Tensor, stream=None) -> None:
+    """twn_ternarize_codes: the coding sweep alone, against the threshold already in `stats`."""
+    _check(lib().twn_ternarize_codes(_ptr(W), C.c_int64(rows), C.c_int64(cols), _ptr(stats), _ptr(packed),
+                                     C.c_int64(ld_codes), _ptr(codes_i8), _ptr(workspace),
+                                     C.c_size_t(workspace.numel() * workspace.element_size()),
+                                     _stream(stream)), "twn_ternarize_codes")
+
+
 class TernarizeItem(C.Structure):
     _fields_ = [("W", C.c_void_p), ("rows", C.c_int64), ("cols", C.c_int64), ("stats", C.c_void_p),
                 ("packed", C.c_void_p), ("ld_codes", C.c_int64), ("codes_i8", C.c_void_p)]
