@@ -446,7 +446,10 @@ class NetWorkload:
         torch.cuda.synchronize()
         net.check_status()
         self.graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(self.graph):
+        # The step is captured on a high-priority stream: the forward / backward-for-data chain is the
+        # critical path, while the weight gradients and the code re-layouts (streams of default
+        # priority forked from it) fill the SMs it leaves free.
+        with torch.cuda.graph(self.graph, stream=torch.cuda.Stream(priority=-1)):
             self._eager()
         # per-kernel device times from one eager pass; a spin keeps the GPU behind the host so
         # that the events bracket kernels only
