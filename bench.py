@@ -706,7 +706,7 @@ def run_ours(args):
                         "ms_per_step": ms_e2e, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
                 "gpu_launches": wl.launches_per_step() * steps,
                 "roofline": wl.roofline(ms, peaks)}
-        if args.workload == DEFAULT_WORKLOAD and not args.no_ternarize_leg:
+        if args.workload == DEFAULT_WORKLOAD and world == 1 and not args.no_ternarize_leg:
             # the second half of the headline metric, measured in the same run: ternarize + pack of
             # one 1e8-weight tensor (larger than L2), in GB/s of algorithmic traffic
             line["ternarize_pack"] = ternarize_leg(torch, twn, peaks)
