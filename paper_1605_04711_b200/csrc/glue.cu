@@ -268,6 +268,28 @@ maxpool_fwd_rows_kernel(const __nv_bfloat16 *__restrict__ X, int B, int H, int W
             int arg[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) { best[e] = -INFINITY; arg[e] = 0; }
+            if (k <= 3) {
+                // all (up to nine) window elements are requested before the first comparison, so
+                // their latencies overlap; an element outside the image reads as -inf and never wins
+                uint4 v[9];
+#pragma unroll
+                for (int q = 0; q < 9; ++q) {
+                    const int r = q / 3, sx = q - 3 * r;
+                    const int h = h_lo + r, w = w_lo + sx;
+                    const bool ok = r < k && sx < k && h >= 0 && h < H && w >= 0 && w < W;
+                    v[q] = ok ? __ldg(reinterpret_cast<const uint4 *>(X + ((size_t)(b * H + h) * W + w) * C + cv * 8))
+                              : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);   // bf16 -inf
+                }
+#pragma unroll
+                for (int q = 0; q < 9; ++q) {
+                    const int r = q / 3, sx = q - 3 * r;
+                    float x[8];
+                    unpack8(v[q], x);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        if (x[e] > best[e]) { best[e] = x[e]; arg[e] = r * k + sx; }
+                }
+            } else
             for (int r = 0; r < k; ++r) {
                 const int h = h_lo + r;
                 if (h < 0 || h >= H) continue;
