@@ -32,22 +32,31 @@ __device__ __forceinline__ unsigned long long warp_sum(unsigned long long v)
     return v;
 }
 
-// Block-wide sum with a fixed order, returned to every thread.
-template <typename T>
-__device__ __forceinline__ T block_sum_all(T v, T *smem /* kWarps + 1 entries */)
+// Block-wide sums with a fixed order: a shuffle tree per warp, one partial per warp in shared
+// memory, and after a single barrier every thread adds the kWarps partials in index order.
+__device__ __forceinline__ double block_sum_all(double v, double *part /* kWarps entries, not in use by a slower warp */)
 {
     v = warp_sum(v);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    __syncthreads();                       // the previous use of `smem` is over
-    if (lane == 0) smem[warp] = v;
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = v;
     __syncthreads();
-    if (warp == 0) {
-        T r = lane < kWarps ? smem[lane] : T(0);
-        r = warp_sum(r);
-        if (lane == 0) smem[kWarps] = r;
-    }
+    double r = 0.0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) r += part[w];
+    return r;
+}
+// The same for a floating-point and an integer quantity at once (one barrier for both).
+__device__ __forceinline__ void block_sum_all2(double &a, unsigned long long &b, double *part_a, unsigned long long *part_b)
+{
+    a = warp_sum(a);
+    b = warp_sum(b);
+    if ((threadIdx.x & 31) == 0) { part_a[threadIdx.x >> 5] = a; part_b[threadIdx.x >> 5] = b; }
     __syncthreads();
-    return smem[kWarps];
+    double ra = 0.0;
+    unsigned long long rb = 0ull;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) { ra += part_a[w]; rb += part_b[w]; }
+    a = ra;
+    b = rb;
 }
 
 // Bit position of element e (0..15) inside its packed word (the layout of twn_ternarize): even
@@ -76,8 +85,8 @@ ternarize_rows_kernel(const float *__restrict__ W, long long rows, long long col
                       int8_t *__restrict__ codes_i8)
 {
     extern __shared__ float4 rowbuf[];
-    __shared__ double red_d[kWarps + 1];
-    __shared__ unsigned long long red_u[kWarps + 1];
+    __shared__ double red_s[kWarps], red_k[kWarps];      // partials of the two sweeps: separate, so that a warp
+    __shared__ unsigned long long red_u[kWarps];         // ahead of the others never overwrites what they still read
     const int tid = threadIdx.x, lane = tid & 31;
     const long long words = (cols + 15) >> 4;         // words that hold codes; the rest of a row is padding
     const int n4 = (int)(cols >> 2);
@@ -91,7 +100,6 @@ ternarize_rows_kernel(const float *__restrict__ W, long long rows, long long col
         double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
         if (MODE >= 1) {
             const float4 *W4 = reinterpret_cast<const float4 *>(Wr);
-            if (MODE == 2) __syncthreads();        // the previous filter's readers are done with the buffer
 #pragma unroll 8
             for (int i = tid; i < n4; i += kThreads) {
                 const float4 x = __ldg(W4 + i);
@@ -101,7 +109,7 @@ ternarize_rows_kernel(const float *__restrict__ W, long long rows, long long col
         } else {
             for (long long i = tid; i < cols; i += kThreads) a0 += (double)fabsf(__ldg(Wr + i));
         }
-        const double S = block_sum_all((a0 + a1) + (a2 + a3), red_d);
+        const double S = block_sum_all((a0 + a1) + (a2 + a3), red_s);
         const double delta = cols > 0 ? factor * (S / (double)cols) : 0.0;
         // a float w satisfies |w| > delta exactly when |w| > the largest float <= delta
         const float thr = __double2float_rd(delta);
@@ -153,9 +161,10 @@ ternarize_rows_kernel(const float *__restrict__ W, long long rows, long long col
         // padding words of the row
         for (long long j = words + tid; j < wpr; j += kThreads) Pr[j] = 0u;
 
-        const double K = block_sum_all(k0 + k1, red_d);
+        double K = k0 + k1;
         // positives in the low, negatives in the high half
-        const unsigned long long c2 = block_sum_all((unsigned long long)(nz - ng) + ((unsigned long long)ng << 32), red_u);
+        unsigned long long c2 = (unsigned long long)(nz - ng) + ((unsigned long long)ng << 32);
+        block_sum_all2(K, c2, red_k, red_u);
         if (tid == 0) {
             const unsigned long long n_pos = c2 & 0xFFFFFFFFull, n_neg = c2 >> 32;
             twn_stats_t st;
@@ -170,6 +179,7 @@ ternarize_rows_kernel(const float *__restrict__ W, long long rows, long long col
             st.reserved = 0;
             stats[row] = st;
         }
+        __syncthreads();       // the partials are free for the next filter of this block
     }
 }
 
