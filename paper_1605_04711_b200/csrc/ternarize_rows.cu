@@ -79,7 +79,7 @@ __device__ __forceinline__ int8_t code_of(uint32_t f) { return (f & 1u) ? ((f & 
 // MODE 1: rows 16-byte aligned and cols % 4 == 0, filter longer than the shared-memory budget: read twice.
 // MODE 2: as 1, and the filter (cols * 4 bytes of dynamic shared memory) stays on chip between the steps.
 template <int MODE>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 6)      // six blocks of 32 KB filters per SM: at most 40 registers
 ternarize_rows_kernel(const float *__restrict__ W, long long rows, long long cols, double factor,
                       twn_stats_t *__restrict__ stats, uint32_t *__restrict__ packed, long long wpr,
                       int8_t *__restrict__ codes_i8)
@@ -123,15 +123,13 @@ ternarize_rows_kernel(const float *__restrict__ W, long long rows, long long col
             // Elements 0 and 2 of the quarter go to the low half-word, 1 and 3 to the high one, the
             // first of each pair two bits above the second.
             const int sh = 12 - 4 * (lane & 3);    // field_pos of element 2 of this lane's quarter
-            for (int i0 = 0; i0 < n4; i0 += kThreads) {
-                const int i = i0 + tid;
-                const float4 x = i < n4 ? rowbuf[i] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            auto quarter = [&](const int i, const float4 x, const bool in_row) {
                 const uint32_t f0 = field_of(x.x, thr, k0), f1 = field_of(x.y, thr, k1);
                 const uint32_t f2 = field_of(x.z, thr, k0), f3 = field_of(x.w, thr, k1);
                 uint32_t part = ((f0 * 4u + f2) | ((f1 * 4u + f3) << 16)) << sh;
                 nz += __popc(part & 0x55555555u);
                 ng += __popc(part & 0xAAAAAAAAu);
-                if (Cr && i < n4) {
+                if (Cr && in_row) {
                     // cols % 4 == 0 and the matrix is aligned: the four codes are one aligned word
                     const uint32_t c4 = (uint32_t)(uint8_t)code_of(f0) | ((uint32_t)(uint8_t)code_of(f1) << 8) |
                                         ((uint32_t)(uint8_t)code_of(f2) << 16) | ((uint32_t)(uint8_t)code_of(f3) << 24);
@@ -139,7 +137,18 @@ ternarize_rows_kernel(const float *__restrict__ W, long long rows, long long col
                 }
                 part |= __shfl_xor_sync(0xffffffffu, part, 1);
                 part |= __shfl_xor_sync(0xffffffffu, part, 2);
-                if ((lane & 3) == 0 && i < n4) Pr[i >> 2] = part;
+                if ((lane & 3) == 0 && in_row) Pr[i >> 2] = part;
+            };
+            // whole sweeps of the block first (no bounds to check), then one ragged sweep
+            const int full = n4 / kThreads;
+#pragma unroll 4
+            for (int it = 0; it < full; ++it) {
+                const int i = it * kThreads + tid;
+                quarter(i, rowbuf[i], true);
+            }
+            if (full * kThreads < n4) {
+                const int i = full * kThreads + tid;
+                quarter(i, i < n4 ? rowbuf[i] : make_float4(0.0f, 0.0f, 0.0f, 0.0f), i < n4);
             }
         } else {
             for (long long j = tid; j < words; j += kThreads) {
