@@ -136,6 +136,10 @@ CONV_CASES = [
     # enough pixels for the 256-pixel kernel
     (8, 64, 64, 64, 256, 3, 1, 1),
     (37, 28, 28, 128, 256, 3, 2, 1),
+    # shapes for which the tile cost model picks the 192-pixel kernel (8 x 8 x 3 pixel tiles): ragged
+    # in width, height (60 of 64) and batch (5 of 6); 64 and 96 channels (half-empty channel tile)
+    (5, 60, 60, 64, 64, 3, 1, 1),
+    (5, 62, 59, 64, 96, 3, 1, 1),
     (64, 14, 14, 64, 384, 3, 1, 1),
 ]
 
