@@ -383,16 +383,20 @@ class NetWorkload:
     def __init__(self, kind):
         self.kind = kind
         self.name = {"resnet18_train": "resnet18_train_step_b64_224", "vgg7_fwd": "vgg7_forward_b128",
-                     "lenet5_fwd": "lenet5_forward_b100", "resnet18b_train": "resnet18b_train_step_b64_224"}[kind]
+                     "lenet5_fwd": "lenet5_forward_b100", "resnet18b_train": "resnet18b_train_step_b64_224",
+                     "resnet18_train_sgd": "resnet18_train_step_with_update_b64_224"}[kind]
 
     def train_kind(self):
-        return self.kind in ("resnet18_train", "resnet18b_train")
+        return self.kind in ("resnet18_train", "resnet18b_train", "resnet18_train_sgd")
 
     def make(self, nets):
         if self.kind == "resnet18_train":
             return nets.resnet18(64, train=True)
         if self.kind == "resnet18b_train":
             return nets.resnet18b(64, train=True)
+        if self.kind == "resnet18_train_sgd":
+            # a learning rate small enough that hundreds of steps on the same synthetic batch stay finite
+            return nets.resnet18(64, train=True, optimizer=dict(lr=1e-12, momentum=0.9, weight_decay=1e-4))
         if self.kind == "vgg7_fwd":
             return nets.vgg7(128)
         return nets.lenet5(100)
@@ -405,6 +409,9 @@ class NetWorkload:
         if self.train_kind():
             c["step"] = ("ternarize+pack 21 tensors, transpose codes, forward, backward for data, "
                          "straight-through dW; synthetic dY N(0,1e-2) at the logits")
+            if self.kind == "resnet18_train_sgd":
+                c["step"] += ("; SGD-momentum update of the master weights (lr 1e-12 so that repeated steps on one "
+                              "synthetic batch stay finite), whose threshold reduction replaces the first ternarization sweep")
         else:
             c["step"] = "forward through ternary conv/FC with packed weights (ternarization done once, untimed)"
             c["l2"] = "L2 flushed between timed steps is not needed: one step per replay, working set noted"
@@ -412,7 +419,8 @@ class NetWorkload:
 
     def host_inputs(self):
         from paper_1605_04711_b200 import datagen as dg
-        shape = {"resnet18_train": (64, 224, 224, 3), "resnet18b_train": (64, 224, 224, 3), "vgg7_fwd": (128, 32, 32, 3),
+        shape = {"resnet18_train": (64, 224, 224, 3), "resnet18b_train": (64, 224, 224, 3),
+                 "resnet18_train_sgd": (64, 224, 224, 3), "vgg7_fwd": (128, 32, 32, 3),
                  "lenet5_fwd": (100, 28, 28, 1)}[self.kind]
         n = 1
         for s in shape:
@@ -526,6 +534,7 @@ class NetWorkload:
                 n += 2 if self.train else 1
         if self.train:
             n += 3 * ((len(net.layers) + 31) // 32)     # batched ternarization (two sweeps) and code transposes
+            # with the update: coding sweep + update instead of the two sweeps, the same count
         return n
 
     def units_per_step(self):
@@ -581,14 +590,16 @@ class NetWorkload:
     def _macs_per_image(self):
         if hasattr(self, "net"):
             return self.net.total_macs() / self.net.B
-        return {"resnet18_train": 340.7e9 / 64, "resnet18b_train": 755.3e9 / 64, "vgg7_fwd": 615.9e6,
+        return {"resnet18_train": 340.7e9 / 64, "resnet18_train_sgd": 340.7e9 / 64, "resnet18b_train": 755.3e9 / 64,
+                "vgg7_fwd": 615.9e6,
                 "lenet5_fwd": 4.27e6}[self.kind]
 
 
 WORKLOADS = {"ternarize": lambda: TernarizeWorkload(), "sgd_ternarize": lambda: SgdTernarizeWorkload(), "ternarize_rows": lambda: TernarizeRowsWorkload(), "resnet18_train": lambda: NetWorkload("resnet18_train"),
              "gemm_16384": lambda: GemmWorkload(16384), "gemm_4096": lambda: GemmWorkload(4096),
              "vgg7_fwd": lambda: NetWorkload("vgg7_fwd"), "lenet5_fwd": lambda: NetWorkload("lenet5_fwd"),
-             "resnet18b_train": lambda: NetWorkload("resnet18b_train")}
+             "resnet18b_train": lambda: NetWorkload("resnet18b_train"),
+             "resnet18_train_sgd": lambda: NetWorkload("resnet18_train_sgd")}
 DEFAULT_WORKLOAD = "resnet18_train"
 
 
@@ -606,7 +617,7 @@ def run_reference(args):
         if i >= args.warmup:
             vals.append(v)
     value = sum(vals) / len(vals)
-    upstep = wl.units_per_step() if isinstance(wl, (TernarizeWorkload, GemmWorkload)) else {"resnet18_train": 64, "resnet18b_train": 64, "vgg7_fwd": 128, "lenet5_fwd": 100}[args.workload]
+    upstep = wl.units_per_step() if isinstance(wl, (TernarizeWorkload, GemmWorkload)) else {"resnet18_train": 64, "resnet18b_train": 64, "resnet18_train_sgd": 64, "vgg7_fwd": 128, "lenet5_fwd": 100}[args.workload]
     line = {"impl": "reference", "metric": wl.metric, "value": value, "unit": wl.unit,
             "n_gpus": args.gpus, "steps": steps, "warmup": args.warmup,
             "ms_per_step": upstep / value * 1e3, "higher_is_better": True,

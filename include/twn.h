@@ -221,6 +221,23 @@ int twn_ternarize_codes(const float *W, int64_t rows, int64_t cols, twn_stats_t 
                         uint32_t *packed, int64_t ld_codes, int8_t *codes_i8,
                         void *workspace, size_t workspace_bytes, twn_stream_t stream);
 
+/* twn_sgd_update and twn_ternarize_codes for up to 32 tensors (the layers of a network) in one
+ * launch each; every tensor gets the bits of a call of its own.  items: HOST arrays, read during
+ * the call only; fields as the arguments of the single-tensor calls.  workspace: at least
+ * twn_ternarize_batch_workspace_bytes(count), 256-byte aligned. */
+typedef struct {
+    float *W;
+    const float *dW;
+    float *V;
+    int64_t n;
+    twn_stats_t *stats_next;   /* optional */
+} twn_sgd_item_t;
+int twn_sgd_update_batch(const twn_sgd_item_t *items, int count, float lr, float momentum,
+                         float weight_decay, double delta_factor, void *workspace,
+                         size_t workspace_bytes, twn_stream_t stream);
+int twn_ternarize_codes_batch(const twn_ternarize_item_t *items, int count, void *workspace,
+                              size_t workspace_bytes, twn_stream_t stream);
+
 /*
  * Per-filter threshold ternarization fused with 2-bit packing: Algorithm 1 as printed,
  * whose first loop runs over the filters of a layer.  Row r of W is one filter and gets

@@ -157,20 +157,21 @@ __device__ __forceinline__ float sgd_one(float w, float g, float &v, float lr, f
     return __fsub_rn(w, __fmul_rn(lr, v));
 }
 
-__global__ void __launch_bounds__(kThreads)
-sgd_update_kernel(float *__restrict__ W, const float *__restrict__ dW, float *__restrict__ V, long long n,
-                  float lr, float mu, float wd, double factor, void *ws_raw, twn_stats_t *__restrict__ stats)
+// `vb` of `vg`: this block's index among the blocks that work on this tensor.
+__device__ __forceinline__ void sgd_update_body(float *__restrict__ W, const float *__restrict__ dW, float *__restrict__ V,
+                                                long long n, float lr, float mu, float wd, double factor,
+                                                const Workspace ws, twn_stats_t *__restrict__ stats, unsigned int vb,
+                                                unsigned int vg)
 {
     __shared__ double red[kWarps];
-    const Workspace ws = carve(ws_raw);
     const long long n4 = n >> 2;
     float4 *W4 = reinterpret_cast<float4 *>(W);
     float4 *V4 = reinterpret_cast<float4 *>(V);
     const float4 *G4 = reinterpret_cast<const float4 *>(dW);
-    const long long stride = (long long)gridDim.x * kThreads;
+    const long long stride = (long long)vg * kThreads;
     double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
 #pragma unroll 2
-    for (long long i = (long long)blockIdx.x * kThreads + threadIdx.x; i < n4; i += stride) {
+    for (long long i = (long long)vb * kThreads + threadIdx.x; i < n4; i += stride) {
         float4 w = W4[i], v = V4[i];
         const float4 g = __ldg(G4 + i);
         w.x = sgd_one(w.x, g.x, v.x, lr, mu, wd);
@@ -181,7 +182,7 @@ sgd_update_kernel(float *__restrict__ W, const float *__restrict__ dW, float *__
         V4[i] = v;
         a0 += (double)fabsf(w.x); a1 += (double)fabsf(w.y); a2 += (double)fabsf(w.z); a3 += (double)fabsf(w.w);
     }
-    if (blockIdx.x == 0) {
+    if (vb == 0) {
         const long long t = (n4 << 2) + threadIdx.x;
         if (t < n) {
             float v = V[t];
@@ -192,10 +193,10 @@ sgd_update_kernel(float *__restrict__ W, const float *__restrict__ dW, float *__
         }
     }
     const double bsum = block_sum((a0 + a1) + (a2 + a3), red);
-    if (threadIdx.x == 0) ws.part_sum[blockIdx.x] = bsum;
-    if (last_block(ws.ticket1, gridDim.x)) {
+    if (threadIdx.x == 0) ws.part_sum[vb] = bsum;
+    if (last_block(ws.ticket1, vg)) {
         double s = 0.0;
-        for (int b = threadIdx.x; b < (int)gridDim.x; b += kThreads) s += __ldcg(ws.part_sum + b);
+        for (int b = threadIdx.x; b < (int)vg; b += kThreads) s += __ldcg(ws.part_sum + b);
         s = block_sum(s, red);
         if (threadIdx.x == 0) {
             if (stats) {
@@ -207,6 +208,13 @@ sgd_update_kernel(float *__restrict__ W, const float *__restrict__ dW, float *__
             *ws.ticket1 = 0u;
         }
     }
+}
+
+__global__ void __launch_bounds__(kThreads)
+sgd_update_kernel(float *__restrict__ W, const float *__restrict__ dW, float *__restrict__ V, long long n,
+                  float lr, float mu, float wd, double factor, void *ws_raw, twn_stats_t *__restrict__ stats)
+{
+    sgd_update_body(W, dW, V, n, lr, mu, wd, factor, carve(ws_raw), stats, blockIdx.x, gridDim.x);
 }
 
 // ---- sweep 2 -------------------------------------------------------------
@@ -448,6 +456,29 @@ code_pack_batch_kernel(const __grid_constant__ BatchParams P, void *ws_raw)
     code_pack_body(it.W, it.rows, it.cols, it.ld_codes, it.fast_units, it.packed, it.codes_i8,
                    carve_batch(ws_raw, t, P.count), it.stats, blockIdx.x - P.first_block[t],
                    P.first_block[t + 1] - P.first_block[t]);
+}
+
+struct SgdItem {
+    float *W;
+    const float *dW;
+    float *V;
+    long long n;
+    twn_stats_t *stats;
+};
+struct SgdBatch {
+    int count;
+    unsigned int first_block[kMaxBatch + 1];
+    SgdItem item[kMaxBatch];
+};
+
+__global__ void __launch_bounds__(kThreads)
+sgd_update_batch_kernel(const __grid_constant__ SgdBatch P, float lr, float mu, float wd, double factor, void *ws_raw)
+{
+    int t = 0;
+    while (t + 1 < P.count && blockIdx.x >= P.first_block[t + 1]) ++t;
+    const SgdItem &it = P.item[t];
+    sgd_update_body(it.W, it.dW, it.V, it.n, lr, mu, wd, factor, carve_batch(ws_raw, t, P.count), it.stats,
+                    blockIdx.x - P.first_block[t], P.first_block[t + 1] - P.first_block[t]);
 }
 
 // ---- standalone pack / unpack / re-layout ----------------------------------
@@ -707,6 +738,84 @@ extern "C" int twn_sgd_update(float *W, const float *dW, float *V, int64_t n, fl
     TWN_CUDA_OK(cudaMemsetAsync(workspace, 0, 128, s));
     const int g = grid_for((n / 4 + 1) / 2, dev.sm_count);
     sgd_update_kernel<<<g, kThreads, 0, s>>>(W, dW, V, n, lr, momentum, weight_decay, delta_factor, workspace, stats_next);
+    TWN_CUDA_OK(cudaGetLastError());
+    return TWN_OK;
+}
+
+extern "C" int twn_sgd_update_batch(const twn_sgd_item_t *items, int count, float lr, float momentum,
+                                    float weight_decay, double delta_factor, void *workspace, size_t workspace_bytes,
+                                    twn_stream_t stream)
+{
+    TWN_REQUIRE(count >= 0 && count <= kMaxBatch, TWN_ERR_INVALID_ARG);
+    if (count == 0) return TWN_OK;
+    TWN_REQUIRE(items != nullptr && workspace != nullptr, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(lr == lr && momentum == momentum && weight_decay == weight_decay, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(delta_factor >= 0.0 && delta_factor == delta_factor, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(workspace_bytes >= twn_ternarize_batch_workspace_bytes(count), TWN_ERR_WORKSPACE);
+    TWN_REQUIRE(twn_aligned(workspace, 256), TWN_ERR_MISALIGNED);
+    twn_device_info dev;
+    const int rc = twn_current_device(&dev);
+    if (rc != TWN_OK) return rc;
+    SgdBatch P;
+    P.count = count;
+    unsigned int g = 0;
+    for (int t = 0; t < count; ++t) {
+        const twn_sgd_item_t &it = items[t];
+        TWN_REQUIRE(it.n >= 0 && (it.n == 0 || (it.W && it.dW && it.V)), TWN_ERR_INVALID_ARG);
+        TWN_REQUIRE(twn_aligned(it.W, 16) && twn_aligned(it.dW, 16) && twn_aligned(it.V, 16) &&
+                        twn_aligned(it.stats_next, 8), TWN_ERR_MISALIGNED);
+        SgdItem si;
+        si.W = it.W; si.dW = it.dW; si.V = it.V; si.n = it.n; si.stats = it.stats_next;
+        P.item[t] = si;
+        P.first_block[t] = g;
+        g += (unsigned int)grid_for((it.n / 4 + 1) / 2, dev.sm_count);     // the grid of a call of its own
+    }
+    P.first_block[count] = g;
+    cudaStream_t s = twn_cu(stream);
+    TWN_CUDA_OK(cudaMemsetAsync(workspace, 0, (size_t)count * 256, s));
+    sgd_update_batch_kernel<<<g, kThreads, 0, s>>>(P, lr, momentum, weight_decay, delta_factor, workspace);
+    TWN_CUDA_OK(cudaGetLastError());
+    return TWN_OK;
+}
+
+extern "C" int twn_ternarize_codes_batch(const twn_ternarize_item_t *items, int count, void *workspace,
+                                         size_t workspace_bytes, twn_stream_t stream)
+{
+    TWN_REQUIRE(count >= 0 && count <= kMaxBatch, TWN_ERR_INVALID_ARG);
+    if (count == 0) return TWN_OK;
+    TWN_REQUIRE(items != nullptr && workspace != nullptr, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(workspace_bytes >= twn_ternarize_batch_workspace_bytes(count), TWN_ERR_WORKSPACE);
+    TWN_REQUIRE(twn_aligned(workspace, 256), TWN_ERR_MISALIGNED);
+    twn_device_info dev;
+    const int rc = twn_current_device(&dev);
+    if (rc != TWN_OK) return rc;
+    BatchParams B;
+    B.count = count;
+    unsigned int gb = 0;
+    for (int t = 0; t < count; ++t) {
+        const twn_ternarize_item_t &it = items[t];
+        TWN_REQUIRE(it.rows >= 0 && it.cols >= 0 && it.stats != nullptr, TWN_ERR_INVALID_ARG);
+        TWN_REQUIRE(it.ld_codes >= it.cols && it.ld_codes % 64 == 0, TWN_ERR_INVALID_ARG);
+        const long long n = (long long)it.rows * it.cols;
+        TWN_REQUIRE(n == 0 || (it.W != nullptr && it.packed != nullptr), TWN_ERR_INVALID_ARG);
+        TWN_REQUIRE(twn_aligned(it.W, 16) && twn_aligned(it.packed, 16) && twn_aligned(it.stats, 8) &&
+                        twn_aligned(it.codes_i8, 16), TWN_ERR_MISALIGNED);
+        const bool flat = (it.rows <= 1) || (it.ld_codes == it.cols);
+        const long long fast_units = flat ? n / 512 : 0;
+        const long long rest_words = (long long)it.rows * (it.ld_codes / 16) - fast_units * 32;
+        long long work = fast_units * 32 / 4;
+        if (rest_words > work) work = rest_words;
+        BatchItem bi;
+        bi.W = it.W; bi.rows = it.rows; bi.cols = it.cols; bi.ld_codes = it.ld_codes; bi.fast_units = fast_units;
+        bi.packed = it.packed; bi.codes_i8 = it.codes_i8; bi.stats = it.stats;
+        B.item[t] = bi;
+        B.first_block[t] = gb;
+        gb += (unsigned int)grid_for(work, dev.sm_count);
+    }
+    B.first_block[count] = gb;
+    cudaStream_t s = twn_cu(stream);
+    TWN_CUDA_OK(cudaMemsetAsync(workspace, 0, (size_t)count * 256, s));
+    code_pack_batch_kernel<<<gb, kThreads, 0, s>>>(B, workspace);
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }

@@ -68,9 +68,14 @@ class TernaryNet:
     """A chain of ternary conv / FC layers with pooling glue, all buffers preallocated."""
 
     def __init__(self, name: str, batch: int, in_shape, ops, seed: int = 0, delta_factor: float = 0.7,
-                 train: bool = False):
+                 train: bool = False, optimizer: dict | None = None):
+        """optimizer: None (the step ends with the weight gradients) or dict(lr, momentum, weight_decay):
+        the step then ends with the SGD update of the master weights (Algorithm 1, UpdateParameters), which
+        also leaves the next iteration's thresholds behind, so that later steps run only the coding sweep."""
         self.name, self.B, self.in_shape, self.ops = name, batch, in_shape, ops
         self.seed, self.delta_factor, self.train = seed, delta_factor, train
+        self.optimizer = optimizer if train else None
+        self._delta_ready = False
         self.layers: dict[str, Layer] = {op[1].name: op[1] for op in ops if op[0] == "layer"}
         self.act: dict[str, torch.Tensor] = {}
         self.aux: dict[str, torch.Tensor] = {}
@@ -123,6 +128,10 @@ class TernaryNet:
                 res = self.act[L.residual] if L.residual else None
                 e["epi"] = twn.epilogue(e["scale"], e["shift"], res, relu=L.relu,
                                         out_dtype=twn.F32 if L.out_f32 else twn.BF16)
+                if self.optimizer:
+                    if L.small_cin and not L.fold:
+                        raise NotImplementedError("the update needs a weight gradient in the layout of the weights")
+                    e["V"] = torch.zeros_like(e["W"])
                 if self.train:
                     first = L.src == "input"
                     if not first:
@@ -188,8 +197,13 @@ class TernaryNet:
             group = layers[i:i + 32]
             items = [(L.extra["W"], L.Cout, L.K, L.extra["stats"], L.extra["packed"], L.extra["ld"], None)
                      for L in group]
-            self._call("ternarize", f"layers {i}..{i + len(group) - 1}", 0,
-                       lambda: twn.ternarize_batch(items, self.delta_factor, self.ws_tern))
+            if self._delta_ready:
+                # the thresholds were left behind by the previous step's update: coding sweep only
+                self._call("ternarize", f"layers {i}..{i + len(group) - 1}", 0,
+                           lambda: twn.ternarize_codes_batch(items, self.ws_tern))
+            else:
+                self._call("ternarize", f"layers {i}..{i + len(group) - 1}", 0,
+                           lambda: twn.ternarize_batch(items, self.delta_factor, self.ws_tern))
         for L in layers:
             if L.fold:
                 twn.fold_codes(L.desc, L.extra["packed"], L.extra["ld"], L.extra["packed_f"], L.fold[2])
@@ -383,11 +397,23 @@ class TernaryNet:
         main.wait_stream(self.dw_stream)
         self.last_grads = acc
 
+    def sgd_step(self):
+        """Algorithm 1, UpdateParameters: SGD with momentum and weight decay on every layer's master
+        weights (one batched launch per 32 layers), which also writes the next thresholds."""
+        o = self.optimizer
+        layers = list(self.layers.values())
+        for i in range(0, len(layers), 32):
+            items = [(L.extra["W"], L.extra["dW"], L.extra["V"], L.extra["stats"]) for L in layers[i:i + 32]]
+            twn.sgd_update_batch(items, o["lr"], o["momentum"], o["weight_decay"], self.delta_factor, self.ws_tern)
+        self._delta_ready = True
+
     def train_step(self, dlogits):
         self.ternarize_all(join=False)
         self.forward()
         self.backward(dlogits)
         self.join_side_streams()
+        if self.optimizer:
+            self.sgd_step()
 
     def check_status(self):
         s = twn.read_status(self.status)
@@ -432,7 +458,8 @@ def vgg7(batch=128, train=False, seed=0):
     return TernaryNet("vgg7", batch, (32, 32, 3), ops, seed, train=train)
 
 
-def resnet18(batch=64, train=True, seed=0, image=224, classes=1000, widths=(64, 128, 256, 512), name="resnet18"):
+def resnet18(batch=64, train=True, seed=0, image=224, classes=1000, widths=(64, 128, 256, 512), name="resnet18",
+             optimizer=None):
     """BasicBlock layout [2, 2, 2, 2] with a 7x7/2 first layer.  `widths` are the channels of the four
     stages; (96, 192, 384, 768) is the 1.5x wider "ResNet-18B" of the paper's ImageNet experiments."""
     w0 = widths[0]
@@ -456,7 +483,7 @@ def resnet18(batch=64, train=True, seed=0, image=224, classes=1000, widths=(64, 
             src, cin, H = p + ".conv2", c, Ho
     ops.append(("avgpool", "gap", src))
     ops.append(("layer", Layer("fc", widths[-1], classes, relu=False, src="gap", out_f32=True)))
-    return TernaryNet(name, batch, (image, image, 3), ops, seed, train=train)
+    return TernaryNet(name, batch, (image, image, 3), ops, seed, train=train, optimizer=optimizer)
 
 
 def resnet18b(batch=64, train=True, seed=0, image=224, classes=1000):

@@ -174,6 +174,34 @@ def ternarize_batch(items, delta_factor: float, workspace: torch.Tensor, stream=
                                      _stream(stream)), "twn_ternarize_batch")
 
 
+class SgdItem(C.Structure):
+    _fields_ = [("W", C.c_void_p), ("dW", C.c_void_p), ("V", C.c_void_p), ("n", C.c_int64), ("stats_next", C.c_void_p)]
+
+
+def sgd_update_batch(items, lr: float, momentum: float, weight_decay: float, delta_factor: float,
+                     workspace: torch.Tensor, stream=None) -> None:
+    """twn_sgd_update_batch.  items: list of (W, dW, V, stats_next or None)."""
+    arr = (SgdItem * max(len(items), 1))()
+    for i, (W, dW, V, st) in enumerate(items):
+        assert dW.numel() == W.numel() == V.numel()
+        arr[i] = SgdItem(_ptr(W).value, _ptr(dW).value, _ptr(V).value, W.numel(), _ptr(st).value)
+    _check(lib().twn_sgd_update_batch(arr, C.c_int(len(items)), C.c_float(lr), C.c_float(momentum),
+                                      C.c_float(weight_decay), C.c_double(delta_factor), _ptr(workspace),
+                                      C.c_size_t(workspace.numel() * workspace.element_size()), _stream(stream)),
+           "twn_sgd_update_batch")
+
+
+def ternarize_codes_batch(items, workspace: torch.Tensor, stream=None) -> None:
+    """twn_ternarize_codes_batch.  items as for ternarize_batch; every stats holds its threshold already."""
+    arr = (TernarizeItem * max(len(items), 1))()
+    for i, (W, rows, cols, stats, packed, ld, codes) in enumerate(items):
+        arr[i] = TernarizeItem(_ptr(W).value, rows, cols, _ptr(stats).value, _ptr(packed).value, ld,
+                               _ptr(codes).value)
+    _check(lib().twn_ternarize_codes_batch(arr, C.c_int(len(items)), _ptr(workspace),
+                                           C.c_size_t(workspace.numel() * workspace.element_size()),
+                                           _stream(stream)), "twn_ternarize_codes_batch")
+
+
 class TransposeItem(C.Structure):
     _fields_ = [("packed_fwd", C.c_void_p), ("ld_fwd", C.c_int64), ("desc", ConvDesc), ("packed_bwd", C.c_void_p),
                 ("ld_bwd", C.c_int64)]

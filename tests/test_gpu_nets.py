@@ -201,6 +201,42 @@ def test_resnet18b_wider_stages_small_train_step(monkeypatch):
     check_backward(net, npix=200, nent=200)
 
 
+def test_resnet18_small_steps_with_parameter_update():
+    """Algorithm 1 end to end, twice: ternarize, forward, backward, SGD update.  The update is checked
+    against the oracle on the GPU's own gradients (bit-exact), and the second step's codes, which come
+    from the coding sweep alone with the thresholds the update left behind, against the oracle's
+    ternarization of the updated weights."""
+    opt = dict(lr=1e-3, momentum=0.9, weight_decay=1e-4)
+    net = nets.resnet18(batch=2, train=True, image=64, classes=24, optimizer=opt)
+    x = dg.draw_bf16(0, "sgdnet.input", net.act["input"].numel(), "normal")
+    net.set_input(x)
+    dy_bits = dg.draw_bf16(0, "sgdnet.dlogits", 2 * 24, "normal", 0.0, 0.1)
+    dY = torch.from_numpy(dy_bits.view(np.int16)).cuda().view(torch.bfloat16).view(2, 24)
+    W = {n: L.extra["W"].cpu().numpy().copy() for n, L in net.layers.items()}
+    V = {n: np.zeros_like(w) for n, w in W.items()}
+    for step in range(2):
+        net.train_step(dY)
+        torch.cuda.synchronize()
+        net.check_status()
+        for n, L in net.layers.items():
+            if step == 1:
+                # this step's codes came from the coding sweep alone
+                st, codes = oracle.ternarize(W[n], net.delta_factor)
+                got = twn.stats_to_host(L.extra["stats"])
+                assert st.n_boundary == 0
+                assert np.array_equal(L.extra["packed"].cpu().numpy().view(np.uint32),
+                                      oracle.pack(codes.reshape(L.Cout, L.K), L.extra["ld"]))
+                assert abs(got["alpha"] - st.alpha) <= 1e-12 * st.alpha
+            dW = L.extra["dW"].cpu().numpy().reshape(W[n].shape)
+            W[n], V[n] = oracle.sgd_update(W[n], dW, V[n], opt["lr"], opt["momentum"], opt["weight_decay"])
+            assert np.array_equal(L.extra["W"].cpu().numpy().view(np.uint32), W[n].view(np.uint32))
+            assert np.array_equal(L.extra["V"].cpu().numpy().view(np.uint32), V[n].view(np.uint32))
+            # the threshold for the next step is already there
+            st_next, _ = oracle.ternarize(W[n], net.delta_factor)
+            got = twn.stats_to_host(L.extra["stats"])
+            assert got["status"] == 0 and abs(got["delta"] - st_next.delta) <= 1e-12 * st_next.delta
+
+
 def test_resnet18_train_step_batch64(monkeypatch):
     net = nets.resnet18(batch=64, train=True)
     run_train_step(net, monkeypatch)
