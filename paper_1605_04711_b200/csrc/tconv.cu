@@ -141,8 +141,10 @@ struct __align__(1024) SmemLayout {
     static constexpr int kStages = Cfg<PIX>::kStages, kSub = Cfg<PIX>::kSub;
     static constexpr int kXBytes = PIX * kBlockK * 2;
     uint8_t x[kStages][kSub][kXBytes];           // swizzled activation tiles
-    unsigned long long full[kStages];      // TMA -> MMA: activation tile landed
-    unsigned long long ready_a[8];         // decode -> MMA: weights of the stage / k-block are in tensor memory
+    // TMA and decode -> MMA: the activation tile has landed (one arrival with its byte count) and the
+    // four decode warps have put the stage's weights into tensor memory (one arrival each).  One
+    // barrier for both: every wait of the issuing warp is latency that the tensor core may sit out.
+    unsigned long long full[kStages];
     unsigned long long empty[kStages];     // MMA commit -> TMA and decode: both operand slots are free
     unsigned long long acc_full[2];        // MMA commit -> epilogue
     unsigned long long acc_empty[2];       // epilogue -> MMA
@@ -187,10 +189,9 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(&sm->full[s], 1);
+            mbar_init(&sm->full[s], 1 + 4);
             mbar_init(&sm->empty[s], 1);
         }
-        for (int s = 0; s < 8; ++s) mbar_init(&sm->ready_a[s], 4);
         for (int b = 0; b < 2; ++b) {
             mbar_init(&sm->acc_full[b], 1);
             mbar_init(&sm->acc_empty[b], kEpiWarps);
@@ -272,10 +273,6 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 for (int st = 0; st < spt; ++st, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
-                    PROF_T(t_r);
-                    if (!mbar_wait_warp(&sm->ready_a[s], ph, abort_flag, P.status, 0)) { ok = false; break; }
-                    PROF_ACC(w_ready, t_r);
-                    if (lane == 0) PROF_TL(2, it);
                     PROF_T(t_x);
                     if (!mbar_wait_warp(&sm->full[s], ph, abort_flag, P.status, 0)) { ok = false; break; }
                     PROF_ACC(w_issue, t_x);
@@ -403,7 +400,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sm->ready_a[s]);
+                if (lane == 0) mbar_arrive(&sm->full[s]);
                 PROF_ACC(d_wst, t_wst);
                 PROF_TL2(2, it);
                 advance(tile_c, st_c, kDecodeSets);
@@ -842,7 +839,7 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     //   128 pixels: max(2000 + 680 kb, 6500): the epilogue overlaps the next tile and bounds short reductions
     //   192 pixels: max(2500 + 790 kb, 10500), floor 7600 when only the lower half of the channel
     //               tile exists: overlapped as well, fewer rounds than 128
-    //   256 pixels: 13500 + 640 kb: one accumulator, so the epilogue is exposed; 8000 when only the
+    //   256 pixels: 8000 + 740 kb: one accumulator, so the epilogue is exposed; 7000 when only the
     //               lower half of the channel tile exists (half of the epilogue warps idle)
     int a, b;
     const long long kb = (long long)P.n_taps * P.n_cblk;
@@ -853,7 +850,7 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     const long long per128 = 2000 + 680 * kb > 6500 ? 2000 + 680 * kb : 6500;
     const long long floor192 = half ? 7600 : 10500;
     const long long per192 = 2500 + 790 * kb > floor192 ? 2500 + 790 * kb : floor192;
-    const long long per256 = (half ? 8000 : 13500) + 640 * kb;
+    const long long per256 = (half ? 7000 : 8000) + 740 * kb;
     const long long c128 = ((t128 + sms - 1) / sms) * per128, c192 = ((t192 + sms - 1) / sms) * per192,
                     c256 = ((t256 + sms - 1) / sms) * per256;
     int choice = c256 < c128 ? 1 : 0;
