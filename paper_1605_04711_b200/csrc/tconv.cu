@@ -837,9 +837,9 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     // Tile shape by a cost model fitted to measured launches (cycles per round of tiles, kb = k-blocks
     // per tile):
     //   128 pixels: max(2000 + 680 kb, 6500): the epilogue overlaps the next tile and bounds short reductions
-    //   192 pixels: max(2500 + 790 kb, 10500), floor 7600 when only the lower half of the channel
+    //   192 pixels: max(2500 + 700 kb, 10500), floor 7600 when only the lower half of the channel
     //               tile exists: overlapped as well, fewer rounds than 128
-    //   256 pixels: 8000 + 740 kb: one accumulator, so the epilogue is exposed; 7000 when only the
+    //   256 pixels: 8000 + 700 kb: one accumulator, so the epilogue is exposed; 7000 when only the
     //               lower half of the channel tile exists (half of the epilogue warps idle)
     int a, b;
     const long long kb = (long long)P.n_taps * P.n_cblk;
@@ -849,8 +849,8 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     const long long t192 = pick_tile(g, 192, &a, &b) * P.n_tiles;
     const long long per128 = 2000 + 680 * kb > 6500 ? 2000 + 680 * kb : 6500;
     const long long floor192 = half ? 7600 : 10500;
-    const long long per192 = 2500 + 790 * kb > floor192 ? 2500 + 790 * kb : floor192;
-    const long long per256 = (half ? 7000 : 8000) + 740 * kb;
+    const long long per192 = 2500 + 700 * kb > floor192 ? 2500 + 700 * kb : floor192;
+    const long long per256 = (half ? 7000 : 8000) + 700 * kb;
     const long long c128 = ((t128 + sms - 1) / sms) * per128, c192 = ((t192 + sms - 1) / sms) * per192,
                     c256 = ((t256 + sms - 1) / sms) * per256;
     int choice = c256 < c128 ? 1 : 0;
