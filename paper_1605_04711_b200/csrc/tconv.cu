@@ -68,10 +68,12 @@ namespace {
 
 constexpr int kChan = 128;          // output channels per tile (UMMA M)
 constexpr int kBlockK = 64;         // reduction elements per k-block (128 bytes of bf16)
-constexpr int kDecodeSets = 1;      // groups of 4 decode warps; a group takes every other stage
-constexpr int kFirstEpiWarp = 2 + 4 * kDecodeSets;
+// Groups of 4 decode warps in a block (template parameter DS): one, or two that take the stages in turn.
+// Two pay where decoding paces an overlapped tile shape on a long reduction; elsewhere the four extra
+// warps cost speed (they cap the block at 112 registers), so each variant is a kernel of its own.
+__host__ __device__ constexpr int first_epi_warp(int ds) { return 2 + 4 * ds; }
 constexpr int kEpiSets = 2;         // epilogue warps per lane quadrant; each drains every other 32-pixel chunk
-constexpr int kThreadsConv = 32 * (kFirstEpiWarp + 4 * kEpiSets);   // kEpiWarps epilogue warps
+__host__ __device__ constexpr int threads_conv(int ds) { return 32 * (first_epi_warp(ds) + 4 * kEpiSets); }
 constexpr int kEpiWarps = 4 * kEpiSets;
 constexpr int kStageBytes = 2048;   // one output staging buffer of a warp: 32 channels x 32 pixels of bf16 or 16 pixels of fp32
 constexpr int kMaxTaps = 64;
@@ -127,6 +129,7 @@ struct ConvParams {
     const void *residual;
     int res_dtype, relu, out_dtype;
     int res_gate;                 // 0: the residual is added; 1: it gates the result (kept where residual > 0)
+    int dsets;                    // host only: decode groups of the kernel variant to launch
     void *Y;
     int32_t *status;
     // output path: 1 = each epilogue warp stages its 32 channels x 32 pixels in shared memory and
@@ -166,8 +169,8 @@ static_assert(offsetof(SmemLayout<128>, stage_res) % 128 == 0 && offsetof(SmemLa
                   offsetof(SmemLayout<128>, stage_out) % 128 == 0 && offsetof(SmemLayout<256>, stage_out) % 128 == 0,
               "TMA and vector accesses need aligned shared-memory regions");
 
-template <int PIX>
-__global__ void __launch_bounds__(kThreadsConv, 1)
+template <int PIX, int DS>
+__global__ void __launch_bounds__(threads_conv(DS), 1)
 tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
              const __grid_constant__ CUtensorMap map_r, const __grid_constant__ ConvParams P)
 {
@@ -202,6 +205,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
     }
     // code-word offset of every k-block, in the order the k-blocks are consumed: taps outer,
     // channel blocks inner
+    constexpr int kFirstEpiWarp = first_epi_warp(DS), kThreadsConv = threads_conv(DS);
     for (int u = threadIdx.x; u < kbpt && u < kWordTab; u += kThreadsConv) {
         const int t = u / P.n_cblk, cb = u - t * P.n_cblk;
         sm->kword[u] = (uint32_t)(P.taps[t].koff >> 4) + cb * (kBlockK / 16);
@@ -299,6 +303,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         // free tensor-memory slot, not on the activation pipeline.
         const int q = warp & 3;                 // tensor-memory lane quadrant of this warp
         const int set = (warp - 2) >> 2;
+        constexpr int dsets = DS;               // groups of this kernel; the loops below are stepped by it
         const int row = q * 32 + lane;          // channel row inside the tile
         const uint32_t lane_base = tmem_a + ((uint32_t)(q * 32) << 16);
 
@@ -331,7 +336,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 }
             }
         };
-        // position of this group's next stages: (tile, st), advanced kDecodeSets stages at a time
+        // position of this group's next stages: (tile, st), advanced dsets stages at a time
         auto advance = [&](int &tile, int &st, int steps) {
             for (int i = 0; i < steps; ++i)
                 if (++st >= spt) { st = 0; tile += gridDim.x; }
@@ -365,9 +370,9 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
             int nt_f = tile_f % P.n_tiles;
             const uint32_t *rowp_f = row_ptr(nt_f);
             Codes c0, c1, c2;
-            fetch(c0, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, kDecodeSets);
-            fetch(c1, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, kDecodeSets);
-            if (PIX == 256) { fetch(c2, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, kDecodeSets); }
+            fetch(c0, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, dsets);
+            fetch(c1, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, dsets);
+            if (PIX == 256) { fetch(c2, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, dsets); }
             uint32_t it = set;
             auto decode_stage = [&](const Codes &cur) -> bool {
                 const int s = it % kStages;
@@ -403,19 +408,19 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 if (lane == 0) mbar_arrive(&sm->full[s]);
                 PROF_ACC(d_wst, t_wst);
                 PROF_TL2(2, it);
-                advance(tile_c, st_c, kDecodeSets);
-                it += kDecodeSets;
+                advance(tile_c, st_c, dsets);
+                it += dsets;
                 return true;
             };
             if (PIX == 256) {
                 // long reductions, no slack for a late code word: three buffers in rotation
                 while (true) {
                     if (tile_c >= P.total_tiles || !decode_stage(c0)) break;
-                    { PROF_T(t0); fetch(c0, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, kDecodeSets); PROF_ACC(d_fetch, t0); PROF_TL2(3, it - kDecodeSets); }
+                    { PROF_T(t0); fetch(c0, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, dsets); PROF_ACC(d_fetch, t0); PROF_TL2(3, it - dsets); }
                     if (tile_c >= P.total_tiles || !decode_stage(c1)) break;
-                    { PROF_T(t1); fetch(c1, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, kDecodeSets); PROF_ACC(d_fetch, t1); }
+                    { PROF_T(t1); fetch(c1, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, dsets); PROF_ACC(d_fetch, t1); }
                     if (tile_c >= P.total_tiles || !decode_stage(c2)) break;
-                    { PROF_T(t2); fetch(c2, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, kDecodeSets); PROF_ACC(d_fetch, t2); }
+                    { PROF_T(t2); fetch(c2, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, dsets); PROF_ACC(d_fetch, t2); }
                 }
             } else {
                 // The overlapped tile shapes are paced by this loop, and a loop that is a third as long
@@ -426,7 +431,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 while (true) {
                     if (tile_c >= P.total_tiles || !decode_stage(c0)) break;
                     c0 = c1;
-                    { PROF_T(t0); fetch(c1, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, kDecodeSets); PROF_ACC(d_fetch, t0); }
+                    { PROF_T(t0); fetch(c1, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, dsets); PROF_ACC(d_fetch, t0); }
                 }
             }
         }
@@ -708,14 +713,14 @@ long long pick_tile(const Geometry &g, int pix, int *lgBW, int *lgBH)
     return best;
 }
 
-template <int PIX>
+template <int PIX, int DS>
 int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const twn_device_info &dev,
                   EncodeTiledFn enc, cudaStream_t s)
 {
     static bool attr_set[64] = {false};
     const int smem_bytes = (int)sizeof(SmemLayout<PIX>) + 1024;
     if (!attr_set[dev.ordinal]) {
-        TWN_CUDA_OK(cudaFuncSetAttribute(tconv_kernel<PIX>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
+        TWN_CUDA_OK(cudaFuncSetAttribute(tconv_kernel<PIX, DS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
         attr_set[dev.ordinal] = true;
     }
     pick_tile(g, PIX, &P.lgBW, &P.lgBH);
@@ -791,7 +796,7 @@ int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const twn_dev
     if (getenv("TWN_NOTMA")) { P.tma_store = 0; }
 #endif
     const int grid = dev.sm_count < P.total_tiles ? dev.sm_count : P.total_tiles;
-    tconv_kernel<PIX><<<grid, kThreadsConv, smem_bytes, s>>>(map_x, map_y, map_r, P);
+    tconv_kernel<PIX, DS><<<grid, threads_conv(DS), smem_bytes, s>>>(map_x, map_y, map_r, P);
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }
@@ -836,8 +841,9 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
 
     // Tile shape by a cost model fitted to measured launches (cycles per round of tiles, kb = k-blocks
     // per tile):
-    //   128 pixels: max(2000 + 680 kb, 6500): the epilogue overlaps the next tile and bounds short reductions
-    //   192 pixels: max(2500 + 700 kb, 10500), floor 7600 when only the lower half of the channel
+    //   128 pixels: max(2000 + 680 kb, 6500), 540 kb with both decode groups: the epilogue overlaps
+    //               the next tile and bounds short reductions
+    //   192 pixels: max(2500 + 700 kb, 10500), 630 kb with both decode groups; floor 7600 when only the lower half of the channel
     //               tile exists: overlapped as well, fewer rounds than 128
     //   256 pixels: 8000 + 700 kb: one accumulator, so the epilogue is exposed; 7000 when only the
     //               lower half of the channel tile exists (half of the epilogue warps idle)
@@ -847,9 +853,13 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     const bool half = g.Cout <= kChan / 2;
     const long long t128 = pick_tile(g, 128, &a, &b) * P.n_tiles, t256 = pick_tile(g, 256, &a, &b) * P.n_tiles;
     const long long t192 = pick_tile(g, 192, &a, &b) * P.n_tiles;
-    const long long per128 = 2000 + 680 * kb > 6500 ? 2000 + 680 * kb : 6500;
+    // a second decode group pays where decoding paces the overlapped shapes: long reductions
+    const bool two = kb >= 18;
+    const long long lin128 = two ? 2000 + 540 * kb : 2000 + 680 * kb;
+    const long long per128 = lin128 > 6500 ? lin128 : 6500;
     const long long floor192 = half ? 7600 : 10500;
-    const long long per192 = 2500 + 700 * kb > floor192 ? 2500 + 700 * kb : floor192;
+    const long long lin192 = two ? 2500 + 630 * kb : 2500 + 700 * kb;
+    const long long per192 = lin192 > floor192 ? lin192 : floor192;
     const long long per256 = (half ? 7000 : 8000) + 700 * kb;
     const long long c128 = ((t128 + sms - 1) / sms) * per128, c192 = ((t192 + sms - 1) / sms) * per192,
                     c256 = ((t256 + sms - 1) / sms) * per256;
@@ -858,9 +868,13 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
 #if defined(TWN_PROFILE) || defined(TWN_TUNE)
     if (const char *force = getenv("TWN_TILE")) choice = atoi(force) % 3;   // profiling and tuning builds: pin the variant
 #endif
-    if (choice == 2) return launch_conv_t<192>(g, P, X, dev, enc, s);
-    if (choice == 1) return launch_conv_t<256>(g, P, X, dev, enc, s);
-    return launch_conv_t<128>(g, P, X, dev, enc, s);
+    P.dsets = (choice != 1 && two) ? 2 : 1;
+#if defined(TWN_PROFILE) || defined(TWN_TUNE)
+    if (const char *force = getenv("TWN_DSETS")) P.dsets = atoi(force) == 2 ? 2 : 1;
+#endif
+    if (choice == 1) return launch_conv_t<256, 1>(g, P, X, dev, enc, s);
+    if (choice == 2) return P.dsets == 2 ? launch_conv_t<192, 2>(g, P, X, dev, enc, s) : launch_conv_t<192, 1>(g, P, X, dev, enc, s);
+    return P.dsets == 2 ? launch_conv_t<128, 2>(g, P, X, dev, enc, s) : launch_conv_t<128, 1>(g, P, X, dev, enc, s);
 }
 
 // Helper streams for launches that are independent of one another (the residue classes of a
