@@ -319,6 +319,103 @@ maxpool_fwd_rows_kernel(const __nv_bfloat16 *__restrict__ X, int B, int H, int W
     }
 }
 
+// bit 7 of each byte of the result is set where that byte of t is zero (exact for every byte value)
+__device__ __forceinline__ uint32_t zero_bytes(uint32_t t)
+{
+    return ~(((t & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | t);
+}
+// bytes of the result, low to high: sign of byte s0 of z twice, sign of byte s1 twice (prmt's replicate mode)
+template <uint32_t SEL>
+__device__ __forceinline__ uint32_t pair_mask(uint32_t z)
+{
+    uint32_t m;
+    asm("prmt.b32 %0, %1, %1, %2;" : "=r"(m) : "r"(z), "r"(SEL));
+    return m;
+}
+// g += the bf16 values of d whose arg-max byte equals the tap (want4 = the tap in all four bytes)
+__device__ __forceinline__ void add_matching(float (&g)[8], const uint2 a, const uint4 d, uint32_t want4)
+{
+    const uint32_t zx = zero_bytes(a.x ^ want4), zy = zero_bytes(a.y ^ want4);
+    const uint32_t v0 = d.x & pair_mask<0x9988u>(zx), v1 = d.y & pair_mask<0xBBAAu>(zx);
+    const uint32_t v2 = d.z & pair_mask<0x9988u>(zy), v3 = d.w & pair_mask<0xBBAAu>(zy);
+    g[0] += __uint_as_float(v0 << 16); g[1] += __uint_as_float(v0 & 0xFFFF0000u);
+    g[2] += __uint_as_float(v1 << 16); g[3] += __uint_as_float(v1 & 0xFFFF0000u);
+    g[4] += __uint_as_float(v2 << 16); g[5] += __uint_as_float(v2 & 0xFFFF0000u);
+    g[6] += __uint_as_float(v3 << 16); g[7] += __uint_as_float(v3 & 0xFFFF0000u);
+}
+// 0xFFFF in each half whose bf16 value is greater than zero (false for NaN)
+__device__ __forceinline__ uint32_t positive_mask(uint32_t pair)
+{
+    const __nv_bfloat162 p = *reinterpret_cast<const __nv_bfloat162 *>(&pair);
+    return __hgt2_mask(p, __float2bfloat162_rn(0.0f));
+}
+
+// k = 3, stride 2, pad 1.  An even input row (column) lies in one window, at tap 1; an odd one in
+// two, at tap 2 of the window before and tap 0 of the window after.  One thread takes a 2 x 2 block
+// of input pixels (8 channels): the four windows around it are loaded once, gated once, and feed
+// 1 + 2 + 2 + 4 pixel-window pairs with no divergence.
+__global__ void __launch_bounds__(kT)
+maxpool_bwd_k3s2_kernel(const __nv_bfloat16 *__restrict__ dY, const uint8_t *__restrict__ idx, int B, int H, int W,
+                        int C, int Ho, int Wo, __nv_bfloat16 *__restrict__ dX,
+                        const __nv_bfloat16 *__restrict__ pooled, const float *__restrict__ scale)
+{
+    const int Cv = C >> 3, Hb = (H + 1) >> 1, Wb = (W + 1) >> 1;
+    const int items = B * Hb * Wb * Cv;
+    for (int it = blockIdx.x * kT + threadIdx.x; it < items; it += gridDim.x * kT) {
+        int t = it / Cv;
+        const int cv = it - t * Cv;
+        const int i = t % Wb;
+        t /= Wb;
+        const int j = t % Hb, b = t / Hb;
+        uint2 a[4];
+        uint4 d[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int ho = j + (q >> 1), wo = i + (q & 1);
+            const bool ok = ho < Ho && wo < Wo;
+            const size_t o = ok ? ((size_t)(b * Ho + ho) * Wo + wo) * C + cv * 8 : 0;
+            // an absent window's 0xFF bytes match no tap
+            a[q] = ok ? __ldg(reinterpret_cast<const uint2 *>(idx + o)) : make_uint2(0xFFFFFFFFu, 0xFFFFFFFFu);
+            d[q] = ok ? __ldg(reinterpret_cast<const uint4 *>(dY + o)) : make_uint4(0u, 0u, 0u, 0u);
+            if (pooled) {
+                const uint4 pl = ok ? __ldg(reinterpret_cast<const uint4 *>(pooled + o)) : make_uint4(0u, 0u, 0u, 0u);
+                d[q].x &= positive_mask(pl.x); d[q].y &= positive_mask(pl.y);
+                d[q].z &= positive_mask(pl.z); d[q].w &= positive_mask(pl.w);
+            }
+        }
+        float4 s0 = make_float4(1.0f, 1.0f, 1.0f, 1.0f), s1 = s0;
+        if (scale) {
+            s0 = __ldg(reinterpret_cast<const float4 *>(scale + cv * 8));
+            s1 = __ldg(reinterpret_cast<const float4 *>(scale + cv * 8 + 4));
+        }
+#pragma unroll
+        for (int pr = 0; pr < 2; ++pr) {
+#pragma unroll
+            for (int pc = 0; pc < 2; ++pc) {
+                const int h = 2 * j + pr, w = 2 * i + pc;
+                float g[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) g[e] = 0.0f;
+                // later windows first, as the general kernels add them
+#pragma unroll
+                for (int dj = pr; dj >= 0; --dj) {
+#pragma unroll
+                    for (int di = pc; di >= 0; --di) {
+                        const int r = pr == 0 ? 1 : (dj == 0 ? 2 : 0), sx = pc == 0 ? 1 : (di == 0 ? 2 : 0);
+                        add_matching(g, a[dj * 2 + di], d[dj * 2 + di], (uint32_t)(r * 3 + sx) * 0x01010101u);
+                    }
+                }
+                if (scale) {
+                    g[0] *= s0.x; g[1] *= s0.y; g[2] *= s0.z; g[3] *= s0.w;
+                    g[4] *= s1.x; g[5] *= s1.y; g[6] *= s1.z; g[7] *= s1.w;
+                }
+                if (h < H && w < W)
+                    *reinterpret_cast<uint4 *>(dX + ((size_t)(b * H + h) * W + w) * C + cv * 8) = pack8(g);
+            }
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kT)
 maxpool_bwd_rows_kernel(const __nv_bfloat16 *__restrict__ dY, const uint8_t *__restrict__ idx, int B, int H, int W,
                         int C, int k, int stride, int lg_stride, int pad, int Ho, int Wo,
@@ -646,7 +743,12 @@ int maxpool_bwd_launch(const void *dY, const uint8_t *argmax, const void *pooled
     const bool vec = C % 8 == 0 && twn_aligned(dY, 16) && twn_aligned(dX, 16) && twn_aligned(argmax, 8) &&
                      twn_aligned(pooled_v, 16) && twn_aligned(scale, 16);
     cudaStream_t s = twn_cu(stream);
-    if (vec && small) {
+    if (vec && small && k == 3 && stride == 2 && pad == 1) {
+        const long long items = B * ((H + 1) / 2) * ((W + 1) / 2) * (C / 8);
+        maxpool_bwd_k3s2_kernel<<<blocks_for(items, dev.sm_count * 4), kT, 0, s>>>(
+            dy, argmax, (int)B, (int)H, (int)W, (int)C, (int)Ho, (int)Wo, dx, pooled, scale);
+    }
+    else if (vec && small) {
         const long long rows = B * H;
         const int grid = (int)(rows < dev.sm_count * 16LL ? rows : dev.sm_count * 16LL);
         int lg = -1;
