@@ -249,72 +249,102 @@ maxpool_bwd_kernel(const __nv_bfloat16 *__restrict__ dY, const uint8_t *__restri
     }
 }
 
-// Row variants of the two pooling kernels for the common case (8 channels per thread, 32-bit
-// indices): a block walks whole image rows, so a thread needs one integer division instead of
-// ten, and a power-of-two stride turns the window search of the backward pass into shifts.  These
-// sweeps are otherwise bound by their index arithmetic, not by memory.
+// 0xFFFF in each half where the bf16 value of a is greater than (equal to) that of b; false for NaN
+__device__ __forceinline__ uint32_t greater_mask(uint32_t a, uint32_t b)
+{
+    return __hgt2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&a), *reinterpret_cast<const __nv_bfloat162 *>(&b));
+}
+__device__ __forceinline__ uint32_t equal_mask(uint32_t a, uint32_t b)
+{
+    return __heq2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&a), *reinterpret_cast<const __nv_bfloat162 *>(&b));
+}
+
+// Variants of the two pooling kernels for the common case (8 channels per thread, 32-bit
+// indices).  The forward one takes one window per thread over the flat index; in the backward one
+// a block walks whole image rows, and a power-of-two stride turns the window search into shifts.
+// These sweeps are otherwise bound by their index arithmetic, not by memory.
 __global__ void __launch_bounds__(kT)
-maxpool_fwd_rows_kernel(const __nv_bfloat16 *__restrict__ X, int B, int H, int W, int C, int k, int stride, int pad,
+maxpool_fwd_vec_kernel(const __nv_bfloat16 *__restrict__ X, int B, int H, int W, int C, int k, int stride, int pad,
                         int Ho, int Wo, __nv_bfloat16 *__restrict__ Y, uint8_t *__restrict__ idx)
 {
-    const int Cv = C >> 3, per_row = Wo * Cv;
-    for (int row = blockIdx.x; row < B * Ho; row += gridDim.x) {
+    const int Cv = C >> 3, per_row = Wo * Cv, total = B * Ho * per_row;
+    // one window (8 channels) per thread over the flat index: every block has the same work
+    for (int it = blockIdx.x * kT + threadIdx.x; it < total; it += gridDim.x * kT) {
+        const int row = it / per_row, i = it - row * per_row;
         const int b = row / Ho, ho = row - b * Ho;
         const int h_lo = ho * stride - pad;
-        for (int i = threadIdx.x; i < per_row; i += kT) {
-            const int wo = i / Cv, cv = i - wo * Cv;
-            const int w_lo = wo * stride - pad;
-            float best[8];
-            int arg[8];
+        const int wo = i / Cv, cv = i - wo * Cv;
+        const int w_lo = wo * stride - pad;
+        float best[8];
+        int arg[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) { best[e] = -INFINITY; arg[e] = 0; }
-            if (k <= 3) {
-                // all (up to nine) window elements are requested before the first comparison, so
-                // their latencies overlap; an element outside the image reads as -inf and never wins
-                uint4 v[9];
+        for (int e = 0; e < 8; ++e) { best[e] = -INFINITY; arg[e] = 0; }
+        if (k <= 3) {
+            // all (up to nine) window elements are requested before the first comparison, so
+            // their latencies overlap; an element outside the image reads as -inf and never wins
+            uint4 v[9];
 #pragma unroll
-                for (int q = 0; q < 9; ++q) {
-                    const int r = q / 3, sx = q - 3 * r;
-                    const int h = h_lo + r, w = w_lo + sx;
-                    const bool ok = r < k && sx < k && h >= 0 && h < H && w >= 0 && w < W;
-                    v[q] = ok ? __ldg(reinterpret_cast<const uint4 *>(X + ((size_t)(b * H + h) * W + w) * C + cv * 8))
-                              : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);   // bf16 -inf
-                }
+            for (int q = 0; q < 9; ++q) {
+                const int r = q / 3, sx = q - 3 * r;
+                const int h = h_lo + r, w = w_lo + sx;
+                const bool ok = r < k && sx < k && h >= 0 && h < H && w >= 0 && w < W;
+                v[q] = ok ? __ldg(reinterpret_cast<const uint4 *>(X + ((size_t)(b * H + h) * W + w) * C + cv * 8))
+                          : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);   // bf16 -inf
+            }
+            // two channels per register: the comparison yields a mask per bf16 half, and the
+            // maximum and its tap (16 bits each until the end) are selected with it
+            uint32_t bp[4], ap[4];
 #pragma unroll
-                for (int q = 0; q < 9; ++q) {
-                    const int r = q / 3, sx = q - 3 * r;
-                    float x[8];
-                    unpack8(v[q], x);
+            for (int p = 0; p < 4; ++p) { bp[p] = 0xFF80FF80u; ap[p] = 0u; }
 #pragma unroll
-                    for (int e = 0; e < 8; ++e)
-                        if (x[e] > best[e]) { best[e] = x[e]; arg[e] = r * k + sx; }
-                }
-            } else
-            for (int r = 0; r < k; ++r) {
-                const int h = h_lo + r;
-                if (h < 0 || h >= H) continue;
-                const __nv_bfloat16 *rowp = X + ((size_t)(b * H + h) * W) * C + cv * 8;
-                for (int sx = 0; sx < k; ++sx) {
-                    const int w = w_lo + sx;
-                    if (w < 0 || w >= W) continue;
-                    float x[8];
-                    unpack8(__ldg(reinterpret_cast<const uint4 *>(rowp + (size_t)w * C)), x);
+            for (int q = 0; q < 9; ++q) {
+                const int r = q / 3, sx = q - 3 * r;
+                const uint32_t tap2 = (uint32_t)(r * k + sx) * 0x00010001u;
+                const uint32_t x4[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
 #pragma unroll
-                    for (int e = 0; e < 8; ++e)
-                        if (x[e] > best[e]) { best[e] = x[e]; arg[e] = r * k + sx; }
+                for (int p = 0; p < 4; ++p) {
+                    const uint32_t m = greater_mask(x4[p], bp[p]);      // false for NaN, as x > best is
+                    bp[p] = (x4[p] & m) | (bp[p] & ~m);
+                    ap[p] = (tap2 & m) | (ap[p] & ~m);
                 }
             }
-            const size_t o = ((size_t)row * Wo + wo) * C + cv * 8;
-            float t8[8];
+            // a maximum still at -inf is written as zero
 #pragma unroll
-            for (int e = 0; e < 8; ++e) t8[e] = best[e] == -INFINITY ? 0.0f : best[e];
-            *reinterpret_cast<uint4 *>(Y + o) = pack8(t8);     // exact: the values are bf16 already
+            for (int p = 0; p < 4; ++p) bp[p] &= ~equal_mask(bp[p], 0xFF80FF80u);
+            const size_t o = ((size_t)row * Wo + wo) * C + cv * 8;
+            *reinterpret_cast<uint4 *>(Y + o) = make_uint4(bp[0], bp[1], bp[2], bp[3]);
             if (idx) {
-                uint2 a;
-                a.x = arg[0] | (arg[1] << 8) | (arg[2] << 16) | (arg[3] << 24);
-                a.y = arg[4] | (arg[5] << 8) | (arg[6] << 16) | (arg[7] << 24);
+                uint2 a;        // the low byte of each 16-bit tap
+                asm("prmt.b32 %0, %1, %2, 0x6420;" : "=r"(a.x) : "r"(ap[0]), "r"(ap[1]));
+                asm("prmt.b32 %0, %1, %2, 0x6420;" : "=r"(a.y) : "r"(ap[2]), "r"(ap[3]));
                 *reinterpret_cast<uint2 *>(idx + o) = a;
             }
+            continue;
+        } else
+        for (int r = 0; r < k; ++r) {
+            const int h = h_lo + r;
+            if (h < 0 || h >= H) continue;
+            const __nv_bfloat16 *rowp = X + ((size_t)(b * H + h) * W) * C + cv * 8;
+            for (int sx = 0; sx < k; ++sx) {
+                const int w = w_lo + sx;
+                if (w < 0 || w >= W) continue;
+                float x[8];
+                unpack8(__ldg(reinterpret_cast<const uint4 *>(rowp + (size_t)w * C)), x);
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                    if (x[e] > best[e]) { best[e] = x[e]; arg[e] = r * k + sx; }
+            }
+        }
+        const size_t o = ((size_t)row * Wo + wo) * C + cv * 8;
+        float t8[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) t8[e] = best[e] == -INFINITY ? 0.0f : best[e];
+        *reinterpret_cast<uint4 *>(Y + o) = pack8(t8);     // exact: the values are bf16 already
+        if (idx) {
+            uint2 a;
+            a.x = arg[0] | (arg[1] << 8) | (arg[2] << 16) | (arg[3] << 24);
+            a.y = arg[4] | (arg[5] << 8) | (arg[6] << 16) | (arg[7] << 24);
+            *reinterpret_cast<uint2 *>(idx + o) = a;
         }
     }
 }
@@ -346,8 +376,7 @@ __device__ __forceinline__ void add_matching(float (&g)[8], const uint2 a, const
 // 0xFFFF in each half whose bf16 value is greater than zero (false for NaN)
 __device__ __forceinline__ uint32_t positive_mask(uint32_t pair)
 {
-    const __nv_bfloat162 p = *reinterpret_cast<const __nv_bfloat162 *>(&pair);
-    return __hgt2_mask(p, __float2bfloat162_rn(0.0f));
+    return greater_mask(pair, 0u);
 }
 
 // k = 3, stride 2, pad 1.  An even input row (column) lies in one window, at tap 1; an odd one in
@@ -709,9 +738,7 @@ extern "C" int twn_maxpool2d_fwd(const void *X, int64_t B, int64_t H, int64_t W,
     const bool vec = C % 8 == 0 && twn_aligned(X, 16) && twn_aligned(Y, 16) && twn_aligned(argmax, 8);
     cudaStream_t s = twn_cu(stream);
     if (vec && small) {
-        const long long rows = B * Ho;
-        const int grid = (int)(rows < dev.sm_count * 16LL ? rows : dev.sm_count * 16LL);
-        maxpool_fwd_rows_kernel<<<grid, kT, 0, s>>>(x, (int)B, (int)H, (int)W, (int)C, k, stride, pad, (int)Ho, (int)Wo,
+        maxpool_fwd_vec_kernel<<<blocks_for(B * Ho * Wo * (C / 8), dev.sm_count * 4), kT, 0, s>>>(x, (int)B, (int)H, (int)W, (int)C, k, stride, pad, (int)Ho, (int)Wo,
                                                     y, argmax);
     }
     else if (vec)
