@@ -556,24 +556,33 @@ maxpool_bwd_rows_kernel(const __nv_bfloat16 *__restrict__ dY, const uint8_t *__r
 // the 2 x 2 pixel block at (2i - pad_h, 2j - pad_w) becomes the 4*Cin <= 16 channels of folded
 // pixel (i, j), so that the stride-2 k x k layer is a stride-1 ceil(k/2) x ceil(k/2) layer and the
 // four folded pixels a filter row touches are 64 consecutive bf16 (one tensor-core k-block).
+// CIN > 0 fixes the channel count at compile time (the 16 values then stay in registers)
+template <int CIN>
 __global__ void __launch_bounds__(kT)
-fold_input_kernel(const __nv_bfloat16 *__restrict__ X, int B, int H, int W, int Cin, int pad_h, int pad_w, int Hf,
+fold_input_kernel(const __nv_bfloat16 *__restrict__ X, int B, int H, int W, int Cin_rt, int pad_h, int pad_w, int Hf,
                   int Wf, __nv_bfloat16 *__restrict__ Xf)
 {
+    const int Cin = CIN > 0 ? CIN : Cin_rt;
     const int total = B * Hf * Wf;
     for (int p = blockIdx.x * kT + threadIdx.x; p < total; p += gridDim.x * kT) {
         const int j = p % Wf, t = p / Wf, i = t % Hf, b = t / Hf;
         __align__(16) __nv_bfloat16 v[16];
 #pragma unroll
         for (int e = 0; e < 16; ++e) v[e] = __float2bfloat16_rn(0.0f);
+#pragma unroll
         for (int dy = 0; dy < 2; ++dy) {
             const int h = 2 * i + dy - pad_h;
-            if (h < 0 || h >= H) continue;
+#pragma unroll
             for (int dx = 0; dx < 2; ++dx) {
                 const int w = 2 * j + dx - pad_w;
-                if (w < 0 || w >= W) continue;
+                if (h < 0 || h >= H || w < 0 || w >= W) continue;
                 const __nv_bfloat16 *src = X + ((size_t)(b * H + h) * W + w) * Cin;
-                for (int c = 0; c < Cin; ++c) v[(dy * 2 + dx) * Cin + c] = src[c];
+                if (CIN > 0) {
+#pragma unroll
+                    for (int c = 0; c < CIN; ++c) v[(dy * 2 + dx) * CIN + c] = src[c];
+                } else {
+                    for (int c = 0; c < Cin; ++c) v[(dy * 2 + dx) * Cin + c] = src[c];
+                }
             }
         }
         uint4 *dst = reinterpret_cast<uint4 *>(Xf + (size_t)p * 16);
@@ -605,6 +614,53 @@ avgpool_bwd_kernel(const __nv_bfloat16 *__restrict__ dY, long long B, long long 
     for (long long i = (long long)blockIdx.x * kT + threadIdx.x; i < total; i += (long long)gridDim.x * kT) {
         const long long c = i % C, b = i / (C * HW);
         dX[i] = __float2bfloat16_rn(__bfloat162float(dY[b * C + c]) * inv);
+    }
+}
+
+// 8 channels per thread (C a multiple of 8, 32-bit indices).  Forward: a block takes 32 channel
+// groups of one image, its 8 warps share the pixels, the partial sums meet in shared memory in a
+// fixed order.  Backward: one 16-byte store per thread.
+__global__ void __launch_bounds__(kT)
+avgpool_fwd_vec_kernel(const __nv_bfloat16 *__restrict__ X, int HW, int C, int groups, __nv_bfloat16 *__restrict__ Y)
+{
+    __shared__ float part[kT / 32][32][9];
+    const int Cv = C >> 3, b = blockIdx.x / groups, cv = (blockIdx.x - b * groups) * 32 + (threadIdx.x & 31);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float s[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) s[e] = 0.0f;
+    if (cv < Cv)
+        for (int p = warp; p < HW; p += kT / 32) {
+            float x[8];
+            unpack8(__ldg(reinterpret_cast<const uint4 *>(X + ((size_t)b * HW + p) * C + cv * 8)), x);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) s[e] += x[e];
+        }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) part[warp][lane][e] = s[e];
+    __syncthreads();
+    const int col = threadIdx.x & 31, e = threadIdx.x >> 5;     // 256 threads = 32 groups x 8 channels
+    const int c = ((blockIdx.x - b * groups) * 32 + col) * 8 + e;
+    if (c < C) {
+        float t = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kT / 32; ++w) t += part[w][col][e];
+        Y[(size_t)b * C + c] = __float2bfloat16_rn(t / (float)HW);
+    }
+}
+
+__global__ void __launch_bounds__(kT)
+avgpool_bwd_vec_kernel(const __nv_bfloat16 *__restrict__ dY, int total, int HW, int C, __nv_bfloat16 *__restrict__ dX)
+{
+    const int Cv = C >> 3;
+    const float inv = 1.0f / (float)HW;
+    for (int i = blockIdx.x * kT + threadIdx.x; i < total; i += gridDim.x * kT) {
+        const int pix = i / Cv, cv = i - pix * Cv, b = pix / HW;
+        float g[8];
+        unpack8(__ldg(reinterpret_cast<const uint4 *>(dY + (size_t)b * C + cv * 8)), g);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) g[e] *= inv;
+        *reinterpret_cast<uint4 *>(dX + (size_t)i * 8) = pack8(g);
     }
 }
 
@@ -715,9 +771,15 @@ extern "C" int twn_fold_input(const twn_conv_desc_t *d, const void *X, void *Xf,
     twn_device_info dev;
     rc = twn_current_device(&dev);
     if (rc != TWN_OK) return rc;
-    fold_input_kernel<<<blocks_for(d->B * Hf * Wf, dev.sm_count), kT, 0, twn_cu(stream)>>>(
-        static_cast<const __nv_bfloat16 *>(X), (int)d->B, (int)d->H, (int)d->W, (int)d->Cin, d->pad_h, d->pad_w, (int)Hf,
-        (int)Wf, static_cast<__nv_bfloat16 *>(Xf));
+    const int grid = blocks_for(d->B * Hf * Wf, dev.sm_count * 4);
+    if (d->Cin == 3)
+        fold_input_kernel<3><<<grid, kT, 0, twn_cu(stream)>>>(
+            static_cast<const __nv_bfloat16 *>(X), (int)d->B, (int)d->H, (int)d->W, 3, d->pad_h, d->pad_w, (int)Hf,
+            (int)Wf, static_cast<__nv_bfloat16 *>(Xf));
+    else
+        fold_input_kernel<0><<<grid, kT, 0, twn_cu(stream)>>>(
+            static_cast<const __nv_bfloat16 *>(X), (int)d->B, (int)d->H, (int)d->W, (int)d->Cin, d->pad_h, d->pad_w,
+            (int)Hf, (int)Wf, static_cast<__nv_bfloat16 *>(Xf));
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }
@@ -816,8 +878,13 @@ extern "C" int twn_avgpool_fwd(const void *X, int64_t B, int64_t HW, int64_t C, 
     twn_device_info dev;
     const int rc = twn_current_device(&dev);
     if (rc != TWN_OK) return rc;
-    avgpool_fwd_kernel<<<blocks_for(B * C, dev.sm_count), kT, 0, twn_cu(stream)>>>(
-        static_cast<const __nv_bfloat16 *>(X), B, HW, C, static_cast<__nv_bfloat16 *>(Y));
+    const long long groups = (C / 8 + 31) / 32;
+    if (C % 8 == 0 && twn_aligned(X, 16) && B * HW * C < 0x7fffffffLL && B * groups < 0x7fffffffLL)
+        avgpool_fwd_vec_kernel<<<(int)(B * groups), kT, 0, twn_cu(stream)>>>(
+            static_cast<const __nv_bfloat16 *>(X), (int)HW, (int)C, (int)groups, static_cast<__nv_bfloat16 *>(Y));
+    else
+        avgpool_fwd_kernel<<<blocks_for(B * C, dev.sm_count), kT, 0, twn_cu(stream)>>>(
+            static_cast<const __nv_bfloat16 *>(X), B, HW, C, static_cast<__nv_bfloat16 *>(Y));
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }
@@ -828,8 +895,13 @@ extern "C" int twn_avgpool_bwd(const void *dY, int64_t B, int64_t HW, int64_t C,
     twn_device_info dev;
     const int rc = twn_current_device(&dev);
     if (rc != TWN_OK) return rc;
-    avgpool_bwd_kernel<<<blocks_for(B * HW * C, dev.sm_count), kT, 0, twn_cu(stream)>>>(
-        static_cast<const __nv_bfloat16 *>(dY), B, HW, C, static_cast<__nv_bfloat16 *>(dX));
+    if (C % 8 == 0 && twn_aligned(dY, 16) && twn_aligned(dX, 16) && B * HW * C < 0x7fffffffLL)
+        avgpool_bwd_vec_kernel<<<blocks_for(B * HW * C / 8, dev.sm_count), kT, 0, twn_cu(stream)>>>(
+            static_cast<const __nv_bfloat16 *>(dY), (int)(B * HW * C / 8), (int)HW, (int)C,
+            static_cast<__nv_bfloat16 *>(dX));
+    else
+        avgpool_bwd_kernel<<<blocks_for(B * HW * C, dev.sm_count), kT, 0, twn_cu(stream)>>>(
+            static_cast<const __nv_bfloat16 *>(dY), B, HW, C, static_cast<__nv_bfloat16 *>(dX));
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }

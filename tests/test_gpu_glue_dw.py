@@ -197,8 +197,8 @@ def test_maxpool_forward_and_backward(k, s, p, H, W, C):
     assert np.all(np.abs(gotz - dzr) <= 2.0 ** -8 * np.abs(dzr) + 1e-30)
 
 
-def test_avgpool_and_activation_backward():
-    B, H, W, C = 4, 7, 7, 512
+@pytest.mark.parametrize("B,H,W,C", [(4, 7, 7, 512), (3, 5, 4, 320), (2, 3, 3, 20)])
+def test_avgpool_and_activation_backward(B, H, W, C):
     xb = dg.draw_bf16(4, "ap", B * H * W * C, "normal").reshape(B, H, W, C)
     Y = torch.empty((B, C), dtype=torch.bfloat16, device="cuda")
     twn.avgpool_fwd(dev_bf16(xb), B, H * W, C, Y)
