@@ -168,7 +168,7 @@ def test_fold_rejects_layers_it_cannot_take():
 
 
 @pytest.mark.parametrize("k,s,p,H,W,C", [(2, 2, 0, 24, 24, 32), (3, 2, 1, 112, 112, 8), (3, 2, 1, 7, 9, 5), (2, 2, 0, 8, 8, 512),
-                                          (3, 2, 1, 7, 9, 16), (3, 2, 1, 10, 13, 64), (3, 2, 1, 1, 1, 8), (3, 1, 1, 9, 6, 16)])
+                                          (3, 2, 1, 7, 9, 16), (3, 2, 1, 10, 13, 64), (3, 2, 1, 1, 1, 8), (3, 1, 1, 9, 6, 16), (3, 2, 1, 112, 112, 64)])
 def test_maxpool_forward_and_backward(k, s, p, H, W, C):
     B = 2
     xb = dg.draw_bf16(3, f"mp{H}{C}", B * H * W * C, "normal").reshape(B, H, W, C)
