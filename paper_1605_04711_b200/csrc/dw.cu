@@ -20,19 +20,6 @@
 #include "common.cuh"
 #include "tc_ptx.cuh"
 
-// Optional cycle counters (compiled in with -DTWN_PROFILE, read back with twn_dwprof_read).
-#ifdef TWN_PROFILE
-__device__ long long g_dwprof[256 * 8];
-#define DWPROF_DECL(v) long long v = 0
-#define DWPROF_T(v) const long long v = clock64()
-#define DWPROF_ACC(acc, t0) acc += clock64() - (t0)
-#define DWPROF_OUT(slot, val) g_dwprof[blockIdx.x * 8 + (slot)] = (val)
-#else
-#define DWPROF_DECL(v)
-#define DWPROF_T(v)
-#define DWPROF_ACC(acc, t0)
-#define DWPROF_OUT(slot, val)
-#endif
 
 namespace {
 
@@ -174,26 +161,20 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
     } else if (warp == 1) {
         uint32_t it = 0, lu = 0;     // lu counts the units that accumulate something
         bool ok = true;
-        DWPROF_DECL(w_full); DWPROF_DECL(w_acc);
-        DWPROF_T(t_all);
         for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
             int ot, gi, nb, sp, p0, p1;
             unit_range(u, ot, gi, nb, sp, p0, p1);
             if (p1 <= p0) continue;                      // the epilogue writes zeros for an empty split
             const uint32_t idesc = make_idesc_mn(128, 64 * nb);
             const int buf = lu & 1;
-            DWPROF_T(t_a);
             if (!mbar_wait_warp(&sm->acc_empty[buf], ((lu >> 1) & 1u) ^ 1u, abort_flag, P.status, 0)) break;
-            DWPROF_ACC(w_acc, t_a);
             tc_fence_after();
             const uint32_t d_tmem = tmem + buf * kDwAccCols;
             int s = it % P.stages;
             uint32_t ph = (it / P.stages) & 1u;
             for (int p = p0; p < p1; ++p, ++it) {
                 const uint32_t st = smem_u32(sm->pool) + s * P.stage_bytes;
-                DWPROF_T(t_f);
                 if (!mbar_wait_warp(&sm->full[s], ph, abort_flag, P.status, 0)) { ok = false; break; }
-                DWPROF_ACC(w_full, t_f);
                 tc_fence_after();
                 const uint64_t adesc = smem_desc_mn_sw128(st, kDwBlockBytes);
                 // 16 pixels per MMA = 16 rows of 128 bytes = 2048 bytes
@@ -222,18 +203,15 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
             if (ok) tc_commit(&sm->acc_full[buf]);
             ++lu;
         }
-        if (lane == 0) { DWPROF_OUT(0, clock64() - t_all); DWPROF_OUT(1, w_full); DWPROF_OUT(2, w_acc); DWPROF_OUT(3, (long long)it); DWPROF_OUT(4, (long long)lu); }
     } else {
         const int q = warp & 3;
         uint32_t lu = 0;
-        DWPROF_DECL(e_busy);
         for (int u = blockIdx.x; u < P.total_units; u += gridDim.x) {
             int ot, gi, nb, sp, p0, p1;
             unit_range(u, ot, gi, nb, sp, p0, p1);
             const bool have = p1 > p0;
             const int buf = lu & 1;
             if (have && !mbar_wait_warp(&sm->acc_full[buf], (lu >> 1) & 1u, abort_flag, P.status, 32)) break;
-            DWPROF_T(t_e);
             tc_fence_after();
             const int o = ot * 128 + q * 32 + lane;
             float *row = P.partial + (long long)sp * P.split_stride + (long long)o * P.K;
@@ -293,9 +271,7 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
                 if (lane == 0) mbar_arrive(&sm->acc_empty[buf]);
                 ++lu;
             }
-            DWPROF_ACC(e_busy, t_e);
         }
-        if (warp == 2 && lane == 0) DWPROF_OUT(5, e_busy);
     }
 
     tc_fence_before();
@@ -571,6 +547,3 @@ extern "C" int twn_conv2d_bwd_weight_folded(const twn_conv_desc_t *d, const void
     return TWN_OK;
 }
 
-#ifdef TWN_PROFILE
-extern "C" int twn_dwprof_read(long long *host) { return cudaMemcpyFromSymbol(host, g_dwprof, sizeof(long long) * 256 * 8); }
-#endif

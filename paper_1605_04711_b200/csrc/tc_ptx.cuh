@@ -12,10 +12,7 @@
 namespace {
 
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;
-#ifndef TWN_CONVERGED_TRIES
-#define TWN_CONVERGED_TRIES 16
-#endif
-constexpr int kConvergedTries = TWN_CONVERGED_TRIES;   // warp-wide blocking probes before a single lane takes over
+constexpr int kConvergedTries = 16;   // warp-wide blocking probes before a single lane takes over
 
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -121,14 +118,6 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap *map, const void 
         : "memory");
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
-// named barrier of the four warps of an epilogue group
-__device__ __forceinline__ void epi_bar(int set)
-{
-    // immediate barrier numbers: a register operand would make the compiler reserve all sixteen
-    if (set == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
-    else asm volatile("bar.sync 2, 128;" ::: "memory");
-}
-
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 

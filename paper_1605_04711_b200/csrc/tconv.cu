@@ -16,18 +16,25 @@
 // owns one channel, so alpha, the per-channel affine and ReLU cost one register each,
 // and a warp's store of one pixel covers 32 consecutive channels (128 contiguous bytes).
 //
-//   warp 0        TMA producer: activation tile per k-block
-//   warp 1        allocates tensor memory, issues tcgen05.mma, commits to mbarriers
-//   warps 2-9     decode: packed codes (global, L2) -> bf16 pairs -> tensor memory
-//   warps 10-13   epilogue: tensor memory -> registers -> global
+//   warp 0            TMA producer: one activation tile per k-block
+//   warp 1            allocates tensor memory, issues tcgen05.mma, commits to mbarriers
+//   warps 2-5 (2-9)   decode: packed codes (global, L2) -> bf16 pairs -> tensor memory; one group
+//                     of four warps (one per lane quadrant), or two groups that take the stages
+//                     in turn (template parameter DS)
+//   last eight warps  epilogue, two per lane quadrant: tensor memory -> registers -> per-warp
+//                     staging buffer -> TMA store
 //
-// Two tile shapes.  Measured on B200: one thread can issue a tcgen05.mma about every
-// 50-90 cycles whatever its size, and waits or commits between MMAs are not hidden
-// unless the MMA itself is long.  A 128x256x16 MMA (128 cycles) hides that; a 128x128x16
-// one (64 cycles) does not.  So the large shape uses 256-pixel tiles with a single
-// accumulator (tensor memory holds 512 columns: 256 for it, the rest for the decoded
-// weights), and the epilogue of a tile is not overlapped with the next tile's MMAs.
-// Small problems use 128-pixel tiles, two accumulators and two k-blocks per stage.
+// Three tile shapes (template parameter PIX = pixels per tile; the channel tile is always 128).
+// Measured on B200: one thread can issue a tcgen05.mma about every 50-90 cycles whatever its
+// size, and waits or commits between MMAs are not hidden unless the MMA itself is long.  A
+// 128x256x16 MMA (128 cycles) hides that; a 128x128x16 one (64 cycles) does not.
+//   PIX = 256: one accumulator (256 of the 512 tensor-memory columns, the rest holds decoded
+//              weights), five stages; the epilogue of a tile is not overlapped with the next
+//              tile's MMAs.  Long reductions with many tiles.
+//   PIX = 192: two accumulators and four stages fill the tensor memory exactly; the epilogue
+//              overlaps the next tile.
+//   PIX = 128: two accumulators, four stages of two k-blocks each.  Small problems.
+// The host picks the shape and the number of decode groups per launch with a cost model.
 //
 // Every wait on an mbarrier is bounded (about a second); on expiry the kernel records
 // TWN_ERR_TIMEOUT, all roles leave their loops, tensor memory is freed and the grid exits.
@@ -36,33 +43,11 @@
 
 #include <cstddef>
 
-#include "common.cuh"
-#include <cstdlib>
 #include <mutex>
+
+#include "common.cuh"
 #include "tc_ptx.cuh"
 
-// Optional cycle counters per role (compiled in with -DTWN_PROFILE, read back with
-// twn_prof_read; absent from the normal build).
-#ifdef TWN_PROFILE
-__device__ long long g_prof[256 * 32];
-__device__ long long g_tl2[4 * 1024];  // block 0, first decode warp: [0] slot free seen, [1] stores issued, [2] arrived, [3] next codes fetched
-#define PROF_TL2(row, it) do { if (blockIdx.x == 0 && warp == 2 && lane == 0 && (it) < 1024) g_tl2[(row) * 1024 + (it)] = clock64(); } while (0)
-__device__ long long g_tl[4 * 1024];   // block 0: [0] TMA issue, [1] X seen by MMA, [2] A ready seen, [3] commit, per stage
-#define PROF_TL(row, it) do { if (blockIdx.x == 0 && (it) < 1024) g_tl[(row) * 1024 + (it)] = clock64(); } while (0)
-#define PROF_DECL(v) long long v = 0
-#define PROF_NOW() clock64()
-#define PROF_T(v) const long long v = clock64()
-#define PROF_ACC(acc, t0) acc += clock64() - (t0)
-#define PROF_OUT(slot, val) g_prof[blockIdx.x * 32 + (slot)] = (val)
-#else
-#define PROF_TL(row, it)
-#define PROF_TL2(row, it)
-#define PROF_DECL(v)
-#define PROF_NOW() 0
-#define PROF_T(v)
-#define PROF_ACC(acc, t0)
-#define PROF_OUT(slot, val)
-#endif
 
 namespace {
 
@@ -226,7 +211,6 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            PROF_DECL(w_empty);
             const uint32_t block_bytes = kXBytes;
             for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x) {
                 int pt = tile / P.n_tiles;
@@ -241,10 +225,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
                     const int nsb = (kbpt - st * kSub) < kSub ? (kbpt - st * kSub) : kSub;
-                    PROF_T(t_e);
                     if (!mbar_wait(&sm->empty[s], ph ^ 1u, abort_flag, P.status)) { ok = false; break; }
-                    PROF_ACC(w_empty, t_e);
-                    PROF_TL(0, it);
                     mbar_expect_tx(&sm->full[s], nsb * block_bytes);
                     for (int sb = 0; sb < nsb; ++sb) {
                         const Tap tap = P.taps[t];
@@ -253,7 +234,6 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     }
                 }
             }
-            PROF_OUT(5, w_empty);
         }
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer (whole warp, converged)
@@ -264,23 +244,16 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
             const uint64_t bdesc0 = smem_desc_sw128(smem_u32(sm->x[0][0]));
             uint32_t it = 0, lt = 0;
             bool ok = true;
-            PROF_DECL(w_acc); PROF_DECL(w_ready); PROF_DECL(w_issue);
-            PROF_T(t_start);
             for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x, ++lt) {
                 const int buf = lt % kAccBufs;
                 const uint32_t aph = (lt / kAccBufs) & 1u;
-                PROF_T(t_a);
                 if (!mbar_wait_warp(&sm->acc_empty[buf], aph ^ 1u, abort_flag, P.status, 0)) break;
-                PROF_ACC(w_acc, t_a);
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_acc + buf * PIX;
                 for (int st = 0; st < spt; ++st, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
-                    PROF_T(t_x);
                     if (!mbar_wait_warp(&sm->full[s], ph, abort_flag, P.status, 0)) { ok = false; break; }
-                    PROF_ACC(w_issue, t_x);
-                    if (lane == 0) PROF_TL(1, it);
                     tc_fence_after();
                     const uint64_t bdesc = bdesc0 + (uint64_t)(s * ((kSub * kXBytes) >> 4));
                     const uint32_t a_tmem = tmem_a + s * kAColsPerStage;
@@ -289,11 +262,9 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     if (kSub > 1 && kbpt - st * kSub > 1)
                         tc_mma_block<false>(d_tmem, a_tmem + kAColsPerBlock, bdesc + (kXBytes >> 4), idesc);
                     tc_commit(&sm->empty[s]);
-                    if (lane == 0) PROF_TL(3, it);
                 }
                 if (ok) tc_commit(&sm->acc_full[buf]);
             }
-            if (lane == 0) { PROF_OUT(0, PROF_NOW() - t_start); PROF_OUT(1, w_acc); PROF_OUT(2, w_issue); PROF_OUT(3, w_ready); PROF_OUT(4, (long long)it); }
         }
     } else if (warp < kFirstEpiWarp) {
         // ------------------------------------------------ decode: codes -> bf16 -> tensor memory
@@ -358,8 +329,6 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     rowp = row_ptr(nt);
                 }
         };
-        PROF_DECL(w_full); PROF_DECL(d_alu); PROF_DECL(d_wst); PROF_DECL(d_fetch); PROF_DECL(d_st);
-        PROF_T(t_dec);
         if (spt > 0) {
             // 256-pixel tiles: three code buffers in rotation, each refilled right after use for the
             // stage three of this group's stages ahead: no register is copied while its load is still
@@ -379,11 +348,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 const uint32_t ph = (it / kStages) & 1u;
                 const int nsb = (kbpt - st_c * kSub) < kSub ? (kbpt - st_c * kSub) : kSub;
                 // the MMAs that read this slot's previous contents have completed
-                PROF_T(t_f);
                 if (!mbar_wait_warp(&sm->empty[s], ph ^ 1u, abort_flag, P.status, 32)) return false;
-                PROF_ACC(w_full, t_f);
-                PROF_TL2(0, it);
-                PROF_T(t_alu);
                 tc_fence_after();
 #pragma unroll
                 for (int sb = 0; sb < kSub; ++sb) {
@@ -394,20 +359,13 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                         for (int g = 0; g < 4; ++g)
 #pragma unroll
                             for (int e = 0; e < 8; ++e) out[g * 8 + e] = pair_to_bf16x2(wv[g], e);
-                        PROF_T(t_st);
                         tmem_st32(lane_base + s * kAColsPerStage + sb * kAColsPerBlock, out);
-                        PROF_ACC(d_st, t_st);
                     }
                 }
-                PROF_ACC(d_alu, t_alu);
-                PROF_TL2(1, it);
-                PROF_T(t_wst);
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sm->full[s]);
-                PROF_ACC(d_wst, t_wst);
-                PROF_TL2(2, it);
                 advance(tile_c, st_c, dsets);
                 it += dsets;
                 return true;
@@ -416,11 +374,11 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 // long reductions, no slack for a late code word: three buffers in rotation
                 while (true) {
                     if (tile_c >= P.total_tiles || !decode_stage(c0)) break;
-                    { PROF_T(t0); fetch(c0, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, dsets); PROF_ACC(d_fetch, t0); PROF_TL2(3, it - dsets); }
+                    { fetch(c0, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, dsets); }
                     if (tile_c >= P.total_tiles || !decode_stage(c1)) break;
-                    { PROF_T(t1); fetch(c1, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, dsets); PROF_ACC(d_fetch, t1); }
+                    { fetch(c1, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, dsets); }
                     if (tile_c >= P.total_tiles || !decode_stage(c2)) break;
-                    { PROF_T(t2); fetch(c2, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, dsets); PROF_ACC(d_fetch, t2); }
+                    { fetch(c2, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, dsets); }
                 }
             } else {
                 // The overlapped tile shapes are paced by this loop, and a loop that is a third as long
@@ -431,11 +389,10 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 while (true) {
                     if (tile_c >= P.total_tiles || !decode_stage(c0)) break;
                     c0 = c1;
-                    { PROF_T(t0); fetch(c1, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, dsets); PROF_ACC(d_fetch, t0); }
+                    { fetch(c1, rowp_f, st_f); advance_f(tile_f, st_f, nt_f, rowp_f, dsets); }
                 }
             }
         }
-        if (warp == 2 && lane == 0) { PROF_OUT(6, w_full); PROF_OUT(8, PROF_NOW() - t_dec); PROF_OUT(12, d_alu); PROF_OUT(13, d_wst); PROF_OUT(14, d_fetch); PROF_OUT(15, d_st); }
     } else {
         // ------------------------------------------------ epilogue
         // Eight warps, two per tensor-memory lane quadrant; the two warps of a quadrant take
@@ -465,7 +422,6 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         uint32_t nst = 0;      // staging buffers this warp has filled so far (selects the buffer)
         uint32_t nres = 0;     // residual chunks this warp has consumed so far (buffer and phase)
         bool alive = true;
-        PROF_DECL(e_wait); PROF_DECL(e_drain); PROF_DECL(e_ld); PROF_DECL(e_grp); PROF_DECL(e_math); PROF_DECL(e_st);
         for (int tile = blockIdx.x; tile < P.total_tiles && alive; tile += gridDim.x, ++lt) {
             const int nt = tile % P.n_tiles;
             int pt = tile / P.n_tiles;
@@ -496,10 +452,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 if (kMine > 1) res_load(es + kEpiSets, (nres + 1) & 1u);
             }
             const int buf = lt % kAccBufs;
-            PROF_T(t_w);
             if (kbpt > 0 && !mbar_wait_warp(&sm->acc_full[buf], (lt / kAccBufs) & 1u, abort_flag, P.status, 32)) break;
-            PROF_ACC(e_wait, t_w);
-            PROF_T(t_d);
             tc_fence_after();
             float *const y32 = reinterpret_cast<float *>(P.Y) + n;
             __nv_bfloat16 *const y16 = reinterpret_cast<__nv_bfloat16 *>(P.Y) + n;
@@ -510,7 +463,6 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
 #pragma unroll 1
             for (int i = 0; i < kMine; ++i) {
                 const int c = es + i * kEpiSets;
-                PROF_T(t_ld);
                 if (kbpt > 0) {
                     if (warp_on) {
                         tmem_ld32(t_acc + c * 32, v);
@@ -521,13 +473,11 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&sm->acc_empty[buf]);
-                        PROF_ACC(e_drain, t_d);
                     }
                 } else {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
                 }
-                PROF_ACC(e_ld, t_ld);
                 if (!warp_on) continue;
                 // output offset of pixel `lane` of this chunk (per-thread stores and residual loads
                 // exchange them by shuffle), ~0 = outside the output
@@ -540,12 +490,9 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     if (wv < P.Wv && hv < P.Hv && bv < P.Bv)
                         my_off = (uint32_t)((((long long)bv * P.OH + (hv * P.osh + P.ooh)) * P.OW + (wv * P.osw + P.oow)) * P.ldy);
                 }
-                PROF_T(t_grp);
                 if (use_res_tma) {
                     if (!mbar_wait_warp(&my_res_full[nres & 1u], (nres >> 1) & 1u, abort_flag, P.status, 32)) { alive = false; break; }
                 }
-                PROF_ACC(e_grp, t_grp);
-                PROF_T(t_math);
                 // The inner loops are kept free of conditionals: every instruction issued here is
                 // exposed latency of this warp's chunk.
                 if (use_res_tma) {
@@ -581,8 +528,6 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(fmaxf(fmaf(__uint_as_float(v[j]), sc, sf), floor_v));
                 }
-                PROF_ACC(e_math, t_math);
-                PROF_T(t_st);
                 if (P.tma_store) {
                     // a staging buffer holds 32 pixels of bf16 or 16 of fp32: one or two rounds per chunk
                     const int rounds = out_bf16 ? 1 : 2;
@@ -635,11 +580,9 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                         }
                     }
                 }
-                PROF_ACC(e_st, t_st);
             }
             __syncwarp();
         }
-        if (q == 0 && lane == 0 && es == 0) { PROF_OUT(9, e_wait); PROF_OUT(10, e_drain); PROF_OUT(11, (long long)lt); PROF_OUT(16, e_ld); PROF_OUT(17, e_grp); PROF_OUT(18, e_math); PROF_OUT(19, e_st); }
         // all bulk stores of this thread have been written before the block may exit
         if (P.tma_store && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
@@ -792,9 +735,6 @@ int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const twn_dev
             }
         }
     }
-#if defined(TWN_PROFILE) || defined(TWN_TUNE)
-    if (getenv("TWN_NOTMA")) { P.tma_store = 0; }
-#endif
     const int grid = dev.sm_count < P.total_tiles ? dev.sm_count : P.total_tiles;
     tconv_kernel<PIX, DS><<<grid, threads_conv(DS), smem_bytes, s>>>(map_x, map_y, map_r, P);
     TWN_CUDA_OK(cudaGetLastError());
@@ -865,13 +805,7 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
                     c256 = ((t256 + sms - 1) / sms) * per256;
     int choice = c256 < c128 ? 1 : 0;
     if (c192 < (choice ? c256 : c128)) choice = 2;
-#if defined(TWN_PROFILE) || defined(TWN_TUNE)
-    if (const char *force = getenv("TWN_TILE")) choice = atoi(force) % 3;   // profiling and tuning builds: pin the variant
-#endif
     P.dsets = (choice != 1 && two) ? 2 : 1;
-#if defined(TWN_PROFILE) || defined(TWN_TUNE)
-    if (const char *force = getenv("TWN_DSETS")) P.dsets = atoi(force) == 2 ? 2 : 1;
-#endif
     if (choice == 1) return launch_conv_t<256, 1>(g, P, X, dev, enc, s);
     if (choice == 2) return P.dsets == 2 ? launch_conv_t<192, 2>(g, P, X, dev, enc, s) : launch_conv_t<192, 1>(g, P, X, dev, enc, s);
     return P.dsets == 2 ? launch_conv_t<128, 2>(g, P, X, dev, enc, s) : launch_conv_t<128, 1>(g, P, X, dev, enc, s);
@@ -1109,15 +1043,3 @@ extern "C" int twn_conv2d_bwd_data(const twn_conv_desc_t *d, const void *dZ, con
     return first_error;
 }
 
-#ifdef TWN_PROFILE
-extern "C" int twn_tl2_read(long long *host) { return cudaMemcpyFromSymbol(host, g_tl2, sizeof(long long) * 4 * 1024); }
-extern "C" int twn_tl_read(long long *host) { return cudaMemcpyFromSymbol(host, g_tl, sizeof(long long) * 4 * 1024); }
-extern "C" int twn_prof_read(long long *host, int zero)
-{
-    if (zero) {
-        static long long z[256 * 32];
-        return cudaMemcpyToSymbol(g_prof, z, sizeof(z));
-    }
-    return cudaMemcpyFromSymbol(host, g_prof, sizeof(long long) * 256 * 32);
-}
-#endif

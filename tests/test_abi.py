@@ -21,9 +21,21 @@ def declared_functions():
     return sorted(set(re.findall(r"\b(twn_[a-z0-9_]+)\s*\(", text)))
 
 
-def test_header_declares_the_north_star_entry_points_once_built():
+REQUIRED = [
+    # the five entry points the contract names
+    "twn_ternarize", "twn_pack", "twn_gemm", "twn_conv2d_fwd", "twn_conv2d_bwd_data",
+    # their companions: inverse of pack, code re-layout for the backward pass, weight gradient
+    "twn_unpack", "twn_transpose_codes", "twn_conv2d_bwd_weight",
+    # library helpers: error text, device status, scratch sizes
+    "twn_strerror", "twn_read_status", "twn_ternarize_workspace_bytes",
+    "twn_ternarize_batch_workspace_bytes", "twn_conv2d_bwd_weight_workspace_bytes",
+]
+
+
+def test_header_declares_every_contract_entry_point_by_name():
     names = declared_functions()
-    assert "twn_ternarize" in names and "twn_pack" in names
+    for name in REQUIRED:
+        assert name in names, f"{name} is missing from include/twn.h"
 
 
 def test_every_declared_symbol_is_exported(lib):
@@ -48,6 +60,46 @@ def test_host_side_argument_checks_need_no_device(lib):
     assert bad == -1
     bad = lib.twn_unpack(None, C.c_int64(-1), C.c_int64(1), C.c_int64(64), None, None, None)
     assert bad == -1
+
+
+class _Desc(C.Structure):
+    _fields_ = [("B", C.c_int64), ("H", C.c_int64), ("W", C.c_int64), ("Cin", C.c_int64),
+                ("Cout", C.c_int64), ("kh", C.c_int32), ("kw", C.c_int32),
+                ("stride_h", C.c_int32), ("stride_w", C.c_int32),
+                ("pad_h", C.c_int32), ("pad_w", C.c_int32)]
+
+
+def test_contractions_refuse_bad_arguments_on_the_host(lib):
+    """twn_gemm, twn_conv2d_fwd and twn_conv2d_bwd_data through raw ctypes with arguments the host can
+    see are wrong: each returns its error code before any CUDA call, so no device is needed."""
+    i64, null = C.c_int64, None
+    # negative extent / NULL operands with work to do / row pitch smaller than K / pitch not a multiple of 64
+    assert lib.twn_gemm(null, i64(64), null, i64(64), null, i64(-1), i64(8), i64(64), null, null, i64(8), null, null) == -1
+    assert lib.twn_gemm(null, i64(64), null, i64(64), null, i64(4), i64(8), i64(64), null, null, i64(8), null, null) == -1
+    fake = C.c_void_p(4096)          # never dereferenced: every call below fails a host check first
+    assert lib.twn_gemm(fake, i64(32), fake, i64(64), null, i64(4), i64(8), i64(64), null, fake, i64(8), null, null) == -1
+    assert lib.twn_gemm(fake, i64(64), fake, i64(100), null, i64(4), i64(8), i64(64), null, fake, i64(8), null, null) == -1
+    # an empty product is fine and launches nothing
+    assert lib.twn_gemm(null, i64(64), null, i64(64), null, i64(0), i64(8), i64(64), null, null, i64(8), null, null) == 0
+    # operand pitch not a multiple of 8 elements, misaligned pointer
+    assert lib.twn_gemm(fake, i64(68), fake, i64(64), null, i64(4), i64(8), i64(64), null, fake, i64(8), null, null) == -2
+    assert lib.twn_gemm(C.c_void_p(4098), i64(64), fake, i64(64), null, i64(4), i64(8), i64(64), null, fake, i64(8), null, null) == -2
+    for fn in (lib.twn_conv2d_fwd, lib.twn_conv2d_bwd_data):
+        assert fn(null, fake, fake, i64(64), null, null, fake, null, null) == -1            # no descriptor
+        d = _Desc(2, 8, 8, 16, 16, 3, 3, 1, 1, 1, 1)
+        assert fn(C.byref(d), null, fake, i64(192), null, null, fake, null, null) == -1     # NULL input
+        assert fn(C.byref(d), fake, fake, i64(64), null, null, fake, null, null) == -1      # pitch < kh*kw*C
+        bad = _Desc(2, 8, 8, 16, 16, 3, 3, 0, 1, 1, 1)
+        assert fn(C.byref(bad), fake, fake, i64(192), null, null, fake, null, null) == -1   # stride 0
+        bad = _Desc(2, 2, 2, 16, 16, 7, 7, 1, 1, 0, 0)
+        assert fn(C.byref(bad), fake, fake, i64(1024), null, null, fake, null, null) == -1  # window larger than the image
+    # channel counts the tensor copies cannot address: the reduction runs over Cin in the forward pass
+    # and over Cout in the backward pass, and needs runs of 16 codes (8 for a 1x1 filter)
+    d = _Desc(2, 8, 8, 24, 40, 3, 3, 1, 1, 1, 1)
+    assert lib.twn_conv2d_fwd(C.byref(d), fake, fake, i64(256), null, null, fake, null, null) == -2
+    assert lib.twn_conv2d_bwd_data(C.byref(d), fake, fake, i64(384), null, null, fake, null, null) == -2
+    d = _Desc(2, 8, 8, 32, 130, 1, 1, 1, 1, 0, 0)
+    assert lib.twn_conv2d_bwd_data(C.byref(d), fake, fake, i64(192), null, null, fake, null, null) == -2
 
 
 def test_binding_names_match_the_header():

@@ -167,9 +167,10 @@ def test_sweep_small_and_medium(dist, seed, n):
 
 
 @pytest.mark.parametrize("dist", ["normal", "laplace", "uniform"])
-def test_sweep_full_size_1e8(dist):
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_sweep_full_size_1e8(dist, seed):
     n = 100_000_000
-    st = check_against_oracle(dg.draw(0, f"sweep-{dist}", n, dist).reshape(1, n), want_i8=False)
+    st = check_against_oracle(dg.draw(seed, f"sweep-{dist}", n, dist).reshape(1, n), want_i8=False)
     assert st["n_neg"] + st["n_zero"] + st["n_pos"] == n
 
 

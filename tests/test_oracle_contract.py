@@ -108,6 +108,44 @@ def test_conv_fwd_equals_torch_conv2d(case):
     np.testing.assert_array_equal(Ap, A.reshape(-1, Cout)[pix])
 
 
+@pytest.mark.parametrize("case", CONV_CASES)
+def test_conv_fwd_epilogue_equals_torch_conv2d_then_the_same_epilogue(case):
+    """Per-channel scale and shift, an fp64 residual of the output's shape and ReLU, applied by the
+    oracle inside both convolution entry points (full tensor and pixel list), against torch's fp64
+    conv2d followed by the same four steps written out with numpy.  The scale and shift differ per
+    channel and the residual per element, so a wrong channel or a wrong residual index shows."""
+    B, H, W, Cin, Cout, k, s, p = case
+    d = oracle.conv_desc(B, H, W, Cin, Cout, k, s, p)
+    X = _x(20, "cx", (B, H, W, Cin)); T = _rand_codes(21, (Cout, k, k, Cin))
+    alpha = 0.55
+    scale = dg.draw(22, "s", Cout, "normal", 1.0, 0.4)
+    shift = dg.draw(22, "b", Cout, "normal", 0.0, 0.5)
+    res = dg.draw(23, "r", B * d.Ho * d.Wo * Cout, "normal").astype(np.float64).reshape(B, d.Ho, d.Wo, Cout)
+    xd, wd = _torch_conv(d, X, T, alpha)
+    z = alpha * F.conv2d(xd, wd, stride=s, padding=p).permute(0, 2, 3, 1).numpy()
+    pre = z * scale.astype(np.float64)[None, None, None, :] + shift.astype(np.float64)[None, None, None, :] + res
+    want = np.maximum(pre, 0.0)
+    assert (pre < 0).any() and (pre > 0).any()          # the ReLU must matter
+    Y, _ = oracle.conv2d_fwd(d, X, T, alpha, scale, shift, res, relu=True)
+    np.testing.assert_allclose(Y, want, rtol=1e-12, atol=1e-12)
+    # without ReLU, and each step alone
+    Y, _ = oracle.conv2d_fwd(d, X, T, alpha, scale, shift, res, relu=False)
+    np.testing.assert_allclose(Y, pre, rtol=1e-12, atol=1e-12)
+    Y, _ = oracle.conv2d_fwd(d, X, T, alpha, residual=res)
+    np.testing.assert_allclose(Y, z + res, rtol=1e-12, atol=1e-12)
+    Y, _ = oracle.conv2d_fwd(d, X, T, alpha, shift=shift)
+    np.testing.assert_allclose(Y, z + shift.astype(np.float64), rtol=1e-12, atol=1e-12)
+    # the pixel-list form, in an order that is not the tensor's: the residual is still indexed by
+    # the flat position in the full output
+    npix = B * d.Ho * d.Wo
+    pix = np.array(sorted(set([0, npix - 1, npix // 2, npix // 3, 1, max(npix - 2, 0)])))[::-1].copy()
+    Yp, Ap = oracle.conv2d_fwd(d, X, T, alpha, scale, shift, res, relu=True, pixels=pix)
+    np.testing.assert_allclose(Yp, want.reshape(-1, Cout)[pix], rtol=1e-12, atol=1e-12)
+    Yf, Af = oracle.conv2d_fwd(d, X, T, alpha, scale, shift, res, relu=True)
+    np.testing.assert_array_equal(Yp, Yf.reshape(-1, Cout)[pix])
+    np.testing.assert_array_equal(Ap, Af.reshape(-1, Cout)[pix])
+
+
 def test_conv_1x1_is_the_gemm():
     d = oracle.conv_desc(2, 3, 5, 16, 9, 1, 1, 0)
     X = _x(2, "cx", (2, 3, 5, 16)); T = _rand_codes(3, (9, 1, 1, 16))

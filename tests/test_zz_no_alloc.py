@@ -14,6 +14,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_1605_04711_b200 import datagen as dg
 from paper_1605_04711_b200 import twn
 
@@ -56,6 +57,42 @@ def test_two_calls_in_a_row_match_the_allocating_entry_point():
             assert got[0] == want[0], call
             assert np.array_equal(got[1], want[1]), call
             assert np.array_equal(got[2], want[2]), call
+
+
+def test_matches_the_oracle_and_leaves_device_memory_as_it_found_it():
+    """The results are checked against the CPU oracle directly (codes and packed words to the bit,
+    threshold and scale to 1e-12), and the device memory in use is the same before and after a
+    call: neither torch's allocator nor the driver hands out anything on its behalf.  The second
+    call is the one measured at the driver level, because the first launch of a kernel in a process
+    may make the driver load its code."""
+    rows, cols = 96, 2000
+    W = dg.draw(13, "noalloc-oracle", rows * cols, "normal").reshape(rows, cols)
+    Wd = torch.from_numpy(W).cuda()
+    ld = twn.ld_for(cols)
+    stats = twn.new_stats()
+    packed = torch.full((rows, ld // 16), -1, dtype=torch.int32, device="cuda")
+    codes = torch.full((rows, cols), 7, dtype=torch.int8, device="cuda")
+    ref, ref_codes = oracle.ternarize(W, 0.7)
+    assert ref.n_boundary == 0
+    want_packed = oracle.pack(ref_codes.reshape(rows, cols), ld)
+    for call in range(2):
+        torch.cuda.synchronize()
+        torch_before = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+        free_before, _ = torch.cuda.mem_get_info()
+        twn.ternarize_static(Wd, 0.7, stats, packed, ld, codes, rows=rows, cols=cols)
+        torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
+        assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == torch_before
+        if call == 1:
+            assert free_after == free_before
+        st = twn.stats_to_host(stats)
+        assert st["status"] == 0
+        assert abs(st["delta"] - ref.delta) <= 1e-12 * ref.delta
+        assert abs(st["alpha"] - ref.alpha) <= 1e-12 * ref.alpha
+        assert (st["n_neg"], st["n_zero"], st["n_pos"]) == (ref.n_neg, ref.n_zero, ref.n_pos)
+        assert np.array_equal(codes.cpu().numpy(), ref_codes.reshape(rows, cols))
+        assert np.array_equal(packed.cpu().numpy().view(np.uint32), want_packed)
+        packed.fill_(-1); codes.fill_(7)
 
 
 def test_a_small_tensor_after_a_large_one_sees_no_stale_partials():
