@@ -47,6 +47,9 @@
 
 #include "common.cuh"
 #include "tc_ptx.cuh"
+#include "tconv_host.cuh"
+
+using namespace twn_detail;
 
 
 namespace {
@@ -61,7 +64,6 @@ constexpr int kEpiSets = 2;         // epilogue warps per lane quadrant; each dr
 __host__ __device__ constexpr int threads_conv(int ds) { return 32 * (first_epi_warp(ds) + 4 * kEpiSets); }
 constexpr int kEpiWarps = 4 * kEpiSets;
 constexpr int kStageBytes = 2048;   // one output staging buffer of a warp: 32 channels x 32 pixels of bf16 or 16 pixels of fp32
-constexpr int kMaxTaps = 64;
 constexpr int kWordTab = 128;       // k-blocks per tile whose code offsets are tabulated in shared memory
 constexpr int kAColsPerBlock = kBlockK / 2;    // 32 columns of bf16 pairs per k-block
 constexpr uint32_t kTmemCols = 512;
@@ -86,11 +88,6 @@ template <> struct Cfg<192> {
     static constexpr int kSub = 1;
     static constexpr int kAccBufs = 2;
     static constexpr int kOutBufs = 4;
-};
-
-struct Tap {
-    int16_t dh, dw;   // input pixel offset of this tap
-    int32_t koff;     // first code column of this tap in a packed row
 };
 
 struct ConvParams {
@@ -602,60 +599,6 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
 }
 
 // ---------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult qr;
-        if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &p, 12000, cudaEnableDefault, &qr) == cudaSuccess &&
-            qr == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
-struct Geometry {
-    // input tensor X: NHWC [XB, XH, XW, XC] with pixel pitch ldx (elements)
-    long long XB, XH, XW, XC, ldx;
-    long long x_row_pitch, x_img_pitch;   // elements between rows / images; 0 = dense (XW*ldx, XH*XW*ldx)
-    // virtual output grid and embedding
-    int Bv, Hv, Wv, OH, OW, osh, osw, ooh, oow;
-    long long ldy;
-    int sh, sw;      // input step per virtual output pixel
-    int Cout;
-    long long ld_codes, code_cols;  // packed row pitch and used columns
-    int n_taps;
-    Tap taps[kMaxTaps];
-    long long Cin;   // channels per tap
-};
-
-// Picks the pixel-tile shape BW x BH x BB (BW and BH powers of two, product `pix`) that needs the
-// fewest tiles.
-long long pick_tile(const Geometry &g, int pix, int *lgBW, int *lgBH)
-{
-    int lg = 0;
-    while (((pix >> lg) & 1) == 0) ++lg;      // BW * BH divides the power-of-two part of `pix`
-    long long best = -1;
-    int bw = 0, bh = 0;
-    for (int a = 0; a <= lg; ++a)
-        for (int b = 0; a + b <= lg; ++b) {
-            const int BW = 1 << a, BH = 1 << b, BB = pix >> (a + b);
-            if (BW * g.sw > 256 || BH * g.sh > 256 || BB > 256) continue;
-            const long long tiles = ((g.Wv + BW - 1) / BW) * (long long)((g.Hv + BH - 1) / BH) * ((g.Bv + BB - 1) / BB);
-            // prefer fewer tiles, then wider rows
-            if (best < 0 || tiles < best || (tiles == best && a > bw)) { best = tiles; bw = a; bh = b; }
-        }
-    *lgBW = bw; *lgBH = bh;
-    return best;
-}
-
 template <int PIX, int DS>
 int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const twn_device_info &dev,
                   EncodeTiledFn enc, cudaStream_t s)
@@ -752,6 +695,21 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
 
     // the epilogue keeps output offsets in 32 bits
     if ((long long)g.Bv * g.OH * g.OW * g.ldy >= 0xFFFFFFFFLL) return TWN_ERR_INVALID_ARG;
+    {
+        // narrow layers: the kernel that decodes the layer's codes once per block
+        EpilogueArgs ea;
+        ea.alpha = stats ? &stats->alpha : nullptr;
+        ea.scale = epi ? epi->scale : nullptr;
+        ea.shift = epi ? epi->shift : nullptr;
+        ea.residual = epi ? epi->residual : nullptr;
+        ea.res_dtype = epi ? epi->residual_dtype : TWN_F32;
+        ea.res_gate = (epi && epi->residual) ? epi->residual_op : 0;
+        ea.relu = epi ? epi->relu : 0;
+        ea.out_dtype = epi ? epi->out_dtype : out_dtype_default;
+        bool handled = false;
+        rc = launch_conv_resident(g, X, T, ea, Y, dev_status, dev, s, &handled);
+        if (rc != TWN_OK || handled) return rc;
+    }
     ConvParams P;
     memset(&P, 0, sizeof P);
     P.n_tiles = (g.Cout + kChan - 1) / kChan;
