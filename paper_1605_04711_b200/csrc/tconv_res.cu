@@ -24,9 +24,10 @@
 // the same way, one tile ahead.
 //
 //   warp 0      TMA producer: one activation tile (with halo) per tile and 64-channel block
-//   warp 1      allocates tensor memory, issues tcgen05.mma, commits to mbarriers
+//   warp 1      allocates tensor memory; one thread issues the tcgen05.mma of the even tiles of the block
 //   warps 2-9   epilogue: two sets of four (one warp per tensor-memory lane quadrant), the sets
 //               take alternate tiles
+//   warp 10     one thread issues the tcgen05.mma of the odd tiles
 // All warps decode the weights before the roles start.
 //
 // Every wait on an mbarrier is bounded; on expiry the kernel records TWN_ERR_TIMEOUT, all roles
@@ -50,7 +51,8 @@ constexpr int kNMax = 64;                 // output channels (UMMA N)
 constexpr int kAccBufs = 4;
 constexpr uint32_t kTmemCols = kAccBufs * kNMax;
 constexpr int kEpiWarps = 8;
-constexpr int kThreads = 32 * (2 + kEpiWarps);
+constexpr int kIssuerB = 2 + kEpiWarps;    // the warp of the second MMA-issuing thread
+constexpr int kThreads = 32 * (3 + kEpiWarps);
 constexpr int kMaxStages = 8;
 constexpr int kStageBuf = 4096;           // per-warp staging: 32 pixels x 128 bytes
 constexpr int kSmemLimit = 232448;
@@ -59,7 +61,9 @@ struct Ctl {
     unsigned long long full[kMaxStages], empty[kMaxStages];
     unsigned long long acc_full[kAccBufs], acc_empty[kAccBufs];
     unsigned long long res_full[kEpiWarps];
+    unsigned long long turn[2];           // issuer -> issuer: "every stage up to the end of my tile has landed"
     float sc[kNMax], sf[kNMax];           // per-channel scale (alpha and the decode factor folded in) and shift
+    uint2 tap[kMaxTaps + 1];              // per tap: operand offsets of its first k-block (A inside a stage, B inside the weights), 16-byte units
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -68,7 +72,6 @@ struct ResParams {
     int total_tiles, tw, th;
     int lgBW, lgBH;               // pixel tile = BB x BH x BW, powers of two, product 128
     int n_taps, n_cblk, kbpt;     // k-blocks per tile = n_taps * n_cblk
-    int last_k16;                 // K = 16 steps of the last channel block that hold real channels (1..4)
     int N;                        // UMMA N: Cout rounded up to 16
     int Cout;
     const uint32_t *T;            // packed codes, one row of `wpr` words per output channel
@@ -100,16 +103,35 @@ __device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t saddr, uint32_t s
     return d;
 }
 
-// D[tmem] (+)= A[smem] * B[smem]^T with the accumulate flag in a register.
-__device__ __forceinline__ void tc_mma_ss_flag(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc)
+// D[tmem] (+)= A[smem] * B[smem]^T, issued by the calling thread alone.  The descriptors arrive as
+// halves: the upper words never change and the lower ones advance by 32-bit additions, so an MMA
+// costs its issuing thread two additions and the instruction itself.
+template <bool ACC>
+__device__ __forceinline__ void tc_mma_ss_1t(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                             uint32_t idesc)
 {
     asm volatile(
-        "{\n\t.reg .pred p, pe;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "elect.sync _|pe, 0xffffffff;\n\t"
-        "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(ACC ? 1 : 0)
         : "memory");
+}
+// One k-block of one tap: four K = 16 steps, 32 bytes apart in both operands.
+template <bool FIRST>
+__device__ __forceinline__ void tc_mma_tap(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                           uint32_t idesc)
+{
+    tc_mma_ss_1t<!FIRST>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc);
+    tc_mma_ss_1t<true>(d_tmem, a_lo + 2, a_hi, b_lo + 2, b_hi, idesc);
+    tc_mma_ss_1t<true>(d_tmem, a_lo + 4, a_hi, b_lo + 4, b_hi, idesc);
+    tc_mma_ss_1t<true>(d_tmem, a_lo + 6, a_hi, b_lo + 6, b_hi, idesc);
+}
+__device__ __forceinline__ void tc_commit_1t(void *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
@@ -146,6 +168,8 @@ tconv_res_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         for (int s = 0; s < kMaxStages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
         for (int b = 0; b < kAccBufs; ++b) { mbar_init(&ctl->acc_full[b], 1); mbar_init(&ctl->acc_empty[b], 4); }
         for (int w = 0; w < kEpiWarps; ++w) mbar_init(&ctl->res_full[w], 1);
+        mbar_init(&ctl->turn[0], 1);
+        mbar_init(&ctl->turn[1], 1);
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -161,6 +185,8 @@ tconv_res_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         ctl->sc[c] = ((P.scale && c_ok) ? __ldg(P.scale + c) : 1.0f) * alpha;
         ctl->sf[c] = (P.shift && c_ok) ? __ldg(P.shift + c) : 0.0f;
     }
+    for (int t = threadIdx.x; t <= P.n_taps && t <= kMaxTaps; t += kThreads)
+        ctl->tap[t] = make_uint2(t < P.n_taps ? (uint32_t)P.a_off[t] : 0u, (uint32_t)(t * P.n_cblk) * ((uint32_t)(P.N * 128) >> 4));
     // Decode the layer: item (channel n, k-block u) = 64 codes = 16 bytes -> 128 bytes of bf16, written as
     // row n of k-block u in the K-major layout the MMA reads (16-byte chunk j of row n at chunk j ^ (n & 7)).
     // Code words past the end of a row are clamped into it: they only ever meet activations that the TMA
@@ -220,39 +246,62 @@ tconv_res_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 }
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------ MMA issuer (whole warp, converged)
-        if (P.kbpt > 0) {
+    } else if (warp == 1 || warp == kIssuerB) {
+        // ------------------------------------------------ MMA issuers: two threads, alternate tiles
+        // Measured on B200: a 128x64x16 MMA with both operands in shared memory occupies the tensor core
+        // for 48 cycles, and tcgen05.mma holds its issuing thread until the tensor core accepts it, so every
+        // instruction that thread runs between two MMAs (address arithmetic, waits) is time the tensor core
+        // idles: one issuer reached 59 to 76 cycles per MMA, two issuers on different accumulators 48 whatever
+        // they execute in between.  Tiles alternate between the two threads; each works on the accumulator and
+        // the activation stages of its own tiles, so the two instruction streams never touch the same data.
+        // The stages form one ring that both threads consume, and an mbarrier wait only tells a phase from
+        // its neighbours: a thread may wait for "stage s, parity p" only once every earlier phase of that
+        // barrier is known to be over.  So the threads pass a token: after seeing the last stage of its tile
+        // land, a thread lets the other one start waiting for the stages of the next tile.
+        if (lane == 0 && P.kbpt > 0) {
+            const uint32_t me = warp == 1 ? 0u : 1u;
             const uint32_t idesc = make_idesc(kPix, P.N);
             const uint64_t adesc0 = smem_desc_k_sw128(base_u32, P.a_sbo);
             const uint64_t bdesc0 = smem_desc_sw128(base_u32 + P.wts_off);
+            const uint32_t a_hi = (uint32_t)(adesc0 >> 32), b_hi = (uint32_t)(bdesc0 >> 32);
+            const uint32_t a_lo0 = (uint32_t)adesc0, b_lo0 = (uint32_t)bdesc0;
             const uint32_t b_step = (uint32_t)(P.N * 128) >> 4;      // one k-block of weights, 16-byte units
             const uint32_t a_step = (uint32_t)P.stage_bytes >> 4;
-            uint32_t s = 0, ph = 0, lt = 0;
+            const int n_taps = P.n_taps;
+            uint32_t s = 0, ph = 0;
+            // stage position of this thread's first tile, then of every other tile
+            auto skip_tile = [&]() {
+                for (int cb = 0; cb < P.n_cblk; ++cb)
+                    if (++s == (uint32_t)P.n_stages) { s = 0; ph ^= 1u; }
+            };
+            if (me) skip_tile();
             bool ok = true;
-            for (int tile = blockIdx.x; tile < P.total_tiles && ok; tile += gridDim.x, ++lt) {
+            uint32_t lt = me;
+            for (int tile = blockIdx.x + (int)me * (int)gridDim.x; tile < P.total_tiles && ok; tile += 2 * (int)gridDim.x, lt += 2) {
                 const uint32_t buf = lt & (kAccBufs - 1);
-                if (!mbar_wait_warp(&ctl->acc_empty[buf], ((lt / kAccBufs) & 1u) ^ 1u, abort_flag, P.status, 0)) break;
+                if (!mbar_wait(&ctl->acc_empty[buf], ((lt / kAccBufs) & 1u) ^ 1u, abort_flag, P.status, 0)) break;
+                if (lt > 0 && !mbar_wait(&ctl->turn[me], ((lt - 1) >> 1) & 1u, abort_flag, P.status, 0)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem + buf * kNMax;
-                uint32_t acc = 0;
                 for (int cb = 0; cb < P.n_cblk; ++cb) {
-                    if (!mbar_wait_warp(&ctl->full[s], ph, abort_flag, P.status, 0)) { ok = false; break; }
+                    if (!mbar_wait(&ctl->full[s], ph, abort_flag, P.status, 0)) { ok = false; break; }
+                    if (cb == P.n_cblk - 1) mbar_arrive(&ctl->turn[me ^ 1u]);
                     tc_fence_after();
-                    const uint64_t a_s = adesc0 + (uint64_t)(s * a_step);
-                    const int nk = (cb == P.n_cblk - 1) ? P.last_k16 : 4;
-                    for (int t = 0; t < P.n_taps; ++t) {
-                        const uint64_t a = a_s + (uint64_t)(uint32_t)P.a_off[t];
-                        const uint64_t b = bdesc0 + (uint64_t)((uint32_t)(t * P.n_cblk + cb) * b_step);
-                        for (int k = 0; k < nk; ++k) {
-                            tc_mma_ss_flag(d_tmem, a + 2 * k, b + 2 * k, idesc, acc);
-                            acc = 1;
-                        }
+                    const uint32_t a_s = a_lo0 + s * a_step, b_s = b_lo0 + (uint32_t)cb * b_step;
+                    uint2 cur = ctl->tap[0];
+                    uint2 nxt = ctl->tap[1];
+                    if (cb == 0) tc_mma_tap<true>(d_tmem, a_s + cur.x, a_hi, b_s + cur.y, b_hi, idesc);
+                    else tc_mma_tap<false>(d_tmem, a_s + cur.x, a_hi, b_s + cur.y, b_hi, idesc);
+#pragma unroll 1
+                    for (int t = 1; t < n_taps; ++t) {
+                        cur = nxt;
+                        nxt = ctl->tap[t + 1];
+                        tc_mma_tap<false>(d_tmem, a_s + cur.x, a_hi, b_s + cur.y, b_hi, idesc);
                     }
-                    tc_commit(&ctl->empty[s]);
+                    tc_commit_1t(&ctl->empty[s]);
                     if (++s == (uint32_t)P.n_stages) { s = 0; ph ^= 1u; }
                 }
-                if (ok) tc_commit(&ctl->acc_full[buf]);
+                if (ok) { tc_commit_1t(&ctl->acc_full[buf]); skip_tile(); }
             }
         }
     } else {
@@ -429,9 +478,6 @@ int twn_detail::launch_conv_resident(const Geometry &g, const void *X, const uin
     P.kbpt = P.n_taps * P.n_cblk;
     P.N = (g.Cout + 15) / 16 * 16;
     P.Cout = g.Cout;
-    P.last_k16 = (int)((g.Cin - (long long)(P.n_cblk - 1) * kBlockK + 15) / 16);
-    if (P.last_k16 > 4) P.last_k16 = 4;
-    if (P.last_k16 < 1) P.last_k16 = 1;
     P.codes_aligned = 1;
     int w_lo = 0, w_hi = 0, h_lo = 0, h_hi = 0;
     for (int t = 0; t < g.n_taps; ++t) {
@@ -480,7 +526,7 @@ int twn_detail::launch_conv_resident(const Geometry &g, const void *X, const uin
     P.stage_tx = 128 * row_pix * (BH + hh) * BB;
     P.stage_bytes = (P.stage_tx + 1023) / 1024 * 1024;
     const long long wts_bytes = (long long)P.kbpt * P.N * 128;
-    const long long fixed = 1024 + wts_bytes + kEpiWarps * kStageBuf * (epi.residual ? 2 : 1) + 1024;
+    const long long fixed = 1024 + wts_bytes + kEpiWarps * kStageBuf * (epi.residual ? 2 : 1) + 2048;
     if (fixed > kSmemLimit) return TWN_OK;
     int n_stages = P.kbpt > 0 ? (int)((kSmemLimit - fixed) / P.stage_bytes) : 0;
     if (n_stages > kMaxStages) n_stages = kMaxStages;
@@ -490,8 +536,8 @@ int twn_detail::launch_conv_resident(const Geometry &g, const void *X, const uin
     P.stg_off = P.wts_off + (uint32_t)wts_bytes;
     P.res_off = P.stg_off + kEpiWarps * kStageBuf;
     P.ctl_off = P.res_off + (epi.residual ? kEpiWarps * kStageBuf : 0);
-    static_assert(sizeof(Ctl) <= 1024, "control block");
-    const int smem_bytes = 1024 + (int)P.ctl_off + 1024;
+    static_assert(sizeof(Ctl) <= 2048, "control block");
+    const int smem_bytes = 1024 + (int)P.ctl_off + 2048;
 
     P.T = T;
     P.wpr = g.ld_codes / 16;

@@ -90,6 +90,10 @@ BWD_CASES = [
     (5, 28, 28, 64, 64, 3, 1, 1, "gate", True),
     (2, 9, 9, 16, 96, 3, 1, 1, None, False),
     (9, 56, 56, 64, 64, 3, 1, 1, "add", True),
+    # two 64-channel blocks per tap and room for only two activation stages: both MMA-issuing threads
+    # walk the same small ring, several times per block
+    (6, 40, 40, 64, 96, 3, 1, 1, "add", True),
+    (16, 44, 40, 64, 128, 3, 1, 1, None, True),
 ]
 
 
