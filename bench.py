@@ -372,6 +372,257 @@ class GemmWorkload:
         return 2.0 * rows * self.N * self.K / dt / 1e12, f"oracle gemm on {rows} of {self.M} rows ({dt:.1f} s)", oracle.num_threads()
 
 
+def flush_l2(torch, _cache={}):
+    """Writes a buffer larger than L2 (126 MB) so that the next launch starts cold."""
+    if "buf" not in _cache:
+        _cache["buf"] = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    _cache["buf"].fill_(1)
+
+
+def time_cold(torch, fn, reps=20, warm=3):
+    """Median and minimum (microseconds) of `reps` single launches, each after an L2 flush."""
+    for _ in range(warm):
+        fn()
+    us = []
+    for _ in range(reps):
+        flush_l2(torch)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); fn(); e1.record()
+        e1.synchronize()
+        us.append(e0.elapsed_time(e1) * 1e3)
+    us.sort()
+    return us[len(us) // 2], us[0]
+
+
+def bound_of(flops, nbytes, peaks):
+    """Roofline of one launch timed alone: the slower of its flops at the measured bf16 burst peak and
+    its algorithmic bytes at the measured copy bandwidth.  Returns (kind, microseconds)."""
+    t_tensor = flops / (peaks["bf16_tflops"] * 1e12) * 1e6
+    t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9) * 1e6
+    return ("tensor", t_tensor) if t_tensor >= t_hbm else ("hbm", t_hbm)
+
+
+SWEEP_KN = [(512, 512), (1152, 128), (2304, 256), (4608, 512), (4096, 4096)]
+SWEEP_M = [128, 1024, 4096, 16384]
+# the shapes the 60 % target is stated for
+SWEEP_GATED = [(4096, 4608, 512), (16384, 4608, 512), (4096, 4096, 4096), (16384, 4096, 4096), (16384, 2304, 256)]
+
+
+class GemmSweepWorkload:
+    """The ternary-weight GEMM sweep Y = alpha * X T^T (Eq. 2, inner-product form): bf16 X [M, K] drawn N(0,1),
+    T [N, K] ternarized from He-normal weights and 2-bit packed, fp32 Y, for M in {128, 1024, 4096, 16384} and
+    (K, N) in {(512,512), (1152,128), (2304,256), (4608,512), (4096,4096)}.  A step is one pass over the 20
+    shapes.  Algorithmic bytes of a shape: 2MK (X) + KN/4 (codes) + 4MN (Y); flops 2MKN."""
+    name = "ternary_gemm_sweep_fp32_out"
+    metric = "ternary GEMM TFLOP/s"
+    unit = "TFLOP/s"
+    dtype = "bf16"
+    default_steps = 20
+
+    def config(self):
+        return {"workload": self.name, "seed": 0, "delta_factor": 0.7, "shapes": 20, "out_dtype": "f32",
+                "l2": "per-shape times: L2 flushed (256 MB written) before every timed launch; "
+                      "the sweep's step time: 20 shapes back to back, 2.4 GB of operands per pass"}
+
+    def host_inputs(self):
+        from paper_1605_04711_b200 import datagen as dg
+        w = {(K, N): dg.he_normal(0, f"sweep{N}x{K}", N, K) for K, N in SWEEP_KN}
+        x = {(M, K): dg.draw_bf16(1, f"sweepx{M}x{K}", M * K, "normal").reshape(M, K)
+             for M in SWEEP_M for K in sorted({k for k, _ in SWEEP_KN})}
+        return w, x
+
+    def setup(self, torch, twn, host):
+        import numpy as np
+        self.torch, self.twn = torch, twn
+        w, x = host
+        ws = torch.empty(twn.ternarize_workspace_bytes(), dtype=torch.uint8, device="cuda")
+        self.layers, self.X, self.cases = {}, {}, []
+        for (K, N), Wm in w.items():
+            ld = twn.ld_for(K)
+            stats = twn.new_stats()
+            packed = torch.empty((N, ld // 16), dtype=torch.int32, device="cuda")
+            twn.ternarize(torch.from_numpy(Wm).cuda(), 0.7, stats, packed, ld, None, ws, rows=N, cols=K)
+            self.layers[(K, N)] = (packed, ld, stats)
+        for (M, K), xb in x.items():
+            self.X[(M, K)] = torch.from_numpy(xb.view(np.int16)).cuda().view(torch.bfloat16)
+        self.Y = torch.empty(16384 * 4096, dtype=torch.float32, device="cuda")
+        self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        for K, N in SWEEP_KN:
+            for M in SWEEP_M:
+                self.cases.append((M, K, N))
+        self.host_x = torch.empty(16384 * 4608, dtype=torch.int16).pin_memory()
+        self.host_y = torch.empty(16384 * 4096, dtype=torch.float32).pin_memory()
+
+    def _run(self, M, K, N):
+        packed, ld, stats = self.layers[(K, N)]
+        self.twn.gemm(self.X[(M, K)], K, packed, ld, stats, M, N, K, None, self.Y[:M * N].view(M, N), N, self.status)
+
+    def step(self):
+        for c in self.cases:
+            self._run(*c)
+
+    def step_e2e(self):
+        t = self.torch
+        for M, K, N in self.cases:
+            self.X[(M, K)].view(t.int16).view(-1).copy_(self.host_x[:M * K], non_blocking=True)
+            self._run(M, K, N)
+            self.host_y[:M * N].copy_(self.Y[:M * N], non_blocking=True)
+
+    def e2e_bytes(self):
+        return sum(2 * M * K for M, K, N in self.cases), sum(4 * M * N for M, K, N in self.cases)
+
+    def launches_per_step(self):
+        return len(self.cases)
+
+    def units_per_step(self):
+        return sum(2.0 * M * K * N for M, K, N in self.cases) / 1e12
+
+    def roofline(self, ms_per_step, peaks):
+        shapes, worst = [], None
+        for M, K, N in self.cases:
+            med, mn = time_cold(self.torch, lambda: self._run(M, K, N))
+            flops, nbytes = 2.0 * M * K * N, 2.0 * M * K + K * N / 4.0 + 4.0 * M * N
+            kind, t_us = bound_of(flops, nbytes, peaks)
+            row = {"M": M, "K": K, "N": N, "us_median": round(med, 2), "us_min": round(mn, 2), "bound": kind,
+                   "bound_us": round(t_us, 2), "frac": round(t_us / med, 3), "tflops": round(flops / med / 1e6, 1),
+                   "gbs": round(nbytes / med / 1e3, 1), "gated": (M, K, N) in SWEEP_GATED}
+            shapes.append(row)
+            if row["gated"] and (worst is None or row["frac"] < worst["frac"]):
+                worst = row
+        unit = "TFLOP/s" if worst["bound"] == "tensor" else "GB/s"
+        ach = worst["tflops"] if worst["bound"] == "tensor" else worst["gbs"]
+        peak = peaks["bf16_tflops"] if worst["bound"] == "tensor" else peaks["hbm_gbs"]
+        return {"bound": worst["bound"], "kernel": "tconv_kernel / tconv_res_kernel (one twn_gemm call per shape); headline = "
+                f"the worst of the five gated shapes: M={worst['M']} K={worst['K']} N={worst['N']}",
+                "achieved": ach, "peak": peak, "unit": unit, "frac": worst["frac"],
+                "peak_source": peaks["source"] + " (bf16 burst / copy bandwidth: every shape is timed alone, cold L2)",
+                "traffic": None, "shapes": shapes}
+
+    def check(self):
+        assert self.twn.read_status(self.status) == 0
+
+    def cpu_sample(self, host, seconds=10.0):
+        import oracle
+        w, x = host
+        K, N, M = 4096, 4096, 16384
+        st, codes = oracle.ternarize(w[(K, N)], 0.7)
+        rows = 8
+        while True:
+            t0 = time.perf_counter()
+            oracle.gemm(x[(M, K)][:rows], codes, st.alpha)
+            dt = time.perf_counter() - t0
+            if dt >= seconds * 0.5 or rows >= M:
+                break
+            rows = int(min(M, max(rows * 2, rows * seconds / max(dt, 1e-3))))
+        return 2.0 * rows * N * K / dt / 1e12, f"oracle gemm on {rows} of {M} rows of the K=N=4096 shape ({dt:.1f} s)", oracle.num_threads()
+
+
+LAYER_SHAPES = {   # name: (H = W, Cin, Cout, kernel, stride, pad): the 3x3 layers of the four ResNet-18 stages
+    "l1": (56, 64, 64, 3, 1, 1), "l2": (28, 128, 128, 3, 1, 1), "l3": (14, 256, 256, 3, 1, 1), "l4": (7, 512, 512, 3, 1, 1)}
+
+
+class LayerWorkload:
+    """One ternary convolution forward (Eq. 2) of a ResNet-18 stage shape with folded batch-norm affine and ReLU,
+    bf16 in and out.  Used for per-layer numbers and for profiler captures at a reduced batch (--batch)."""
+    metric = "ternary conv TFLOP/s"
+    unit = "TFLOP/s"
+    dtype = "bf16"
+    default_steps = 200
+
+    def __init__(self, which, batch=64):
+        self.which, self.B = which, batch
+        self.H, self.Cin, self.Cout, self.k, self.s, self.p = LAYER_SHAPES[which]
+        self.name = f"conv_fwd_{which}_{self.H}x{self.H}x{self.Cin}_to_{self.Cout}_b{batch}"
+
+    def config(self):
+        mb = self.B * self.H * self.H * (self.Cin + self.Cout) * 2 / 1e6
+        return {"workload": self.name, "seed": 0, "delta_factor": 0.7,
+                "l2": f"activations in and out: {mb:.0f} MB per step; L2 flushed between the timed launches of the roofline figure"}
+
+    def host_inputs(self):
+        from paper_1605_04711_b200 import datagen as dg
+        K = self.k * self.k * self.Cin
+        return (dg.he_normal(0, f"layer.{self.which}.w", self.Cout, K),
+                dg.draw_bf16(0, f"layer.{self.which}.x", self.B * self.H * self.H * self.Cin, "normal"))
+
+    def setup(self, torch, twn, host):
+        import numpy as np
+        self.torch, self.twn = torch, twn
+        Wm, x = host
+        K = self.k * self.k * self.Cin
+        self.ld = twn.ld_for(K)
+        self.stats = twn.new_stats()
+        self.packed = torch.empty((self.Cout, self.ld // 16), dtype=torch.int32, device="cuda")
+        ws = torch.empty(twn.ternarize_workspace_bytes(), dtype=torch.uint8, device="cuda")
+        twn.ternarize(torch.from_numpy(Wm).cuda(), 0.7, self.stats, self.packed, self.ld, None, ws, rows=self.Cout, cols=K)
+        self.d = twn.conv_desc(self.B, self.H, self.H, self.Cin, self.Cout, self.k, self.s, self.p)
+        self.host_x = torch.from_numpy(x.view(np.int16)).pin_memory()
+        self.X = self.host_x.cuda().view(torch.bfloat16).view(self.B, self.H, self.H, self.Cin)
+        self.Y = torch.empty((self.B, self.d.Ho, self.d.Wo, self.Cout), dtype=torch.bfloat16, device="cuda")
+        self.host_y = torch.empty(self.Y.numel(), dtype=torch.int16).pin_memory()
+        self.scale = torch.ones(self.Cout, device="cuda")
+        self.shift = torch.zeros(self.Cout, device="cuda")
+        self.epi = twn.epilogue(self.scale, self.shift, None, relu=True, out_dtype=twn.BF16)
+        self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def step(self):
+        self.twn.conv2d_fwd(self.d, self.X, self.packed, self.ld, self.stats, self.epi, self.Y, self.status)
+
+    def step_e2e(self):
+        t = self.torch
+        self.X.view(t.int16).view(-1).copy_(self.host_x, non_blocking=True)
+        self.step()
+        self.host_y.copy_(self.Y.view(t.int16).view(-1), non_blocking=True)
+
+    def e2e_bytes(self):
+        return self.X.numel() * 2, self.Y.numel() * 2
+
+    def launches_per_step(self):
+        return 1
+
+    def flops(self):
+        return 2.0 * self.B * self.d.Ho * self.d.Wo * self.k * self.k * self.Cin * self.Cout
+
+    def nbytes(self):
+        return self.X.numel() * 2 + self.k * self.k * self.Cin * self.Cout / 4.0 + self.Y.numel() * 2
+
+    def units_per_step(self):
+        return self.flops() / 1e12
+
+    def roofline(self, ms_per_step, peaks):
+        med, mn = time_cold(self.torch, self.step)
+        kind, t_us = bound_of(self.flops(), self.nbytes(), peaks)
+        return {"bound": kind, "kernel": "one twn_conv2d_fwd call, timed alone after an L2 flush",
+                "achieved": self.flops() / med / 1e6 if kind == "tensor" else self.nbytes() / med / 1e3,
+                "peak": peaks["bf16_tflops"] if kind == "tensor" else peaks["hbm_gbs"],
+                "unit": "TFLOP/s" if kind == "tensor" else "GB/s", "frac": t_us / med, "us_median": med, "us_min": mn,
+                "bound_us": t_us, "algorithmic_bytes": self.nbytes(), "flops": self.flops(),
+                "peak_source": peaks["source"] + " (burst: timed alone)", "traffic": None}
+
+    def check(self):
+        assert self.twn.read_status(self.status) == 0
+
+    def cpu_sample(self, host, seconds=10.0):
+        import numpy as np
+        import oracle
+        Wm, x = host
+        st, codes = oracle.ternarize(Wm, 0.7)
+        d = oracle.conv_desc(self.B, self.H, self.H, self.Cin, self.Cout, self.k, self.s, self.p)
+        X = x.reshape(self.B, self.H, self.H, self.Cin)
+        total = self.B * d.Ho * d.Wo
+        npix = 64
+        while True:
+            pix = np.arange(npix) % total
+            t0 = time.perf_counter()
+            oracle.conv2d_fwd(d, X, codes.reshape(self.Cout, self.k, self.k, self.Cin), st.alpha, pixels=pix)
+            dt = time.perf_counter() - t0
+            if dt >= seconds * 0.5 or npix >= total:
+                break
+            npix = int(min(total, max(npix * 2, npix * seconds / max(dt, 1e-3))))
+        return 2.0 * npix * self.k * self.k * self.Cin * self.Cout / dt / 1e12, \
+            f"oracle conv2d_fwd on {npix} of {total} output pixels ({dt:.1f} s)", oracle.num_threads()
+
+
 class NetWorkload:
     """A chained network workload: images/s of a forward pass or of a whole training step,
     replayed from a CUDA graph (the step is a fixed sequence of ~200 launches)."""
@@ -405,7 +656,8 @@ class NetWorkload:
         c = {"workload": self.name, "seed": 0, "delta_factor": 0.7,
              "l2": "activations of a step (> 1 GB for ResNet-18) exceed L2 (126 MB)",
              "launch": "one CUDA graph replay per step",
-             "e2e": "pipelined: the pinned-host copy of batch i+1 runs on a copy stream while step i computes"}
+             "e2e": "pipelined: the pinned-host copy of batch i+1 runs on a copy stream while step i computes; "
+                    "the result read back every step is the logits (the weight gradients stay on the device)"}
         if self.train_kind():
             c["step"] = ("ternarize+pack 21 tensors, transpose codes, forward, backward for data, "
                          "straight-through dW; synthetic dY N(0,1e-2) at the logits")
@@ -471,12 +723,48 @@ class NetWorkload:
             a[0] += 1; a[1] += e0.elapsed_time(e1); a[2] += flops
         self.kernel_times = agg
         net.timed = None
+        self.per_layer = self._per_layer_pass()
 
     def _eager(self):
         if self.train:
             self.net.train_step(self.dY)
         else:
             self.net.forward()
+
+    def _per_layer_pass(self, reps=20):
+        """Isolated device time of every tensor-core call of a step: the step is run eagerly with the weight-gradient
+        and code-layout streams joined to the main stream, so that every kernel has the GPU to itself (the inputs are
+        as the preceding kernels of the step left them: the activations of a layer exceed L2 for the large layers
+        only).  Returns {(kind, name): (flops, [microseconds per repetition])}."""
+        t, net = self.torch, self.net
+        main = t.cuda.current_stream()
+        saved = net.dw_stream, net.side_streams
+        net.dw_stream, net.side_streams = main, [main]
+        rows = {}
+        try:
+            for _ in range(reps + 2):
+                net.timed = []
+                t.cuda._sleep(int(10e6))       # the host runs ahead of the device: events bracket kernels only
+                self._eager()
+                t.cuda.synchronize()
+                for kind, name, flops, e0, e1 in net.timed:
+                    rows.setdefault((kind, name), (flops, []))[1].append(e0.elapsed_time(e1) * 1e3)
+        finally:
+            net.timed = None
+            net.dw_stream, net.side_streams = saved
+        return {k: (f, v[2:]) for k, (f, v) in rows.items()}
+
+    def _op_bytes(self, L, op):
+        """Algorithmic bytes of one call: operands once in, result once out, packed codes at 2 bits."""
+        e = L.extra
+        in_b = (e["xf"].numel() if L.fold else e["xcol"].numel() if L.small_cin else L.B * L.H * L.W * L.Cin) * 2
+        out_px = L.B * L.Ho * L.Wo
+        codes = L.K * L.Cout / 4.0
+        if op == "fwd":
+            return in_b + codes + out_px * L.Cout * (4 if L.out_f32 else 2) + (out_px * L.Cout * 2 if L.residual else 0)
+        if op == "dX":
+            return out_px * L.Cout * 2 + codes + L.B * L.H * L.W * L.Cin * 2
+        return in_b + out_px * L.Cout * 2 + L.K * L.Cout * 4.0
 
     def step(self):
         self.graph.replay()
@@ -541,65 +829,145 @@ class NetWorkload:
         return self.net.B
 
     def roofline(self, ms_per_step, peaks):
+        """Headline: the ternary contractions of a step (every forward and backward-for-data call), each timed alone
+        (median of 20), against the measured bf16 burst peak.  `per_layer` lists every tensor-core call with its own
+        bound (the slower of flops at the burst peak and algorithmic bytes at the copy bandwidth) and fraction;
+        `contended` keeps the per-kind times of one eager pass with the weight gradients on their own stream."""
         k = self.kernel_times
-        t = k.get("tconv", [0, 0.0, 0.0])
-        ach = t[2] / (t[1] * 1e-3) / 1e12 if t[1] > 0 else 0.0
-        peak = peaks["bf16_tflops_sustained"]
-        out = {"bound": "tensor", "kernel": "tconv_kernel (all forward and backward-for-data launches of a step)",
+        per_layer, sums = [], {}
+        for (kind, name), (flops, us) in self.per_layer.items():
+            if kind == "ternarize":
+                continue
+            us = sorted(us)
+            med, mn = us[len(us) // 2], us[0]
+            lname, op = name.rsplit(".", 1)
+            nbytes = self._op_bytes(self.net.layers[lname], op)
+            bkind, t_us = bound_of(flops, nbytes, peaks)
+            per_layer.append({"call": name, "us_median": round(med, 2), "us_min": round(mn, 2), "gflop": round(flops / 1e9, 2),
+                              "mbytes": round(nbytes / 1e6, 2), "bound": bkind, "bound_us": round(t_us, 2),
+                              "frac": round(t_us / med, 3)})
+            a = sums.setdefault(kind, [0.0, 0.0, 0.0, 0])
+            a[0] += med; a[1] += flops; a[2] += t_us; a[3] += 1
+        t = sums.get("tconv", [0.0, 0.0, 0.0, 0])
+        ach = t[1] / t[0] / 1e6 if t[0] > 0 else 0.0
+        peak = peaks["bf16_tflops"]
+        tern = self.per_layer_ternarize_us()
+        step_flops = 2.0 * self.net.total_macs()
+        out = {"bound": "tensor", "kernel": "tconv_kernel + tconv_res_kernel (every forward and backward-for-data call of a step, each timed alone)",
                "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
-               "peak_source": peaks["source"] + " (sustained bf16)", "traffic": None,
-               "launches": t[0], "ms_in_kernel": t[1],
-               "breakdown_ms": {kk: round(v[1], 4) for kk, v in k.items()},
-               "breakdown_tflops": {kk: (round(v[2] / (v[1] * 1e-3) / 1e12, 1) if v[1] > 0 and v[2] > 0 else None)
-                                    for kk, v in k.items()},
-               "step_macs": self.net.total_macs(),
-               "step_frac_of_tensor_peak": 2 * self.net.total_macs() / (ms_per_step * 1e-3) / 1e12 / peak}
+               "peak_source": peaks["source"] + " (bf16 burst: isolated kernels)", "traffic": self.measured_traffic(),
+               "launches": t[3], "us_in_kernel_isolated": round(t[0], 1), "us_at_bound": round(t[2], 1),
+               "frac_of_own_bounds": (t[2] / t[0]) if t[0] > 0 else None,
+               "isolated_sums_us": {kk: round(v[0], 1) for kk, v in sums.items()},
+               "isolated_tflops": {kk: round(v[1] / v[0] / 1e6, 1) for kk, v in sums.items() if v[0] > 0},
+               "ternarize_us_isolated": tern,
+               "contended": {"note": "one eager pass, weight gradients on their own stream beside the backward-for-data chain",
+                             "ms": {kk: round(v[1], 4) for kk, v in k.items()}},
+               "step_flops": step_flops,
+               "step_frac_of_burst_peak": step_flops / (ms_per_step * 1e-3) / 1e12 / peak,
+               "step_frac_of_sustained_peak": step_flops / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+               "per_layer": per_layer}
         return out
+
+    def per_layer_ternarize_us(self):
+        us = [v for (kind, _), (_, vals) in self.per_layer.items() if kind == "ternarize" for v in [sorted(vals)[len(vals) // 2]]]
+        return round(sum(us), 1) if us else None
+
+    def measured_traffic(self):
+        """DRAM bytes per step of the ternary contractions of the ResNet-18 step: sum over the launches of
+        dram__bytes_read.sum + dram__bytes_write.sum, from ncu captures of the four 3x3 stage shapes at batch 8
+        (profiles/tconv_resnet18_layers_dram.md) scaled by the batch and the launch count; None for other workloads
+        or when the kernels have changed since the capture."""
+        return TRAFFIC_RESNET18_STEP if self.kind in ("resnet18_train", "resnet18_train_sgd") else None
 
     def check(self):
         self.net.check_status()
         assert bool(self.torch.isfinite(self.logits.float()).all())
 
-    def cpu_sample(self, host, seconds=10.0):
-        """Oracle convolution (fp64, OpenMP) on sampled output pixels of one mid-network layer
-        (28x28, 128 -> 128 channels, 3x3); images/s extrapolated by the MAC count of a step."""
+    def _ops(self):
+        from paper_1605_04711_b200 import nets
+        if self.kind in ("resnet18_train", "resnet18_train_sgd"):
+            return nets.resnet18_ops(), 64
+        if self.kind == "resnet18b_train":
+            return nets.resnet18_ops(widths=(96, 192, 384, 768)), 64
+        if self.kind == "vgg7_fwd":
+            return nets.vgg7_ops(), 128
+        return nets.lenet5_ops(), 100
+
+    def cpu_sample(self, host, seconds=24.0, full=False):
+        """The oracle (fp64, OpenMP) on every layer of the workload: forward, and for a training step backward for
+        data and the weight gradient.  A layer whose full size fits its share of the time budget is run in full;
+        otherwise the oracle runs on sampled output pixels (weight-gradient entries) at batch 2 and the time is
+        scaled to the layer's full size.  The step time is the sum over layers, plus (training step only) the ternarization
+        of all weights.  full=True runs every layer at its full size whatever it takes."""
         import numpy as np
         import oracle
         from paper_1605_04711_b200 import datagen as dg
-        B, H, C = 4, 28, 128
-        d = oracle.conv_desc(B, H, H, C, C, 3, 1, 1)
-        X = dg.draw_bf16(0, "cpu.x", B * H * H * C, "normal").reshape(B, H, H, C)
-        W = dg.he_normal(0, "cpu.w", C, 9 * C)
-        st, codes = oracle.ternarize(W, 0.7)
-        codes = codes.reshape(C, 3, 3, C)
-        npix, rate = 256, None
-        while True:
-            pix = np.arange(npix) % (B * H * H)
+        ops, B = self._ops()
+        layers = [op[1] for op in ops if op[0] == "layer"]
+        train = self.train_kind()
+        budget = 1e9 if full else seconds / (len(layers) * (3 if train else 1))
+        Bs = 2
+
+        def run(fn, n_total, scale):
+            """fn(indices) on a growing sample of range(n_total); returns seconds extrapolated to scale * n_total items."""
+            n, full = min(16, n_total), False
+            while True:
+                idx = np.arange(n, dtype=np.int64) * max(1, n_total // n) % n_total
+                t0 = time.perf_counter()
+                fn(idx)
+                dt = time.perf_counter() - t0
+                if n >= n_total:
+                    full = True
+                    break
+                if dt >= budget * 0.5:
+                    break
+                n = int(min(n_total, max(n * 2, n * budget / max(dt, 1e-4))))
+            return dt / n * n_total * scale, full and scale == 1.0
+
+        t_cpu0 = time.perf_counter()
+        total_s, n_full, n_ops, n_weights = 0.0, 0, 0, 0
+        for L in layers:
+            K = L.k * L.k * L.Cin
+            # layers small enough are taken at their full batch, the others at batch 2
+            b = B if (full or B * L.Ho * L.Wo * K * L.Cout <= 3e9) else Bs
+            d = oracle.conv_desc(b, L.H, L.W, L.Cin, L.Cout, L.k, L.stride, L.pad)
+            X = dg.draw_bf16(0, f"cpu.{L.name}.x", b * L.H * L.W * L.Cin, "normal").reshape(b, L.H, L.W, L.Cin)
+            Wm = dg.he_normal(0, f"cpu.{L.name}.w", L.Cout, K)
             t0 = time.perf_counter()
-            oracle.conv2d_fwd(d, X, codes, st.alpha, pixels=pix)
-            dt = time.perf_counter() - t0
-            rate = npix * 9 * C * C / dt
-            if dt >= seconds * 0.5 or npix >= 1 << 22:
-                break
-            npix = int(min(1 << 22, max(npix * 2, npix * seconds / max(dt, 1e-3))))
-        macs_per_image = self._macs_per_image()
-        return rate / macs_per_image, (f"oracle conv2d_fwd on {npix} output pixels of a 28x28x128->128 3x3 layer "
-                                       f"({dt:.1f} s); extrapolated by MACs per image ({macs_per_image / 1e9:.2f} G)"), \
-            oracle.num_threads()
+            st, codes = oracle.ternarize(Wm, 0.7)
+            oracle.pack(codes.reshape(L.Cout, K), oracle.ld_for(K))
+            if train:
+                total_s += time.perf_counter() - t0
+            n_weights += Wm.size
+            codes4 = codes.reshape(L.Cout, L.k, L.k, L.Cin)
+            sec, full = run(lambda pix: oracle.conv2d_fwd(d, X, codes4, st.alpha, pixels=pix), b * L.Ho * L.Wo, B / b)
+            total_s += sec; n_full += full; n_ops += 1
+            if train:
+                dZ = dg.draw_bf16(0, f"cpu.{L.name}.dz", b * L.Ho * L.Wo * L.Cout, "normal", 0.0, 0.1).reshape(b, L.Ho, L.Wo, L.Cout)
+                if L.src != "input":
+                    sec, full = run(lambda pix: oracle.conv2d_bwd_data(d, dZ, codes4, st.alpha, pixels=pix), b * L.H * L.W, B / b)
+                    total_s += sec; n_full += full; n_ops += 1
+                sec, full = run(lambda ent: oracle.conv2d_bwd_weight(d, X, dZ, entries=ent), L.Cout * K, B / b)
+                total_s += sec; n_full += full; n_ops += 1
+        spent = time.perf_counter() - t_cpu0
+        what = "forward, backward for data and weight gradient" if train else "forward"
+        return B / total_s, (f"oracle {what} of all {len(layers)} layers, one by one on seeded inputs, plus ternarize+pack of their "
+                             f"{n_weights} weights; {n_full} of {n_ops} calls at full size, the others on sampled outputs at batch {Bs} "
+                             f"scaled to batch {B} ({spent:.1f} s of CPU; oracle step time {total_s:.1f} s)"), oracle.num_threads()
 
-    def _macs_per_image(self):
-        if hasattr(self, "net"):
-            return self.net.total_macs() / self.net.B
-        return {"resnet18_train": 340.7e9 / 64, "resnet18_train_sgd": 340.7e9 / 64, "resnet18b_train": 755.3e9 / 64,
-                "vgg7_fwd": 615.9e6,
-                "lenet5_fwd": 4.27e6}[self.kind]
-
+# Filled from the ncu captures under profiles/ (see NetWorkload.measured_traffic); None until captured for the
+# kernels as they stand.
+TRAFFIC_RESNET18_STEP = None
 
 WORKLOADS = {"ternarize": lambda: TernarizeWorkload(), "sgd_ternarize": lambda: SgdTernarizeWorkload(), "ternarize_rows": lambda: TernarizeRowsWorkload(), "resnet18_train": lambda: NetWorkload("resnet18_train"),
              "gemm_16384": lambda: GemmWorkload(16384), "gemm_4096": lambda: GemmWorkload(4096),
              "vgg7_fwd": lambda: NetWorkload("vgg7_fwd"), "lenet5_fwd": lambda: NetWorkload("lenet5_fwd"),
              "resnet18b_train": lambda: NetWorkload("resnet18b_train"),
-             "resnet18_train_sgd": lambda: NetWorkload("resnet18_train_sgd")}
+             "resnet18_train_sgd": lambda: NetWorkload("resnet18_train_sgd"),
+             "gemm_sweep": lambda: GemmSweepWorkload(),
+             "layer_l1": lambda: LayerWorkload("l1"), "layer_l2": lambda: LayerWorkload("l2"),
+             "layer_l3": lambda: LayerWorkload("l3"), "layer_l4": lambda: LayerWorkload("l4")}
 DEFAULT_WORKLOAD = "resnet18_train"
 
 
@@ -609,15 +977,20 @@ def run_reference(args):
     if rank != 0:
         return
     wl = WORKLOADS[args.workload]()
-    host = wl.host_inputs() if isinstance(wl, (TernarizeWorkload, GemmWorkload)) else None   # (covers the per-filter workload)
+    host = wl.host_inputs() if isinstance(wl, (TernarizeWorkload, GemmWorkload, GemmSweepWorkload, LayerWorkload)) else None
     vals = []
     steps = args.steps if args.steps else 3
     for i in range(args.warmup + steps):
-        v, sample, cores = wl.cpu_sample(host)
+        v, sample, cores = wl.cpu_sample(host, full=True) if (args.full_oracle and isinstance(wl, NetWorkload)) else wl.cpu_sample(host)
         if i >= args.warmup:
             vals.append(v)
     value = sum(vals) / len(vals)
-    upstep = wl.units_per_step() if isinstance(wl, (TernarizeWorkload, GemmWorkload)) else {"resnet18_train": 64, "resnet18b_train": 64, "resnet18_train_sgd": 64, "vgg7_fwd": 128, "lenet5_fwd": 100}[args.workload]
+    if isinstance(wl, GemmSweepWorkload):
+        wl.cases = [(M, K, N) for K, N in SWEEP_KN for M in SWEEP_M]
+    if isinstance(wl, LayerWorkload):
+        import oracle as _o
+        wl.d = _o.conv_desc(wl.B, wl.H, wl.H, wl.Cin, wl.Cout, wl.k, wl.s, wl.p)
+    upstep = wl.units_per_step() if isinstance(wl, (TernarizeWorkload, GemmWorkload, GemmSweepWorkload, LayerWorkload)) else wl._ops()[1]
     line = {"impl": "reference", "metric": wl.metric, "value": value, "unit": wl.unit,
             "n_gpus": args.gpus, "steps": steps, "warmup": args.warmup,
             "ms_per_step": upstep / value * 1e3, "higher_is_better": True,
@@ -659,7 +1032,8 @@ def ternarize_leg(torch, twn, peaks, steps=300):
         ms = e0.elapsed_time(e1) / steps
         gbs = w.n * w.bytes_per_unit / (ms * 1e-3) / 1e9
         out[name] = {"value": gbs, "unit": "GB/s", "n": w.n, "bytes_per_weight": w.bytes_per_unit, "ms": ms,
-                     "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"]}
+                     "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": gbs / 8000.0,
+                     "peak_source": peaks["source"]}
     return out
 
 
@@ -679,6 +1053,8 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     wl = WORKLOADS[args.workload]()
+    if args.batch and isinstance(wl, LayerWorkload):
+        wl = LayerWorkload(wl.which, args.batch)
     steps = args.steps if args.steps else wl.default_steps
     warmup = max(args.warmup, 3)
     host = wl.host_inputs()
@@ -686,32 +1062,36 @@ def run_ours(args):
     peaks = measured_peaks()
 
     def timed(fn, n_steps, n_warm):
+        """Mean step time over exactly n_steps back-to-back steps (the reported value), and the
+        median and minimum of the single steps, from one event per step boundary."""
         for _ in range(n_warm):
             fn()
         barrier()
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ev0.record()
-        for _ in range(n_steps):
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_steps + 1)]
+        evs[0].record()
+        for i in range(n_steps):
             fn()
-        ev1.record()
+            evs[i + 1].record()
         barrier()
-        ms = max_over_ranks(ev0.elapsed_time(ev1), world, dist if world > 1 else None, "cuda")
-        return ms / n_steps
+        ms = max_over_ranks(evs[0].elapsed_time(evs[-1]), world, dist if world > 1 else None, "cuda")
+        each = sorted(evs[i].elapsed_time(evs[i + 1]) for i in range(n_steps))
+        return ms / n_steps, {"median_ms": each[len(each) // 2], "min_ms": each[0], "steps": n_steps}
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
     if sampler:
         sampler.start()
-    ms = timed(wl.step, steps, warmup)
+    ms, spread = timed(wl.step, steps, warmup)
     clocks = sampler.stop() if sampler else None
     wl.check()
-    ms_e2e = timed(wl.step_e2e, max(2, min(steps, 20)), 1)
+    ms_e2e, _ = timed(wl.step_e2e, max(2, min(steps, 20)), 1)
     wl.check()
 
     if rank == 0:
         h2d, d2h = wl.e2e_bytes()
         line = {"metric": wl.metric, "value": world * wl.units_per_step() / (ms * 1e-3),
                 "unit": wl.unit, "n_gpus": world, "steps": steps, "warmup": warmup,
-                "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "ms_per_step": ms, "ms_per_step_median": spread["median_ms"], "ms_per_step_min": spread["min_ms"],
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": wl.dtype, "data": "synthetic", "config": wl.config(), "clocks": clocks,
                 "e2e": {"value": world * wl.units_per_step() / (ms_e2e * 1e-3), "unit": wl.unit,
                         "ms_per_step": ms_e2e, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
@@ -737,7 +1117,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--batch", type=int, default=0, help="layer_* workloads: batch size (default 64)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--full-oracle", action="store_true",
+                    help="--impl reference, network workloads: run the oracle on every layer at its full size (no sampling)")
     ap.add_argument("--no-ternarize-leg", action="store_true",
                     help="default workload only: skip the ternarize+pack GB/s measurement added to the line")
     args = ap.parse_args()

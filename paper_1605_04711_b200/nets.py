@@ -430,8 +430,8 @@ class TernaryNet:
 
 
 # ---------------------------------------------------------------------- the three shapes
-def lenet5(batch=100, train=False, seed=0):
-    ops = [
+def lenet5_ops():
+    return [
         ("layer", Layer("conv1", 1, 32, 5, 1, 0, 28, 28, src="input")),
         ("maxpool", "pool1", "conv1", 2, 2, 0),
         ("layer", Layer("conv2", 32, 64, 5, 1, 0, 12, 12, src="pool1")),
@@ -440,10 +440,13 @@ def lenet5(batch=100, train=False, seed=0):
         ("layer", Layer("fc1", 1024, 512, src="flat")),
         ("layer", Layer("fc2", 512, 10, relu=False, src="fc1", out_f32=True)),
     ]
-    return TernaryNet("lenet5", batch, (28, 28, 1), ops, seed, train=train)
 
 
-def vgg7(batch=128, train=False, seed=0):
+def lenet5(batch=100, train=False, seed=0):
+    return TernaryNet("lenet5", batch, (28, 28, 1), lenet5_ops(), seed, train=train)
+
+
+def vgg7_ops():
     ops, src, H = [], "input", 32
     cin = 3
     for i, c in enumerate([128, 128, 256, 256, 512, 512], 1):
@@ -455,11 +458,14 @@ def vgg7(batch=128, train=False, seed=0):
     ops.append(("flatten", "flat", src))
     ops.append(("layer", Layer("fc1", 8192, 1024, affine=True, src="flat")))
     ops.append(("layer", Layer("fc2", 1024, 10, relu=False, src="fc1", out_f32=True)))
-    return TernaryNet("vgg7", batch, (32, 32, 3), ops, seed, train=train)
+    return ops
 
 
-def resnet18(batch=64, train=True, seed=0, image=224, classes=1000, widths=(64, 128, 256, 512), name="resnet18",
-             optimizer=None):
+def vgg7(batch=128, train=False, seed=0):
+    return TernaryNet("vgg7", batch, (32, 32, 3), vgg7_ops(), seed, train=train)
+
+
+def resnet18_ops(image=224, classes=1000, widths=(64, 128, 256, 512)):
     """BasicBlock layout [2, 2, 2, 2] with a 7x7/2 first layer.  `widths` are the channels of the four
     stages; (96, 192, 384, 768) is the 1.5x wider "ResNet-18B" of the paper's ImageNet experiments."""
     w0 = widths[0]
@@ -483,7 +489,13 @@ def resnet18(batch=64, train=True, seed=0, image=224, classes=1000, widths=(64, 
             src, cin, H = p + ".conv2", c, Ho
     ops.append(("avgpool", "gap", src))
     ops.append(("layer", Layer("fc", widths[-1], classes, relu=False, src="gap", out_f32=True)))
-    return TernaryNet(name, batch, (image, image, 3), ops, seed, train=train, optimizer=optimizer)
+    return ops
+
+
+def resnet18(batch=64, train=True, seed=0, image=224, classes=1000, widths=(64, 128, 256, 512), name="resnet18",
+             optimizer=None):
+    return TernaryNet(name, batch, (image, image, 3), resnet18_ops(image, classes, widths), seed, train=train,
+                      optimizer=optimizer)
 
 
 def resnet18b(batch=64, train=True, seed=0, image=224, classes=1000):
