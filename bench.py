@@ -875,9 +875,9 @@ class NetWorkload:
 
     def measured_traffic(self):
         """DRAM bytes per step of the ternary contractions of the ResNet-18 step: sum over the launches of
-        dram__bytes_read.sum + dram__bytes_write.sum, from ncu captures of the four 3x3 stage shapes at batch 8
-        (profiles/tconv_resnet18_layers_dram.md) scaled by the batch and the launch count; None for other workloads
-        or when the kernels have changed since the capture."""
+        dram__bytes_read.sum + dram__bytes_write.sum over the 59 forward and backward-for-data launches of one step,
+        from one ncu capture of this workload at its full size (profiles/tconv_resnet18_step_dram.md); None for the
+        other workloads."""
         return TRAFFIC_RESNET18_STEP if self.kind in ("resnet18_train", "resnet18_train_sgd") else None
 
     def check(self):
@@ -956,9 +956,8 @@ class NetWorkload:
                              f"{n_weights} weights; {n_full} of {n_ops} calls at full size, the others on sampled outputs at batch {Bs} "
                              f"scaled to batch {B} ({spent:.1f} s of CPU; oracle step time {total_s:.1f} s)"), oracle.num_threads()
 
-# Filled from the ncu captures under profiles/ (see NetWorkload.measured_traffic); None until captured for the
-# kernels as they stand.
-TRAFFIC_RESNET18_STEP = None
+# From the ncu capture summarised in profiles/tconv_resnet18_step_dram.md (see NetWorkload.measured_traffic).
+TRAFFIC_RESNET18_STEP = 907.9e6
 
 WORKLOADS = {"ternarize": lambda: TernarizeWorkload(), "sgd_ternarize": lambda: SgdTernarizeWorkload(), "ternarize_rows": lambda: TernarizeRowsWorkload(), "resnet18_train": lambda: NetWorkload("resnet18_train"),
              "gemm_16384": lambda: GemmWorkload(16384), "gemm_4096": lambda: GemmWorkload(4096),
