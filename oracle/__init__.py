@@ -196,6 +196,50 @@ def bruteforce_enum(W):
     return codes, a.value, j.value
 
 
+# ---------------------------------------------------------------- binary weights
+def binarize(W):
+    """Binary precision weights (Sec. 3): codes = sign(W) with sign(0) = +1, alpha = mean |W|.
+    Returns (Stats, int8 codes shaped like W); delta = 0 and n_zero = 0 in the Stats."""
+    w = _f32(W)
+    st = _Stats()
+    codes = np.empty(w.shape, dtype=np.int8)
+    lib().ref_binarize(_p(w), C.c_int64(w.size), C.byref(st), _p(codes))
+    return Stats(st.delta, st.alpha, st.sum_abs, st.sum_abs_kept, st.n_neg, st.n_zero, st.n_pos,
+                 st.n_boundary, bool(st.nonfinite)), codes
+
+
+def bruteforce_enum2(W):
+    """Minimiser of ||W - alpha B||^2 over all 2^n sign vectors B and alpha >= 0 (n <= 16)."""
+    w = _f32(W)
+    codes = np.zeros(w.size, dtype=np.int8)
+    a, j = C.c_double(), C.c_double()
+    rc = lib().ref_bruteforce_enum2(_p(w), C.c_int64(w.size), _p(codes), C.byref(a), C.byref(j))
+    assert rc == 0
+    return codes, a.value, j.value
+
+
+def pack1(codes, ld_codes: int | None = None):
+    """1-bit packing of codes in {-1, +1}: uint32 [rows, ld_codes/32]."""
+    c = _i8(codes)
+    c2 = c.reshape(1, -1) if c.ndim == 1 else c.reshape(c.shape[0], -1)
+    rows, cols = c2.shape
+    ld = ld_for(cols, 128) if ld_codes is None else ld_codes
+    out = np.empty((rows, ld // 32), dtype=np.uint32)
+    rc = lib().ref_pack1(_p(c2), C.c_int64(rows), C.c_int64(cols), C.c_int64(ld), _p(out))
+    if rc != 0:
+        raise ValueError(f"ref_pack1 failed ({rc})")
+    return out
+
+
+def unpack1(packed, rows: int, cols: int, ld_codes: int):
+    p = np.ascontiguousarray(packed, dtype=np.uint32)
+    out = np.empty((rows, cols), dtype=np.int8)
+    rc = lib().ref_unpack1(_p(p), C.c_int64(rows), C.c_int64(cols), C.c_int64(ld_codes), _p(out))
+    if rc != 0:
+        raise ValueError(f"ref_unpack1 failed ({rc})")
+    return out
+
+
 # --------------------------------------------------------------------- pack
 def ld_for(cols: int, multiple: int = 64) -> int:
     return (cols + multiple - 1) // multiple * multiple

@@ -18,6 +18,8 @@
  * quotient (per layer and per filter), a hand-worked per-filter example, 3^n enumeration of Eq. 1, threshold sweeps vs. the paper's
  * closed forms for uniform / normal weights, pack round trip over all 3^16
  * words, numpy/torch fp64 matmul and conv2d, adjoint identities.
+ * The binary-weight functions (ref_binarize, ref_pack1): a hand-worked example, the 2^n enumeration, the
+ * closed form of alpha, every bit position of a word.
  * Parity unpinned: none of the functions below.
  */
 #include <math.h>
@@ -293,6 +295,99 @@ int ref_bruteforce_enum(const float *W, int64_t n, int8_t *best_codes, double *b
         }
     }
     *best_J = bJ;
+    return 0;
+}
+
+/* ------------------------------------------------------------------------
+ * Binary precision weights (Section 3: the BPWN baseline "uses the sign
+ * function to binarize the weights"), scaled like the ternary ones:
+ *   B_i   = +1 if W_i >= 0, -1 if W_i < 0     (a two-valued code has no zero;
+ *           the reading taken for W_i = 0, and for -0.0, is +1)
+ *   alpha = (1/n) * sum |W_i|                  (the minimiser of ||W - alpha B||^2
+ *           for B = sign(W): a 1-D quadratic in alpha, as Eq. 4 is for Eq. 1)
+ * st: alpha, sum_abs, n_pos, n_neg and nonfinite are written; delta = 0,
+ * n_zero = 0, sum_abs_kept = sum_abs.  Returns 0, or 1 when a weight is not finite.
+ * ---------------------------------------------------------------------- */
+int ref_binarize(const float *W, int64_t n, ref_stats *st, int8_t *codes)
+{
+    memset(st, 0, sizeof *st);
+    csum S = {0.0, 0.0};
+    for (int64_t i = 0; i < n; ++i) {
+        double w = (double)W[i];
+        if (!isfinite(w)) st->nonfinite = 1;
+        csum_add(&S, fabs(w));
+        int8_t b = (w < 0.0) ? -1 : +1;
+        if (b > 0) st->n_pos++; else st->n_neg++;
+        if (codes) codes[i] = b;
+    }
+    st->sum_abs = S.s + S.c;
+    st->sum_abs_kept = st->sum_abs;
+    if (st->nonfinite) return 1;
+    st->alpha = n > 0 ? st->sum_abs / (double)n : 0.0;
+    return 0;
+}
+
+/* Full enumeration of min over alpha >= 0 and B in {-1,+1}^n of ||W - alpha B||^2 for n <= 16: all 2^n
+ * sign vectors, each with its best alpha = max(0, W.B / n).  Writes the minimiser. */
+int ref_bruteforce_enum2(const float *W, int64_t n, int8_t *best_codes, double *best_alpha, double *best_J)
+{
+    if (n <= 0 || n > 16) return -1;
+    int8_t b[16];
+    double bJ = INFINITY;
+    for (int64_t v = 0; v < ((int64_t)1 << n); ++v) {
+        double num = 0.0;
+        for (int64_t i = 0; i < n; ++i) {
+            b[i] = ((v >> i) & 1) ? -1 : +1;
+            num += (double)W[i] * b[i];
+        }
+        double alpha = num / (double)n;
+        if (alpha < 0.0) alpha = 0.0;
+        double J = 0.0;
+        for (int64_t i = 0; i < n; ++i) {
+            double d = (double)W[i] - alpha * b[i];
+            J += d * d;
+        }
+        if (J < bJ) {
+            bJ = J; *best_alpha = alpha;
+            memcpy(best_codes, b, (size_t)n);
+        }
+    }
+    *best_J = bJ;
+    return 0;
+}
+
+/* 1-bit storage of binary codes (the paper's model-compression argument with one bit per weight,
+ * 32x smaller than fp32).  The paper fixes no encoding; this library's mirrors the 2-bit one:
+ *   bit     1 for -1, 0 for +1;
+ *   word    a row is cut into groups of 32 codes, one 32-bit word per group.  The even elements fill
+ *           the low half-word and the odd elements the high half-word, each from its top bit down:
+ *           element e (0..31) sits at bit position 15 - e/2 + 16*(e%2);
+ *   row     ld_codes/32 words (ld_codes a multiple of 32 here); the padding bits are 0.
+ * ---------------------------------------------------------------------- */
+static int bit_pos(int64_t e) { return (int)(15 - (e / 2) + 16 * (e % 2)); }
+
+int ref_pack1(const int8_t *codes, int64_t rows, int64_t cols, int64_t ld_codes, uint32_t *packed)
+{
+    if (ld_codes % 32 != 0 || ld_codes < cols) return -1;
+    int64_t wpr = ld_codes / 32;
+    for (int64_t r = 0; r < rows; ++r) {
+        for (int64_t w = 0; w < wpr; ++w) packed[r * wpr + w] = 0u;
+        for (int64_t j = 0; j < cols; ++j) {
+            int8_t t = codes[r * cols + j];
+            if (t != 1 && t != -1) return -2;
+            if (t == -1) packed[r * wpr + j / 32] |= 1u << bit_pos(j % 32);
+        }
+    }
+    return 0;
+}
+
+int ref_unpack1(const uint32_t *packed, int64_t rows, int64_t cols, int64_t ld_codes, int8_t *codes)
+{
+    if (ld_codes % 32 != 0 || ld_codes < cols) return -1;
+    int64_t wpr = ld_codes / 32;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t j = 0; j < cols; ++j)
+            codes[r * cols + j] = ((packed[r * wpr + j / 32] >> bit_pos(j % 32)) & 1u) ? -1 : +1;
     return 0;
 }
 
