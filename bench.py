@@ -237,6 +237,57 @@ class TernarizeRowsWorkload(TernarizeWorkload):
         return rows * self.cols * self.bytes_per_unit / dt / 1e9, f"oracle on {rows} of {self.rows} filters ({dt:.1f} s)", 1
 
 
+class BinarizeWorkload(TernarizeWorkload):
+    """Binary precision weights (the paper's BPWN baseline, Sec. 3): sign codes, alpha = mean |W|, 1-bit packing of
+    one fp32 tensor of 1e8 weights drawn N(0,1).  No threshold is needed, so one sweep: 4 bytes read and 1/32 byte
+    written per weight."""
+    name = "binarize_pack_n1e8_normal"
+    metric = "binarize+pack GB/s"
+    bytes_per_unit = 4.03125
+
+    def __init__(self, n=100_000_000 // 128 * 128, seed=0):
+        super().__init__(n, seed)
+
+    def config(self):
+        c = super().config()
+        c.pop("delta_factor", None)
+        return c
+
+    def setup(self, torch, twn, host_W):
+        self.torch, self.twn = torch, twn
+        self.ld = twn.ld_for_b1(self.n)
+        self.W = torch.from_numpy(host_W).cuda()
+        self.stats = twn.new_stats()
+        self.packed = torch.empty(self.ld // 32, dtype=torch.int32, device="cuda")
+        self.ws = torch.empty(twn.binarize_workspace_bytes(), dtype=torch.uint8, device="cuda")
+        self.host_W = torch.from_numpy(host_W).pin_memory()
+        self.host_packed = torch.empty(self.ld // 32, dtype=torch.int32).pin_memory()
+        self.host_stats = torch.empty(8, dtype=torch.int64).pin_memory()
+
+    def step(self):
+        self.twn.binarize(self.W, self.stats, self.packed, self.ld, self.ws, rows=1, cols=self.n)
+
+    def e2e_bytes(self):
+        return self.n * 4, self.ld // 8 + 64
+
+    def launches_per_step(self):
+        return 1
+
+    def roofline(self, ms_per_step, peaks):
+        r = super().roofline(ms_per_step, peaks)
+        r["kernel"] = "binarize_kernel (one twn_binarize call)"
+        r["traffic"] = None
+        return r
+
+    def cpu_sample(self, host_W):
+        import oracle
+        t0 = time.perf_counter()
+        st, codes = oracle.binarize(host_W)
+        oracle.pack1(codes, self.ld)
+        dt = time.perf_counter() - t0
+        return self.n * self.bytes_per_unit / dt / 1e9, f"full tensor, n={self.n}", 1
+
+
 class SgdTernarizeWorkload(TernarizeWorkload):
     """End of one iteration and start of the next (Algorithm 1): SGD-with-momentum update of 1e8 fp32
     master weights fused with the threshold reduction of the updated weights, then the coding sweep
@@ -959,7 +1010,7 @@ class NetWorkload:
 # From the ncu capture summarised in profiles/tconv_resnet18_step_dram.md (see NetWorkload.measured_traffic).
 TRAFFIC_RESNET18_STEP = 907.9e6
 
-WORKLOADS = {"ternarize": lambda: TernarizeWorkload(), "sgd_ternarize": lambda: SgdTernarizeWorkload(), "ternarize_rows": lambda: TernarizeRowsWorkload(), "resnet18_train": lambda: NetWorkload("resnet18_train"),
+WORKLOADS = {"ternarize": lambda: TernarizeWorkload(), "binarize": lambda: BinarizeWorkload(), "sgd_ternarize": lambda: SgdTernarizeWorkload(), "ternarize_rows": lambda: TernarizeRowsWorkload(), "resnet18_train": lambda: NetWorkload("resnet18_train"),
              "gemm_16384": lambda: GemmWorkload(16384), "gemm_4096": lambda: GemmWorkload(4096),
              "vgg7_fwd": lambda: NetWorkload("vgg7_fwd"), "lenet5_fwd": lambda: NetWorkload("lenet5_fwd"),
              "resnet18b_train": lambda: NetWorkload("resnet18b_train"),

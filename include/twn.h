@@ -373,6 +373,54 @@ int twn_conv2d_bwd_weight(const twn_conv_desc_t *desc, const void *X, const void
                           void *workspace, size_t workspace_bytes, int32_t *dev_status,
                           twn_stream_t stream);
 
+/* ---- binary precision weights (Sec. 3: the BPWN baseline of the experiments) -------- */
+
+/*
+ * The paper compares ternary weights with binary precision weights, which "use the sign function to
+ * binarize the weights" and, like the ternary ones, carry one scale per layer.  The same contraction
+ * kernels run on them from a 1-bit packing:
+ *   B_i   = +1 if W_i >= 0, -1 if W_i < 0   (a two-valued code has no zero: W_i = 0 and -0.0 give +1)
+ *   alpha = (1/n) * sum_i |W_i|               (the scale that minimises ||W - alpha B||^2 for B = sign W)
+ * One sweep over the weights (no threshold is needed): 4 bytes read, 1/32 byte written per weight.
+ *   W       fp32 [rows, cols], contiguous, 4-byte aligned.
+ *   stats   one twn_stats_t: alpha, sum_abs (= sum_abs_kept), n_pos, n_neg, status are written;
+ *           delta = 0 and n_zero = 0.  TWN_ERR_NONFINITE as for twn_ternarize.
+ *   packed  uint32 [rows][ld_codes/32].  A bit is 1 for -1 and 0 for +1.  Code j of a row lives in
+ *           word j/32; inside the word the even elements fill the low half-word and the odd elements
+ *           the high half-word, each from its top bit down: element e = j%32 is bit 15 - e/2 + 16*(e%2)
+ *           (a left shift by e/2 and one mask turn elements e, e+1 into the sign bits of a bf16 pair).
+ *           ld_codes is a multiple of 128 (rows start 16-byte aligned), ld_codes >= cols; padding bits
+ *           are 0.  16-byte aligned.
+ *   workspace  at least twn_binarize_workspace_bytes(), 256-byte aligned, as for twn_ternarize.
+ * Deterministic (fixed-order fp64 sum).
+ */
+size_t twn_binarize_workspace_bytes(void);
+int twn_binarize(const float *W, int64_t rows, int64_t cols, twn_stats_t *stats, uint32_t *packed,
+                 int64_t ld_codes, void *workspace, size_t workspace_bytes, twn_stream_t stream);
+
+/* int8 codes (+1 / -1) from 1-bit packed rows; [Cout][kh][kw][Cin] -> [Cin][kh][kw][Cout] re-layout of
+ * 1-bit codes for the backward-for-data pass (as twn_unpack and twn_transpose_codes for ternary codes). */
+int twn_unpack_b1(const uint32_t *packed, int64_t rows, int64_t cols, int64_t ld_codes, int8_t *codes,
+                  twn_stream_t stream);
+int twn_transpose_codes_b1(const uint32_t *packed_fwd, int64_t ld_fwd, const twn_conv_desc_t *desc,
+                           uint32_t *packed_bwd, int64_t ld_bwd, twn_stream_t stream);
+
+/* twn_gemm, twn_conv2d_fwd and twn_conv2d_bwd_data on 1-bit binary codes: Y = epi(alpha * X (*) B), the
+ * forward block of Eq. 2 and the backward pass of Algorithm 1 with B = sign(W) in place of the ternary
+ * W~.  Arguments as for the ternary calls, except that the packed rows are in the 1-bit layout above
+ * (row pitch a multiple of 128 codes) and that a filter with more than one tap needs channel runs of
+ * 32 codes (Cin % 32 == 0 forward, Cout % 32 == 0 backward) instead of 16. */
+int twn_gemm_b1(const void *X, int64_t ldx, const uint32_t *B_packed, int64_t ld_codes,
+                const twn_stats_t *stats, int64_t M, int64_t N, int64_t K,
+                const twn_epilogue_t *epi, void *Y, int64_t ldy, int32_t *dev_status,
+                twn_stream_t stream);
+int twn_conv2d_fwd_b1(const twn_conv_desc_t *desc, const void *X, const uint32_t *B_fwd, int64_t ld_codes,
+                      const twn_stats_t *stats, const twn_epilogue_t *epi, void *Y,
+                      int32_t *dev_status, twn_stream_t stream);
+int twn_conv2d_bwd_data_b1(const twn_conv_desc_t *desc, const void *dZ, const uint32_t *B_bwd, int64_t ld_codes,
+                           const twn_stats_t *stats, const twn_epilogue_t *epi, void *dX,
+                           int32_t *dev_status, twn_stream_t stream);
+
 /* ---- layer glue (Sec. 2.4: conv, affine, ReLU, pooling; standard back-propagation) ---- */
 
 /*

@@ -164,6 +164,10 @@ __device__ __forceinline__ void ld_nc_v4(uint4 &v, const uint32_t *p)
 {
     asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
 }
+__device__ __forceinline__ void ld_nc_v2(uint32_t &x, uint32_t &y, const uint32_t *p)
+{
+    asm volatile("ld.global.nc.v2.u32 {%0, %1}, [%2];" : "=r"(x), "=r"(y) : "l"(p));
+}
 __device__ __forceinline__ void ld_nc_u32(uint32_t &v, const uint32_t *p)
 {
     asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v) : "l"(p));
@@ -242,6 +246,33 @@ __device__ __forceinline__ uint32_t pair_to_bf16x2(uint32_t w, int j)
 {
     return (w << (2 * j)) & 0xC000C000u;
 }
+
+// Binary codes, one bit per weight (1 = -1): element pair j (0..15) of a word has its two bits j below the
+// top of the two half-words; shifted to the top they are the sign bits of a bf16 pair, and 0x3F80 is 1.0.
+// One shift and one three-input logic operation per pair; the decoded values are exactly +-1.
+__device__ __forceinline__ uint32_t pair_to_bf16x2_b1(uint32_t w, int j)
+{
+    return ((w << j) & 0x80008000u) | 0x3F803F80u;
+}
+// The 64 codes of one k-block -> 32 bf16 pairs.  BITS = 2: four words of ternary codes (values +-2 / 0);
+// BITS = 1: two words of binary codes (values +-1).
+template <int BITS>
+__device__ __forceinline__ void decode_kblock(const uint32_t (&wv)[4], uint32_t (&out)[32])
+{
+    if (BITS == 2) {
+#pragma unroll
+        for (int g = 0; g < 4; ++g)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) out[g * 8 + e] = pair_to_bf16x2(wv[g], e);
+    } else {
+#pragma unroll
+        for (int g = 0; g < 2; ++g)
+#pragma unroll
+            for (int e = 0; e < 16; ++e) out[g * 16 + e] = pair_to_bf16x2_b1(wv[g], e);
+    }
+}
+// what a decoded +1 is worth: taken out again with the scale of the epilogue
+template <int BITS> __host__ __device__ constexpr float decoded_unit() { return BITS == 2 ? kDecodedUnit : 1.0f; }
 
 // ---------------------------------------------------------------- the kernel
 

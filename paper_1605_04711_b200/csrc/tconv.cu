@@ -151,7 +151,7 @@ static_assert(offsetof(SmemLayout<128>, stage_res) % 128 == 0 && offsetof(SmemLa
                   offsetof(SmemLayout<128>, stage_out) % 128 == 0 && offsetof(SmemLayout<256>, stage_out) % 128 == 0,
               "TMA and vector accesses need aligned shared-memory regions");
 
-template <int PIX, int DS>
+template <int PIX, int DS, int BITS>
 __global__ void __launch_bounds__(threads_conv(DS), 1)
 tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
              const __grid_constant__ CUtensorMap map_r, const __grid_constant__ ConvParams P)
@@ -161,6 +161,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
     constexpr int kOutBufs = Cfg<PIX>::kOutBufs;
     constexpr int kXBytes = L::kXBytes;
     constexpr int kAColsPerStage = kSub * kAColsPerBlock;
+    constexpr int kCodesPerWord = 32 / BITS, kWordsPerBlock = kBlockK / kCodesPerWord;   // 16 and 4, or 32 and 2
     static_assert(kAccBufs * PIX + kStages * kAColsPerStage <= (int)kTmemCols, "tensor memory budget");
     
 
@@ -190,7 +191,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
     constexpr int kFirstEpiWarp = first_epi_warp(DS), kThreadsConv = threads_conv(DS);
     for (int u = threadIdx.x; u < kbpt && u < kWordTab; u += kThreadsConv) {
         const int t = u / P.n_cblk, cb = u - t * P.n_cblk;
-        sm->kword[u] = (uint32_t)(P.taps[t].koff >> 4) + cb * (kBlockK / 16);
+        sm->kword[u] = (uint32_t)(P.taps[t].koff / kCodesPerWord) + cb * kWordsPerBlock;
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)), "r"(kTmemCols) : "memory");
@@ -291,16 +292,26 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     word = sm->kword[u];
                 } else {
                     const int t = u / P.n_cblk, cb = u - t * P.n_cblk;
-                    word = (P.taps[t].koff >> 4) + cb * (kBlockK / 16);
+                    word = (P.taps[t].koff / kCodesPerWord) + cb * kWordsPerBlock;
                 }
-                if (P.codes_aligned) {
-                    ld_nc_v4(c.v[sb], rowp + word);
+                if (BITS == 2) {
+                    if (P.codes_aligned) {
+                        ld_nc_v4(c.v[sb], rowp + word);
+                    } else {
+                        const long long last = P.wpr - 1;
+                        ld_nc_u32(c.v[sb].x, rowp + (word + 0 < last ? word + 0 : last));
+                        ld_nc_u32(c.v[sb].y, rowp + (word + 1 < last ? word + 1 : last));
+                        ld_nc_u32(c.v[sb].z, rowp + (word + 2 < last ? word + 2 : last));
+                        ld_nc_u32(c.v[sb].w, rowp + (word + 3 < last ? word + 3 : last));
+                    }
                 } else {
-                    const long long last = P.wpr - 1;
-                    ld_nc_u32(c.v[sb].x, rowp + (word + 0 < last ? word + 0 : last));
-                    ld_nc_u32(c.v[sb].y, rowp + (word + 1 < last ? word + 1 : last));
-                    ld_nc_u32(c.v[sb].z, rowp + (word + 2 < last ? word + 2 : last));
-                    ld_nc_u32(c.v[sb].w, rowp + (word + 3 < last ? word + 3 : last));
+                    if (P.codes_aligned) {
+                        ld_nc_v2(c.v[sb].x, c.v[sb].y, rowp + word);
+                    } else {
+                        const long long last = P.wpr - 1;
+                        ld_nc_u32(c.v[sb].x, rowp + (word + 0 < last ? word + 0 : last));
+                        ld_nc_u32(c.v[sb].y, rowp + (word + 1 < last ? word + 1 : last));
+                    }
                 }
             }
         };
@@ -352,10 +363,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     if (sb < nsb) {
                         const uint32_t wv[4] = {cur.v[sb].x, cur.v[sb].y, cur.v[sb].z, cur.v[sb].w};
                         uint32_t out[32];
-#pragma unroll
-                        for (int g = 0; g < 4; ++g)
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) out[g * 8 + e] = pair_to_bf16x2(wv[g], e);
+                        decode_kblock<BITS>(wv, out);
                         tmem_st32(lane_base + s * kAColsPerStage + sb * kAColsPerBlock, out);
                     }
                 }
@@ -403,8 +411,8 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         const int q = warp & 3;
         const int es = (warp - kFirstEpiWarp) >> 2;          // which of the two warps of the quadrant
         const int ewi = warp - kFirstEpiWarp;                // buffer set of this warp
-        // decoded weights are +-2, so half of alpha scales the accumulators
-        const float alpha = (P.alpha ? (float)(*P.alpha) : 1.0f) * (1.0f / kDecodedUnit);
+        // decoded ternary weights are +-2, so half of alpha scales the accumulators
+        const float alpha = (P.alpha ? (float)(*P.alpha) : 1.0f) * (1.0f / decoded_unit<BITS>());
         const int BWm = (1 << P.lgBW) - 1, BHm = (1 << P.lgBH) - 1;
         const bool out_bf16 = P.out_dtype == TWN_BF16, res_bf16 = P.res_dtype == TWN_BF16;
         const bool need_off = !P.tma_store || (P.residual && !P.res_tma);
@@ -599,14 +607,14 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
 }
 
 // ---------------------------------------------------------------- host side
-template <int PIX, int DS>
+template <int PIX, int DS, int BITS>
 int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const twn_device_info &dev,
                   EncodeTiledFn enc, cudaStream_t s)
 {
     static bool attr_set[64] = {false};
     const int smem_bytes = (int)sizeof(SmemLayout<PIX>) + 1024;
     if (!attr_set[dev.ordinal]) {
-        TWN_CUDA_OK(cudaFuncSetAttribute(tconv_kernel<PIX, DS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
+        TWN_CUDA_OK(cudaFuncSetAttribute(tconv_kernel<PIX, DS, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
         attr_set[dev.ordinal] = true;
     }
     pick_tile(g, PIX, &P.lgBW, &P.lgBH);
@@ -679,7 +687,7 @@ int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const twn_dev
         }
     }
     const int grid = dev.sm_count < P.total_tiles ? dev.sm_count : P.total_tiles;
-    tconv_kernel<PIX, DS><<<grid, threads_conv(DS), smem_bytes, s>>>(map_x, map_y, map_r, P);
+    tconv_kernel<PIX, DS, BITS><<<grid, threads_conv(DS), smem_bytes, s>>>(map_x, map_y, map_r, P);
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }
@@ -719,7 +727,7 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     for (int t = 0; t < g.n_taps; ++t)
         if (g.taps[t].koff % kBlockK != 0) P.codes_aligned = 0;
     P.T = T;
-    P.wpr = g.ld_codes / 16;
+    P.wpr = g.ld_codes / (g.code_bits == 1 ? 32 : 16);
     P.sw = g.sw; P.sh = g.sh;
     P.Bv = g.Bv; P.Hv = g.Hv; P.Wv = g.Wv;
     P.OH = g.OH; P.OW = g.OW; P.osh = g.osh; P.osw = g.osw; P.ooh = g.ooh; P.oow = g.oow;
@@ -764,9 +772,14 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     int choice = c256 < c128 ? 1 : 0;
     if (c192 < (choice ? c256 : c128)) choice = 2;
     P.dsets = (choice != 1 && two) ? 2 : 1;
-    if (choice == 1) return launch_conv_t<256, 1>(g, P, X, dev, enc, s);
-    if (choice == 2) return P.dsets == 2 ? launch_conv_t<192, 2>(g, P, X, dev, enc, s) : launch_conv_t<192, 1>(g, P, X, dev, enc, s);
-    return P.dsets == 2 ? launch_conv_t<128, 2>(g, P, X, dev, enc, s) : launch_conv_t<128, 1>(g, P, X, dev, enc, s);
+    if (g.code_bits == 1) {
+        if (choice == 1) return launch_conv_t<256, 1, 1>(g, P, X, dev, enc, s);
+        if (choice == 2) return P.dsets == 2 ? launch_conv_t<192, 2, 1>(g, P, X, dev, enc, s) : launch_conv_t<192, 1, 1>(g, P, X, dev, enc, s);
+        return P.dsets == 2 ? launch_conv_t<128, 2, 1>(g, P, X, dev, enc, s) : launch_conv_t<128, 1, 1>(g, P, X, dev, enc, s);
+    }
+    if (choice == 1) return launch_conv_t<256, 1, 2>(g, P, X, dev, enc, s);
+    if (choice == 2) return P.dsets == 2 ? launch_conv_t<192, 2, 2>(g, P, X, dev, enc, s) : launch_conv_t<192, 1, 2>(g, P, X, dev, enc, s);
+    return P.dsets == 2 ? launch_conv_t<128, 2, 2>(g, P, X, dev, enc, s) : launch_conv_t<128, 1, 2>(g, P, X, dev, enc, s);
 }
 
 // Helper streams for launches that are independent of one another (the residue classes of a
@@ -810,15 +823,18 @@ int check_epilogue(const twn_epilogue_t *e)
 
 }  // namespace
 
-extern "C" int twn_gemm(const void *X, int64_t ldx, const uint32_t *T_packed, int64_t ld_codes,
-                        const twn_stats_t *stats, int64_t M, int64_t N, int64_t K,
-                        const twn_epilogue_t *epi, void *Y, int64_t ldy, int32_t *dev_status,
-                        twn_stream_t stream)
+namespace {
+
+// Shared by the ternary (bits = 2) and binary (bits = 1) entry points.
+int gemm_impl(const void *X, int64_t ldx, const uint32_t *T_packed, int64_t ld_codes,
+              const twn_stats_t *stats, int64_t M, int64_t N, int64_t K,
+              const twn_epilogue_t *epi, void *Y, int64_t ldy, int32_t *dev_status,
+              twn_stream_t stream, int bits)
 {
     TWN_REQUIRE(M >= 0 && N >= 0 && K >= 0, TWN_ERR_INVALID_ARG);
     if (M == 0 || N == 0) return TWN_OK;
     TWN_REQUIRE(X && T_packed && Y && K > 0, TWN_ERR_INVALID_ARG);
-    TWN_REQUIRE(ldx >= K && ldy >= N && ld_codes >= K && ld_codes % 64 == 0, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(ldx >= K && ldy >= N && ld_codes >= K && ld_codes % (bits == 1 ? 128 : 64) == 0, TWN_ERR_INVALID_ARG);
     TWN_REQUIRE(M <= 0x7fffffffLL && N <= 0x7fffffffLL && K <= 0x7fffffffLL, TWN_ERR_INVALID_ARG);
     TWN_REQUIRE(ldx % 8 == 0, TWN_ERR_MISALIGNED);
     TWN_REQUIRE(twn_aligned(X, 16) && twn_aligned(T_packed, 16) && twn_aligned(Y, 4) && twn_aligned(stats, 8) &&
@@ -834,7 +850,26 @@ extern "C" int twn_gemm(const void *X, int64_t ldx, const uint32_t *T_packed, in
     g.Cout = (int)N; g.ld_codes = ld_codes; g.code_cols = K;
     g.n_taps = 1; g.taps[0] = Tap{0, 0, 0};
     g.Cin = K;
+    g.code_bits = bits;
     return launch_conv(g, X, T_packed, stats, epi, Y, TWN_F32, dev_status, twn_cu(stream));
+}
+
+}  // namespace
+
+extern "C" int twn_gemm(const void *X, int64_t ldx, const uint32_t *T_packed, int64_t ld_codes,
+                        const twn_stats_t *stats, int64_t M, int64_t N, int64_t K,
+                        const twn_epilogue_t *epi, void *Y, int64_t ldy, int32_t *dev_status,
+                        twn_stream_t stream)
+{
+    return gemm_impl(X, ldx, T_packed, ld_codes, stats, M, N, K, epi, Y, ldy, dev_status, stream, 2);
+}
+
+extern "C" int twn_gemm_b1(const void *X, int64_t ldx, const uint32_t *B_packed, int64_t ld_codes,
+                           const twn_stats_t *stats, int64_t M, int64_t N, int64_t K,
+                           const twn_epilogue_t *epi, void *Y, int64_t ldy, int32_t *dev_status,
+                           twn_stream_t stream)
+{
+    return gemm_impl(X, ldx, B_packed, ld_codes, stats, M, N, K, epi, Y, ldy, dev_status, stream, 1);
 }
 
 namespace {
@@ -855,17 +890,19 @@ int conv_common_checks(const twn_conv_desc_t *d)
 
 }  // namespace
 
-extern "C" int twn_conv2d_fwd(const twn_conv_desc_t *d, const void *X, const uint32_t *T_fwd, int64_t ld_codes,
-                              const twn_stats_t *stats, const twn_epilogue_t *epi, void *Y,
-                              int32_t *dev_status, twn_stream_t stream)
+namespace {
+
+int conv_fwd_impl(const twn_conv_desc_t *d, const void *X, const uint32_t *T_fwd, int64_t ld_codes,
+                  const twn_stats_t *stats, const twn_epilogue_t *epi, void *Y,
+                  int32_t *dev_status, twn_stream_t stream, int bits)
 {
     int rc = conv_common_checks(d);
     if (rc != TWN_OK) return rc;
     TWN_REQUIRE(X && T_fwd && Y, TWN_ERR_INVALID_ARG);
     const long long taps = (long long)d->kh * d->kw;
-    TWN_REQUIRE(ld_codes % 64 == 0 && ld_codes >= taps * d->Cin, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(ld_codes % (bits == 1 ? 128 : 64) == 0 && ld_codes >= taps * d->Cin, TWN_ERR_INVALID_ARG);
     // channel runs must start on 16-byte boundaries for TMA, tap columns on word boundaries
-    TWN_REQUIRE(d->Cin % 8 == 0 && (taps == 1 || d->Cin % 16 == 0), TWN_ERR_MISALIGNED);
+    TWN_REQUIRE(d->Cin % 8 == 0 && (taps == 1 || d->Cin % (bits == 1 ? 32 : 16) == 0), TWN_ERR_MISALIGNED);
     TWN_REQUIRE(twn_aligned(X, 16) && twn_aligned(T_fwd, 16) && twn_aligned(Y, 4) && twn_aligned(stats, 8) &&
                     twn_aligned(dev_status, 4), TWN_ERR_MISALIGNED);
     rc = check_epilogue(epi);
@@ -887,7 +924,24 @@ extern "C" int twn_conv2d_fwd(const twn_conv_desc_t *d, const void *X, const uin
             t.dw = (int16_t)(s - d->pad_w);
             t.koff = (int32_t)((r * d->kw + s) * d->Cin);
         }
+    g.code_bits = bits;
     return launch_conv(g, X, T_fwd, stats, epi, Y, TWN_F32, dev_status, twn_cu(stream));
+}
+
+}  // namespace
+
+extern "C" int twn_conv2d_fwd(const twn_conv_desc_t *d, const void *X, const uint32_t *T_fwd, int64_t ld_codes,
+                              const twn_stats_t *stats, const twn_epilogue_t *epi, void *Y,
+                              int32_t *dev_status, twn_stream_t stream)
+{
+    return conv_fwd_impl(d, X, T_fwd, ld_codes, stats, epi, Y, dev_status, stream, 2);
+}
+
+extern "C" int twn_conv2d_fwd_b1(const twn_conv_desc_t *d, const void *X, const uint32_t *B_fwd, int64_t ld_codes,
+                                 const twn_stats_t *stats, const twn_epilogue_t *epi, void *Y,
+                                 int32_t *dev_status, twn_stream_t stream)
+{
+    return conv_fwd_impl(d, X, B_fwd, ld_codes, stats, epi, Y, dev_status, stream, 1);
 }
 
 extern "C" int twn_conv2d_fwd_folded(const twn_conv_desc_t *d, const void *Xf, const uint32_t *Tf, int64_t ld_folded,
@@ -920,19 +974,22 @@ extern "C" int twn_conv2d_fwd_folded(const twn_conv_desc_t *d, const void *Xf, c
         t.dw = 0;
         t.koff = (int32_t)(r * 64);
     }
+    g.code_bits = 2;
     return launch_conv(g, Xf, Tf, stats, epi, Y, TWN_F32, dev_status, twn_cu(stream));
 }
 
-extern "C" int twn_conv2d_bwd_data(const twn_conv_desc_t *d, const void *dZ, const uint32_t *T_bwd, int64_t ld_codes,
-                                   const twn_stats_t *stats, const twn_epilogue_t *epi, void *dX,
-                                   int32_t *dev_status, twn_stream_t stream)
+namespace {
+
+int conv_bwd_data_impl(const twn_conv_desc_t *d, const void *dZ, const uint32_t *T_bwd, int64_t ld_codes,
+                       const twn_stats_t *stats, const twn_epilogue_t *epi, void *dX,
+                       int32_t *dev_status, twn_stream_t stream, int bits)
 {
     int rc = conv_common_checks(d);
     if (rc != TWN_OK) return rc;
     TWN_REQUIRE(dZ && T_bwd && dX, TWN_ERR_INVALID_ARG);
     const long long taps = (long long)d->kh * d->kw;
-    TWN_REQUIRE(ld_codes % 64 == 0 && ld_codes >= taps * d->Cout, TWN_ERR_INVALID_ARG);
-    TWN_REQUIRE(d->Cout % 8 == 0 && (taps == 1 || d->Cout % 16 == 0), TWN_ERR_MISALIGNED);
+    TWN_REQUIRE(ld_codes % (bits == 1 ? 128 : 64) == 0 && ld_codes >= taps * d->Cout, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(d->Cout % 8 == 0 && (taps == 1 || d->Cout % (bits == 1 ? 32 : 16) == 0), TWN_ERR_MISALIGNED);
     TWN_REQUIRE(twn_aligned(dZ, 16) && twn_aligned(T_bwd, 16) && twn_aligned(dX, 4) && twn_aligned(stats, 8) &&
                     twn_aligned(dev_status, 4), TWN_ERR_MISALIGNED);
     rc = check_epilogue(epi);
@@ -988,6 +1045,7 @@ extern "C" int twn_conv2d_bwd_data(const twn_conv_desc_t *d, const void *dZ, con
                     t.koff = (int32_t)((r * d->kw + s) * d->Cout);
                 }
             }
+            g.code_bits = bits;
             rc = launch_conv(g, dZ, T_bwd, stats, epi, dX, TWN_F32, dev_status, s);
             if (rc != TWN_OK && first_error == TWN_OK) first_error = rc;
         }
@@ -999,5 +1057,21 @@ extern "C" int twn_conv2d_bwd_data(const twn_conv_desc_t *d, const void *dZ, con
         }
     }
     return first_error;
+}
+
+}  // namespace
+
+extern "C" int twn_conv2d_bwd_data(const twn_conv_desc_t *d, const void *dZ, const uint32_t *T_bwd, int64_t ld_codes,
+                                   const twn_stats_t *stats, const twn_epilogue_t *epi, void *dX,
+                                   int32_t *dev_status, twn_stream_t stream)
+{
+    return conv_bwd_data_impl(d, dZ, T_bwd, ld_codes, stats, epi, dX, dev_status, stream, 2);
+}
+
+extern "C" int twn_conv2d_bwd_data_b1(const twn_conv_desc_t *d, const void *dZ, const uint32_t *B_bwd, int64_t ld_codes,
+                                      const twn_stats_t *stats, const twn_epilogue_t *epi, void *dX,
+                                      int32_t *dev_status, twn_stream_t stream)
+{
+    return conv_bwd_data_impl(d, dZ, B_bwd, ld_codes, stats, epi, dX, dev_status, stream, 1);
 }
 

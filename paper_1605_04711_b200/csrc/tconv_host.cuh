@@ -47,6 +47,7 @@ struct Geometry {
     int sh, sw;      // input step per virtual output pixel
     int Cout;
     long long ld_codes, code_cols;  // packed row pitch and used columns
+    int code_bits;   // 2: ternary codes, 16 per word; 1: binary codes, 32 per word
     int n_taps;
     Tap taps[kMaxTaps];
     long long Cin;   // channels per tap

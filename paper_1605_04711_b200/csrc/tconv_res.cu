@@ -76,7 +76,8 @@ struct ResParams {
     int Cout;
     const uint32_t *T;            // packed codes, one row of `wpr` words per output channel
     long long wpr;
-    int codes_aligned;            // 1: every k-block starts on a 16-byte boundary of the packed row
+    int codes_aligned;            // 1: every k-block starts on a 64-code boundary of the packed row
+    int code_bits;                // 2: ternary codes; 1: binary codes
     int w_lo, h_lo;               // smallest tap offsets: origin of the halo
     int stage_bytes, stage_tx;    // pitch of an activation stage (multiple of 1024), bytes one load delivers
     int n_stages;
@@ -180,7 +181,7 @@ tconv_res_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     // per-channel scale and shift; the decoded weights are +-2, so half of alpha scales the accumulators
     if (threadIdx.x < kNMax) {
         const int c = threadIdx.x;
-        const float alpha = (P.alpha ? (float)(*P.alpha) : 1.0f) * (1.0f / kDecodedUnit);
+        const float alpha = (P.alpha ? (float)(*P.alpha) : 1.0f) * (P.code_bits == 2 ? 1.0f / kDecodedUnit : 1.0f);
         const bool c_ok = c < P.Cout;
         ctl->sc[c] = ((P.scale && c_ok) ? __ldg(P.scale + c) : 1.0f) * alpha;
         ctl->sf[c] = (P.shift && c_ok) ? __ldg(P.shift + c) : 0.0f;
@@ -197,27 +198,35 @@ tconv_res_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         for (int i = threadIdx.x; i < items; i += kThreads) {
             const int u = i / P.N, n = i - u * P.N;
             const int t = u / P.n_cblk, cb = u - t * P.n_cblk;
-            const long long word = (P.koff[t] >> 4) + cb * (kBlockK / 16);
             const uint32_t *rowp = P.T + (long long)(n < P.Cout ? n : P.Cout - 1) * P.wpr;
-            uint32_t wv[4];
-            if (P.codes_aligned) {
-                uint4 c;
-                ld_nc_v4(c, rowp + word);
-                wv[0] = c.x; wv[1] = c.y; wv[2] = c.z; wv[3] = c.w;
-            } else {
-                const long long last = P.wpr - 1;
+            uint32_t wv[4] = {0u, 0u, 0u, 0u};
+            const long long last = P.wpr - 1;
+            if (P.code_bits == 2) {
+                const long long word = (P.koff[t] >> 4) + cb * (kBlockK / 16);
+                if (P.codes_aligned) {
+                    uint4 c;
+                    ld_nc_v4(c, rowp + word);
+                    wv[0] = c.x; wv[1] = c.y; wv[2] = c.z; wv[3] = c.w;
+                } else {
 #pragma unroll
-                for (int g = 0; g < 4; ++g) ld_nc_u32(wv[g], rowp + (word + g < last ? word + g : last));
+                    for (int g = 0; g < 4; ++g) ld_nc_u32(wv[g], rowp + (word + g < last ? word + g : last));
+                }
+            } else {
+                const long long word = (P.koff[t] >> 5) + cb * (kBlockK / 32);
+#pragma unroll
+                for (int g = 0; g < 2; ++g) ld_nc_u32(wv[g], rowp + (word + g < last ? word + g : last));
             }
-            if (n >= P.Cout) wv[0] = wv[1] = wv[2] = wv[3] = 0u;
+            uint32_t out[32];
+            if (P.code_bits == 2) decode_kblock<2>(wv, out);
+            else decode_kblock<1>(wv, out);
+            if (n >= P.Cout) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) out[j] = 0u;
+            }
             const uint32_t dst = wts + (uint32_t)(u * P.N + n) * 128u;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const uint32_t w = wv[j >> 1];
-                const int e0 = (j & 1) * 4;
-                st_shared_v4(dst + (uint32_t)((j ^ (n & 7)) << 4), pair_to_bf16x2(w, e0), pair_to_bf16x2(w, e0 + 1),
-                             pair_to_bf16x2(w, e0 + 2), pair_to_bf16x2(w, e0 + 3));
-            }
+            for (int j = 0; j < 8; ++j)
+                st_shared_v4(dst + (uint32_t)((j ^ (n & 7)) << 4), out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
         }
         // the tensor core reads shared memory through the async proxy
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -481,7 +490,7 @@ int twn_detail::launch_conv_resident(const Geometry &g, const void *X, const uin
     P.codes_aligned = 1;
     int w_lo = 0, w_hi = 0, h_lo = 0, h_hi = 0;
     for (int t = 0; t < g.n_taps; ++t) {
-        if (g.taps[t].koff % 16 != 0) return TWN_OK;          // code words must not straddle taps
+        if (g.taps[t].koff % (g.code_bits == 1 ? 32 : 16) != 0) return TWN_OK;   // code words must not straddle taps
         if (g.taps[t].koff % kBlockK != 0) P.codes_aligned = 0;
         P.koff[t] = g.taps[t].koff;
         if (t == 0) { w_lo = w_hi = g.taps[t].dw; h_lo = h_hi = g.taps[t].dh; }
@@ -540,7 +549,8 @@ int twn_detail::launch_conv_resident(const Geometry &g, const void *X, const uin
     const int smem_bytes = 1024 + (int)P.ctl_off + 2048;
 
     P.T = T;
-    P.wpr = g.ld_codes / 16;
+    P.wpr = g.ld_codes / (g.code_bits == 1 ? 32 : 16);
+    P.code_bits = g.code_bits == 1 ? 1 : 2;
     P.osw = g.osw; P.osh = g.osh;
     P.alpha = epi.alpha;
     P.scale = epi.scale; P.shift = epi.shift;

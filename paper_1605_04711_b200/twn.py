@@ -68,6 +68,7 @@ def lib() -> C.CDLL:
         l.twn_ternarize_batch_workspace_bytes.restype = C.c_size_t
         l.twn_conv2d_bwd_weight_workspace_bytes.restype = C.c_size_t
         l.twn_conv2d_bwd_weight_folded_workspace_bytes.restype = C.c_size_t
+        l.twn_binarize_workspace_bytes.restype = C.c_size_t
         _lib = l
     return _lib
 
@@ -322,6 +323,58 @@ def conv2d_bwd_data(desc: ConvDesc, dZ: torch.Tensor, T_bwd: torch.Tensor, ld_co
     _check(lib().twn_conv2d_bwd_data(C.byref(desc), _ptr(dZ), _ptr(T_bwd), C.c_int64(ld_codes),
                                      _ptr(stats), C.byref(epi) if epi is not None else None, _ptr(dX),
                                      _ptr(dev_status), _stream(stream)), "twn_conv2d_bwd_data")
+
+
+# ---- binary precision weights: the same calls on 1-bit codes
+def ld_for_b1(cols: int) -> int:
+    """Smallest legal row pitch (in codes) for 1-bit rows of `cols` codes."""
+    return (cols + 127) // 128 * 128
+
+
+def binarize_workspace_bytes() -> int:
+    return int(lib().twn_binarize_workspace_bytes())
+
+
+def binarize(W: torch.Tensor, stats: torch.Tensor, packed: torch.Tensor, ld_codes: int, workspace: torch.Tensor,
+             stream=None, rows: int | None = None, cols: int | None = None) -> None:
+    if rows is None:
+        rows, cols = (W.shape[0], W.numel() // W.shape[0]) if W.dim() > 1 else (1, W.numel())
+    _check(lib().twn_binarize(_ptr(W), C.c_int64(rows), C.c_int64(cols), _ptr(stats), _ptr(packed),
+                              C.c_int64(ld_codes), _ptr(workspace), C.c_size_t(workspace.numel()), _stream(stream)),
+           "twn_binarize")
+
+
+def unpack_b1(packed: torch.Tensor, rows: int, cols: int, ld_codes: int, codes: torch.Tensor, stream=None) -> None:
+    _check(lib().twn_unpack_b1(_ptr(packed), C.c_int64(rows), C.c_int64(cols), C.c_int64(ld_codes), _ptr(codes),
+                               _stream(stream)), "twn_unpack_b1")
+
+
+def transpose_codes_b1(packed_fwd: torch.Tensor, ld_fwd: int, desc: ConvDesc, packed_bwd: torch.Tensor, ld_bwd: int,
+                       stream=None) -> None:
+    _check(lib().twn_transpose_codes_b1(_ptr(packed_fwd), C.c_int64(ld_fwd), C.byref(desc), _ptr(packed_bwd),
+                                        C.c_int64(ld_bwd), _stream(stream)), "twn_transpose_codes_b1")
+
+
+def gemm_b1(X: torch.Tensor, ldx: int, B_packed: torch.Tensor, ld_codes: int, stats, M: int, N: int,
+            K: int, epi, Y: torch.Tensor, ldy: int, dev_status=None, stream=None) -> None:
+    _check(lib().twn_gemm_b1(_ptr(X), C.c_int64(ldx), _ptr(B_packed), C.c_int64(ld_codes), _ptr(stats),
+                             C.c_int64(M), C.c_int64(N), C.c_int64(K),
+                             C.byref(epi) if epi is not None else None, _ptr(Y), C.c_int64(ldy),
+                             _ptr(dev_status), _stream(stream)), "twn_gemm_b1")
+
+
+def conv2d_fwd_b1(desc: ConvDesc, X: torch.Tensor, B_fwd: torch.Tensor, ld_codes: int, stats, epi,
+                  Y: torch.Tensor, dev_status=None, stream=None) -> None:
+    _check(lib().twn_conv2d_fwd_b1(C.byref(desc), _ptr(X), _ptr(B_fwd), C.c_int64(ld_codes), _ptr(stats),
+                                   C.byref(epi) if epi is not None else None, _ptr(Y), _ptr(dev_status),
+                                   _stream(stream)), "twn_conv2d_fwd_b1")
+
+
+def conv2d_bwd_data_b1(desc: ConvDesc, dZ: torch.Tensor, B_bwd: torch.Tensor, ld_codes: int, stats, epi,
+                       dX: torch.Tensor, dev_status=None, stream=None) -> None:
+    _check(lib().twn_conv2d_bwd_data_b1(C.byref(desc), _ptr(dZ), _ptr(B_bwd), C.c_int64(ld_codes),
+                                        _ptr(stats), C.byref(epi) if epi is not None else None, _ptr(dX),
+                                        _ptr(dev_status), _stream(stream)), "twn_conv2d_bwd_data_b1")
 
 
 def im2col(desc: ConvDesc, X: torch.Tensor, Xcol: torch.Tensor, ldk: int, stream=None) -> None:
