@@ -339,6 +339,32 @@ int twn_conv2d_fwd(const twn_conv_desc_t *desc, const void *X, const uint32_t *T
                    int32_t *dev_status, twn_stream_t stream);
 
 /*
+ * twn_conv2d_fwd that also returns the batch statistics of its output, for the batch normalisation
+ * that follows every ternary convolution while the network is trained (Sec. 2.4; the block of Fig. 1):
+ *   bn_sum[o]   = sum over (b, ho, wo) of z[b,ho,wo,o]
+ *   bn_sumsq[o] = sum over (b, ho, wo) of z[b,ho,wo,o]^2
+ * with z = alpha * acc * scale[o] + shift[o], the value before the residual and the ReLU of the
+ * epilogue (with scale = shift = NULL: the plain convolution output).  The sums are taken of the
+ * fp32 values in the kernel's epilogue, not of a rounded copy: per thread in fp32 over at most a
+ * tile's pixels, across tiles in fp64 and in a fixed order (deterministic).
+ *   bn_sum, bn_sumsq  fp64 [Cout], overwritten; 8-byte aligned.
+ *   workspace         at least twn_conv2d_fwd_bn_workspace_bytes(desc) bytes, 16-byte aligned: per-tile
+ *                     partial sums.
+ * Everything else as in twn_conv2d_fwd.  twn_bn_finalize turns the sums over n = B*Ho*Wo values into the
+ * mean, the biased variance and the affine of the normalisation:
+ *   scale[o] = gamma[o] / sqrt(var[o] + eps),  shift[o] = beta[o] - mean[o] * scale[o]
+ * (gamma / beta NULL: 1 / 0; scale, shift fp32 [C]; mean, var fp64 [C]; any output may be NULL).
+ */
+size_t twn_conv2d_fwd_bn_workspace_bytes(const twn_conv_desc_t *desc);
+int twn_conv2d_fwd_bn(const twn_conv_desc_t *desc, const void *X, const uint32_t *T_fwd, int64_t ld_codes,
+                      const twn_stats_t *stats, const twn_epilogue_t *epi, void *Y, double *bn_sum,
+                      double *bn_sumsq, void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                      twn_stream_t stream);
+int twn_bn_finalize(const double *sum, const double *sumsq, int64_t n, int64_t C, const float *gamma,
+                    const float *beta, double eps, float *scale, float *shift, double *mean, double *var,
+                    twn_stream_t stream);
+
+/*
  * Convolution backward for data (Algorithm 1: ordinary back-propagation with
  * T = alpha * W~ in place of W), the adjoint of twn_conv2d_fwd:
  *   dX[b,h,w,c] = epi( alpha * sum over (r,s,o) with ho*stride_h - pad_h + r == h,

@@ -331,6 +331,28 @@ def conv2d_bwd_weight(d: ConvDesc, X, dZ, entries=None):
     return dW, A
 
 
+# ------------------------------------------- batch statistics (Sec. 2.4, Fig. 1)
+def bn_stats(Z):
+    """Per-channel sum and sum of squares of a pre-activation tensor Z (fp64, channels last), the two
+    statistics a batch normalisation in training mode needs.  Exactly rounded sums (math.fsum)."""
+    import math
+    z = np.asarray(Z, dtype=np.float64).reshape(-1, Z.shape[-1])
+    s = np.array([math.fsum(z[:, c]) for c in range(z.shape[1])])
+    ss = np.array([math.fsum(z[:, c] * z[:, c]) for c in range(z.shape[1])])
+    return s, ss
+
+
+def bn_affine(s, ss, n, gamma=None, beta=None, eps=1e-5):
+    """mean, biased variance, and the affine y = z * scale + shift of the normalisation
+    gamma * (z - mean) / sqrt(var + eps) + beta."""
+    mean = s / n
+    var = np.maximum(ss / n - mean * mean, 0.0)
+    g = np.ones_like(mean) if gamma is None else np.asarray(gamma, dtype=np.float64)
+    b = np.zeros_like(mean) if beta is None else np.asarray(beta, dtype=np.float64)
+    scale = g / np.sqrt(var + eps)
+    return mean, var, scale, b - mean * scale
+
+
 # --------------------------------------------------- glue (textbook, numpy)
 def maxpool(x, k: int, stride: int, pad: int = 0):
     """x: fp64 [B,H,W,C]; window k x k, -inf padding.  Returns (y, argmax flat

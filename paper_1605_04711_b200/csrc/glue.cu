@@ -927,3 +927,44 @@ extern "C" int twn_act_bwd(const void *dY, const void *Y, const float *scale, in
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }
+
+namespace {
+
+// Batch normalisation in training mode, from the sums the convolution's epilogue produced:
+// mean = sum/n, var = sumsq/n - mean^2 (biased), scale = gamma / sqrt(var + eps), shift = beta - mean * scale.
+__global__ void __launch_bounds__(kT)
+bn_finalize_kernel(const double *__restrict__ sum, const double *__restrict__ sumsq, long long n, int C,
+                   const float *__restrict__ gamma, const float *__restrict__ beta, double eps,
+                   float *__restrict__ scale, float *__restrict__ shift, double *__restrict__ mean,
+                   double *__restrict__ var)
+{
+    const int c = blockIdx.x * kT + threadIdx.x;
+    if (c >= C) return;
+    const double m = sum[c] / (double)n;
+    double v = sumsq[c] / (double)n - m * m;
+    if (v < 0.0) v = 0.0;
+    const double sc = (gamma ? (double)gamma[c] : 1.0) / sqrt(v + eps);
+    if (scale) scale[c] = (float)sc;
+    if (shift) shift[c] = (float)((beta ? (double)beta[c] : 0.0) - m * sc);
+    if (mean) mean[c] = m;
+    if (var) var[c] = v;
+}
+
+}  // namespace
+
+extern "C" int twn_bn_finalize(const double *sum, const double *sumsq, int64_t n, int64_t C, const float *gamma,
+                               const float *beta, double eps, float *scale, float *shift, double *mean, double *var,
+                               twn_stream_t stream)
+{
+    TWN_REQUIRE(sum && sumsq && n > 0 && C > 0 && C <= 0x7fffffffLL && eps >= 0.0, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(twn_aligned(sum, 8) && twn_aligned(sumsq, 8) && twn_aligned(mean, 8) && twn_aligned(var, 8) &&
+                    twn_aligned(gamma, 4) && twn_aligned(beta, 4) && twn_aligned(scale, 4) && twn_aligned(shift, 4),
+                TWN_ERR_MISALIGNED);
+    twn_device_info dev;
+    const int rc = twn_current_device(&dev);
+    if (rc != TWN_OK) return rc;
+    bn_finalize_kernel<<<(int)((C + kT - 1) / kT), kT, 0, twn_cu(stream)>>>(sum, sumsq, n, (int)C, gamma, beta, eps, scale,
+                                                                          shift, mean, var);
+    TWN_CUDA_OK(cudaGetLastError());
+    return TWN_OK;
+}

@@ -114,6 +114,8 @@ struct ConvParams {
     int dsets;                    // host only: decode groups of the kernel variant to launch
     void *Y;
     int32_t *status;
+    // optional batch statistics: [tile][epilogue warp of the quadrant][128 channels][sum, sum of squares]
+    float *bn_partial;
     // output path: 1 = each epilogue warp stages its 32 channels x 32 pixels in shared memory and
     // writes them with a TMA store (box = 32 channels x sbw x sbh x sbb pixels); 0 = per-thread stores
     int tma_store, lg_sbw, lg_sbh;
@@ -463,6 +465,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
             __nv_bfloat16 *const y16 = reinterpret_cast<__nv_bfloat16 *>(P.Y) + n;
             const uint32_t t_acc = tmem_acc + ((uint32_t)(q * 32) << 16) + buf * PIX;
             uint32_t v[32];
+            float bn_s1 = 0.0f, bn_s2 = 0.0f;      // this thread's channel: sum and sum of squares over its pixels of the tile
             // the chunk loop stays rolled: the epilogue is straight-line code that every warp walks
             // once per chunk, so its size is instruction-fetch time
 #pragma unroll 1
@@ -497,6 +500,20 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                 }
                 if (use_res_tma) {
                     if (!mbar_wait_warp(&my_res_full[nres & 1u], (nres >> 1) & 1u, abort_flag, P.status, 32)) { alive = false; break; }
+                }
+                if (P.bn_partial) {
+                    // Batch statistics of z = acc * scale' + shift, the value before the residual and the ReLU,
+                    // over the pixels that exist (a ragged tile computes on zero-filled pixels too).  Lane j
+                    // decides for pixel j of the chunk, a vote makes the mask warp-wide.
+                    const int p = c * 32 + lane;
+                    const bool in_range = (p_w0 + (p & BWm)) < P.Wv && (p_h0 + ((p >> P.lgBW) & BHm)) < P.Hv &&
+                                          (p_b0 + (p >> (P.lgBW + P.lgBH))) < P.Bv;
+                    const uint32_t live = __ballot_sync(0xffffffffu, in_range);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float z = fmaf(__uint_as_float(v[j]), sc, sf);
+                        if ((live >> j) & 1u) { bn_s1 += z; bn_s2 = fmaf(z, z, bn_s2); }
+                    }
                 }
                 // The inner loops are kept free of conditionals: every instruction issued here is
                 // exposed latency of this warp's chunk.
@@ -586,6 +603,9 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     }
                 }
             }
+            if (P.bn_partial && warp_on)
+                *reinterpret_cast<float2 *>(P.bn_partial + ((size_t)tile * kEpiSets + es) * (2 * kChan) + (q * 32 + lane) * 2) =
+                    make_float2(bn_s1, bn_s2);
             __syncwarp();
         }
         // all bulk stores of this thread have been written before the block may exit
@@ -604,6 +624,31 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
+}
+
+// Totals of the per-tile statistics: one warp per channel, the lanes take the tiles in turn and a shuffle tree
+// adds the 32 partial totals: a fixed order, so the result is the same bits on every run.
+__global__ void __launch_bounds__(256)
+bn_reduce_kernel(const float *__restrict__ partial, int total_tiles, int n_tiles, int Cout,
+                 double *__restrict__ sum, double *__restrict__ sumsq)
+{
+    const int lane = threadIdx.x & 31;
+    const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (c >= Cout) return;
+    const int nt = c / kChan, within = c - nt * kChan;
+    double s1 = 0.0, s2 = 0.0;
+    for (int tile = nt + lane * n_tiles; tile < total_tiles; tile += 32 * n_tiles)
+#pragma unroll
+        for (int es = 0; es < kEpiSets; ++es) {
+            const float2 v = __ldg(reinterpret_cast<const float2 *>(partial + ((size_t)tile * kEpiSets + es) * (2 * kChan) + within * 2));
+            s1 += (double)v.x; s2 += (double)v.y;
+        }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        s1 += __shfl_down_sync(0xffffffffu, s1, o);
+        s2 += __shfl_down_sync(0xffffffffu, s2, o);
+    }
+    if (lane == 0) { sum[c] = s1; sumsq[c] = s2; }
 }
 
 // ---------------------------------------------------------------- host side
@@ -687,7 +732,10 @@ int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const twn_dev
         }
     }
     const int grid = dev.sm_count < P.total_tiles ? dev.sm_count : P.total_tiles;
+    if (P.bn_partial && (size_t)P.total_tiles * kEpiSets * 2 * kChan * sizeof(float) > g.bn_partial_bytes) return TWN_ERR_WORKSPACE;
     tconv_kernel<PIX, DS, BITS><<<grid, threads_conv(DS), smem_bytes, s>>>(map_x, map_y, map_r, P);
+    if (P.bn_partial)
+        bn_reduce_kernel<<<(g.Cout + 7) / 8, 256, 0, s>>>(P.bn_partial, P.total_tiles, P.n_tiles, g.Cout, g.bn_sum, g.bn_sumsq);
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }
@@ -743,6 +791,7 @@ int launch_conv(const Geometry &g, const void *X, const uint32_t *T, const twn_s
     P.out_dtype = epi ? epi->out_dtype : out_dtype_default;
     P.Y = Y;
     P.status = dev_status;
+    P.bn_partial = g.bn_partial;
     for (int t = 0; t < g.n_taps; ++t) P.taps[t] = g.taps[t];
 
     // Tile shape by a cost model fitted to measured launches (cycles per round of tiles, kb = k-blocks
@@ -892,9 +941,11 @@ int conv_common_checks(const twn_conv_desc_t *d)
 
 namespace {
 
+struct BnArgs { double *sum, *sumsq; void *ws; size_t ws_bytes; };
+
 int conv_fwd_impl(const twn_conv_desc_t *d, const void *X, const uint32_t *T_fwd, int64_t ld_codes,
                   const twn_stats_t *stats, const twn_epilogue_t *epi, void *Y,
-                  int32_t *dev_status, twn_stream_t stream, int bits)
+                  int32_t *dev_status, twn_stream_t stream, int bits, const BnArgs *bn = nullptr)
 {
     int rc = conv_common_checks(d);
     if (rc != TWN_OK) return rc;
@@ -925,10 +976,42 @@ int conv_fwd_impl(const twn_conv_desc_t *d, const void *X, const uint32_t *T_fwd
             t.koff = (int32_t)((r * d->kw + s) * d->Cin);
         }
     g.code_bits = bits;
+    if (bn) {
+        g.bn_partial = static_cast<float *>(bn->ws);
+        g.bn_partial_bytes = bn->ws_bytes;
+        g.bn_sum = bn->sum; g.bn_sumsq = bn->sumsq;
+    }
     return launch_conv(g, X, T_fwd, stats, epi, Y, TWN_F32, dev_status, twn_cu(stream));
 }
 
 }  // namespace
+
+extern "C" size_t twn_conv2d_fwd_bn_workspace_bytes(const twn_conv_desc_t *d)
+{
+    if (conv_common_checks(d) != TWN_OK) return 0;
+    // the smallest pixel tile gives the most tiles: 128 pixels, whatever shape the launch then picks
+    Geometry g;
+    memset(&g, 0, sizeof g);
+    g.Bv = (int)d->B;
+    g.Hv = (int)((d->H + 2 * d->pad_h - d->kh) / d->stride_h + 1);
+    g.Wv = (int)((d->W + 2 * d->pad_w - d->kw) / d->stride_w + 1);
+    g.sh = d->stride_h; g.sw = d->stride_w;
+    int a, b;
+    const long long tiles = pick_tile(g, 128, &a, &b) * ((d->Cout + kChan - 1) / kChan);
+    return (size_t)tiles * kEpiSets * 2 * kChan * sizeof(float);
+}
+
+extern "C" int twn_conv2d_fwd_bn(const twn_conv_desc_t *d, const void *X, const uint32_t *T_fwd, int64_t ld_codes,
+                                 const twn_stats_t *stats, const twn_epilogue_t *epi, void *Y, double *bn_sum,
+                                 double *bn_sumsq, void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                 twn_stream_t stream)
+{
+    TWN_REQUIRE(bn_sum && bn_sumsq && workspace, TWN_ERR_INVALID_ARG);
+    TWN_REQUIRE(twn_aligned(bn_sum, 8) && twn_aligned(bn_sumsq, 8) && twn_aligned(workspace, 16), TWN_ERR_MISALIGNED);
+    TWN_REQUIRE(workspace_bytes >= twn_conv2d_fwd_bn_workspace_bytes(d) && workspace_bytes > 0, TWN_ERR_WORKSPACE);
+    const BnArgs bn = {bn_sum, bn_sumsq, workspace, workspace_bytes};
+    return conv_fwd_impl(d, X, T_fwd, ld_codes, stats, epi, Y, dev_status, stream, 2, &bn);
+}
 
 extern "C" int twn_conv2d_fwd(const twn_conv_desc_t *d, const void *X, const uint32_t *T_fwd, int64_t ld_codes,
                               const twn_stats_t *stats, const twn_epilogue_t *epi, void *Y,

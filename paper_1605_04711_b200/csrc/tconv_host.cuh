@@ -48,6 +48,10 @@ struct Geometry {
     int Cout;
     long long ld_codes, code_cols;  // packed row pitch and used columns
     int code_bits;   // 2: ternary codes, 16 per word; 1: binary codes, 32 per word
+    // batch statistics of the pre-activation output (optional): per-tile partial sums, then the totals
+    float *bn_partial;
+    size_t bn_partial_bytes;
+    double *bn_sum, *bn_sumsq;
     int n_taps;
     Tap taps[kMaxTaps];
     long long Cin;   // channels per tap

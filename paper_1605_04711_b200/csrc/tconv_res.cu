@@ -470,6 +470,7 @@ int twn_detail::launch_conv_resident(const Geometry &g, const void *X, const uin
 {
     *handled = false;
     if (g.sw != 1 || g.sh != 1 || g.Cout > kNMax || g.Cout < 1) return TWN_OK;
+    if (g.bn_partial) return TWN_OK;      // batch statistics come out of the general kernel's epilogue
     const bool out_bf16 = epi.out_dtype == TWN_BF16;
     const int es = out_bf16 ? 2 : 4;
     // the output (and a residual) must be addressable by TMA

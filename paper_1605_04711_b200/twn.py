@@ -69,6 +69,7 @@ def lib() -> C.CDLL:
         l.twn_conv2d_bwd_weight_workspace_bytes.restype = C.c_size_t
         l.twn_conv2d_bwd_weight_folded_workspace_bytes.restype = C.c_size_t
         l.twn_binarize_workspace_bytes.restype = C.c_size_t
+        l.twn_conv2d_fwd_bn_workspace_bytes.restype = C.c_size_t
         _lib = l
     return _lib
 
@@ -316,6 +317,26 @@ def conv2d_fwd(desc: ConvDesc, X: torch.Tensor, T_fwd: torch.Tensor, ld_codes: i
     _check(lib().twn_conv2d_fwd(C.byref(desc), _ptr(X), _ptr(T_fwd), C.c_int64(ld_codes), _ptr(stats),
                                 C.byref(epi) if epi is not None else None, _ptr(Y), _ptr(dev_status),
                                 _stream(stream)), "twn_conv2d_fwd")
+
+
+def conv2d_fwd_bn_workspace_bytes(desc: ConvDesc) -> int:
+    return int(lib().twn_conv2d_fwd_bn_workspace_bytes(C.byref(desc)))
+
+
+def conv2d_fwd_bn(desc: ConvDesc, X: torch.Tensor, T_fwd: torch.Tensor, ld_codes: int, stats, epi, Y: torch.Tensor,
+                  bn_sum: torch.Tensor, bn_sumsq: torch.Tensor, workspace: torch.Tensor, dev_status=None,
+                  stream=None) -> None:
+    _check(lib().twn_conv2d_fwd_bn(C.byref(desc), _ptr(X), _ptr(T_fwd), C.c_int64(ld_codes), _ptr(stats),
+                                   C.byref(epi) if epi is not None else None, _ptr(Y), _ptr(bn_sum), _ptr(bn_sumsq),
+                                   _ptr(workspace), C.c_size_t(workspace.numel()), _ptr(dev_status), _stream(stream)),
+           "twn_conv2d_fwd_bn")
+
+
+def bn_finalize(bn_sum: torch.Tensor, bn_sumsq: torch.Tensor, n: int, C_: int, gamma, beta, eps: float, scale, shift,
+                mean=None, var=None, stream=None) -> None:
+    _check(lib().twn_bn_finalize(_ptr(bn_sum), _ptr(bn_sumsq), C.c_int64(n), C.c_int64(C_), _ptr(gamma), _ptr(beta),
+                                 C.c_double(eps), _ptr(scale), _ptr(shift), _ptr(mean), _ptr(var), _stream(stream)),
+           "twn_bn_finalize")
 
 
 def conv2d_bwd_data(desc: ConvDesc, dZ: torch.Tensor, T_bwd: torch.Tensor, ld_codes: int, stats, epi,

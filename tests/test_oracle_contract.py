@@ -217,3 +217,29 @@ def test_avgpool():
     np.testing.assert_allclose(y, x.reshape(3, 49, 4).sum(1) / 49, rtol=1e-14)
     dx = oracle.global_avgpool_bwd(y, 7, 7)
     assert dx.shape == x.shape and np.allclose(dx[:, 3, 2, :], y / 49)
+
+
+# ------------------------------------------------------------------- batch statistics
+def test_bn_statistics_and_affine_match_torch_batch_norm_in_training_mode():
+    """The two per-channel sums and the affine derived from them against torch's batch_norm in training mode
+    (batch statistics, biased variance), on the output of an oracle convolution."""
+    B, H, W, Cin, Cout, k, s, p = 3, 9, 8, 4, 6, 3, 1, 1
+    d = oracle.conv_desc(B, H, W, Cin, Cout, k, s, p)
+    X = _x(30, "bnx", (B, H, W, Cin)); T = _rand_codes(31, (Cout, k, k, Cin))
+    Z, _ = oracle.conv2d_fwd(d, X, T, 0.7)
+    ssum, ssq = oracle.bn_stats(Z)
+    n = B * d.Ho * d.Wo
+    zt = torch.from_numpy(Z).permute(0, 3, 1, 2)
+    var_t, mean_t = torch.var_mean(zt, dim=(0, 2, 3), unbiased=False)
+    gamma = dg.draw(32, "bng", Cout, "normal", 1.0, 0.2).astype(np.float64)
+    beta = dg.draw(32, "bnb", Cout, "normal", 0.0, 0.3).astype(np.float64)
+    mean, var, scale, shift = oracle.bn_affine(ssum, ssq, n, gamma, beta, eps=1e-5)
+    np.testing.assert_allclose(mean, mean_t.numpy(), rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(var, var_t.numpy(), rtol=1e-10)
+    want = F.batch_norm(zt, None, None, torch.from_numpy(gamma), torch.from_numpy(beta), training=True, eps=1e-5)
+    got = Z * scale[None, None, None, :] + shift[None, None, None, :]
+    np.testing.assert_allclose(got, want.permute(0, 2, 3, 1).numpy(), rtol=1e-9, atol=1e-10)
+    # a constant channel has zero variance; sums are plain sums
+    C2 = np.zeros((2, 3, 3, 2)); C2[..., 0] = 1.5; C2[..., 1] = np.arange(18).reshape(2, 3, 3)
+    s2, q2 = oracle.bn_stats(C2)
+    assert s2.tolist() == [27.0, 153.0] and q2.tolist() == [40.5, float(sum(i * i for i in range(18)))]
