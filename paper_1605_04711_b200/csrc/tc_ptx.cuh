@@ -61,7 +61,7 @@ __device__ __forceinline__ unsigned long long global_ns()
 // off with nanosleep instead of polling flat out (`backoff_ns` = 0 for the latency-critical
 // waits of the MMA warp, which rely on the suspend time of try_wait alone).
 __device__ __forceinline__ bool mbar_wait(void *bar, uint32_t parity, volatile int *abort_flag, int32_t *status,
-                                          uint32_t backoff_ns = 64)
+                                          uint32_t backoff_ns = 64, unsigned long long limit_ns = kWaitLimitNs)
 {
     if (mbar_try(bar, parity)) return true;
     unsigned long long t0 = 0;
@@ -72,7 +72,7 @@ __device__ __forceinline__ bool mbar_wait(void *bar, uint32_t parity, volatile i
             if (*abort_flag) return false;
             const unsigned long long now = global_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) {
+            else if (now - t0 > limit_ns) {
                 *abort_flag = 1;
                 if (status) atomicMin(status, (int)TWN_ERR_TIMEOUT);
                 return false;
@@ -84,7 +84,7 @@ __device__ __forceinline__ bool mbar_wait(void *bar, uint32_t parity, volatile i
 // Warp-wide wait: lane 0 polls, the result is broadcast.  One polling lane instead of 32
 // keeps the shared-memory pipe free for the warps that are working.
 __device__ __forceinline__ bool mbar_wait_warp(void *bar, uint32_t parity, volatile int *abort_flag, int32_t *status,
-                                               uint32_t backoff_ns = 64)
+                                               uint32_t backoff_ns = 64, unsigned long long limit_ns = kWaitLimitNs)
 {
     // fast path: the phase is already over.  One non-blocking probe by the whole warp and one vote:
     // measured at 16 cycles, against 46 for the potentially blocking try_wait and 129 when a single
@@ -96,7 +96,7 @@ __device__ __forceinline__ bool mbar_wait_warp(void *bar, uint32_t parity, volat
     for (int i = 0; i < kConvergedTries; ++i)
         if (__all_sync(0xffffffffu, mbar_try(bar, parity))) return true;
     int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status, backoff_ns) ? 1 : 0;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status, backoff_ns, limit_ns) ? 1 : 0;
     ok = __shfl_sync(0xffffffffu, ok, 0);
     __syncwarp();
     return ok != 0;
