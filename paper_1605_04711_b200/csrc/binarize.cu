@@ -60,23 +60,37 @@ binarize_kernel(const float *__restrict__ W, long long rows, long long cols, lon
 
     double acc = 0.0;
     unsigned long long negs = 0;
-    for (long long w = warp_id; w < total_words; w += n_warps) {
-        long long idx;
-        bool valid;
-        if (flat) {
-            idx = (w << 5) + e;
-            valid = true;
-        } else {
-            const long long r = w / wpr, c = ((w - r * wpr) << 5) + e;
-            valid = c < cols;
-            idx = r * cols + c;
+    if (flat) {
+        // sixteen words per warp and iteration, their loads issued before any is used: the sweep is bound by the
+        // bytes a warp keeps in flight
+        constexpr int kU = 16;
+        double a1 = 0.0;
+        for (long long w0 = warp_id * kU; w0 < total_words; w0 += n_warps * kU) {
+            float x[kU];
+#pragma unroll
+            for (int u = 0; u < kU; ++u) x[u] = (w0 + u < total_words) ? __ldg(W + ((w0 + u) << 5) + e) : 0.0f;
+#pragma unroll
+            for (int u = 0; u < kU; ++u) {
+                if (u & 1) a1 += (double)fabsf(x[u]); else acc += (double)fabsf(x[u]);
+                const unsigned int word = __ballot_sync(0xffffffffu, x[u] < 0.0f);     // -0.0 and NaN vote "not negative"
+                if (lane == u && w0 + u < total_words) {
+                    packed[w0 + u] = word;
+                    negs += (unsigned long long)__popc(word);
+                }
+            }
         }
-        const float x = valid ? __ldg(W + idx) : 0.0f;
-        acc += (double)fabsf(x);
-        const unsigned int word = __ballot_sync(0xffffffffu, x < 0.0f);     // -0.0 and NaN vote "not negative"
-        if (lane == 0) {
-            packed[w] = word;
-            negs += (unsigned long long)__popc(word);
+        acc += a1;
+    } else {
+        for (long long w = warp_id; w < total_words; w += n_warps) {
+            const long long r = w / wpr, c = ((w - r * wpr) << 5) + e;
+            const bool valid = c < cols;
+            const float x = valid ? __ldg(W + r * cols + c) : 0.0f;
+            acc += (double)fabsf(x);
+            const unsigned int word = __ballot_sync(0xffffffffu, x < 0.0f);
+            if (lane == 0) {
+                packed[w] = word;
+                negs += (unsigned long long)__popc(word);
+            }
         }
     }
     // block partials
