@@ -5,7 +5,9 @@
 // A dense bf16 x bf16 -> fp32 contraction whose reduction runs over the pixels, i.e. over the
 // slow dimension of both NHWC operands.  tcgen05 takes such operands directly ("MN-major"
 // shared-memory descriptors), so the dZ tile and the tap-shifted X tile go from TMA straight
-// into the MMA: D[o, c] += dZ_tile^T * X_tile, 64 pixels per k-block.
+// into the MMA: D[o, c] += dZ_tile^T * X_tile, 64 or 128 pixels per k-block (a tensor copy of 128 rows
+// moves its bytes almost twice as fast as one of 64, so the larger k-block is taken wherever its padding
+// and the ring depth allow).
 //
 // One MMA covers up to four 64-channel column blocks of dW, taken in (tap, channel block)
 // order, so narrow layers (Cin = 64) process four taps per pass over the dZ tile.
@@ -13,8 +15,9 @@
 // so the pixels are split across CTAs; each CTA writes its fp32 partial tile to the workspace
 // and a second kernel adds the partials in split order (deterministic, no atomics).
 //
-//   warp 0     TMA producer        warp 1     MMA issuer (whole warp, elected lane issues)
-//   warps 2-5  epilogue: tensor memory -> workspace
+//   warp 0     TMA producer: lane j issues copy j of a k-block (gradient blocks, activation blocks)
+//   warps 1, 6 one MMA-issuing thread each, alternate k-blocks, an accumulator each
+//   warps 2-5  epilogue: sum of the two accumulators -> workspace
 #include <cstddef>
 
 #include "common.cuh"
@@ -23,12 +26,12 @@
 
 namespace {
 
-constexpr int kDwMaxStages = 8;
-constexpr int kDwPoolBytes = 176 * 1024;         // operand ring: stages of 16 KB of dZ plus the X blocks
-constexpr int kDwPix = 64;                       // pixels per k-block
-constexpr int kDwBlockBytes = kDwPix * 128;      // one 64-channel x 64-pixel swizzled block: 8 KB
+constexpr int kDwMaxStages = 12;
+constexpr int kDwPoolBytes = 208 * 1024;         // operand ring: stages of one or two blocks of dZ plus the X blocks
+constexpr int kDwMaxMma = 8;                     // K = 16 pixels per MMA: 4 or 8 MMAs per k-block of 64 or 128 pixels
 constexpr int kDwMaxCb = 4;                      // up to 256 input channels per tile
-constexpr int kDwThreads = 192;
+constexpr int kDwThreads = 224;
+constexpr int kDwIssuerB = 6;                    // the warp of the second MMA-issuing thread
 constexpr int kDwMaxTaps = 64;
 constexpr int kDwAccCols = 256;
 
@@ -50,7 +53,9 @@ struct DwParams {
     // columns: tap s is the tile one pixel (128 bytes) further, so a single MMA of N = 64 kw
     // covers the row and the tile is loaded once instead of kw times.
     int row_mode, kw, x_bytes, k_group_bytes;
-    int mma_off[4];              // byte offset of the 16 pixels of MMA i inside the activation tile
+    int x_off;                   // byte offset of the activation blocks inside a stage (after the blocks of dZ)
+    int kpix, n_mma, blk_bytes;  // pixels per k-block (64 or 128), its MMAs (K = 16 pixels each), bytes of one 64-channel block of it
+    int mma_off[kDwMaxMma];      // byte offset of the 16 pixels of MMA i inside the activation tile
     int stages, stage_bytes;
     DwTap taps[kDwMaxTaps];
 };
@@ -62,10 +67,25 @@ struct __align__(1024) DwSmem {
     // per epilogue warp: 32 rows x 32 fp32 of the accumulator, 16-byte chunks XOR-swizzled by the
     // row so that row-wise writes and the transposed reads are both free of bank conflicts
     float4 stg[4][32][8];
-    unsigned long long full[kDwMaxStages], empty[kDwMaxStages], acc_full[2], acc_empty[2];
+    unsigned long long full[kDwMaxStages], empty[kDwMaxStages], acc_full, acc_empty;
     uint32_t tmem_base;
     volatile int abort_flag;
 };
+
+// D[tmem] (+)= A[smem] * B[smem]^T issued by the calling thread alone, accumulate flag in a register.
+__device__ __forceinline__ void dw_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+__device__ __forceinline__ void dw_commit(void *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
 
 __global__ void __launch_bounds__(kDwThreads, 1)
 dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CUtensorMap map_x,
@@ -78,7 +98,8 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kDwMaxStages; ++s) { mbar_init(&sm->full[s], 1); mbar_init(&sm->empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&sm->acc_full[b], 1); mbar_init(&sm->acc_empty[b], 4); }
+        mbar_init(&sm->acc_full, 2);
+        mbar_init(&sm->acc_empty, 4);
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -107,136 +128,188 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
         if (p1 > P.pix_tiles) p1 = P.pix_tiles;
         if (p0 > p1) p0 = p1;
     };
+    // row mode: filter row and 64-channel block of group gi
+    auto row_group = [&](int gi, int &r, int &cb0) {
+        r = gi / P.cblocks;
+        cb0 = gi - r * P.cblocks;
+    };
+    const int x_slot = (P.x_bytes + 1023) & ~1023;     // row mode: one activation tile
 
     if (warp == 0) {
-        if (lane == 0) {
-            uint32_t it = 0;
-            bool ok = true;
-            for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
-                int ot, gi, nb, sp, p0, p1;
-                unit_range(u, ot, gi, nb, sp, p0, p1);
-                // the second 64-channel block of dZ is not loaded when it lies past Cout: what the MMA
-                // then reads there lands in accumulator rows that are never stored
-                const bool a1 = ot * 128 + 64 < P.Cout;
-                const uint32_t bytes = (a1 ? 2 : 1) * kDwBlockBytes + (P.row_mode ? P.x_bytes : nb * kDwBlockBytes);
-                // Everything that does not change along the pixel tiles is worked out here: this one
-                // thread paces the pipeline, and an integer division costs it hundreds of cycles.
-                int xc[kDwMaxCb], xdw[kDwMaxCb], xdh[kDwMaxCb];
-                int nx = nb;
-                if (P.row_mode) {
-                    // filter row r = gi / cblocks of channel block gi % cblocks: one box, kw - 1 pixels wider
-                    const int r = gi / P.cblocks, cb = gi - r * P.cblocks;
-                    const DwTap tap = P.taps[r * P.kw];
-                    xc[0] = cb * 64; xdw[0] = tap.dw; xdh[0] = tap.dh;
-                    nx = 1;
-                } else {
-                    for (int j = 0; j < nb; ++j) {
-                        const int i = gi * kDwMaxCb + j, t = i / P.cblocks, cb = i - t * P.cblocks;
-                        const DwTap tap = P.taps[t];
-                        xc[j] = cb * 64; xdw[j] = tap.dw; xdh[j] = tap.dh;
-                    }
-                }
-                // pixel tile p0 as (column tile, row tile, image tile), stepped without divisions
-                int twi = p0 % P.tw, thi = (p0 / P.tw) % P.th, tbi = p0 / (P.tw * P.th);
-                const int bstep = kDwPix >> (P.lgBW + P.lgBH);
-                int s = it % P.stages;
-                uint32_t ph = (it / P.stages) & 1u;
-                for (int p = p0; p < p1; ++p, ++it) {
-                    uint8_t *const st = sm->pool + s * P.stage_bytes;
-                    const int w0 = twi << P.lgBW, h0 = thi << P.lgBH, b0 = tbi * bstep;
-                    if (!mbar_wait(&sm->empty[s], ph ^ 1u, abort_flag, P.status, 32)) { ok = false; break; }
-                    mbar_expect_tx(&sm->full[s], bytes);
-                    tma_load_4d(st, &map_dz, &sm->full[s], ot * 128, w0, h0, b0);
-                    if (a1) tma_load_4d(st + kDwBlockBytes, &map_dz, &sm->full[s], ot * 128 + 64, w0, h0, b0);
-#pragma unroll
-                    for (int j = 0; j < kDwMaxCb; ++j)
-                        if (j < nx)
-                            tma_load_4d(st + (2 + j) * kDwBlockBytes, &map_x, &sm->full[s], xc[j], w0 * P.sw + xdw[j],
-                                        h0 * P.sh + xdh[j], b0);
-                    if (++twi == P.tw) { twi = 0; if (++thi == P.th) { thi = 0; ++tbi; } }
-                    if (++s == P.stages) { s = 0; ph ^= 1u; }
-                }
-            }
-        }
-    } else if (warp == 1) {
-        uint32_t it = 0, lu = 0;     // lu counts the units that accumulate something
+        // ------------------------------------------------ TMA producer: the whole warp
+        // Issuing a tensor copy holds its thread for roughly a hundred cycles, and a k-block needs up to six
+        // of them (two gradient blocks, up to four activation blocks); here lane j issues copy j, all in the
+        // same instruction.
+        uint32_t it = 0;
         bool ok = true;
         for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
             int ot, gi, nb, sp, p0, p1;
             unit_range(u, ot, gi, nb, sp, p0, p1);
-            if (p1 <= p0) continue;                      // the epilogue writes zeros for an empty split
-            const uint32_t idesc = make_idesc_mn(128, 64 * nb);
-            const int buf = lu & 1;
-            if (!mbar_wait_warp(&sm->acc_empty[buf], ((lu >> 1) & 1u) ^ 1u, abort_flag, P.status, 0)) break;
-            tc_fence_after();
-            const uint32_t d_tmem = tmem + buf * kDwAccCols;
+            // the second 64-channel block of dZ is not loaded when it lies past Cout: what the MMA
+            // then reads there lands in accumulator rows that are never stored
+            const bool a1 = ot * 128 + 64 < P.Cout;
+            const int nx = P.row_mode ? 1 : nb;
+            const uint32_t bytes = (a1 ? 2 : 1) * P.blk_bytes + (P.row_mode ? P.x_bytes : nb * P.blk_bytes);
+            // this lane's copy: lanes 0, 1 the two gradient blocks, lanes 2.. the activation blocks.
+            // Everything that does not change along the pixel tiles is worked out here.
+            bool active;
+            const CUtensorMap *my_map;
+            int my_c0, my_dw = 0, my_dh = 0, my_sw = 1, my_sh = 1;
+            uint32_t my_off;
+            if (lane < 2) {
+                active = lane == 0 || a1;
+                my_map = &map_dz;
+                my_c0 = ot * 128 + lane * 64;
+                my_off = (uint32_t)(lane * P.blk_bytes);
+            } else {
+                const int j = lane - 2;
+                active = j < nx;
+                my_map = &map_x;
+                my_sw = P.sw; my_sh = P.sh;
+                int t = 0, cb = 0;
+                if (P.row_mode) {
+                    // one box per 64-channel block, kw - 1 pixels wider than the tile
+                    int r, cb0;
+                    row_group(gi, r, cb0);
+                    t = r * P.kw; cb = cb0 + j;
+                    my_off = (uint32_t)(P.x_off + j * x_slot);
+                } else {
+                    const int i = gi * kDwMaxCb + (active ? j : 0);
+                    t = i / P.cblocks; cb = i - t * P.cblocks;
+                    my_off = (uint32_t)(P.x_off + j * P.blk_bytes);
+                }
+                const DwTap tap = P.taps[active ? t : 0];
+                my_c0 = cb * 64; my_dw = tap.dw; my_dh = tap.dh;
+            }
+            // pixel tile p0 as (column tile, row tile, image tile), stepped without divisions
+            int twi = p0 % P.tw, thi = (p0 / P.tw) % P.th, tbi = p0 / (P.tw * P.th);
+            const int bstep = P.kpix >> (P.lgBW + P.lgBH);
             int s = it % P.stages;
             uint32_t ph = (it / P.stages) & 1u;
             for (int p = p0; p < p1; ++p, ++it) {
-                const uint32_t st = smem_u32(sm->pool) + s * P.stage_bytes;
-                if (!mbar_wait_warp(&sm->full[s], ph, abort_flag, P.status, 0)) { ok = false; break; }
-                tc_fence_after();
-                const uint64_t adesc = smem_desc_mn_sw128(st, kDwBlockBytes);
-                // 16 pixels per MMA = 16 rows of 128 bytes = 2048 bytes
-                if (P.row_mode) {
-                    const uint32_t xt = st + 2 * kDwBlockBytes;
-                    const uint64_t b0d = smem_desc_mn_sw128_groups(xt + P.mma_off[0], 128, P.k_group_bytes);
-                    const uint64_t b1d = smem_desc_mn_sw128_groups(xt + P.mma_off[1], 128, P.k_group_bytes);
-                    const uint64_t b2d = smem_desc_mn_sw128_groups(xt + P.mma_off[2], 128, P.k_group_bytes);
-                    const uint64_t b3d = smem_desc_mn_sw128_groups(xt + P.mma_off[3], 128, P.k_group_bytes);
-                    if (p == p0) tc_mma_ss<false>(d_tmem, adesc, b0d, idesc);
-                    else tc_mma_ss<true>(d_tmem, adesc, b0d, idesc);
-                    tc_mma_ss<true>(d_tmem, adesc + 128, b1d, idesc);
-                    tc_mma_ss<true>(d_tmem, adesc + 256, b2d, idesc);
-                    tc_mma_ss<true>(d_tmem, adesc + 384, b3d, idesc);
-                } else {
-                    const uint64_t bdesc = smem_desc_mn_sw128(st + 2 * kDwBlockBytes, kDwBlockBytes);
-                    if (p == p0) tc_mma_ss<false>(d_tmem, adesc, bdesc, idesc);
-                    else tc_mma_ss<true>(d_tmem, adesc, bdesc, idesc);
-                    tc_mma_ss<true>(d_tmem, adesc + 128, bdesc + 128, idesc);
-                    tc_mma_ss<true>(d_tmem, adesc + 256, bdesc + 256, idesc);
-                    tc_mma_ss<true>(d_tmem, adesc + 384, bdesc + 384, idesc);
-                }
-                tc_commit(&sm->empty[s]);
+                uint8_t *const st = sm->pool + s * P.stage_bytes;
+                const int w0 = twi << P.lgBW, h0 = thi << P.lgBH, b0 = tbi * bstep;
+                if (!mbar_wait_warp(&sm->empty[s], ph ^ 1u, abort_flag, P.status, 32)) { ok = false; break; }
+                if (lane == 0) mbar_expect_tx(&sm->full[s], bytes);
+                __syncwarp();
+                if (active) tma_load_4d(st + my_off, my_map, &sm->full[s], my_c0, w0 * my_sw + my_dw, h0 * my_sh + my_dh, b0);
+                if (++twi == P.tw) { twi = 0; if (++thi == P.th) { thi = 0; ++tbi; } }
                 if (++s == P.stages) { s = 0; ph ^= 1u; }
             }
-            if (ok) tc_commit(&sm->acc_full[buf]);
-            ++lu;
+        }
+    } else if (warp == 1 || warp == kDwIssuerB) {
+        // Two MMA-issuing threads, each with an accumulator of its own (256 tensor-memory columns).
+        // tcgen05.mma holds its issuing thread until the tensor core accepts the instruction, so whatever one
+        // thread executes between two MMAs (waits, descriptor arithmetic, commits) is time the tensor core
+        // idles unless another thread has work queued.  The threads take alternate k-blocks and the epilogue
+        // adds the two accumulators; the ring has an even number of stages, so a stage always belongs to the
+        // same thread and each full barrier has one waiter that sees every phase in turn.
+        if (lane == 0) {
+            const uint32_t me = warp == 1 ? 0u : 1u;
+            uint32_t it = 0, lu = 0;     // lu counts the units that accumulate something
+            bool ok = true;
+            const uint32_t pool = smem_u32(sm->pool);
+            const uint32_t st_step = (uint32_t)P.stage_bytes >> 4;
+            for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
+                int ot, gi, nb, sp, p0, p1;
+                unit_range(u, ot, gi, nb, sp, p0, p1);
+                if (p1 <= p0) continue;                      // the epilogue writes zeros for an empty split
+                const uint32_t idesc = make_idesc_mn(128, 64 * nb);
+                if (!mbar_wait(&sm->acc_empty, (lu & 1u) ^ 1u, abort_flag, P.status, 0)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem + me * kDwAccCols;
+                // descriptors of stage 0; a stage further is st_step more in the address field.
+                // 16 pixels per MMA = 16 rows of 128 bytes = 2048 bytes
+                const uint64_t adesc0 = smem_desc_mn_sw128(pool, (uint32_t)P.blk_bytes);
+                uint64_t bd[kDwMaxMma];
+                if (P.row_mode) {
+                    const uint32_t xt = pool + (uint32_t)P.x_off;
+#pragma unroll
+                    for (int j = 0; j < kDwMaxMma; ++j) bd[j] = smem_desc_mn_sw128_groups(xt + P.mma_off[j], 128, P.k_group_bytes);
+                } else {
+                    const uint64_t b0 = smem_desc_mn_sw128(pool + (uint32_t)P.x_off, (uint32_t)P.blk_bytes);
+#pragma unroll
+                    for (int j = 0; j < kDwMaxMma; ++j) bd[j] = b0 + 128 * j;
+                }
+                uint32_t s = it % P.stages;
+                uint32_t ph = (it / P.stages) & 1u;
+                uint32_t acc = 0;
+                for (int p = p0; p < p1; ++p, ++it) {
+                    if ((it & 1u) == me) {
+                        if (!mbar_wait(&sm->full[s], ph, abort_flag, P.status, 0)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint64_t so = (uint64_t)(s * st_step);
+                        dw_mma(d_tmem, adesc0 + so, bd[0] + so, idesc, acc);
+                        dw_mma(d_tmem, adesc0 + so + 128, bd[1] + so, idesc, 1u);
+                        dw_mma(d_tmem, adesc0 + so + 256, bd[2] + so, idesc, 1u);
+                        dw_mma(d_tmem, adesc0 + so + 384, bd[3] + so, idesc, 1u);
+                        if (P.n_mma > 4) {
+                            dw_mma(d_tmem, adesc0 + so + 512, bd[4] + so, idesc, 1u);
+                            dw_mma(d_tmem, adesc0 + so + 640, bd[5] + so, idesc, 1u);
+                            dw_mma(d_tmem, adesc0 + so + 768, bd[6] + so, idesc, 1u);
+                            dw_mma(d_tmem, adesc0 + so + 896, bd[7] + so, idesc, 1u);
+                        }
+                        acc = 1u;
+                        dw_commit(&sm->empty[s]);
+                    }
+                    if (++s == (uint32_t)P.stages) { s = 0; ph ^= 1u; }
+                }
+                if (ok) dw_commit(&sm->acc_full);
+                ++lu;
+            }
         }
     } else {
         const int q = warp & 3;
-        uint32_t lu = 0;
+        uint32_t lu = 0, it = 0;
         for (int u = blockIdx.x; u < P.total_units; u += gridDim.x) {
             int ot, gi, nb, sp, p0, p1;
             unit_range(u, ot, gi, nb, sp, p0, p1);
             const bool have = p1 > p0;
-            const int buf = lu & 1;
-            if (have && !mbar_wait_warp(&sm->acc_full[buf], (lu >> 1) & 1u, abort_flag, P.status, 32)) break;
+            // which of the two accumulators hold something: the threads took the k-blocks in turn, starting
+            // with the one whose number is the parity of `it`
+            const uint32_t len = (uint32_t)(p1 - p0);
+            const bool have0 = have && ((len + ((it & 1u) == 0u ? 1u : 0u)) >> 1) > 0u;
+            const bool have1 = have && ((len + ((it & 1u) == 1u ? 1u : 0u)) >> 1) > 0u;
+            it += len;
+            if (have && !mbar_wait_warp(&sm->acc_full, lu & 1u, abort_flag, P.status, 32)) break;
             tc_fence_after();
             const int o = ot * 128 + q * 32 + lane;
             float *row = P.partial + (long long)sp * P.split_stride + (long long)o * P.K;
+            int rr_ = 0, cb0 = 0;
+            if (P.row_mode) row_group(gi, rr_, cb0);
+            const int n_chunks = nb * 2;
 #pragma unroll 1
-            for (int c = 0; c < nb * 2; ++c) {
-                // columns [32c, 32c+32) of the accumulator: half of column block c/2
+            for (int c = 0; c < n_chunks; ++c) {
+                // columns [32cc, 32cc+32) of an accumulator: half of column block cc/2
+                const int cc = c;
                 int t, cb;
                 if (P.row_mode) {
-                    const int r = gi / P.cblocks;
-                    cb = gi - r * P.cblocks;
-                    t = r * P.kw + (c >> 1);
+                    cb = cb0;
+                    t = rr_ * P.kw + (cc >> 1);
                 } else {
-                    const int i = gi * kDwMaxCb + (c >> 1);
+                    const int i = gi * kDwMaxCb + (cc >> 1);
                     t = i / P.cblocks;
                     cb = i - t * P.cblocks;
                 }
-                const int ch0 = cb * 64 + (c & 1) * 32;          // first input channel of this chunk
+                const int ch0 = cb * 64 + (cc & 1) * 32;          // first input channel of this chunk
                 float *dst = row + P.taps[t].koff + ch0;
                 uint32_t v[32];
-                if (have) {
-                    tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + buf * kDwAccCols + c * 32, v);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                } else {
+                const uint32_t t_lane = tmem + ((uint32_t)(q * 32) << 16) + cc * 32;
+                {
+                    // the sum of the two threads' accumulators (fixed order: deterministic)
+                    uint32_t w[32];
+                    if (have0) tmem_ld32(t_lane, v);
+                    if (have1) tmem_ld32(t_lane + kDwAccCols, w);
+                    if (have0) tmem_wait_ld(v);
+                    if (have1) tmem_wait_ld(w);
+                    if (!have0) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = 0u;
+                        for (int j = 0; j < 32; ++j) v[j] = 0u;
+                    }
+                    if (have1) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(w[j]));
+                    }
                 }
                 if (P.vec_ok && ch0 + 32 <= P.Cin) {
                     // through shared memory, so that a store instruction writes four whole 128-byte
@@ -268,7 +341,7 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
             if (have) {
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sm->acc_empty[buf]);
+                if (lane == 0) mbar_arrive(&sm->acc_empty);
                 ++lu;
             }
         }
@@ -286,12 +359,22 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
     }
 }
 
+// dW = sum over the splits of their partial tiles, added in split order (deterministic).  A thread owns one
+// output; the loads of eight splits are in flight before the first is added.
 __global__ void __launch_bounds__(256)
 dw_reduce_kernel(const float *__restrict__ partial, long long n, int splits, float *__restrict__ dW)
 {
     for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256) {
         float s = 0.0f;
-        for (int k = 0; k < splits; ++k) s += __ldg(partial + (long long)k * n + i);
+        int k = 0;
+        for (; k + 8 <= splits; k += 8) {
+            float v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = __ldg(partial + (long long)(k + j) * n + i);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) s += v[j];
+        }
+        for (; k < splits; ++k) s += __ldg(partial + (long long)k * n + i);
         dW[i] = s;
     }
 }
@@ -333,43 +416,85 @@ int dw_plan(const twn_conv_desc_t *d, int sm_count, DwPlan *plan)
     plan->Ho = (d->H + 2 * d->pad_h - d->kh) / d->stride_h + 1;
     plan->Wo = (d->W + 2 * d->pad_w - d->kw) / d->stride_w + 1;
     TWN_REQUIRE(plan->Ho > 0 && plan->Wo > 0, TWN_ERR_INVALID_ARG);
-    // pixel box: 64 = BB x BH x BW, fewest tiles
-    long long best = -1;
-    for (int a = 0; a <= 6; ++a)
-        for (int b = 0; a + b <= 6; ++b) {
-            const int BW = 1 << a, BH = 1 << b, BB = kDwPix >> (a + b);
-            if (BW * d->stride_w > 256 || BH * d->stride_h > 256) continue;
-            const long long tiles = ((plan->Wo + BW - 1) / BW) * ((plan->Ho + BH - 1) / BH) * ((d->B + BB - 1) / BB);
-            if (best < 0 || tiles < best || (tiles == best && a > P.lgBW)) { best = tiles; P.lgBW = a; P.lgBH = b; }
-        }
-    const int BW = 1 << P.lgBW, BH = 1 << P.lgBH, BB = kDwPix >> (P.lgBW + P.lgBH);
-    P.tw = (int)((plan->Wo + BW - 1) / BW);
-    P.th = (int)((plan->Ho + BH - 1) / BH);
-    P.tb = (int)((d->B + BB - 1) / BB);
-    TWN_REQUIRE(best > 0 && best <= 0x7fffffffLL, TWN_ERR_INVALID_ARG);
-    P.pix_tiles = (int)best;
     P.n_otiles = (int)((d->Cout + 127) / 128);
     P.n_taps = d->kh * d->kw;
     P.cblocks = (int)((d->Cin + 63) / 64);
     P.n_colblocks = P.n_taps * P.cblocks;
-    P.n_groups = (P.n_colblocks + kDwMaxCb - 1) / kDwMaxCb;
     P.kw = d->kw;
-    P.stage_bytes = (2 + kDwMaxCb) * kDwBlockBytes;
-    // row mode: stride 1, 2..4 taps per filter row, the tile inside one image and at least 8 pixels wide
-    if (d->stride_h == 1 && d->stride_w == 1 && d->kw >= 2 && d->kw <= kDwMaxCb && BB == 1 && BW >= 8) {
-        P.row_mode = 1;
-        P.n_groups = d->kh * P.cblocks;
-        const int pitch = BW + d->kw - 1;                 // pixels per row of the widened tile
-        P.x_bytes = pitch * BH * 128;
-        P.k_group_bytes = BW == 8 ? pitch * 128 : 1024;   // second 8-pixel run of an MMA: next row, or same row
-        for (int i = 0; i < 4; ++i) {
-            const int h = (16 * i) / BW, w = (16 * i) % BW;
-            P.mma_off[i] = (h * pitch + w) * 128;
+    memset(P.mma_off, 0, sizeof P.mma_off);
+    const bool row_ok = d->stride_h == 1 && d->stride_w == 1 && d->kw >= 2 && d->kw <= kDwMaxCb;
+    // Pixel box of a k-block: kpix = BB x BH x BW, fewest tiles.  Row mode (see DwParams) needs a box at least 8
+    // pixels wide (its extra columns are a halo in w only, so the box may span several images).  Two sizes: a copy of 128 rows moves its bytes almost twice as fast as one
+    // of 64 (measured: 1.75 against 3.25 cycles per 128-byte row), so 128-pixel k-blocks are taken unless their
+    // padding costs more than a fifth (small images).
+    struct Box { long long tiles; int lgBW, lgBH; bool row; };
+    auto best_box = [&](int kpix) {
+        Box best = {-1, 0, 0, false};
+        int lg = 0;
+        while ((1 << lg) < kpix) ++lg;
+        for (int pass = 0; pass < 2; ++pass) {          // first among the boxes row mode can use, then among all
+            for (int a = 0; a <= lg; ++a)
+                for (int b = 0; a + b <= lg; ++b) {
+                    const int BW = 1 << a, BH = 1 << b, BB = kpix >> (a + b);
+                    if (BW * d->stride_w > 256 || BH * d->stride_h > 256 || BB > 256) continue;
+                    const bool row = row_ok && BW >= 8 && BW + d->kw - 1 <= 256;
+                    if (pass == 0 && !row) continue;
+                    const long long tiles = ((plan->Wo + BW - 1) / BW) * ((plan->Ho + BH - 1) / BH) * ((d->B + BB - 1) / BB);
+                    if (best.tiles < 0 || tiles < best.tiles || (tiles == best.tiles && a > best.lgBW)) best = {tiles, a, b, row};
+                }
+            if (best.tiles >= 0) break;
         }
-        P.stage_bytes = 2 * kDwBlockBytes + ((P.x_bytes + 1023) & ~1023);
+        return best;
+    };
+    const Box b64 = best_box(64), b128 = best_box(128);
+    TWN_REQUIRE(b64.tiles > 0 && b64.tiles <= 0x7fffffffLL, TWN_ERR_INVALID_ARG);
+    // a box that row mode can use beats one it cannot (three copies per k-block instead of up to six)
+    bool use128 = b128.tiles > 0 && b128.tiles * 2 * 5 <= b64.tiles * 6 && (b128.row || !b64.row);
+    int BW = 0, BH = 0, BB = 0;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        const Box bx = use128 ? b128 : b64;
+        P.kpix = use128 ? 128 : 64;
+        P.n_mma = P.kpix / 16;
+        P.blk_bytes = P.kpix * 128;
+        P.lgBW = bx.lgBW; P.lgBH = bx.lgBH;
+        BW = 1 << P.lgBW; BH = 1 << P.lgBH; BB = P.kpix >> (P.lgBW + P.lgBH);
+        P.tw = (int)((plan->Wo + BW - 1) / BW);
+        P.th = (int)((plan->Ho + BH - 1) / BH);
+        P.tb = (int)((d->B + BB - 1) / BB);
+        P.pix_tiles = (int)bx.tiles;
+        P.n_groups = (P.n_colblocks + kDwMaxCb - 1) / kDwMaxCb;
+        // a layer of at most 64 output channels has one block of dZ per stage: rows 64..127 of the MMA then read
+        // whatever follows in the stage, into accumulator rows that are never stored
+        P.x_off = (d->Cout > 64 ? 2 : 1) * P.blk_bytes;
+        {
+            const int nb_max = P.n_colblocks < kDwMaxCb ? P.n_colblocks : kDwMaxCb;
+            P.stage_bytes = P.x_off + nb_max * P.blk_bytes;
+        }
+        P.row_mode = 0;
+        // row mode: stride 1, 2..4 taps per filter row, the tile at least 8 pixels wide
+        if (bx.row) {
+            P.row_mode = 1;
+            P.n_groups = d->kh * P.cblocks;
+            const int pitch = BW + d->kw - 1;                 // pixels per row of the widened tile
+            P.x_bytes = pitch * BH * BB * 128;       // rows of consecutive images follow each other: no halo in h
+            P.k_group_bytes = BW == 8 ? pitch * 128 : 1024;   // second 8-pixel run of an MMA: next row, or same row
+            for (int i = 0; i < P.n_mma; ++i) {
+                const int h = (16 * i) / BW, w = (16 * i) % BW;
+                P.mma_off[i] = (h * pitch + w) * 128;
+            }
+            P.stage_bytes = P.x_off + ((P.x_bytes + 1023) & ~1023);
+        }
+        // the MMA reads two blocks of dZ whatever Cout is: the stage must hold that many bytes
+        if (P.stage_bytes < 2 * P.blk_bytes) P.stage_bytes = 2 * P.blk_bytes;
+        P.stages = kDwPoolBytes / P.stage_bytes;
+        if (P.stages > kDwMaxStages) P.stages = kDwMaxStages;
+        // the two issuing threads take alternate stages of the ring: an even count
+        P.stages &= ~1;
+        // large k-blocks only with a ring of at least four of them
+        if (!use128 || P.stages >= 4) break;
+        use128 = false;
     }
-    P.stages = kDwPoolBytes / P.stage_bytes;
-    if (P.stages > kDwMaxStages) P.stages = kDwMaxStages;
+    TWN_REQUIRE(P.stages >= 2, TWN_ERR_INVALID_ARG);
     const long long units = (long long)P.n_otiles * P.n_groups;
     // as many splits as keep the unit count within two full rounds of the grid (never a third,
     // nearly empty round)
@@ -434,7 +559,7 @@ int dw_run(const twn_conv_desc_t *d, const void *X, long long x_pix, long long x
     DwParams &P = plan.P;
     P.partial = static_cast<float *>(workspace);
     P.status = dev_status;
-    const int BW = 1 << P.lgBW, BH = 1 << P.lgBH, BB = kDwPix >> (P.lgBW + P.lgBH);
+    const int BW = 1 << P.lgBW, BH = 1 << P.lgBH, BB = P.kpix >> (P.lgBW + P.lgBH);
 
     CUtensorMap map_dz, map_x;
     {
