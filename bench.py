@@ -866,9 +866,19 @@ class NetWorkload:
                 n += 1 + (1 if L.small_cin else 0)                       # forward (+ im2col or input fold)
                 if self.train:
                     n += 1 if L.fold else 0                              # folded codes
-                    n += 1 + 2 + (1 if L.fold else 0)                    # act_bwd, dW + reduce (+ unfold)
+                    n += 1 + 1 + (1 if L.fold else 0)                    # act_bwd, dW (+ unfold)
+                    # the reduction of the pixel splits of dW runs only when there is more than one split
+                    if L.fold:
+                        n += 1
+                    else:
+                        d = L.extra["dw_desc"]
+                        splits = self.twn.conv2d_bwd_weight_workspace_bytes(d) // (d.Cout * d.kh * d.kw * d.Cin * 4)
+                        n += 1 if splits > 1 else 0
                     if L.src != "input":
-                        n += L.stride * L.stride                         # backward for data
+                        # backward for data: one launch per residue class of the stride that a tap reaches
+                        # (a 1x1 projection shortcut adds into the dense gradient in place: one class)
+                        shortcut = L.k == 1 and L.stride > 1 and not L.relu and not L.residual
+                        n += 1 if shortcut else L.stride * L.stride
             elif op[0] in ("maxpool", "avgpool"):
                 n += 2 if self.train else 1
         if self.train:

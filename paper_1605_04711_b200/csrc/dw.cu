@@ -557,7 +557,8 @@ int dw_run(const twn_conv_desc_t *d, const void *X, long long x_pix, long long x
     EncodeTiledFn enc = dw_encode_fn();
     if (!enc) return TWN_ERR_CUDA;
     DwParams &P = plan.P;
-    P.partial = static_cast<float *>(workspace);
+    // a single split needs no reduction: its tile is the result
+    P.partial = P.splits == 1 ? dW : static_cast<float *>(workspace);
     P.status = dev_status;
     const int BW = 1 << P.lgBW, BH = 1 << P.lgBH, BB = P.kpix >> (P.lgBW + P.lgBH);
 
@@ -597,7 +598,7 @@ int dw_run(const twn_conv_desc_t *d, const void *X, long long x_pix, long long x
     const long long n = P.split_stride;
     long long rb = (n + 255) / 256;
     if (rb > dev.sm_count * 8) rb = dev.sm_count * 8;
-    dw_reduce_kernel<<<(int)rb, 256, 0, s>>>(P.partial, n, P.splits, dW);
+    if (P.splits > 1) dw_reduce_kernel<<<(int)rb, 256, 0, s>>>(P.partial, n, P.splits, dW);
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }

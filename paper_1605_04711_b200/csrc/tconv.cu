@@ -1129,6 +1129,13 @@ int conv_bwd_data_impl(const twn_conv_desc_t *d, const void *dZ, const uint32_t 
                 }
             }
             g.code_bits = bits;
+            // A residue class no tap reaches gets epilogue(0); when the epilogue only adds a second gradient
+            // branch that already lives in dX (in place), that leaves the class as it is: nothing to launch.
+            if (g.n_taps == 0 && epi && epi->residual == dX && epi->residual_op == TWN_RESIDUAL_ADD && !epi->scale &&
+                !epi->shift && !epi->relu && epi->residual_dtype == epi->out_dtype) {
+                --cls;              // the class takes no stream slot
+                continue;
+            }
             rc = launch_conv(g, dZ, T_bwd, stats, epi, dX, TWN_F32, dev_status, s);
             if (rc != TWN_OK && first_error == TWN_OK) first_error = rc;
         }

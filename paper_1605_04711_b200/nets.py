@@ -315,9 +315,28 @@ class TernaryNet:
                 return None
             return P if consumers.get(P.name) == [L] else None
 
+        # A projection shortcut (a layer read only as the residual input of another layer) shares its input with
+        # the first convolution of its block.  Its backward pass is taken after that convolution's: the dense
+        # gradient is written first, and the strided shortcut then adds into it in place, which lets
+        # twn_conv2d_bwd_data skip the residue classes its single tap never reaches.
+        def is_shortcut(L):
+            if L.relu or L.residual or L.fold or L.small_cin or L.src == "input":
+                return False
+            users = consumers.get(L.name, [])
+            return users == [None]
+        order, deferred = [], {}
+        for op in reversed(self.ops):
+            if op[0] == "layer" and is_shortcut(op[1]):
+                deferred[op[1].src] = op
+                continue
+            order.append(op)
+            if op[0] == "layer" and op[1].src in deferred:
+                order.append(deferred.pop(op[1].src))
+        order.extend(deferred.values())
+
         main = torch.cuda.current_stream()
         self.dw_stream.wait_stream(main)
-        for op in reversed(self.ops):
+        for op in order:
             kind = op[0]
             if kind == "layer":
                 L: Layer = op[1]
