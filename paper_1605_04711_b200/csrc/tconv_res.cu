@@ -28,7 +28,7 @@
 //   warps 2-9   epilogue: two sets of four (one warp per tensor-memory lane quadrant), the sets
 //               take alternate tiles
 //   warp 10     one thread issues the tcgen05.mma of the odd tiles
-// All warps decode the weights before the roles start.
+// All warps but the producer decode the weights before their roles start; the producer fetches meanwhile.
 //
 // Every wait on an mbarrier is bounded; on expiry the kernel records TWN_ERR_TIMEOUT, all roles
 // leave their loops, tensor memory is freed and the grid exits.
@@ -178,62 +178,71 @@ tconv_res_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // per-channel scale and shift; the decoded weights are +-2, so half of alpha scales the accumulators
-    if (threadIdx.x < kNMax) {
-        const int c = threadIdx.x;
-        const float alpha = (P.alpha ? (float)(*P.alpha) : 1.0f) * (P.code_bits == 2 ? 1.0f / kDecodedUnit : 1.0f);
-        const bool c_ok = c < P.Cout;
-        ctl->sc[c] = ((P.scale && c_ok) ? __ldg(P.scale + c) : 1.0f) * alpha;
-        ctl->sf[c] = (P.shift && c_ok) ? __ldg(P.shift + c) : 0.0f;
-    }
-    for (int t = threadIdx.x; t <= P.n_taps && t <= kMaxTaps; t += kThreads)
-        ctl->tap[t] = make_uint2(t < P.n_taps ? (uint32_t)P.a_off[t] : 0u, (uint32_t)(t * P.n_cblk) * ((uint32_t)(P.N * 128) >> 4));
-    // Decode the layer: item (channel n, k-block u) = 64 codes = 16 bytes -> 128 bytes of bf16, written as
-    // row n of k-block u in the K-major layout the MMA reads (16-byte chunk j of row n at chunk j ^ (n & 7)).
-    // Code words past the end of a row are clamped into it: they only ever meet activations that the TMA
-    // zero-fills.  Rows past Cout are zero.
-    {
-        const uint32_t wts = base_u32 + P.wts_off;
-        const int items = P.N * P.kbpt;
-        for (int i = threadIdx.x; i < items; i += kThreads) {
-            const int u = i / P.N, n = i - u * P.N;
-            const int t = u / P.n_cblk, cb = u - t * P.n_cblk;
-            const uint32_t *rowp = P.T + (long long)(n < P.Cout ? n : P.Cout - 1) * P.wpr;
-            uint32_t wv[4] = {0u, 0u, 0u, 0u};
-            const long long last = P.wpr - 1;
-            if (P.code_bits == 2) {
-                const long long word = (P.koff[t] >> 4) + cb * (kBlockK / 16);
-                if (P.codes_aligned) {
-                    uint4 c;
-                    ld_nc_v4(c, rowp + word);
-                    wv[0] = c.x; wv[1] = c.y; wv[2] = c.z; wv[3] = c.w;
-                } else {
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) ld_nc_u32(wv[g], rowp + (word + g < last ? word + g : last));
-                }
-            } else {
-                const long long word = (P.koff[t] >> 5) + cb * (kBlockK / 32);
-#pragma unroll
-                for (int g = 0; g < 2; ++g) ld_nc_u32(wv[g], rowp + (word + g < last ? word + g : last));
-            }
-            uint32_t out[32];
-            if (P.code_bits == 2) decode_kblock<2>(wv, out);
-            else decode_kblock<1>(wv, out);
-            if (n >= P.Cout) {
-#pragma unroll
-                for (int j = 0; j < 32; ++j) out[j] = 0u;
-            }
-            const uint32_t dst = wts + (uint32_t)(u * P.N + n) * 128u;
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                st_shared_v4(dst + (uint32_t)((j ^ (n & 7)) << 4), out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
+    // The producer warp does not take part in the set-up below: it signals the barriers it has initialised
+    // and starts fetching the first activation tiles at once, so that their latency (the operands come from
+    // DRAM) runs beside the decoding of the weights instead of after it.
+    if (warp == 0) {
+        asm volatile("bar.arrive 1, %0;" ::"n"(kThreads) : "memory");
+    } else {
+        constexpr int kWorkers = kThreads - 32;
+        const int tid = threadIdx.x - 32;
+        // per-channel scale and shift; the decoded weights are +-2, so half of alpha scales the accumulators
+        if (tid < kNMax) {
+            const int c = tid;
+            const float alpha = (P.alpha ? (float)(*P.alpha) : 1.0f) * (P.code_bits == 2 ? 1.0f / kDecodedUnit : 1.0f);
+            const bool c_ok = c < P.Cout;
+            ctl->sc[c] = ((P.scale && c_ok) ? __ldg(P.scale + c) : 1.0f) * alpha;
+            ctl->sf[c] = (P.shift && c_ok) ? __ldg(P.shift + c) : 0.0f;
         }
-        // the tensor core reads shared memory through the async proxy
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        for (int t = tid; t <= P.n_taps && t <= kMaxTaps; t += kWorkers)
+            ctl->tap[t] = make_uint2(t < P.n_taps ? (uint32_t)P.a_off[t] : 0u, (uint32_t)(t * P.n_cblk) * ((uint32_t)(P.N * 128) >> 4));
+        // Decode the layer: item (channel n, k-block u) = 64 codes = 16 bytes -> 128 bytes of bf16, written as
+        // row n of k-block u in the K-major layout the MMA reads (16-byte chunk j of row n at chunk j ^ (n & 7)).
+        // Code words past the end of a row are clamped into it: they only ever meet activations that the TMA
+        // zero-fills.  Rows past Cout are zero.
+        {
+            const uint32_t wts = base_u32 + P.wts_off;
+            const int items = P.N * P.kbpt;
+            for (int i = tid; i < items; i += kWorkers) {
+                const int u = i / P.N, n = i - u * P.N;
+                const int t = u / P.n_cblk, cb = u - t * P.n_cblk;
+                const uint32_t *rowp = P.T + (long long)(n < P.Cout ? n : P.Cout - 1) * P.wpr;
+                uint32_t wv[4] = {0u, 0u, 0u, 0u};
+                const long long last = P.wpr - 1;
+                if (P.code_bits == 2) {
+                    const long long word = (P.koff[t] >> 4) + cb * (kBlockK / 16);
+                    if (P.codes_aligned) {
+                        uint4 c;
+                        ld_nc_v4(c, rowp + word);
+                        wv[0] = c.x; wv[1] = c.y; wv[2] = c.z; wv[3] = c.w;
+                    } else {
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) ld_nc_u32(wv[g], rowp + (word + g < last ? word + g : last));
+                    }
+                } else {
+                    const long long word = (P.koff[t] >> 5) + cb * (kBlockK / 32);
+#pragma unroll
+                    for (int g = 0; g < 2; ++g) ld_nc_u32(wv[g], rowp + (word + g < last ? word + g : last));
+                }
+                uint32_t out[32];
+                if (P.code_bits == 2) decode_kblock<2>(wv, out);
+                else decode_kblock<1>(wv, out);
+                if (n >= P.Cout) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) out[j] = 0u;
+                }
+                const uint32_t dst = wts + (uint32_t)(u * P.N + n) * 128u;
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    st_shared_v4(dst + (uint32_t)((j ^ (n & 7)) << 4), out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
+            }
+            // the tensor core reads shared memory through the async proxy
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+        tc_fence_before();
+        asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
+        tc_fence_after();
     }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
     const uint32_t tmem = ctl->tmem_base;
 
     if (warp == 0) {
