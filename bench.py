@@ -936,7 +936,7 @@ class NetWorkload:
 
     def measured_traffic(self):
         """DRAM bytes per step of the ternary contractions of the ResNet-18 step: sum over the launches of
-        dram__bytes_read.sum + dram__bytes_write.sum over the 59 forward and backward-for-data launches of one step,
+        dram__bytes_read.sum + dram__bytes_write.sum over the 50 forward and backward-for-data launches of one step,
         from one ncu capture of this workload at its full size (profiles/tconv_resnet18_step_dram.md); None for the
         other workloads."""
         return TRAFFIC_RESNET18_STEP if self.kind in ("resnet18_train", "resnet18_train_sgd") else None
@@ -1018,7 +1018,7 @@ class NetWorkload:
                              f"scaled to batch {B} ({spent:.1f} s of CPU; oracle step time {total_s:.1f} s)"), oracle.num_threads()
 
 # From the ncu capture summarised in profiles/tconv_resnet18_step_dram.md (see NetWorkload.measured_traffic).
-TRAFFIC_RESNET18_STEP = 907.9e6
+TRAFFIC_RESNET18_STEP = 873.1e6
 
 WORKLOADS = {"ternarize": lambda: TernarizeWorkload(), "binarize": lambda: BinarizeWorkload(), "sgd_ternarize": lambda: SgdTernarizeWorkload(), "ternarize_rows": lambda: TernarizeRowsWorkload(), "resnet18_train": lambda: NetWorkload("resnet18_train"),
              "gemm_16384": lambda: GemmWorkload(16384), "gemm_4096": lambda: GemmWorkload(4096),
