@@ -40,16 +40,42 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples the SM clock and the clock event reasons of one GPU while the timed region runs: through NVML
+    from a thread every 2 ms (a timed region of a few tens of milliseconds still gets samples), else with an
+    nvidia-smi loop.  Reads only; no setting of the GPU is touched."""
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
-    def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
+    def __init__(self, index: int, uuid: str = ""):
+        self.index, self.uuid, self.rows, self.proc, self.nvml = index, uuid, [], None, None
+        self.first, self.halt, self.max_mhz = 0, threading.Event(), None
+
+    def _nvml_handle(self):
+        import pynvml
+        pynvml.nvmlInit()
+        if self.uuid:
+            try:
+                return pynvml, pynvml.nvmlDeviceGetHandleByUUID(self.uuid if self.uuid.startswith("GPU-") else "GPU-" + self.uuid)
+            except pynvml.NVMLError:
+                pass
+        return pynvml, pynvml.nvmlDeviceGetHandleByIndex(self.index)
 
     def start(self):
         try:
+            self.nvml, self.handle = self._nvml_handle()
+            self.max_mhz = float(self.nvml.nvmlDeviceGetMaxClockInfo(self.handle, self.nvml.NVML_CLOCK_SM))
+            self.source = "nvml, every 2 ms"
+            self.t = threading.Thread(target=self._poll, daemon=True)
+            self.t.start()
+            time.sleep(0.05)
+            self.first = len(self.rows)
+            return
+        except Exception:                     # no NVML binding or no permission: the nvidia-smi loop
+            self.nvml = None
+        try:
+            self.source = "nvidia-smi -lms 50"
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
                  "-i", str(self.index), "-lms", "50"], stdout=subprocess.PIPE, text=True)
@@ -60,32 +86,49 @@ class ClockSampler:
         except OSError:
             self.proc = None
 
+    def _poll(self):
+        n = self.nvml
+        bits = [(n.nvmlClocksEventReasonHwSlowdown, "hw_slowdown"), (n.nvmlClocksEventReasonHwThermalSlowdown, "hw_thermal_slowdown"),
+                (n.nvmlClocksEventReasonSwThermalSlowdown, "sw_thermal_slowdown"), (n.nvmlClocksEventReasonSwPowerCap, "sw_power_cap")]
+        while not self.halt.is_set():
+            try:
+                mhz = n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM)
+                r = n.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
+                self.rows.append([str(mhz), str(self.max_mhz)] + ["Active" if r & b else "Not Active" for b, _ in bits])
+            except Exception:
+                pass
+            time.sleep(0.002)
+
     def _read(self):
         for line in self.proc.stdout:
             self.rows.append([c.strip() for c in line.split(",")])
 
     def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-        self.t.join(timeout=2)
+        if self.nvml is not None:
+            self.halt.set()
+            self.t.join(timeout=2)
+        elif self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+            self.t.join(timeout=2)
+        else:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no NVML binding and no nvidia-smi"]}
         sm, mx, reasons = [], None, set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in self.rows[self.first:]:
             try:
                 sm.append(float(r[0])); mx = float(r[1])
             except (ValueError, IndexError):
                 continue
-            for nm, v in zip(names, r[2:6]):
+            for nm, v in zip(self.NAMES, r[2:6]):
                 if v.lower().startswith("active"):
                     reasons.add(nm)
+        lo = min(sm) if sm else None
         sm.sort()
-        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_min_mhz": lo, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(sm), "source": self.source}
 
 
 def max_over_ranks(ms: float, world: int, dist=None, device=None) -> float:
@@ -1137,7 +1180,7 @@ def run_ours(args):
         each = sorted(evs[i].elapsed_time(evs[i + 1]) for i in range(n_steps))
         return ms / n_steps, {"median_ms": each[len(each) // 2], "min_ms": each[0], "steps": n_steps}
 
-    sampler = ClockSampler(local_rank) if rank == 0 else None
+    sampler = ClockSampler(local_rank, str(getattr(torch.cuda.get_device_properties(local_rank), 'uuid', ''))) if rank == 0 else None
     if sampler:
         sampler.start()
     ms, spread = timed(wl.step, steps, warmup)
