@@ -243,3 +243,12 @@ def test_resnet18_train_step_batch64(monkeypatch):
     check_forward(net, npix=96)
     check_pools(net, images=1)
     check_backward(net, npix=64, nent=96)
+
+
+def test_resnet18b_train_step_batch64(monkeypatch):
+    """The wider variant at the size the benchmark runs it: batch 64, 224 x 224."""
+    net = nets.resnet18b(batch=64, train=True)
+    run_train_step(net, monkeypatch)
+    check_forward(net, npix=64)
+    check_pools(net, images=1)
+    check_backward(net, npix=48, nent=64)
