@@ -236,6 +236,31 @@ __device__ __forceinline__ void tmem_wait_ld(uint32_t (&r)[32])
         :: "memory");
 }
 
+// Two fp32 values -> one bf16x2 word (round to nearest even), `lo` in the low half.
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    uint32_t pk;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(hi), "f"(lo));
+    return pk;
+}
+// Same, negative values clamped to zero (a NaN stays a NaN).
+__device__ __forceinline__ uint32_t pack_bf16x2_relu(float lo, float hi)
+{
+    uint32_t pk;
+    asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(hi), "f"(lo));
+    return pk;
+}
+// (x0, x1) <- (x0 * a0 + b0, x1 * a1 + b1), both lanes in one instruction.
+__device__ __forceinline__ void fma_f32x2(uint32_t &x0, uint32_t &x1, float a0, float a1, float b0, float b1)
+{
+    unsigned long long x, a, b;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(x) : "r"(x0), "r"(x1));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(a) : "f"(a0), "f"(a1));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(b) : "f"(b0), "f"(b1));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(x) : "l"(x), "l"(a), "l"(b));
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(x0), "=r"(x1) : "l"(x));
+}
+
 // Element pair j (0..7) of a packed code word -> two bf16 values in {-2, 0, +2}.  The pair's
 // fields sit 2*j bits below the top of the two half-words (bit 0 of a field = non-zero, bit 1 =
 // sign); shifted to the top they are the sign and the high exponent bit of a bf16, and

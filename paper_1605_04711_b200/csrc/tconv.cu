@@ -418,7 +418,9 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
         const int BWm = (1 << P.lgBW) - 1, BHm = (1 << P.lgBH) - 1;
         const bool out_bf16 = P.out_dtype == TWN_BF16, res_bf16 = P.res_dtype == TWN_BF16;
         const bool need_off = !P.tma_store || (P.residual && !P.res_tma);
-        const float floor_v = P.relu ? 0.0f : -INFINITY;
+        // the ReLU of a bf16 output rides on the conversion (a NaN stays a NaN); every other path clamps explicitly
+        const bool relu_in_cvt = P.relu && out_bf16 && P.tma_store;
+        const bool relu_here = P.relu && !relu_in_cvt;
         constexpr int kChunks = PIX / 32;
         constexpr int kMine = kChunks / kEpiSets;            // chunks of a tile this warp drains
         static_assert(kChunks % kEpiSets == 0, "the chunks of a tile are split evenly over the warps of a quadrant");
@@ -522,13 +524,13 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                     if (P.res_gate) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
-                            const float y = fmaxf(fmaf(__uint_as_float(v[j]), sc, sf), floor_v);
+                            const float y = fmaf(__uint_as_float(v[j]), sc, sf);
                             v[j] = __float_as_uint(__bfloat162float(rs[j * 32]) > 0.0f ? y : 0.0f);
                         }
                     } else {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
-                            v[j] = __float_as_uint(fmaxf(fmaf(__uint_as_float(v[j]), sc, sf) + __bfloat162float(rs[j * 32]), floor_v));
+                            v[j] = __float_as_uint(fmaf(__uint_as_float(v[j]), sc, sf) + __bfloat162float(rs[j * 32]));
                     }
                     // the buffer is free again: fetch the residual of the chunk after the next
                     __syncwarp();
@@ -544,11 +546,16 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
                             r = res_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(P.residual)[(size_t)o + n])
                                          : reinterpret_cast<const float *>(P.residual)[(size_t)o + n];
                         const float y = fmaf(__uint_as_float(v[j]), sc, sf);
-                        v[j] = __float_as_uint(P.res_gate ? (r > 0.0f ? fmaxf(y, floor_v) : 0.0f) : fmaxf(y + r, floor_v));
+                        v[j] = __float_as_uint(P.res_gate ? (r > 0.0f ? y : 0.0f) : y + r);
                     }
                 } else {
+                    // two pixels per instruction
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(fmaxf(fmaf(__uint_as_float(v[j]), sc, sf), floor_v));
+                    for (int j = 0; j < 32; j += 2) fma_f32x2(v[j], v[j + 1], sc, sc, sf, sf);
+                }
+                if (relu_here) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(fmaxf(__uint_as_float(v[j]), 0.0f));
                 }
                 if (P.tma_store) {
                     // a staging buffer holds 32 pixels of bf16 or 16 of fp32: one or two rounds per chunk
@@ -563,8 +570,8 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
 #pragma unroll
                             for (int j = 0; j < 32; j += 2) {
                                 // one packed conversion per two pixels
-                                uint32_t pk;
-                                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(__uint_as_float(v[j + 1])), "f"(__uint_as_float(v[j])));
+                                const uint32_t pk = relu_in_cvt ? pack_bf16x2_relu(__uint_as_float(v[j]), __uint_as_float(v[j + 1]))
+                                                                : pack_bf16x2(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
                                 st16[j * 32] = (uint16_t)pk;
                                 st16[(j + 1) * 32] = (uint16_t)(pk >> 16);
                             }

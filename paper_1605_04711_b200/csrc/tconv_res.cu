@@ -24,10 +24,10 @@
 // the same way, one tile ahead.
 //
 //   warp 0      TMA producer: one activation tile (with halo) per tile and 64-channel block
-//   warp 1      allocates tensor memory; one thread issues the tcgen05.mma of the even tiles of the block
+//   warp 1      allocates tensor memory; one thread issues the tcgen05.mma of every third tile of the block
 //   warps 2-9   epilogue: two sets of four (one warp per tensor-memory lane quadrant), the sets
 //               take alternate tiles
-//   warp 10     one thread issues the tcgen05.mma of the odd tiles
+//   warps 10-11 one thread each issues the tcgen05.mma of the other tiles, in turn
 // All warps but the producer decode the weights before their roles start; the producer fetches meanwhile.
 //
 // Every wait on an mbarrier is bounded; on expiry the kernel records TWN_ERR_TIMEOUT, all roles
@@ -51,8 +51,9 @@ constexpr int kNMax = 64;                 // output channels (UMMA N)
 constexpr int kAccBufs = 4;
 constexpr uint32_t kTmemCols = kAccBufs * kNMax;
 constexpr int kEpiWarps = 8;
+constexpr int kIssuers = 3;                // MMA-issuing threads: warp 1 and the warps after the epilogue warps
 constexpr int kIssuerB = 2 + kEpiWarps;    // the warp of the second MMA-issuing thread
-constexpr int kThreads = 32 * (3 + kEpiWarps);
+constexpr int kThreads = 32 * (2 + kEpiWarps + (kIssuers - 1));
 constexpr int kMaxStages = 8;
 constexpr int kStageBuf = 4096;           // per-warp staging: 32 pixels x 128 bytes
 constexpr int kSmemLimit = 232448;
@@ -61,8 +62,9 @@ struct Ctl {
     unsigned long long full[kMaxStages], empty[kMaxStages];
     unsigned long long acc_full[kAccBufs], acc_empty[kAccBufs];
     unsigned long long res_full[kEpiWarps];
-    unsigned long long turn[2];           // issuer -> issuer: "every stage up to the end of my tile has landed"
-    float sc[kNMax], sf[kNMax];           // per-channel scale (alpha and the decode factor folded in) and shift
+    unsigned long long turn[kIssuers];           // issuer -> issuer: "every stage up to the end of my tile has landed"
+    alignas(16) float sc[kNMax];          // read with 16-byte loads
+    alignas(16) float sf[kNMax];          // per-channel scale (alpha and the decode factor folded in) and shift
     uint2 tap[kMaxTaps + 1];              // per tap: operand offsets of its first k-block (A inside a stage, B inside the weights), 16-byte units
     uint32_t tmem_base;
     volatile int abort_flag;
@@ -145,14 +147,12 @@ __device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr)
     asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
     return v;
 }
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
-{
-    uint32_t pk;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(hi), "f"(lo));
-    return pk;
-}
 
-__global__ void __launch_bounds__(kThreads, 1)
+// The register cap is below what one block per SM would allow (65536 / 384 = 170): the block then leaves room
+// on its SM for a small block of another stream.  In a training step the reduction kernels of the weight-
+// gradient stream run in that room beside this kernel; with 168 registers per thread they had to wait for it
+// (ResNet-18 step, batch 64: 1.424 ms against 1.387 ms with the cap; no spills either way).
+__global__ void __maxnreg__(144)
 tconv_res_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
                  const __grid_constant__ CUtensorMap map_r, const __grid_constant__ ResParams P)
 {
@@ -169,8 +169,7 @@ tconv_res_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         for (int s = 0; s < kMaxStages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
         for (int b = 0; b < kAccBufs; ++b) { mbar_init(&ctl->acc_full[b], 1); mbar_init(&ctl->acc_empty[b], 4); }
         for (int w = 0; w < kEpiWarps; ++w) mbar_init(&ctl->res_full[w], 1);
-        mbar_init(&ctl->turn[0], 1);
-        mbar_init(&ctl->turn[1], 1);
+        for (int i = 0; i < kIssuers; ++i) mbar_init(&ctl->turn[i], 1);
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -264,20 +263,23 @@ tconv_res_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 }
             }
         }
-    } else if (warp == 1 || warp == kIssuerB) {
-        // ------------------------------------------------ MMA issuers: two threads, alternate tiles
+    } else if (warp == 1 || warp >= kIssuerB) {
+        // ------------------------------------------------ MMA issuers: three threads, tiles in turn
         // Measured on B200: a 128x64x16 MMA with both operands in shared memory occupies the tensor core
         // for 48 cycles, and tcgen05.mma holds its issuing thread until the tensor core accepts it, so every
         // instruction that thread runs between two MMAs (address arithmetic, waits) is time the tensor core
-        // idles: one issuer reached 59 to 76 cycles per MMA, two issuers on different accumulators 48 whatever
-        // they execute in between.  Tiles alternate between the two threads; each works on the accumulator and
-        // the activation stages of its own tiles, so the two instruction streams never touch the same data.
-        // The stages form one ring that both threads consume, and an mbarrier wait only tells a phase from
+        // idles: one issuer reached 59 to 76 cycles per MMA, two issuers on different accumulators 48 while
+        // both are issuing.  A thread also waits three times per tile (token, accumulator, stage) and commits
+        // twice; with short tiles (16 MMAs in the folded first layer of ResNet-18) two threads spend so much of
+        // their time there that the tensor core idles half of the time, hence three.  The threads take the tiles
+        // in turn; each works on the accumulator and the activation stages of its own tile, so the instruction
+        // streams never touch the same data.
+        // The stages form one ring that all of them consume, and an mbarrier wait only tells a phase from
         // its neighbours: a thread may wait for "stage s, parity p" only once every earlier phase of that
         // barrier is known to be over.  So the threads pass a token: after seeing the last stage of its tile
-        // land, a thread lets the other one start waiting for the stages of the next tile.
+        // land, a thread lets the next one start waiting for the stages of the next tile.
         if (lane == 0 && P.kbpt > 0) {
-            const uint32_t me = warp == 1 ? 0u : 1u;
+            const uint32_t me = warp == 1 ? 0u : (uint32_t)(warp - kIssuerB + 1);
             const uint32_t idesc = make_idesc(kPix, P.N);
             const uint64_t adesc0 = smem_desc_k_sw128(base_u32, P.a_sbo);
             const uint64_t bdesc0 = smem_desc_sw128(base_u32 + P.wts_off);
@@ -292,18 +294,21 @@ tconv_res_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 for (int cb = 0; cb < P.n_cblk; ++cb)
                     if (++s == (uint32_t)P.n_stages) { s = 0; ph ^= 1u; }
             };
-            if (me) skip_tile();
+            for (uint32_t i = 0; i < me; ++i) skip_tile();
             bool ok = true;
             uint32_t lt = me;
-            for (int tile = blockIdx.x + (int)me * (int)gridDim.x; tile < P.total_tiles && ok; tile += 2 * (int)gridDim.x, lt += 2) {
+            for (int tile = blockIdx.x + (int)me * (int)gridDim.x; tile < P.total_tiles && ok; tile += kIssuers * (int)gridDim.x, lt += kIssuers) {
                 const uint32_t buf = lt & (kAccBufs - 1);
+                // The token first: once it is here, the threads of all earlier tiles are past their waits for an
+                // accumulator, so the accumulator barrier (shared by the issuing threads in turn) is at most one
+                // phase behind the one waited for.
+                if (lt > 0 && !mbar_wait(&ctl->turn[me], ((lt - 1) / kIssuers) & 1u, abort_flag, P.status, 0)) break;
                 if (!mbar_wait(&ctl->acc_empty[buf], ((lt / kAccBufs) & 1u) ^ 1u, abort_flag, P.status, 0)) break;
-                if (lt > 0 && !mbar_wait(&ctl->turn[me], ((lt - 1) >> 1) & 1u, abort_flag, P.status, 0)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem + buf * kNMax;
                 for (int cb = 0; cb < P.n_cblk; ++cb) {
                     if (!mbar_wait(&ctl->full[s], ph, abort_flag, P.status, 0)) { ok = false; break; }
-                    if (cb == P.n_cblk - 1) mbar_arrive(&ctl->turn[me ^ 1u]);
+                    if (cb == P.n_cblk - 1) mbar_arrive(&ctl->turn[me + 1 == kIssuers ? 0u : me + 1]);
                     tc_fence_after();
                     const uint32_t a_s = a_lo0 + s * a_step, b_s = b_lo0 + (uint32_t)cb * b_step;
                     uint2 cur = ctl->tap[0];
@@ -319,7 +324,10 @@ tconv_res_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     tc_commit_1t(&ctl->empty[s]);
                     if (++s == (uint32_t)P.n_stages) { s = 0; ph ^= 1u; }
                 }
-                if (ok) { tc_commit_1t(&ctl->acc_full[buf]); skip_tile(); }
+                if (ok) {
+                    tc_commit_1t(&ctl->acc_full[buf]);
+                    for (int i = 1; i < kIssuers; ++i) skip_tile();
+                }
             }
         }
     } else {
@@ -331,11 +339,11 @@ tconv_res_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         const uint32_t res = base_u32 + P.res_off + (uint32_t)ew * kStageBuf;
         const uint32_t my_row = (uint32_t)lane * 128u;
         const uint32_t sw_x = (uint32_t)(lane & 7);
-        const float floor_v = P.relu ? 0.0f : -INFINITY;
         const int chunks = (P.N + 31) >> 5;      // 32-channel chunks of the accumulator
+        const bool per_channel = P.scale != nullptr || P.shift != nullptr;
+        const float sc_all = ctl->sc[0];         // without a per-channel scale every entry is the same
         const int p0 = q * 32;                   // first tile pixel of this warp
         uint32_t nres = 0;
-        bool alive = true;
 
         auto tile_coords = [&](int tile, int &cw, int &ch, int &cbt) {
             int pt = tile;
@@ -356,7 +364,7 @@ tconv_res_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         if (P.has_res && lane == 0 && first_tile < P.total_tiles) res_load(first_tile);
 
         uint32_t lt = set;
-        for (int tile = first_tile; tile < P.total_tiles && alive; tile += 2 * (int)gridDim.x, lt += 2) {
+        for (int tile = first_tile; tile < P.total_tiles; tile += 2 * (int)gridDim.x, lt += 2) {
             int cw, ch, cbt;
             tile_coords(tile, cw, ch, cbt);
             const uint32_t buf = lt & (kAccBufs - 1);
@@ -368,34 +376,46 @@ tconv_res_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 __syncwarp();
             }
-            uint32_t v[32];
-#pragma unroll 1
-            for (int hf = 0; hf < chunks; ++hf) {
-                if (P.kbpt > 0) {
-                    tmem_ld32(t_acc + hf * 32, v);
-                    tmem_wait_ld(v);
-                    if (hf + 1 == chunks) {
-                        // the accumulator is in registers: hand it back
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&ctl->acc_empty[buf]);
+            // The whole accumulator goes to registers at once (one exposed tensor-memory latency per tile
+            // instead of one per 32 channels) and is handed back before any arithmetic.
+            uint32_t va[32], vb[32];
+            if (P.kbpt > 0) {
+                tmem_ld32(t_acc, va);
+                if (chunks > 1) tmem_ld32(t_acc + 32, vb);
+                tmem_wait_ld(va);
+                if (chunks > 1) tmem_wait_ld(vb);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->acc_empty[buf]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) va[j] = vb[j] = 0u;
+            }
+            if (P.has_res && !mbar_wait_warp(&ctl->res_full[ew], nres & 1u, abort_flag, P.status, 32)) break;
+            // 32 channels of this thread's pixel: affine (two channels per instruction), residual or gate, ReLU,
+            // conversion, staging
+            auto chunk = [&](uint32_t (&v)[32], const int hf) {
+                if (per_channel) {
+                    // all sixteen loads of the scales and shifts are issued before the first use
+                    const uint32_t sc_a = smem_u32(ctl->sc + hf * 32), sf_a = smem_u32(ctl->sf + hf * 32);
+                    uint4 a[8], b[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) a[j] = ld_shared_v4(sc_a + j * 16);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) b[j] = ld_shared_v4(sf_a + j * 16);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        fma_f32x2(v[4 * j + 0], v[4 * j + 1], __uint_as_float(a[j].x), __uint_as_float(a[j].y),
+                                  __uint_as_float(b[j].x), __uint_as_float(b[j].y));
+                        fma_f32x2(v[4 * j + 2], v[4 * j + 3], __uint_as_float(a[j].z), __uint_as_float(a[j].w),
+                                  __uint_as_float(b[j].z), __uint_as_float(b[j].w));
                     }
                 } else {
+                    // one factor for every channel (alpha and the decode factor): it lives in a register
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = 0u;
-                }
-                const float4 *sc4 = reinterpret_cast<const float4 *>(ctl->sc + hf * 32);
-                const float4 *sf4 = reinterpret_cast<const float4 *>(ctl->sf + hf * 32);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float4 a = sc4[j], b = sf4[j];
-                    v[4 * j + 0] = __float_as_uint(fmaf(__uint_as_float(v[4 * j + 0]), a.x, b.x));
-                    v[4 * j + 1] = __float_as_uint(fmaf(__uint_as_float(v[4 * j + 1]), a.y, b.y));
-                    v[4 * j + 2] = __float_as_uint(fmaf(__uint_as_float(v[4 * j + 2]), a.z, b.z));
-                    v[4 * j + 3] = __float_as_uint(fmaf(__uint_as_float(v[4 * j + 3]), a.w, b.w));
+                    for (int j = 0; j < 16; ++j) fma_f32x2(v[2 * j], v[2 * j + 1], sc_all, sc_all, 0.0f, 0.0f);
                 }
                 if (P.has_res) {
-                    if (hf == 0 && !mbar_wait_warp(&ctl->res_full[ew], nres & 1u, abort_flag, P.status, 32)) { alive = false; break; }
 #pragma unroll
                     for (int jj = 0; jj < 4; ++jj) {
                         const uint4 r = ld_shared_v4(res + my_row + ((((uint32_t)(hf * 4 + jj)) ^ sw_x) << 4));
@@ -406,30 +426,42 @@ tconv_res_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                             float &y0 = reinterpret_cast<float &>(v[jj * 8 + 2 * i]);
                             float &y1 = reinterpret_cast<float &>(v[jj * 8 + 2 * i + 1]);
                             if (P.res_gate) {
-                                y0 = r0 > 0.0f ? fmaxf(y0, floor_v) : 0.0f;
-                                y1 = r1 > 0.0f ? fmaxf(y1, floor_v) : 0.0f;
+                                y0 = r0 > 0.0f ? y0 : 0.0f;
+                                y1 = r1 > 0.0f ? y1 : 0.0f;
                             } else {
-                                y0 = fmaxf(y0 + r0, floor_v);
-                                y1 = fmaxf(y1 + r1, floor_v);
+                                y0 += r0;
+                                y1 += r1;
                             }
                         }
                     }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(fmaxf(__uint_as_float(v[j]), floor_v));
                 }
                 if (P.out_bf16) {
+                    // the ReLU rides on the conversion
+                    if (P.relu) {
 #pragma unroll
-                    for (int jj = 0; jj < 4; ++jj)
-                        st_shared_v4(stg + my_row + ((((uint32_t)(hf * 4 + jj)) ^ sw_x) << 4),
-                                     pack_bf16x2(__uint_as_float(v[jj * 8 + 0]), __uint_as_float(v[jj * 8 + 1])),
-                                     pack_bf16x2(__uint_as_float(v[jj * 8 + 2]), __uint_as_float(v[jj * 8 + 3])),
-                                     pack_bf16x2(__uint_as_float(v[jj * 8 + 4]), __uint_as_float(v[jj * 8 + 5])),
-                                     pack_bf16x2(__uint_as_float(v[jj * 8 + 6]), __uint_as_float(v[jj * 8 + 7])));
+                        for (int jj = 0; jj < 4; ++jj)
+                            st_shared_v4(stg + my_row + ((((uint32_t)(hf * 4 + jj)) ^ sw_x) << 4),
+                                         pack_bf16x2_relu(__uint_as_float(v[jj * 8 + 0]), __uint_as_float(v[jj * 8 + 1])),
+                                         pack_bf16x2_relu(__uint_as_float(v[jj * 8 + 2]), __uint_as_float(v[jj * 8 + 3])),
+                                         pack_bf16x2_relu(__uint_as_float(v[jj * 8 + 4]), __uint_as_float(v[jj * 8 + 5])),
+                                         pack_bf16x2_relu(__uint_as_float(v[jj * 8 + 6]), __uint_as_float(v[jj * 8 + 7])));
+                    } else {
+#pragma unroll
+                        for (int jj = 0; jj < 4; ++jj)
+                            st_shared_v4(stg + my_row + ((((uint32_t)(hf * 4 + jj)) ^ sw_x) << 4),
+                                         pack_bf16x2(__uint_as_float(v[jj * 8 + 0]), __uint_as_float(v[jj * 8 + 1])),
+                                         pack_bf16x2(__uint_as_float(v[jj * 8 + 2]), __uint_as_float(v[jj * 8 + 3])),
+                                         pack_bf16x2(__uint_as_float(v[jj * 8 + 4]), __uint_as_float(v[jj * 8 + 5])),
+                                         pack_bf16x2(__uint_as_float(v[jj * 8 + 6]), __uint_as_float(v[jj * 8 + 7])));
+                    }
                 } else {
                     // fp32: 32 channels are a 128-byte row of their own box; one store per chunk
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                     __syncwarp();
+                    if (P.relu) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(fmaxf(__uint_as_float(v[j]), 0.0f));
+                    }
 #pragma unroll
                     for (int jj = 0; jj < 8; ++jj)
                         st_shared_v4(stg + my_row + ((((uint32_t)jj) ^ sw_x) << 4), v[jj * 4 + 0], v[jj * 4 + 1], v[jj * 4 + 2],
@@ -438,8 +470,9 @@ tconv_res_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     __syncwarp();
                     if (lane == 0) tma_store_4d(&map_y, base + P.stg_off + (size_t)ew * kStageBuf, hf * 32, cw, ch, cbt);
                 }
-            }
-            if (!alive) break;
+            };
+            chunk(va, 0);
+            if (chunks > 1) chunk(vb, 1);
             if (P.out_bf16) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
