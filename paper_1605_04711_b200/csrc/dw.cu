@@ -17,7 +17,8 @@
 //
 //   warp 0     TMA producer: lane j issues copy j of a k-block (gradient blocks, activation blocks)
 //   warps 1, 6 one MMA-issuing thread each, alternate k-blocks, an accumulator each
-//   warps 2-5  epilogue: sum of the two accumulators -> workspace
+//   warps 2-5, 7-10  epilogue (two per tensor-memory lane quadrant, alternate 32-column chunks): sum of the
+//              two accumulators -> workspace
 #include <cstddef>
 
 #include "common.cuh"
@@ -30,8 +31,9 @@ constexpr int kDwMaxStages = 12;
 constexpr int kDwPoolBytes = 208 * 1024;         // operand ring: stages of one or two blocks of dZ plus the X blocks
 constexpr int kDwMaxMma = 8;                     // K = 16 pixels per MMA: 4 or 8 MMAs per k-block of 64 or 128 pixels
 constexpr int kDwMaxCb = 4;                      // up to 256 input channels per tile
-constexpr int kDwThreads = 224;
+constexpr int kDwThreads = 352;                  // warp 0 producer, 1 and 6 MMA issuers, 2-5 and 7-10 epilogue
 constexpr int kDwIssuerB = 6;                    // the warp of the second MMA-issuing thread
+constexpr int kDwEpiWarps = 8;                   // two per tensor-memory lane quadrant; they take alternate 32-column chunks
 constexpr int kDwMaxTaps = 64;
 constexpr int kDwAccCols = 256;
 
@@ -64,9 +66,9 @@ struct __align__(1024) DwSmem {
     // a stage: dZ as two 64-channel blocks (16 KB), then X: up to four 64-channel blocks, or one
     // tile with its extra columns in row mode
     uint8_t pool[kDwPoolBytes];
-    // per epilogue warp: 32 rows x 32 fp32 of the accumulator, 16-byte chunks XOR-swizzled by the
-    // row so that row-wise writes and the transposed reads are both free of bank conflicts
-    float4 stg[4][32][8];
+    // per epilogue warp: 32 rows x 16 fp32 of the accumulator (half a chunk), 16-byte pieces XOR-swizzled
+    // by the row so that row-wise writes and the transposed reads are both free of bank conflicts
+    float4 stg[kDwEpiWarps][32][4];
     unsigned long long full[kDwMaxStages], empty[kDwMaxStages], acc_full, acc_empty;
     uint32_t tmem_base;
     volatile int abort_flag;
@@ -99,7 +101,7 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
     if (threadIdx.x == 0) {
         for (int s = 0; s < kDwMaxStages; ++s) { mbar_init(&sm->full[s], 1); mbar_init(&sm->empty[s], 1); }
         mbar_init(&sm->acc_full, 2);
-        mbar_init(&sm->acc_empty, 4);
+        mbar_init(&sm->acc_empty, kDwEpiWarps);
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -259,7 +261,10 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
             }
         }
     } else {
+        // The accumulator of a unit is exposed time (a block mostly has one unit), so eight warps drain it: the
+        // two warps of a lane quadrant take alternate 32-column chunks.
         const int q = warp & 3;
+        const int set = warp > kDwIssuerB ? 1 : 0;
         uint32_t lu = 0, it = 0;
         for (int u = blockIdx.x; u < P.total_units; u += gridDim.x) {
             int ot, gi, nb, sp, p0, p1;
@@ -279,7 +284,7 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
             if (P.row_mode) row_group(gi, rr_, cb0);
             const int n_chunks = nb * 2;
 #pragma unroll 1
-            for (int c = 0; c < n_chunks; ++c) {
+            for (int c = set; c < n_chunks; c += 2) {
                 // columns [32cc, 32cc+32) of an accumulator: half of column block cc/2
                 const int cc = c;
                 int t, cb;
@@ -312,24 +317,28 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
                     }
                 }
                 if (P.vec_ok && ch0 + 32 <= P.Cin) {
-                    // through shared memory, so that a store instruction writes four whole 128-byte
-                    // lines (4 rows x 8 lanes x 16 bytes) instead of 16 bytes in each of 32 rows
-                    float4 (*stg)[8] = sm->stg[q];
+                    // through shared memory, half a chunk at a time, so that a store instruction writes eight
+                    // 64-byte runs (8 rows x 4 lanes x 16 bytes) instead of 16 bytes in each of 32 rows
+                    float4 (*stg)[4] = sm->stg[set * 4 + q];
+                    const int rr = lane >> 2, ch = lane & 3;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        stg[lane][j ^ (lane & 7)] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
-                                                                __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
-                    __syncwarp();
-                    const int rr = lane >> 3, ch = lane & 7;
-                    float *const base = P.partial + (long long)sp * P.split_stride + P.taps[t].koff + ch0 + ch * 4;
+                    for (int h = 0; h < 2; ++h) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int r = i * 4 + rr;
-                        const int orow = ot * 128 + q * 32 + r;
-                        if (orow < P.Cout)
-                            *reinterpret_cast<float4 *>(base + (long long)orow * P.K) = stg[r][ch ^ (r & 7)];
+                        for (int j = 0; j < 4; ++j)
+                            stg[lane][j ^ ((lane >> 1) & 3)] =
+                                make_float4(__uint_as_float(v[16 * h + 4 * j]), __uint_as_float(v[16 * h + 4 * j + 1]),
+                                            __uint_as_float(v[16 * h + 4 * j + 2]), __uint_as_float(v[16 * h + 4 * j + 3]));
+                        __syncwarp();
+                        float *const base = P.partial + (long long)sp * P.split_stride + P.taps[t].koff + ch0 + 16 * h + ch * 4;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int r = i * 8 + rr;
+                            const int orow = ot * 128 + q * 32 + r;
+                            if (orow < P.Cout)
+                                *reinterpret_cast<float4 *>(base + (long long)orow * P.K) = stg[r][ch ^ ((r >> 1) & 3)];
+                        }
+                        __syncwarp();
                     }
-                    __syncwarp();
                 } else if (o < P.Cout) {
                     {
 #pragma unroll
