@@ -54,7 +54,11 @@ struct DwParams {
     // 64-channel block.  Its kw column blocks read ONE activation tile with kw - 1 extra pixel
     // columns: tap s is the tile one pixel (128 bytes) further, so a single MMA of N = 64 kw
     // covers the row and the tile is loaded once instead of kw times.
+    // Column mode (row_mode = 2) is the same with the roles of rows and columns swapped, for stride-1 layers with
+    // one tap per filter row and 2..4 filter rows (the folded first layer of ResNet-18): the tile has kh - 1 extra
+    // rows per image and tap r is the tile one row further; `kw` then holds kh.
     int row_mode, kw, x_bytes, k_group_bytes;
+    int tap_stride_bytes;        // row / column mode: bytes between the tiles of consecutive taps (a pixel, or a row of the tile)
     int x_off;                   // byte offset of the activation blocks inside a stage (after the blocks of dZ)
     int kpix, n_mma, blk_bytes;  // pixels per k-block (64 or 128), its MMAs (K = 16 pixels each), bytes of one 64-channel block of it
     int mma_off[kDwMaxMma];      // byte offset of the 16 pixels of MMA i inside the activation tile
@@ -227,7 +231,7 @@ dw_kernel(const __grid_constant__ CUtensorMap map_dz, const __grid_constant__ CU
                 if (P.row_mode) {
                     const uint32_t xt = pool + (uint32_t)P.x_off;
 #pragma unroll
-                    for (int j = 0; j < kDwMaxMma; ++j) bd[j] = smem_desc_mn_sw128_groups(xt + P.mma_off[j], 128, P.k_group_bytes);
+                    for (int j = 0; j < kDwMaxMma; ++j) bd[j] = smem_desc_mn_sw128_groups(xt + P.mma_off[j], (uint32_t)P.tap_stride_bytes, P.k_group_bytes);
                 } else {
                     const uint64_t b0 = smem_desc_mn_sw128(pool + (uint32_t)P.x_off, (uint32_t)P.blk_bytes);
 #pragma unroll
@@ -388,6 +392,43 @@ dw_reduce_kernel(const float *__restrict__ partial, long long n, int splits, flo
     }
 }
 
+// The same sum for many splits of a small tile.  A warp owns 32 consecutive outputs; the eight warps of a
+// block take the splits k = g, g + 8, g + 16, ... (each warp in increasing k, up to eight loads in flight) and
+// warp 0 adds the eight sums in warp order: a fixed order of additions, the same on every run.  (One thread per
+// output is bound by the latency of its chain of loads when the splits are many and the outputs few; with few
+// splits and many outputs it is the faster form.)
+__global__ void __launch_bounds__(256)
+dw_reduce_many_kernel(const float *__restrict__ partial, long long n, int splits, float *__restrict__ dW)
+{
+    __shared__ float sums[8][32];
+    const int ix = threadIdx.x & 31, g = threadIdx.x >> 5;
+    for (long long base = (long long)blockIdx.x * 32; base < n; base += (long long)gridDim.x * 32) {
+        const long long i = base + ix;
+        float s = 0.0f;
+        if (i < n) {
+            for (int k = g; k < splits; k += 64) {
+                float v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int kk = k + 8 * j;
+                    v[j] = kk < splits ? __ldg(partial + (long long)kk * n + i) : 0.0f;
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) s += v[j];
+            }
+        }
+        sums[g][ix] = s;
+        __syncthreads();
+        if (g == 0 && i < n) {
+            float t = sums[0][ix];
+#pragma unroll
+            for (int w = 1; w < 8; ++w) t += sums[w][ix];
+            dW[i] = t;
+        }
+        __syncthreads();
+    }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -432,6 +473,7 @@ int dw_plan(const twn_conv_desc_t *d, int sm_count, DwPlan *plan)
     P.kw = d->kw;
     memset(P.mma_off, 0, sizeof P.mma_off);
     const bool row_ok = d->stride_h == 1 && d->stride_w == 1 && d->kw >= 2 && d->kw <= kDwMaxCb;
+    const bool col_ok = d->stride_h == 1 && d->stride_w == 1 && d->kw == 1 && d->kh >= 2 && d->kh <= kDwMaxCb;
     // Pixel box of a k-block: kpix = BB x BH x BW, fewest tiles.  Row mode (see DwParams) needs a box at least 8
     // pixels wide (its extra columns are a halo in w only, so the box may span several images).  Two sizes: a copy of 128 rows moves its bytes almost twice as fast as one
     // of 64 (measured: 1.75 against 3.25 cycles per 128-byte row), so 128-pixel k-blocks are taken unless their
@@ -446,10 +488,14 @@ int dw_plan(const twn_conv_desc_t *d, int sm_count, DwPlan *plan)
                 for (int b = 0; a + b <= lg; ++b) {
                     const int BW = 1 << a, BH = 1 << b, BB = kpix >> (a + b);
                     if (BW * d->stride_w > 256 || BH * d->stride_h > 256 || BB > 256) continue;
-                    const bool row = row_ok && BW >= 8 && BW + d->kw - 1 <= 256;
+                    // column mode also wants the 16 pixels of an MMA inside one image of the box
+                    const bool row = (row_ok && BW >= 8 && BW + d->kw - 1 <= 256) ||
+                                     (col_ok && BW >= 8 && BW * BH >= 16 && BH + d->kh - 1 <= 256);
                     if (pass == 0 && !row) continue;
                     const long long tiles = ((plan->Wo + BW - 1) / BW) * ((plan->Ho + BH - 1) / BH) * ((d->B + BB - 1) / BB);
-                    if (best.tiles < 0 || tiles < best.tiles || (tiles == best.tiles && a > best.lgBW)) best = {tiles, a, b, row};
+                    // among equally many tiles: wider rows, or in column mode taller boxes (fewer extra rows per pixel)
+                    const bool nicer = (col_ok && row) ? b > best.lgBH : a > best.lgBW;
+                    if (best.tiles < 0 || tiles < best.tiles || (tiles == best.tiles && nicer)) best = {tiles, a, b, row};
                 }
             if (best.tiles >= 0) break;
         }
@@ -480,16 +526,32 @@ int dw_plan(const twn_conv_desc_t *d, int sm_count, DwPlan *plan)
             P.stage_bytes = P.x_off + nb_max * P.blk_bytes;
         }
         P.row_mode = 0;
+        P.kw = d->kw;
+        P.tap_stride_bytes = 0;
         // row mode: stride 1, 2..4 taps per filter row, the tile at least 8 pixels wide
-        if (bx.row) {
+        if (bx.row && row_ok) {
             P.row_mode = 1;
             P.n_groups = d->kh * P.cblocks;
             const int pitch = BW + d->kw - 1;                 // pixels per row of the widened tile
             P.x_bytes = pitch * BH * BB * 128;       // rows of consecutive images follow each other: no halo in h
             P.k_group_bytes = BW == 8 ? pitch * 128 : 1024;   // second 8-pixel run of an MMA: next row, or same row
+            P.tap_stride_bytes = 128;
             for (int i = 0; i < P.n_mma; ++i) {
                 const int h = (16 * i) / BW, w = (16 * i) % BW;
                 P.mma_off[i] = (h * pitch + w) * 128;
+            }
+            P.stage_bytes = P.x_off + ((P.x_bytes + 1023) & ~1023);
+        } else if (bx.row) {
+            P.row_mode = 2;
+            P.kw = d->kh;                                     // taps of a unit
+            P.n_groups = P.cblocks;
+            const int rows = BH + d->kh - 1;                  // rows per image of the heightened tile
+            P.x_bytes = BW * rows * BB * 128;
+            P.k_group_bytes = 1024;                           // second 8-pixel run: same row, or the next row of the image
+            P.tap_stride_bytes = BW * 128;
+            for (int i = 0; i < P.n_mma; ++i) {
+                const int w = (16 * i) % BW, h = ((16 * i) / BW) % BH, b = (16 * i) / (BW * BH);
+                P.mma_off[i] = ((b * rows + h) * BW + w) * 128;
             }
             P.stage_bytes = P.x_off + ((P.x_bytes + 1023) & ~1023);
         }
@@ -588,7 +650,8 @@ int dw_run(const twn_conv_desc_t *d, const void *X, long long x_pix, long long x
         const long long pixp = x_pix ? x_pix : d->Cin, rowp = x_row ? x_row : d->W * pixp, imgp = x_img ? x_img : d->H * rowp;
         cuuint64_t strides[3] = {(cuuint64_t)pixp * 2, (cuuint64_t)rowp * 2, (cuuint64_t)imgp * 2};
         cuuint32_t box[4] = {64, (cuuint32_t)(BW * d->stride_w), (cuuint32_t)(BH * d->stride_h), (cuuint32_t)BB};
-        if (P.row_mode) box[1] = (cuuint32_t)(BW + d->kw - 1);
+        if (P.row_mode == 1) box[1] = (cuuint32_t)(BW + d->kw - 1);
+        if (P.row_mode == 2) box[2] = (cuuint32_t)(BH + d->kh - 1);
         cuuint32_t estr[4] = {1, (cuuint32_t)d->stride_w, (cuuint32_t)d->stride_h, 1};
         if (enc(&map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(X), dims, strides, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -605,9 +668,15 @@ int dw_run(const twn_conv_desc_t *d, const void *X, long long x_pix, long long x
     const int grid = dev.sm_count < P.total_units ? dev.sm_count : P.total_units;
     dw_kernel<<<grid, kDwThreads, smem_bytes, s>>>(map_dz, map_x, P);
     const long long n = P.split_stride;
-    long long rb = (n + 255) / 256;
-    if (rb > dev.sm_count * 8) rb = dev.sm_count * 8;
-    if (P.splits > 1) dw_reduce_kernel<<<(int)rb, 256, 0, s>>>(P.partial, n, P.splits, dW);
+    if (P.splits >= 40) {
+        long long rb = (n + 31) / 32;
+        if (rb > dev.sm_count * 8) rb = dev.sm_count * 8;
+        dw_reduce_many_kernel<<<(int)rb, 256, 0, s>>>(P.partial, n, P.splits, dW);
+    } else if (P.splits > 1) {
+        long long rb = (n + 255) / 256;
+        if (rb > dev.sm_count * 8) rb = dev.sm_count * 8;
+        dw_reduce_kernel<<<(int)rb, 256, 0, s>>>(P.partial, n, P.splits, dW);
+    }
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
 }

@@ -21,6 +21,11 @@ DW_CASES = [
     (1, 20, 20, 320, 72, 3, 1, 1),
     (5, 9, 11, 16, 40, 3, 2, 1),
     (16, 28, 28, 128, 128, 3, 1, 1),
+    # filters of one column (k = (kh, kw)): the tile carries its extra rows and serves all taps
+    (3, 20, 17, 64, 64, (4, 1), 1, 0),
+    (2, 9, 30, 128, 192, (3, 1), 1, 1),
+    (5, 33, 8, 64, 48, (2, 1), 1, 0),
+    (40, 6, 6, 64, 64, (4, 1), 1, 1),
 ]
 
 
@@ -30,7 +35,8 @@ def test_bwd_weight_matches_oracle(case):
     d = twn.conv_desc(B, H, W, Cin, Cout, k, s, p)
     X = dg.draw_bf16(0, f"dwx{case}", B * H * W * Cin, "normal").reshape(B, H, W, Cin)
     dZ = dg.draw_bf16(0, f"dwz{case}", B * d.Ho * d.Wo * Cout, "normal", 0.0, 0.1).reshape(B, d.Ho, d.Wo, Cout)
-    dW = torch.full((Cout, k, k, Cin), float("nan"), dtype=torch.float32, device="cuda")
+    kh, kw = (k, k) if isinstance(k, int) else k
+    dW = torch.full((Cout, kh, kw, Cin), float("nan"), dtype=torch.float32, device="cuda")
     ws = torch.empty(twn.conv2d_bwd_weight_workspace_bytes(d) + 16, dtype=torch.uint8, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     twn.conv2d_bwd_weight(d, dev_bf16(X), dev_bf16(dZ), dW, ws, status)
@@ -152,7 +158,8 @@ def test_folded_layer_is_the_strided_small_channel_conv(case):
     assert np.all(err <= 1e-4 * ref.alpha * A + 1e-6)
     # straight-through weight gradient of the same layer
     dZ = dg.draw_bf16(3, f"foldz{case}", B * d.Ho * d.Wo * Cout, "normal", 0.0, 0.1).reshape(B, d.Ho, d.Wo, Cout)
-    dW = torch.full((Cout, k, k, Cin), float("nan"), dtype=torch.float32, device="cuda")
+    kh, kw = (k, k) if isinstance(k, int) else k
+    dW = torch.full((Cout, kh, kw, Cin), float("nan"), dtype=torch.float32, device="cuda")
     ws = torch.empty(twn.conv2d_bwd_weight_folded_workspace_bytes(d), dtype=torch.uint8, device="cuda")
     twn.conv2d_bwd_weight_folded(d, Xf, dev_bf16(dZ), dW, ws, status)
     assert twn.read_status(status) == 0
