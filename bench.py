@@ -1061,7 +1061,7 @@ class NetWorkload:
                              f"scaled to batch {B} ({spent:.1f} s of CPU; oracle step time {total_s:.1f} s)"), oracle.num_threads()
 
 # From the ncu capture summarised in profiles/tconv_resnet18_step_dram.md (see NetWorkload.measured_traffic).
-TRAFFIC_RESNET18_STEP = 873.1e6
+TRAFFIC_RESNET18_STEP = 873.2e6
 
 WORKLOADS = {"ternarize": lambda: TernarizeWorkload(), "binarize": lambda: BinarizeWorkload(), "sgd_ternarize": lambda: SgdTernarizeWorkload(), "ternarize_rows": lambda: TernarizeRowsWorkload(), "resnet18_train": lambda: NetWorkload("resnet18_train"),
              "gemm_16384": lambda: GemmWorkload(16384), "gemm_4096": lambda: GemmWorkload(4096),
