@@ -236,6 +236,13 @@ __device__ __forceinline__ void tmem_wait_ld(uint32_t (&r)[32])
         :: "memory");
 }
 
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialization attribute may start once
+// every block of the kernel before it in the stream has called pdl_launch_dependents() (or exited); what it does
+// before pdl_wait() must not touch global memory that the earlier kernel writes or reads, and pdl_wait() returns
+// when the earlier kernel has completed and its writes are visible.  Without the attribute both are no-ops.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Two fp32 values -> one bf16x2 word (round to nearest even), `lo` in the low half.
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {

@@ -167,6 +167,7 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
     static_assert(kAccBufs * PIX + kStages * kAColsPerStage <= (int)kTmemCols, "tensor memory budget");
     
 
+    pdl_launch_dependents();
     extern __shared__ uint8_t smem_raw[];
     L *sm = reinterpret_cast<L *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     volatile int *abort_flag = &sm->abort_flag;
@@ -202,6 +203,8 @@ tconv_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    // the set-up above touched no global memory; everything below may read what the previous kernel wrote
+    pdl_wait();
     const uint32_t tmem = sm->tmem_base;
     const uint32_t tmem_acc = tmem;                       // kAccBufs x PIX columns
     const uint32_t tmem_a = tmem + kAccBufs * PIX;        // kStages x kAColsPerStage columns
@@ -740,7 +743,7 @@ int launch_conv_t(const Geometry &g, ConvParams &P, const void *X, const twn_dev
     }
     const int grid = dev.sm_count < P.total_tiles ? dev.sm_count : P.total_tiles;
     if (P.bn_partial && (size_t)P.total_tiles * kEpiSets * 2 * kChan * sizeof(float) > g.bn_partial_bytes) return TWN_ERR_WORKSPACE;
-    tconv_kernel<PIX, DS, BITS><<<grid, threads_conv(DS), smem_bytes, s>>>(map_x, map_y, map_r, P);
+    TWN_CUDA_OK(twn_launch_pdl(tconv_kernel<PIX, DS, BITS>, grid, threads_conv(DS), (size_t)smem_bytes, s, map_x, map_y, map_r, P));
     if (P.bn_partial)
         bn_reduce_kernel<<<(g.Cout + 7) / 8, 256, 0, s>>>(P.bn_partial, P.total_tiles, P.n_tiles, g.Cout, g.bn_sum, g.bn_sumsq);
     TWN_CUDA_OK(cudaGetLastError());

@@ -156,6 +156,7 @@ __global__ void __maxnreg__(144)
 tconv_res_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
                  const __grid_constant__ CUtensorMap map_r, const __grid_constant__ ResParams P)
 {
+    pdl_launch_dependents();
     extern __shared__ uint8_t smem_raw[];
     uint8_t *const base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     Ctl *const ctl = reinterpret_cast<Ctl *>(base + P.ctl_off);
@@ -180,6 +181,8 @@ tconv_res_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     // The producer warp does not take part in the set-up below: it signals the barriers it has initialised
     // and starts fetching the first activation tiles at once, so that their latency (the operands come from
     // DRAM) runs beside the decoding of the weights instead of after it.
+    // nothing above touched global memory; from here on every role reads what earlier kernels wrote
+    pdl_wait();
     if (warp == 0) {
         asm volatile("bar.arrive 1, %0;" ::"n"(kThreads) : "memory");
     } else {
@@ -657,7 +660,7 @@ int twn_detail::launch_conv_resident(const Geometry &g, const void *X, const uin
         attr_set[dev.ordinal] = true;
     }
     const int grid = dev.sm_count < P.total_tiles ? dev.sm_count : P.total_tiles;
-    tconv_res_kernel<<<grid, kThreads, smem_bytes, s>>>(map_x, map_y, map_r, P);
+    TWN_CUDA_OK(twn_launch_pdl(tconv_res_kernel, grid, kThreads, (size_t)smem_bytes, s, map_x, map_y, map_r, P));
     TWN_CUDA_OK(cudaGetLastError());
     *handled = true;
     return TWN_OK;
