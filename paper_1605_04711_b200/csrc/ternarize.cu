@@ -612,11 +612,56 @@ __device__ __forceinline__ void transpose_codes_body(const uint32_t *__restrict_
     }
 }
 
+// The same re-layout for filter banks whose channel counts are whole words on both sides (Cin % 16 == 0,
+// Cout % 64 == 0): a thread takes one tap, 64 output channels and 16 input channels, i.e. 64 input words (word
+// column (t*Cin + c0)/16 of rows o0 .. o0+63, read coalesced across the threads of a warp, which take consecutive
+// c0) and transposes four 16 x 16 blocks of codes in registers into the 16 runs of four output words
+// (rows c0 .. c0+15, word columns (t*Cout + o0)/16 ..).  One load per output word instead of sixteen.
+constexpr int kFastRows = 64;
+__host__ __device__ __forceinline__ bool transpose_fast_ok(int Cout, int Cin) { return Cin % 16 == 0 && Cout % kFastRows == 0; }
+__device__ __forceinline__ void transpose_codes_fast_body(const uint32_t *__restrict__ in, int ld_in, int Cout, int Cin,
+                                                          int taps, uint32_t *__restrict__ out, int ld_out,
+                                                          unsigned int vb, unsigned int vg)
+{
+    const int wpr_out = ld_out >> 4, wpr_in = ld_in >> 4;
+    const int cgs = Cin >> 4, ogs = Cout / kFastRows;
+    const int units = taps * ogs * cgs;
+    for (int u = vb * kThreads + threadIdx.x; u < units; u += vg * kThreads) {
+        const int cg = u % cgs;
+        const int og = (u / cgs) % ogs;
+        const int t = u / (cgs * ogs);
+        const int o0 = og * kFastRows, c0 = cg << 4;
+        const uint32_t *src = in + (size_t)o0 * wpr_in + ((t * Cin + c0) >> 4);
+        uint32_t *dst = out + (size_t)c0 * wpr_out + ((t * Cout + o0) >> 4);
+#pragma unroll 1
+        for (int q = 0; q < kFastRows / 16; ++q) {
+            uint32_t w[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) w[i] = __ldg(src + (size_t)(q * 16 + i) * wpr_in);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                uint32_t word = 0;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) word |= ((w[i] >> field_pos(j)) & 3u) << field_pos(i);
+                dst[(size_t)j * wpr_out + q] = word;
+            }
+        }
+    }
+    // columns past the last tap (a row pitch larger than taps * Cout) read as zero codes
+    const int used = (taps * Cout) >> 4;
+    if (used < wpr_out) {
+        const int pad = wpr_out - used;
+        for (int i = vb * kThreads + threadIdx.x; i < Cin * pad; i += vg * kThreads)
+            out[(size_t)(i / pad) * wpr_out + used + i % pad] = 0u;
+    }
+}
+
 __global__ void __launch_bounds__(kThreads)
 transpose_codes_kernel(const uint32_t *__restrict__ in, int ld_in, int Cout, int Cin,
                        int taps, uint32_t *__restrict__ out, int ld_out)
 {
-    transpose_codes_body(in, ld_in, Cout, Cin, taps, out, ld_out, blockIdx.x, gridDim.x);
+    if (transpose_fast_ok(Cout, Cin)) transpose_codes_fast_body(in, ld_in, Cout, Cin, taps, out, ld_out, blockIdx.x, gridDim.x);
+    else transpose_codes_body(in, ld_in, Cout, Cin, taps, out, ld_out, blockIdx.x, gridDim.x);
 }
 
 // The filter banks of a whole network in one launch (the backward pass of a step needs them all).
@@ -637,8 +682,12 @@ transpose_codes_batch_kernel(const __grid_constant__ TransposeBatch P)
     int t = 0;
     while (t + 1 < P.count && blockIdx.x >= P.first_block[t + 1]) ++t;
     const TransposeItem &it = P.item[t];
-    transpose_codes_body(it.in, it.ld_in, it.Cout, it.Cin, it.taps, it.out, it.ld_out,
-                         blockIdx.x - P.first_block[t], P.first_block[t + 1] - P.first_block[t]);
+    if (transpose_fast_ok(it.Cout, it.Cin))
+        transpose_codes_fast_body(it.in, it.ld_in, it.Cout, it.Cin, it.taps, it.out, it.ld_out,
+                                  blockIdx.x - P.first_block[t], P.first_block[t + 1] - P.first_block[t]);
+    else
+        transpose_codes_body(it.in, it.ld_in, it.Cout, it.Cin, it.taps, it.out, it.ld_out,
+                             blockIdx.x - P.first_block[t], P.first_block[t + 1] - P.first_block[t]);
 }
 
 // Codes of a stride-2 layer re-ordered for the folded input: folded row r' holds 64 columns,
@@ -1025,7 +1074,9 @@ extern "C" int twn_transpose_codes(const uint32_t *packed_fwd, int64_t ld_fwd,
     const long long words = d->Cin * (ld_bwd / 16);
     TWN_REQUIRE(words < 0x7fffffffLL && d->Cout * (ld_fwd / 16) < 0x7fffffffLL && ld_fwd < 0x7fffffffLL &&
                     ld_bwd < 0x7fffffffLL, TWN_ERR_INVALID_ARG);
-    transpose_codes_kernel<<<grid_for(words, dev.sm_count), kThreads, 0, twn_cu(stream)>>>(
+    // threads' worth of work: one output word each, or one tap x 64 x 16 block of codes each
+    const long long work = transpose_fast_ok((int)d->Cout, (int)d->Cin) ? taps * (d->Cout / kFastRows) * (d->Cin / 16) : words;
+    transpose_codes_kernel<<<grid_for(work, dev.sm_count), kThreads, 0, twn_cu(stream)>>>(
         packed_fwd, (int)ld_fwd, (int)d->Cout, (int)d->Cin, (int)taps, packed_bwd, (int)ld_bwd);
     TWN_CUDA_OK(cudaGetLastError());
     return TWN_OK;
@@ -1059,7 +1110,8 @@ extern "C" int twn_transpose_codes_batch(const twn_transpose_item_t *items, int 
         ti.Cout = (int)d->Cout; ti.Cin = (int)d->Cin; ti.taps = (int)taps;
         P.item[t] = ti;
         P.first_block[t] = g;
-        g += (unsigned int)grid_for(words, dev.sm_count);
+        const long long work = transpose_fast_ok(ti.Cout, ti.Cin) ? taps * (d->Cout / kFastRows) * (d->Cin / 16) : words;
+        g += (unsigned int)grid_for(work, dev.sm_count);
     }
     P.first_block[count] = g;
     transpose_codes_batch_kernel<<<g, kThreads, 0, twn_cu(stream)>>>(P);

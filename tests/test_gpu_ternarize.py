@@ -215,11 +215,23 @@ def test_unpack_flags_the_unused_field():
     assert out.cpu().tolist() == [[1, 0]]
 
 
-@pytest.mark.parametrize("Cout,Cin,k", [(64, 64, 3), (128, 64, 1), (10, 512, 1), (32, 8, 5), (6, 3, 3)])
+@pytest.mark.parametrize("Cout,Cin,k", [(64, 64, 3), (128, 64, 1), (10, 512, 1), (32, 8, 5), (6, 3, 3), (512, 256, 3), (192, 96, 3)])
 def test_transpose_codes(Cout, Cin, k):
     u = dg.draw(6, "tr", Cout * k * k * Cin, "uniform")
     codes = (np.where(u > 0.3, 1, 0) - np.where(u < -0.3, 1, 0)).astype(np.int8).reshape(Cout, k, k, Cin)
     ld_f, ld_b = twn.ld_for(k * k * Cin), twn.ld_for(k * k * Cout)
+    pf = dev_u32(oracle.pack(codes.reshape(Cout, -1), ld_f))
+    pb = torch.full((Cin, ld_b // 16), -1, dtype=torch.int32, device="cuda")
+    twn.transpose_codes(pf, ld_f, twn.conv_desc(1, 8, 8, Cin, Cout, k), pb, ld_b)
+    want = oracle.pack(np.ascontiguousarray(codes.transpose(3, 1, 2, 0)).reshape(Cin, -1), ld_b)
+    assert np.array_equal(host_u32(pb), want)
+
+
+def test_transpose_codes_with_a_wider_row_pitch_zeroes_the_rest_of_the_row():
+    Cout, Cin, k = 128, 48, 3
+    u = dg.draw(7, "trp", Cout * k * k * Cin, "uniform")
+    codes = (np.where(u > 0.3, 1, 0) - np.where(u < -0.3, 1, 0)).astype(np.int8).reshape(Cout, k, k, Cin)
+    ld_f, ld_b = twn.ld_for(k * k * Cin) + 64, twn.ld_for(k * k * Cout) + 128
     pf = dev_u32(oracle.pack(codes.reshape(Cout, -1), ld_f))
     pb = torch.full((Cin, ld_b // 16), -1, dtype=torch.int32, device="cuda")
     twn.transpose_codes(pf, ld_f, twn.conv_desc(1, 8, 8, Cin, Cout, k), pb, ld_b)
