@@ -36,7 +36,8 @@ static inline cudaStream_t twn_cu(twn_stream_t s) { return reinterpret_cast<cuda
 // Launch with programmatic stream serialization: the kernel may start while the kernel before it in the stream
 // is still draining (see pdl_wait in tc_ptx.cuh); its blocks run their set-up and wait there.
 template <typename... KArgs, typename... Args>
-static inline cudaError_t twn_launch_pdl(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t s, Args &&...args)
+static inline cudaError_t twn_launch_pdl(bool allow, void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t s,
+                                         Args &&...args)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
@@ -45,7 +46,7 @@ static inline cudaError_t twn_launch_pdl(void (*kernel)(KArgs...), int grid, int
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].val.programmaticStreamSerializationAllowed = allow ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);

@@ -660,7 +660,7 @@ int twn_detail::launch_conv_resident(const Geometry &g, const void *X, const uin
         attr_set[dev.ordinal] = true;
     }
     const int grid = dev.sm_count < P.total_tiles ? dev.sm_count : P.total_tiles;
-    TWN_CUDA_OK(twn_launch_pdl(tconv_res_kernel, grid, kThreads, (size_t)smem_bytes, s, map_x, map_y, map_r, P));
+    TWN_CUDA_OK(twn_launch_pdl(grid * 2 >= dev.sm_count, tconv_res_kernel, grid, kThreads, (size_t)smem_bytes, s, map_x, map_y, map_r, P));
     TWN_CUDA_OK(cudaGetLastError());
     *handled = true;
     return TWN_OK;
