@@ -612,19 +612,23 @@ __device__ __forceinline__ void transpose_codes_body(const uint32_t *__restrict_
     }
 }
 
-// The same re-layout for filter banks whose channel counts are whole words on both sides (Cin % 16 == 0,
-// Cout % 64 == 0): a thread takes one tap, 64 output channels and 16 input channels, i.e. 64 input words (word
+// The same re-layout for filter banks whose taps start on word boundaries on both sides (Cin % 16 == 0, and
+// Cout % 16 == 0 or a single tap): a thread takes one tap, 64 output channels and 16 input channels, i.e. 64 input words (word
 // column (t*Cin + c0)/16 of rows o0 .. o0+63, read coalesced across the threads of a warp, which take consecutive
 // c0) and transposes four 16 x 16 blocks of codes in registers into the 16 runs of four output words
 // (rows c0 .. c0+15, word columns (t*Cout + o0)/16 ..).  One load per output word instead of sixteen.
 constexpr int kFastRows = 64;
-__host__ __device__ __forceinline__ bool transpose_fast_ok(int Cout, int Cin) { return Cin % 16 == 0 && Cout % kFastRows == 0; }
+__host__ __device__ __forceinline__ bool transpose_fast_ok(int Cout, int Cin, int taps)
+{
+    return Cin % 16 == 0 && (Cout % 16 == 0 || taps == 1);
+}
+__host__ __device__ __forceinline__ int transpose_fast_groups(int Cout) { return (Cout + kFastRows - 1) / kFastRows; }
 __device__ __forceinline__ void transpose_codes_fast_body(const uint32_t *__restrict__ in, int ld_in, int Cout, int Cin,
                                                           int taps, uint32_t *__restrict__ out, int ld_out,
                                                           unsigned int vb, unsigned int vg)
 {
     const int wpr_out = ld_out >> 4, wpr_in = ld_in >> 4;
-    const int cgs = Cin >> 4, ogs = Cout / kFastRows;
+    const int cgs = Cin >> 4, ogs = transpose_fast_groups(Cout);
     const int units = taps * ogs * cgs;
     for (int u = vb * kThreads + threadIdx.x; u < units; u += vg * kThreads) {
         const int cg = u % cgs;
@@ -634,10 +638,11 @@ __device__ __forceinline__ void transpose_codes_fast_body(const uint32_t *__rest
         const uint32_t *src = in + (size_t)o0 * wpr_in + ((t * Cin + c0) >> 4);
         uint32_t *dst = out + (size_t)c0 * wpr_out + ((t * Cout + o0) >> 4);
 #pragma unroll 1
-        for (int q = 0; q < kFastRows / 16; ++q) {
+        for (int q = 0; q < kFastRows / 16 && o0 + q * 16 < Cout; ++q) {
+            // rows past Cout (the last group of a bank whose Cout is no multiple of 16) read as zero codes
             uint32_t w[16];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) w[i] = __ldg(src + (size_t)(q * 16 + i) * wpr_in);
+            for (int i = 0; i < 16; ++i) w[i] = o0 + q * 16 + i < Cout ? __ldg(src + (size_t)(q * 16 + i) * wpr_in) : 0u;
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
                 uint32_t word = 0;
@@ -648,7 +653,7 @@ __device__ __forceinline__ void transpose_codes_fast_body(const uint32_t *__rest
         }
     }
     // columns past the last tap (a row pitch larger than taps * Cout) read as zero codes
-    const int used = (taps * Cout) >> 4;
+    const int used = (taps * Cout + 15) >> 4;
     if (used < wpr_out) {
         const int pad = wpr_out - used;
         for (int i = vb * kThreads + threadIdx.x; i < Cin * pad; i += vg * kThreads)
@@ -660,7 +665,7 @@ __global__ void __launch_bounds__(kThreads)
 transpose_codes_kernel(const uint32_t *__restrict__ in, int ld_in, int Cout, int Cin,
                        int taps, uint32_t *__restrict__ out, int ld_out)
 {
-    if (transpose_fast_ok(Cout, Cin)) transpose_codes_fast_body(in, ld_in, Cout, Cin, taps, out, ld_out, blockIdx.x, gridDim.x);
+    if (transpose_fast_ok(Cout, Cin, taps)) transpose_codes_fast_body(in, ld_in, Cout, Cin, taps, out, ld_out, blockIdx.x, gridDim.x);
     else transpose_codes_body(in, ld_in, Cout, Cin, taps, out, ld_out, blockIdx.x, gridDim.x);
 }
 
@@ -682,7 +687,7 @@ transpose_codes_batch_kernel(const __grid_constant__ TransposeBatch P)
     int t = 0;
     while (t + 1 < P.count && blockIdx.x >= P.first_block[t + 1]) ++t;
     const TransposeItem &it = P.item[t];
-    if (transpose_fast_ok(it.Cout, it.Cin))
+    if (transpose_fast_ok(it.Cout, it.Cin, it.taps))
         transpose_codes_fast_body(it.in, it.ld_in, it.Cout, it.Cin, it.taps, it.out, it.ld_out,
                                   blockIdx.x - P.first_block[t], P.first_block[t + 1] - P.first_block[t]);
     else
@@ -1075,7 +1080,7 @@ extern "C" int twn_transpose_codes(const uint32_t *packed_fwd, int64_t ld_fwd,
     TWN_REQUIRE(words < 0x7fffffffLL && d->Cout * (ld_fwd / 16) < 0x7fffffffLL && ld_fwd < 0x7fffffffLL &&
                     ld_bwd < 0x7fffffffLL, TWN_ERR_INVALID_ARG);
     // threads' worth of work: one output word each, or one tap x 64 x 16 block of codes each
-    const long long work = transpose_fast_ok((int)d->Cout, (int)d->Cin) ? taps * (d->Cout / kFastRows) * (d->Cin / 16) : words;
+    const long long work = transpose_fast_ok((int)d->Cout, (int)d->Cin, (int)taps) ? taps * transpose_fast_groups((int)d->Cout) * (d->Cin / 16) : words;
     transpose_codes_kernel<<<grid_for(work, dev.sm_count), kThreads, 0, twn_cu(stream)>>>(
         packed_fwd, (int)ld_fwd, (int)d->Cout, (int)d->Cin, (int)taps, packed_bwd, (int)ld_bwd);
     TWN_CUDA_OK(cudaGetLastError());
@@ -1110,7 +1115,7 @@ extern "C" int twn_transpose_codes_batch(const twn_transpose_item_t *items, int 
         ti.Cout = (int)d->Cout; ti.Cin = (int)d->Cin; ti.taps = (int)taps;
         P.item[t] = ti;
         P.first_block[t] = g;
-        const long long work = transpose_fast_ok(ti.Cout, ti.Cin) ? taps * (d->Cout / kFastRows) * (d->Cin / 16) : words;
+        const long long work = transpose_fast_ok(ti.Cout, ti.Cin, ti.taps) ? taps * transpose_fast_groups(ti.Cout) * (d->Cin / 16) : words;
         g += (unsigned int)grid_for(work, dev.sm_count);
     }
     P.first_block[count] = g;
